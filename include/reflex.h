@@ -1,0 +1,167 @@
+/*
+ * reflex.h -- C ABI of the B200 (sm_100a) hot path of Reflex streaming inference: the
+ * per-denoising-step action-expert layer. Flow-phase-gated AdaRMSNorm, attention of the dynamic
+ * action-token queries over a KV context held in three regions (pinned static prefix, sliding
+ * ring, dynamic suffix), and the Euler flow update of the action chunk.
+ *
+ * Conventions
+ *   - Every function returns an int status: REFLEX_OK (0) or a negative REFLEX_ERR_* code. Nothing
+ *     throws, aborts or exits. reflex_last_error_string() gives a thread-local description of the
+ *     last failure on the calling thread.
+ *   - Arguments are validated on the host before anything is launched: a failing call launches
+ *     nothing and leaves cache state unchanged.
+ *   - All work is enqueued asynchronously on the caller's CUDA stream, passed as void*
+ *     (a cudaStream_t; NULL = the legacy default stream). Calls on one stream are ordered.
+ *   - The five hot-path calls allocate no memory ("zero dynamic allocations during the control
+ *     loop", Sec. 3.4). Device memory -- cache slabs, workspace, tensors -- is allocated by the
+ *     caller and lent as raw pointers; the library owns only the host-side handle.
+ *   - "device" / "host" beside a pointer says where the memory lives. Device tensors are dense,
+ *     row-major in the index order written, and must be 16-byte aligned (REFLEX_ERR_ALIGN).
+ *   - dtype is the storage type of K, V, Q, x, weights: REFLEX_DTYPE_BF16 or REFLEX_DTYPE_F32.
+ *     Accumulation, softmax state and normalisation statistics are always fp32.
+ *   - Symbols: B streams, L layers, Hq / Hkv query / KV heads (G = Hq/Hkv), d head_dim,
+ *     S static-prefix tokens (capacity S_max), N ring capacity in tokens, T dynamic action tokens
+ *     (capacity T_max), D norm width, Cd conditioning width, Hd gate-MLP hidden width, A action width,
+ *     K denoising steps.
+ */
+#ifndef REFLEX_H
+#define REFLEX_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define REFLEX_OK                    0
+#define REFLEX_ERR_INVALID_ARG      (-1)  /* NULL pointer, bad enum, id out of range or duplicated   */
+#define REFLEX_ERR_SHAPE            (-2)  /* a size outside the range the call or the handle accepts  */
+#define REFLEX_ERR_ALIGN            (-3)  /* a device pointer or row pitch not 16-byte aligned        */
+#define REFLEX_ERR_STATE            (-4)  /* e.g. attention on a stream whose prefix was never set    */
+#define REFLEX_ERR_CUDA             (-5)  /* a CUDA runtime/driver call failed                        */
+#define REFLEX_ERR_TIMEOUT          (-6)  /* a bounded device-side wait ran out (status word)         */
+#define REFLEX_ERR_NOT_IMPLEMENTED  (-7)
+
+#define REFLEX_DTYPE_BF16 0
+#define REFLEX_DTYPE_F32  1
+
+/* attention kernel selection (reflex_cache_set_attention_impl) */
+#define REFLEX_ATTN_AUTO   0   /* tensor-core kernel when the shape qualifies, else the SIMT kernel */
+#define REFLEX_ATTN_SIMT   1   /* fp32-FMA split-K kernel, any supported shape and dtype            */
+#define REFLEX_ATTN_TC     2   /* tcgen05 kernel only; REFLEX_ERR_NOT_IMPLEMENTED if it cannot run  */
+
+typedef struct reflex_cache reflex_cache_t; /* opaque, host-side */
+
+/* Geometry of a partitioned KV cache (Sec. 3.1: static prefix / sliding history / dynamic suffix;
+ * Sec. 3.4: one monolithic pre-allocated buffer, here with a stream axis added). */
+typedef struct {
+    int32_t L, B, Hq, Hkv, d;
+    int32_t S_max;   /* capacity of the static-prefix region, tokens            */
+    int32_t N;       /* capacity of the sliding ring, tokens                    */
+    int32_t T_max;   /* largest number of dynamic (action) tokens per call      */
+    int32_t dtype;   /* REFLEX_DTYPE_*                                           */
+} reflex_cache_desc;
+
+const char *reflex_last_error_string(void);
+const char *reflex_version(void);
+
+/* ---- helpers around the five hot-path calls -------------------------------------------------- */
+
+/* Bytes of ONE slab (K or V; the caller allocates two): [L][B][S_max + N][Hkv][d] elements of
+ * dtype. Rows [0, S_max) of a (layer, stream) block are the static region, rows [S_max, S_max+N)
+ * the ring in physical slot order. The dynamic suffix is never copied into the slab: attention
+ * reads it from the caller's tensors in place. Returns 0 for an invalid descriptor. */
+size_t reflex_cache_slab_bytes(const reflex_cache_desc *desc);
+
+/* Bytes of the workspace the caller lends: per-stream ring state, split-K partials, tickets,
+ * status word. Returns 0 for an invalid descriptor. */
+size_t reflex_workspace_bytes(const reflex_cache_desc *desc);
+
+/* Create a handle over caller-owned device memory. k_slab, v_slab (device, slab_bytes each, contents
+ * kept as found -- zero them for the paper's zero-initialised buffer) and workspace (device,
+ * workspace_bytes; its state part is initialised by this call on `stream`). ring_head0: host [B]
+ * initial write positions in [0, N), or NULL for 0. The handle keeps the pointers; the memory must
+ * outlive it. Requirements: Hq % Hkv == 0, d % 32 == 0, d <= 256, all sizes >= 1 (S_max may be 0). */
+int reflex_cache_create(const reflex_cache_desc *desc, void *k_slab, void *v_slab, void *workspace,
+                        const int32_t *ring_head0, void *stream, reflex_cache_t **out);
+int reflex_cache_destroy(reflex_cache_t *cache);
+
+/* Copy the device-side ring state to host arrays (each [B], any may be NULL) and refresh the
+ * handle's host mirror. static_len is -1 for a stream whose prefix was never set. Synchronises
+ * `stream`. The device copy is what kernels read, so replaying a captured CUDA graph of appends
+ * advances it without the host mirror; call this afterwards to resynchronise. */
+int reflex_cache_get_state(reflex_cache_t *cache, int32_t *static_len, int32_t *head, int32_t *count,
+                           int64_t *total_appended, void *stream);
+
+/* slot_of_age (host, [N]): physical ring slot of the token of age j (0 = oldest) for stream b,
+ * -1 beyond the live count, from the host mirror: slot = (head - count + j) mod N. */
+int reflex_cache_slot_map(reflex_cache_t *cache, int b, int32_t *slot_of_age);
+
+int reflex_cache_set_attention_impl(reflex_cache_t *cache, int impl);
+
+/* ---- the five hot-path calls ------------------------------------------------------------------ */
+
+/* Sec. 3.1 "Static Prefix ... computed once and permanently pinned"; timestep invariance of the
+ * encoder makes it valid for every denoising step. Writes K,V of the perception/language prefix of
+ * n_streams streams into rows [0, S[i]) of every layer and sets static_len. Nothing else changes
+ * (ring kept; rows beyond S[i] keep stale bytes and are masked by static_len).
+ *   stream_ids  host [n_streams], distinct, each in [0, B)
+ *   k_static, v_static  device [n_streams][L][S_src][Hkv][d]
+ *   S           host [n_streams], 0 <= S[i] <= min(S_src, S_max); NULL = S_src for all */
+int reflex_cache_init_static(reflex_cache_t *cache, const int32_t *stream_ids, int n_streams,
+                             const void *k_static, const void *v_static, int S_src, const int32_t *S,
+                             void *stream);
+
+/* Sec. 3.1 "Sliding History ... FIFO queue of the last N"; Sec. 3.4 circular pointer arithmetic into
+ * the pre-allocated buffer; App. B.1 "returns eviction count". Appends m tokens per stream in place,
+ * in every layer: token i goes to slot (head + i) mod N; head <- (head + m) mod N;
+ * count <- min(count + m, N). O(m) whatever the history length.
+ *   k_new, v_new  device [n_streams][L][m][Hkv][d]
+ *   m             1..N
+ *   evicted       host [n_streams] out, may be NULL: max(0, count + m - N) per stream (host mirror) */
+int reflex_cache_append_sliding(reflex_cache_t *cache, const int32_t *stream_ids, int n_streams,
+                                const void *k_new, const void *v_new, int m, int32_t *evicted,
+                                void *stream);
+
+/* Eq. 2 / App. B.3: y = x * rsqrt(mean_i x_i^2 + eps) * (1 + W2 SiLU(W1 c + b1) + b2), statistics
+ * and gate accumulation in fp32, one rounding to dtype on store. One gate vector per stream.
+ *   x, y     device [B][R][D], may alias
+ *   cond     device [B][Cd] dtype, or NULL when gate_buf holds a precomputed gate
+ *   W1 [Hd][Cd], b1 [Hd], W2 [D][Hd], b2 [D]  device, dtype (ignored when cond == NULL)
+ *   gate_buf device [B][D] fp32 or NULL.  cond != NULL, gate_buf == NULL: one fused launch.
+ *            cond != NULL, gate_buf != NULL: the gate is written to gate_buf, then used (two launches).
+ *            cond == NULL: gate_buf is an input.
+ * Requirements: D % 8 == 0, Cd % 8 == 0, Hd % 8 == 0, D <= 16384, Cd, Hd <= 4096. */
+int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, const void *b1,
+                      const void *W2, const void *b2, float *gate_buf, int B, int R, int D, int Cd,
+                      int Hd, float eps, int dtype, void *stream);
+
+/* Eq. 1 / App. A Prop. 1: for every stream b, KV head j and its G*T query rows,
+ *   out = softmax(scale * Q [K_pin; K_slide; K_dyn]^T) [V_pin; V_slide; V_dyn]
+ * over static rows [0, static_len[b]), the live ring slots (physical order; softmax does not depend
+ * on key order) and the T dynamic tokens, which are read from k_dyn/v_dyn in place and are new at
+ * every denoising step. Cached regions are only read.
+ *   q, out         device [B][T][Hq][d] dtype
+ *   k_dyn, v_dyn   device [B][T][Hkv][d] dtype
+ *   T              1..T_max
+ *   scale          <= 0 selects 1/sqrt(d)
+ *   dyn_mask       0: every query sees all T dynamic keys (Eq. 1 as printed);
+ *                  1: dynamic key j hidden from dynamic query i when j > i (causal suffix, Prop. 1) */
+int reflex_partitioned_attention(reflex_cache_t *cache, int layer, const void *q, const void *k_dyn,
+                                 const void *v_dyn, void *out, int T, float scale, int dyn_mask,
+                                 void *stream);
+
+/* Sec. 2.1 / App. C: forward Euler step k of K of the flow ODE, x <- x + dt * v with dt = -1/K
+ * (t runs from 1 to 0).
+ *   x       device [B][T][A] fp32 master copy, updated in place
+ *   v       device [B][T][A] dtype
+ *   x_lowp  device [B][T][A] dtype mirror of the updated x, or NULL
+ *   k, K    0 <= k < K (k only validated: dt does not depend on it) */
+int reflex_flow_step(void *x, const void *v, void *x_lowp, int B, int T, int A, int k, int K,
+                     int dtype, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REFLEX_H */

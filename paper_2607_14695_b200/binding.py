@@ -1,0 +1,218 @@
+"""Thin ctypes binding over libreflex_b200.so, same names as the C ABI in include/reflex.h.
+
+Argument marshalling only: every step of the hot path runs in the library's CUDA kernels. torch is
+used for device memory and streams. There is no CPU fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libreflex_b200.so")
+
+DTYPE_BF16 = 0
+DTYPE_F32 = 1
+ATTN_AUTO, ATTN_SIMT, ATTN_TC = 0, 1, 2
+
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_IMPLEMENTED = -1, -2, -3, -4, -5, -6, -7
+
+EXPORTS = [
+    "reflex_last_error_string", "reflex_version", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
+    "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
+    "reflex_cache_set_attention_impl", "reflex_cache_init_static", "reflex_cache_append_sliding",
+    "reflex_adarmsnorm", "reflex_partitioned_attention", "reflex_flow_step",
+]
+
+
+class CacheDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("L", "B", "Hq", "Hkv", "d", "S_max", "N", "T_max", "dtype")]
+
+
+class ReflexError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"reflex error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load():
+    """Load the C-ABI library (raises if it has not been built: there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_14695_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i, f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    i32p, i64p = ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)
+    dp = ctypes.POINTER(CacheDesc)
+    lib.reflex_last_error_string.restype = ctypes.c_char_p
+    lib.reflex_version.restype = ctypes.c_char_p
+    lib.reflex_cache_slab_bytes.argtypes = [dp]; lib.reflex_cache_slab_bytes.restype = ctypes.c_size_t
+    lib.reflex_workspace_bytes.argtypes = [dp]; lib.reflex_workspace_bytes.restype = ctypes.c_size_t
+    lib.reflex_cache_create.argtypes = [dp, vp, vp, vp, i32p, vp, ctypes.POINTER(vp)]
+    lib.reflex_cache_destroy.argtypes = [vp]
+    lib.reflex_cache_get_state.argtypes = [vp, i32p, i32p, i32p, i64p, vp]
+    lib.reflex_cache_slot_map.argtypes = [vp, i, i32p]
+    lib.reflex_cache_set_attention_impl.argtypes = [vp, i]
+    lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
+    lib.reflex_cache_append_sliding.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
+    lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+    lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
+    lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int or fn.restype is None:
+            fn.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(rc: int):
+    if rc != OK:
+        raise ReflexError(rc, load().reflex_last_error_string().decode())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _i32(seq: Optional[Sequence[int]]):
+    if seq is None:
+        return None
+    return (ctypes.c_int32 * len(seq))(*[int(v) for v in seq])
+
+
+def torch_dtype(dtype: int) -> torch.dtype:
+    return torch.bfloat16 if dtype == DTYPE_BF16 else torch.float32
+
+
+def dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    raise ValueError(f"unsupported storage dtype {t.dtype}")
+
+
+def reflex_version() -> str:
+    return load().reflex_version().decode()
+
+
+def reflex_cache_slab_bytes(desc: CacheDesc) -> int:
+    return int(load().reflex_cache_slab_bytes(ctypes.byref(desc)))
+
+
+def reflex_workspace_bytes(desc: CacheDesc) -> int:
+    return int(load().reflex_workspace_bytes(ctypes.byref(desc)))
+
+
+class Cache:
+    """Owns the device memory the library borrows (two slabs + workspace, allocated once through
+    torch) and the opaque handle."""
+
+    def __init__(self, L, B, Hq, Hkv, d, S_max, N, T_max, dtype, device="cuda:0", ring_head0=None, stream=None):
+        lib = load()
+        self.desc = CacheDesc(L, B, Hq, Hkv, d, S_max, N, T_max, dtype)
+        slab = reflex_cache_slab_bytes(self.desc)
+        wsb = reflex_workspace_bytes(self.desc)
+        if slab == 0 or wsb == 0:
+            raise ReflexError(ERR_SHAPE, "invalid cache descriptor")
+        self.device = torch.device(device)
+        tdt = torch_dtype(dtype)
+        self.k_slab = torch.zeros((L, B, S_max + N, Hkv, d), dtype=tdt, device=self.device)
+        self.v_slab = torch.zeros_like(self.k_slab)
+        assert self.k_slab.numel() * self.k_slab.element_size() == slab
+        self.workspace = torch.zeros((wsb,), dtype=torch.uint8, device=self.device)
+        self.handle = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib.reflex_cache_create(ctypes.byref(self.desc), _ptr(self.k_slab), _ptr(self.v_slab), _ptr(self.workspace),
+                                           _i32(ring_head0), _stream(stream), ctypes.byref(self.handle)))
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle:
+            load().reflex_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def reflex_cache_get_state(cache: Cache, stream=None):
+    B = cache.desc.B
+    sl, hd, ct = (ctypes.c_int32 * B)(), (ctypes.c_int32 * B)(), (ctypes.c_int32 * B)()
+    tot = (ctypes.c_int64 * B)()
+    _check(load().reflex_cache_get_state(cache.handle, sl, hd, ct, tot, _stream(stream)))
+    return list(sl), list(hd), list(ct), list(tot)
+
+
+def reflex_cache_slot_map(cache: Cache, b: int):
+    out = (ctypes.c_int32 * cache.desc.N)()
+    _check(load().reflex_cache_slot_map(cache.handle, int(b), out))
+    return list(out)
+
+
+def reflex_cache_set_attention_impl(cache: Cache, impl: int):
+    _check(load().reflex_cache_set_attention_impl(cache.handle, int(impl)))
+
+
+def reflex_cache_init_static(cache: Cache, stream_ids, k_static, v_static, S=None, stream=None):
+    """k_static, v_static: device [n][L][S_src][Hkv][d]."""
+    n = len(stream_ids)
+    S_src = int(k_static.shape[2]) if k_static is not None else 0
+    _check(load().reflex_cache_init_static(cache.handle, _i32(stream_ids), n, _ptr(k_static), _ptr(v_static), S_src,
+                                           _i32(S), _stream(stream)))
+
+
+def reflex_cache_append_sliding(cache: Cache, stream_ids, k_new, v_new, stream=None):
+    """k_new, v_new: device [n][L][m][Hkv][d]. Returns the per-stream eviction counts."""
+    n = len(stream_ids)
+    m = int(k_new.shape[2])
+    ev = (ctypes.c_int32 * n)()
+    _check(load().reflex_cache_append_sliding(cache.handle, _i32(stream_ids), n, _ptr(k_new), _ptr(v_new), m, ev, _stream(stream)))
+    return list(ev)
+
+
+def reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6, stream=None):
+    """x, y [B][R][D]; cond [B][Cd] or None (then gate_buf [B][D] fp32 is the precomputed gate)."""
+    B, R, D = x.shape
+    Hd, Cd = (W1.shape if W1 is not None else (0, 0))
+    _check(load().reflex_adarmsnorm(_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf),
+                                    B, R, D, int(Cd), int(Hd), float(eps), dtype_code(x), _stream(stream)))
+    return y
+
+
+def reflex_partitioned_attention(cache: Cache, layer, q, k_dyn, v_dyn, out, scale=0.0, dyn_mask=0, stream=None):
+    """q, out [B][T][Hq][d]; k_dyn, v_dyn [B][T][Hkv][d]."""
+    T = int(q.shape[1])
+    _check(load().reflex_partitioned_attention(cache.handle, int(layer), _ptr(q), _ptr(k_dyn), _ptr(v_dyn), _ptr(out), T,
+                                               float(scale), int(dyn_mask), _stream(stream)))
+    return out
+
+
+def reflex_flow_step(x, v, x_lowp, k, K, stream=None):
+    """x [B][T][A] fp32 in place; v [B][T][A] storage dtype; x_lowp optional mirror."""
+    B, T, A = x.shape
+    _check(load().reflex_flow_step(_ptr(x), _ptr(v), _ptr(x_lowp), B, T, A, int(k), int(K), dtype_code(v), _stream(stream)))
+    return x

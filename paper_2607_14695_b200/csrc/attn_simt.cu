@@ -1,0 +1,239 @@
+// Partitioned attention (Eq. 1), SIMT form: fp32 FMA, one warp per query row, online softmax over 32-key
+// tiles, optional split over the key range with a merge of (m, l, acc) partials. Serves every supported
+// shape and storage type; the tensor-core kernel takes over where the query tile is large enough.
+//
+// Keys are enumerated in one logical index space per stream:
+//   [0, S)            static rows (S = static_len)
+//   [S, S+N)          ring slots in PHYSICAL order; slot p is live iff ((p - (head-count)) mod N) < count
+//   [S+N, S+N+T)      dynamic tokens, read in place from the caller's tensors
+// Softmax does not depend on key order, so the ring is never unrolled or gathered.
+#include <math.h>
+
+#include "reflex_internal.cuh"
+
+namespace reflex {
+
+template <typename T, int DPL> struct RowIO;
+template <int DPL> struct RowIO<__nv_bfloat16, DPL> {
+    // lane-owned slice of DPL consecutive elements
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&f)[DPL]) {
+        if constexpr (DPL == 8) {
+            uint4 u = *reinterpret_cast<const uint4 *>(p);
+            const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+        } else {
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) f[i] = __bfloat162float(p[i]);
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, const float (&f)[DPL]) {
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) p[i] = __float2bfloat16_rn(f[i]);
+    }
+};
+template <int DPL> struct RowIO<float, DPL> {
+    static __device__ __forceinline__ void load(const float *p, float (&f)[DPL]) {
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) f[i] = p[i];
+    }
+    static __device__ __forceinline__ void store(float *p, const float (&f)[DPL]) {
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) p[i] = f[i];
+    }
+};
+
+template <typename T> __device__ __forceinline__ float ld_f(const T *p);
+template <> __device__ __forceinline__ float ld_f<float>(const float *p) { return *p; }
+template <> __device__ __forceinline__ float ld_f<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+
+// dot of a K row (global, storage type) with a query row (shared, fp32), 8 elements per step
+template <typename T>
+__device__ __forceinline__ float dot_row(const T *__restrict__ k, const float *__restrict__ q_s, int d)
+{
+    float acc0 = 0.f, acc1 = 0.f;
+    for (int e = 0; e < d; e += 8) {
+        float f[8];
+        RowIO<T, 8>::load(k + e, f);
+        const float4 qa = *reinterpret_cast<const float4 *>(q_s + e);
+        const float4 qb = *reinterpret_cast<const float4 *>(q_s + e + 4);
+        acc0 = fmaf(f[0], qa.x, acc0); acc1 = fmaf(f[1], qa.y, acc1);
+        acc0 = fmaf(f[2], qa.z, acc0); acc1 = fmaf(f[3], qa.w, acc1);
+        acc0 = fmaf(f[4], qb.x, acc0); acc1 = fmaf(f[5], qb.y, acc1);
+        acc0 = fmaf(f[6], qb.z, acc0); acc1 = fmaf(f[7], qb.w, acc1);
+    }
+    return acc0 + acc1;
+}
+
+constexpr int kSimtWarps = 4;
+
+// grid = (ceil(T*Hq / kSimtWarps), B, nsplit)
+template <typename T, int DPL>
+__global__ void __launch_bounds__(kSimtWarps * 32)
+attn_simt_kernel(AttnParams p)
+{
+    constexpr int d = DPL * 32;
+    __shared__ __align__(16) float q_s[kSimtWarps][d];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int b = blockIdx.y, split = blockIdx.z;
+    const int rows = p.T * p.Hq;
+    const int r = blockIdx.x * kSimtWarps + warp;
+    if (r >= rows) return;  // no block-wide barrier below
+    const int t = r / p.Hq, h = r % p.Hq;
+    const int kv = h / (p.Hq / p.Hkv);
+
+    const StreamState st = p.state[b];
+    const int S = st.static_len > 0 ? st.static_len : 0;
+    const int N = p.N;
+    const int n_keys = S + N + p.T;
+    const int n_tiles = (n_keys + 31) / 32;
+    const int per = (n_tiles + p.nsplit - 1) / p.nsplit;
+    const int tile0 = split * per;
+    const int tile1 = min(n_tiles, tile0 + per);
+    int oldest = (st.head - st.count) % N;  // physical slot of the oldest live token
+    if (oldest < 0) oldest += N;
+
+    const size_t row_elems = (size_t)p.Hkv * d;
+    const size_t blk = ((size_t)p.layer * p.B + b) * (size_t)(p.S_max + N);
+    const T *k_blk = (const T *)p.k_slab + blk * row_elems + (size_t)kv * d;
+    const T *v_blk = (const T *)p.v_slab + blk * row_elems + (size_t)kv * d;
+    const T *k_dyn = (const T *)p.k_dyn + (size_t)b * p.T * row_elems + (size_t)kv * d;
+    const T *v_dyn = (const T *)p.v_dyn + (size_t)b * p.T * row_elems + (size_t)kv * d;
+
+    const T *q_row = (const T *)p.q + (((size_t)b * p.T + t) * p.Hq + h) * d;
+    {
+        float f[DPL];
+        RowIO<T, DPL>::load(q_row + lane * DPL, f);
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) q_s[warp][lane * DPL + i] = f[i];
+    }
+    __syncwarp();
+
+    float m = -INFINITY, l = 0.f;
+    float acc[DPL];
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+
+    for (int tile = tile0; tile < tile1; ++tile) {
+        const int idx = tile * 32 + lane;
+        const T *kp = nullptr, *vp = nullptr;
+        if (idx < S) {
+            kp = k_blk + (size_t)idx * row_elems; vp = v_blk + (size_t)idx * row_elems;
+        } else if (idx < S + N) {
+            const int slot = idx - S;
+            int age = slot - oldest;
+            if (age < 0) age += N;
+            if (age < st.count) {
+                kp = k_blk + (size_t)(p.S_max + slot) * row_elems; vp = v_blk + (size_t)(p.S_max + slot) * row_elems;
+            }
+        } else if (idx < n_keys) {
+            const int j = idx - S - N;
+            if (!(p.dyn_mask && j > t)) { kp = k_dyn + (size_t)j * row_elems; vp = v_dyn + (size_t)j * row_elems; }
+        }
+        float s = -INFINITY;
+        if (kp) s = dot_row<T>(kp, q_s[warp], d) * p.scale;
+        float tmax = s;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+        const float m_new = fmaxf(m, tmax);
+        if (m_new == -INFINITY) continue;  // nothing live so far (warp-uniform)
+        const float alpha = (m == -INFINITY) ? 0.f : expf(m - m_new);
+        const float pj = kp ? expf(s - m_new) : 0.f;
+        float psum = pj;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, o);
+        l = l * alpha + psum;
+        m = m_new;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] *= alpha;
+        const unsigned long long vaddr = (unsigned long long)vp;
+        for (int j = 0; j < 32; ++j) {
+            const float w = __shfl_sync(0xffffffffu, pj, j);
+            const unsigned long long va = __shfl_sync(0xffffffffu, vaddr, j);
+            if (va == 0ull) continue;  // dead key: its V row is never read (may hold stale or poisoned bytes)
+            float f[DPL];
+            RowIO<T, DPL>::load((const T *)va + lane * DPL, f);
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) acc[i] = fmaf(w, f[i], acc[i]);
+        }
+    }
+
+    if (p.nsplit == 1) {
+        const float inv = 1.f / l;  // l > 0: a dynamic query always sees itself
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] *= inv;
+        T *o = (T *)p.out + (((size_t)b * p.T + t) * p.Hq + h) * d;
+        RowIO<T, DPL>::store(o + lane * DPL, acc);
+    } else {
+        float *part = p.partials + (((size_t)b * rows + r) * p.nsplit + split) * (d + 2);
+        if (lane == 0) { part[0] = m; part[1] = l; }
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) part[2 + lane * DPL + i] = acc[i];
+    }
+}
+
+// grid = (T*Hq, B), block = d threads: merge of split partials, m* = max m_s, l = sum l_s e^{m_s-m*},
+// o = sum acc_s e^{m_s-m*} / l.
+template <typename T>
+__global__ void attn_merge_kernel(AttnParams p)
+{
+    const int d = p.d;
+    const int r = blockIdx.x, b = blockIdx.y, e = threadIdx.x;
+    const int rows = p.T * p.Hq;
+    const float *part = p.partials + ((size_t)b * rows + r) * p.nsplit * (d + 2);
+    float mstar = -INFINITY;
+    for (int s = 0; s < p.nsplit; ++s) mstar = fmaxf(mstar, part[(size_t)s * (d + 2)]);
+    float l = 0.f, o = 0.f;
+    for (int s = 0; s < p.nsplit; ++s) {
+        const float ms = part[(size_t)s * (d + 2)];
+        if (ms == -INFINITY) continue;
+        const float w = expf(ms - mstar);
+        l = fmaf(part[(size_t)s * (d + 2) + 1], w, l);
+        o = fmaf(part[(size_t)s * (d + 2) + 2 + e], w, o);
+    }
+    const int t = r / p.Hq, h = r % p.Hq;
+    T *out = (T *)p.out + (((size_t)b * p.T + t) * p.Hq + h) * d;
+    const float val = o / l;
+    if constexpr (sizeof(T) == 2) out[e] = __float2bfloat16_rn(val);
+    else out[e] = val;
+}
+
+int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
+{
+    const int rows = p.T * p.Hq;
+    const int blocks = ((rows + kSimtWarps - 1) / kSimtWarps) * p.B;
+    const int n_tiles = (p.S_max + p.N + p.T + 31) / 32;
+    int want = (4 * sm_count + blocks - 1) / blocks;  // aim at ~4 blocks per SM
+    if (want > n_tiles / 2) want = n_tiles / 2;       // at least two key tiles per split
+    if (want > kMaxSplits) want = kMaxSplits;
+    const size_t per_split = (size_t)p.B * rows * (p.d + 2) * sizeof(float);
+    if (per_split > 0 && (size_t)want * per_split > partial_bytes) want = (int)(partial_bytes / per_split);
+    if (want < 1) want = 1;
+    return want;
+}
+
+template <typename T>
+static cudaError_t launch_simt_t(const AttnParams &p, cudaStream_t st)
+{
+    const int rows = p.T * p.Hq;
+    dim3 grid((rows + kSimtWarps - 1) / kSimtWarps, p.B, p.nsplit);
+    switch (p.d / 32) {
+        case 1: attn_simt_kernel<T, 1><<<grid, kSimtWarps * 32, 0, st>>>(p); break;
+        case 2: attn_simt_kernel<T, 2><<<grid, kSimtWarps * 32, 0, st>>>(p); break;
+        case 4: attn_simt_kernel<T, 4><<<grid, kSimtWarps * 32, 0, st>>>(p); break;
+        case 8: attn_simt_kernel<T, 8><<<grid, kSimtWarps * 32, 0, st>>>(p); break;
+        default: return cudaErrorInvalidValue;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || p.nsplit == 1) return e;
+    attn_merge_kernel<T><<<dim3(rows, p.B), p.d, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attention_simt(const AttnParams &p, cudaStream_t st)
+{
+    if (p.dtype == REFLEX_DTYPE_BF16) return launch_simt_t<__nv_bfloat16>(p, st);
+    return launch_simt_t<float>(p, st);
+}
+
+}  // namespace reflex

@@ -1,0 +1,225 @@
+// AdaRMSNorm (Eq. 2, App. B.3): y = x * rsqrt(mean x^2 + eps) * (1 + W2 SiLU(W1 c + b1) + b2).
+// Row statistics, the gate MLP accumulation and the product are fp32; the result is rounded once on store.
+#include "reflex_internal.cuh"
+
+namespace reflex {
+
+template <typename T> struct Vec8;
+template <> struct Vec8<__nv_bfloat16> {
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&f)[8]) {
+        uint4 u = *reinterpret_cast<const uint4 *>(p);
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, const float (&f)[8]) {
+        uint4 u;
+        __nv_bfloat162 *h = reinterpret_cast<__nv_bfloat162 *>(&u);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+        *reinterpret_cast<uint4 *>(p) = u;
+    }
+};
+template <> struct Vec8<float> {
+    static __device__ __forceinline__ void load(const float *p, float (&f)[8]) {
+        float4 a = reinterpret_cast<const float4 *>(p)[0], b = reinterpret_cast<const float4 *>(p)[1];
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    }
+    static __device__ __forceinline__ void store(float *p, const float (&f)[8]) {
+        reinterpret_cast<float4 *>(p)[0] = make_float4(f[0], f[1], f[2], f[3]);
+        reinterpret_cast<float4 *>(p)[1] = make_float4(f[4], f[5], f[6], f[7]);
+    }
+};
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// hidden = SiLU(W1 c + b1) for one stream into shared memory; c_s is scratch of Cd floats.
+template <typename T>
+__device__ void gate_hidden(const T *__restrict__ cond_b, const T *__restrict__ W1, const T *__restrict__ b1, int Cd, int Hd,
+                            float *c_s, float *hid_s)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    for (int e = threadIdx.x; e < Cd; e += blockDim.x) c_s[e] = to_f<T>(cond_b[e]);
+    __syncthreads();
+    for (int j = warp; j < Hd; j += nwarp) {
+        const T *w = W1 + (size_t)j * Cd;
+        float acc = 0.f;
+        for (int e = lane * 8; e < Cd; e += 256) {
+            float f[8];
+            Vec8<T>::load(w + e, f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc = fmaf(f[i], c_s[e + i], acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) {
+            const float z = acc + to_f<T>(b1[j]);
+            hid_s[j] = z / (1.f + expf(-z));
+        }
+    }
+    __syncthreads();
+}
+
+// gate[i] = 1 + b2[i] + W2[i] . hidden for columns [i0, i1): one warp per column.
+template <typename T>
+__device__ void gate_columns(const T *__restrict__ W2, const T *__restrict__ b2, int Hd, int i0, int i1, const float *hid_s,
+                             float *gate_out /* indexed by i - i0 */)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    for (int i = i0 + warp; i < i1; i += nwarp) {
+        const T *w = W2 + (size_t)i * Hd;
+        float acc = 0.f;
+        for (int e = lane * 8; e < Hd; e += 256) {
+            float f[8];
+            Vec8<T>::load(w + e, f);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc = fmaf(f[k], hid_s[e + k], acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) gate_out[i - i0] = 1.f + (acc + to_f<T>(b2[i]));
+    }
+}
+
+// grid = (column chunks, B): writes gate_buf[b][i].
+template <typename T>
+__global__ void __launch_bounds__(256)
+gate_kernel(const T *__restrict__ cond, const T *__restrict__ W1, const T *__restrict__ b1, const T *__restrict__ W2,
+            const T *__restrict__ b2, float *__restrict__ gate_buf, int D, int Cd, int Hd, int cols_per_block)
+{
+    extern __shared__ float smem[];
+    float *c_s = smem, *hid_s = smem + Cd;
+    const int b = blockIdx.y;
+    gate_hidden<T>(cond + (size_t)b * Cd, W1, b1, Cd, Hd, c_s, hid_s);
+    const int i0 = blockIdx.x * cols_per_block;
+    const int i1 = min(D, i0 + cols_per_block);
+    gate_columns<T>(W2, b2, Hd, i0, i1, hid_s, gate_buf + (size_t)b * D + i0);
+}
+
+// grid = (row chunks, B); one warp per row. FUSED: the block computes its stream's gate itself.
+template <typename T, bool FUSED>
+__global__ void __launch_bounds__(256)
+adarmsnorm_kernel(const T *x, T *y, const T *__restrict__ cond, const T *__restrict__ W1,
+                  const T *__restrict__ b1, const T *__restrict__ W2, const T *__restrict__ b2,
+                  const float *__restrict__ gate_buf, int R, int D, int Cd, int Hd, float eps, int rows_per_block)
+{
+    extern __shared__ float smem[];
+    float *gate_s = smem;  // D floats
+    const int b = blockIdx.y;
+    if (FUSED) {
+        float *c_s = smem + D, *hid_s = c_s + Cd;
+        gate_hidden<T>(cond + (size_t)b * Cd, W1, b1, Cd, Hd, c_s, hid_s);
+        gate_columns<T>(W2, b2, Hd, 0, D, hid_s, gate_s);
+    } else {
+        for (int i = threadIdx.x; i < D; i += blockDim.x) gate_s[i] = gate_buf[(size_t)b * D + i];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    const int r0 = blockIdx.x * rows_per_block;
+    const int r1 = min(R, r0 + rows_per_block);
+    const float inv_D = 1.f / (float)D;
+    for (int r = r0 + warp; r < r1; r += nwarp) {
+        const T *xr = x + ((size_t)b * R + r) * D;
+        T *yr = y + ((size_t)b * R + r) * D;
+        float ss = 0.f;
+        for (int e = lane * 8; e < D; e += 256) {
+            float f[8];
+            Vec8<T>::load(xr + e, f);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
+        }
+        ss = warp_sum(ss);
+        const float rinv = 1.f / sqrtf(ss * inv_D + eps);
+        for (int e = lane * 8; e < D; e += 256) {
+            float f[8];
+            Vec8<T>::load(xr + e, f);  // second read hits L1/L2; x and y may alias, each lane rewrites only what it read
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = f[i] * rinv * gate_s[e + i];
+            Vec8<T>::store(yr + e, f);
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, const T *b1, const T *W2, const T *b2,
+                                 float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, cudaStream_t st)
+{
+    if (cond && gate_buf) {
+        const int cols = 64;
+        dim3 grid((D + cols - 1) / cols, B);
+        gate_kernel<T><<<grid, 256, (size_t)(Cd + Hd) * 4, st>>>(cond, W1, b1, W2, b2, gate_buf, D, Cd, Hd, cols);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    // enough blocks to cover the SMs about twice, at least one row per warp
+    int chunks = (296 + B - 1) / B;
+    const int max_chunks = (R + 7) / 8;
+    if (chunks > max_chunks) chunks = max_chunks;
+    if (chunks < 1) chunks = 1;
+    const int rows_per_block = (R + chunks - 1) / chunks;
+    chunks = (R + rows_per_block - 1) / rows_per_block;
+    dim3 grid(chunks, B);
+    if (cond && !gate_buf) {
+        size_t smem = (size_t)(D + Cd + Hd) * 4;
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(adarmsnorm_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        adarmsnorm_kernel<T, true><<<grid, 256, smem, st>>>(x, y, cond, W1, b1, W2, b2, nullptr, R, D, Cd, Hd, eps, rows_per_block);
+    } else {
+        size_t smem = (size_t)D * 4;
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(adarmsnorm_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        adarmsnorm_kernel<T, false><<<grid, 256, smem, st>>>(x, y, nullptr, nullptr, nullptr, nullptr, nullptr, gate_buf, R, D, Cd, Hd, eps, rows_per_block);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, const void *b1, const void *W2,
+                              const void *b2, float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, int dtype,
+                              cudaStream_t st)
+{
+    if (dtype == REFLEX_DTYPE_BF16)
+        return launch_norm_t<__nv_bfloat16>((const __nv_bfloat16 *)x, (__nv_bfloat16 *)y, (const __nv_bfloat16 *)cond,
+                                            (const __nv_bfloat16 *)W1, (const __nv_bfloat16 *)b1, (const __nv_bfloat16 *)W2,
+                                            (const __nv_bfloat16 *)b2, gate_buf, B, R, D, Cd, Hd, eps, st);
+    return launch_norm_t<float>((const float *)x, (float *)y, (const float *)cond, (const float *)W1, (const float *)b1,
+                                (const float *)W2, (const float *)b2, gate_buf, B, R, D, Cd, Hd, eps, st);
+}
+
+// Euler update (Sec. 2.1; App. C): x <- x + dt * v on the fp32 master, optional low-precision mirror.
+template <typename T>
+__global__ void flow_step_kernel(float *__restrict__ x, const T *__restrict__ v, T *__restrict__ x_lowp, size_t n, float dt)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float nx = fmaf(dt, to_f<T>(v[i]), x[i]);
+        x[i] = nx;
+        if (x_lowp) {
+            if constexpr (sizeof(T) == 2) x_lowp[i] = __float2bfloat16_rn(nx);
+            else x_lowp[i] = nx;
+        }
+    }
+}
+
+cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, float dt, int dtype, cudaStream_t st)
+{
+    int blocks = (int)((n + 255) / 256);
+    if (blocks > 1184) blocks = 1184;
+    if (blocks < 1) blocks = 1;
+    if (dtype == REFLEX_DTYPE_BF16)
+        flow_step_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(x, (const __nv_bfloat16 *)v, (__nv_bfloat16 *)x_lowp, n, dt);
+    else
+        flow_step_kernel<float><<<blocks, 256, 0, st>>>(x, (const float *)v, (float *)x_lowp, n, dt);
+    return cudaGetLastError();
+}
+
+}  // namespace reflex

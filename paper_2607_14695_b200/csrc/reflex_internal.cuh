@@ -1,0 +1,72 @@
+// Internal declarations shared by the translation units of libreflex_b200 (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "reflex.h"
+
+namespace reflex {
+
+// Per-stream cache state as the kernels read it (device memory, one int4-sized record per stream).
+struct StreamState {
+    int32_t static_len;  // valid prefix rows, -1 = never initialised
+    int32_t head;        // next ring slot to write
+    int32_t count;       // live ring tokens
+    int32_t ticket;      // arrival counter of the append kernel (always 0 between launches)
+};
+
+// Layout of the caller-lent workspace.
+struct WorkspaceLayout {
+    size_t state_off;     // StreamState[B]
+    size_t total_off;     // int64 total_appended[B]
+    size_t status_off;    // uint32 status word (bounded-wait failures)
+    size_t partial_off;   // split-K partials
+    size_t partial_bytes;
+    size_t bytes;
+};
+
+constexpr int kMaxSplits = 32;
+constexpr int kStreamsPerLaunch = 64;  // stream ids / lengths passed by value per launch
+
+struct StreamBatch {
+    int32_t id[kStreamsPerLaunch];
+    int32_t len[kStreamsPerLaunch];
+};
+
+WorkspaceLayout workspace_layout(const reflex_cache_desc &d);
+
+inline size_t elem_size(int dtype) { return dtype == REFLEX_DTYPE_BF16 ? 2 : 4; }
+
+// Geometry every attention kernel needs.
+struct AttnParams {
+    const void *k_slab, *v_slab;   // [L][B][S_max+N][Hkv][d]
+    const void *q, *k_dyn, *v_dyn; // [B][T][Hq][d], [B][T][Hkv][d]
+    void *out;
+    const StreamState *state;
+    float *partials;               // split-K scratch
+    int L, B, Hq, Hkv, d, S_max, N, T, layer;
+    int dyn_mask;
+    float scale;
+    int nsplit;
+    int dtype;
+};
+
+// ---- launchers (each returns the cudaError_t of its launch) ----
+cudaError_t launch_state_init(StreamState *state, int64_t *total, uint32_t *status, const int32_t *head0_dev_or_null,
+                              int B, int N, cudaStream_t st);
+cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
+                               const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max, int N, int S_src,
+                               size_t row_bytes, cudaStream_t st);
+cudaError_t launch_append_sliding(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
+                                  int64_t *total, const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max,
+                                  int N, int m, size_t row_bytes, cudaStream_t st);
+cudaError_t launch_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, const void *b1, const void *W2,
+                              const void *b2, float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, int dtype,
+                              cudaStream_t st);
+cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, float dt, int dtype, cudaStream_t st);
+cudaError_t launch_attention_simt(const AttnParams &p, cudaStream_t st);
+int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
+
+}  // namespace reflex

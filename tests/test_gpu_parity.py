@@ -1,0 +1,306 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element on the
+same seeded inputs. Integer / byte work is compared exactly, floating point within the contract
+tolerances (bf16: max-abs 2e-2, mean-abs 2e-3 against the fp64 oracle; fp32 storage: 2e-5 / 2e-6)."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2607_14695_b200 import synth  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def U():
+    from paper_2607_14695_b200 import build as rbuild
+    rbuild.build()
+    import gpu_util
+    return gpu_util
+
+
+def _norm_case(U, w, x, cond, layer=0, eps=1e-6, gate_buf=False, alias=False, what="adarmsnorm"):
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    W1, b1, W2, b2 = synth.gate_weights(w, layer)
+    dx = U.to_dev(x, w.dtype)
+    dy = dx if alias else torch.full_like(dx, float("nan"))
+    gb = torch.empty((x.shape[0], w.D), dtype=torch.float32, device=U.DEV) if gate_buf else None
+    rb.reflex_adarmsnorm(dx, dy, U.to_dev(cond, w.dtype), U.to_dev(W1, w.dtype), U.to_dev(b1, w.dtype), U.to_dev(W2, w.dtype),
+                         U.to_dev(b2, w.dtype), gate_buf=gb, eps=eps)
+    want = orc.adarmsnorm_batched(x, cond, W1, b1, W2, b2, eps)
+    U.check_close(U.to_host(dy), want, w.dtype, what, rel_clause=True)
+    if gate_buf:  # the gate itself, fp32, and the precomputed-gate entry
+        _, g0 = orc.adarmsnorm(x[0], cond[0], W1, b1, W2, b2, eps, return_gate=True)
+        assert np.max(np.abs(U.to_host(gb[0]) - g0)) <= 1e-5
+        dy2 = torch.full_like(dx, float("nan"))
+        rb.reflex_adarmsnorm(U.to_dev(x, w.dtype), dy2, None, None, None, None, None, gate_buf=gb, eps=eps)
+        assert torch.equal(dy2, dy)
+    return dy
+
+
+# ------------------------------------------------------------------------------------------------
+# config 1: tiny fp32 layer, 40 ticks x 4 Euler steps, every call of every tick compared
+# ------------------------------------------------------------------------------------------------
+def test_cfg1_full_trace(U):
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    w = synth.CONFIGS["cfg1"]
+    tw = U.Twin(w)
+    tw.init_static([0], [w.S])
+    W1, b1, W2, b2 = synth.gate_weights(w, 0, std=0.2)
+    dW = [U.to_dev(a, w.dtype) for a in (W1, b1, W2, b2)]
+    evicted_total = 0
+    for tick in range(w.ticks):
+        evicted_total += tw.append([0], 1, tick)[0]
+        tw.check_state()
+        assert tw.o.head[0] == (tick + 1) % 16 and tw.o.count[0] == min(tick + 1, 16)
+        x0 = synth.normal(w, "noise", (w.B, w.T, w.A), 0, tick)
+        x_or = x0.astype(np.float64).copy()
+        x_gpu = torch.from_numpy(x0).to(U.DEV)
+        for k in range(w.K):
+            variant = tick * w.K + k
+            t_k = orc.flow_time(k, w.K)
+            # norm -> attention chained literally: D = Hq*d = 128, so Q = y viewed [T][2][64], K_d = y[:, :64], V_d = y[:, 64:]
+            x = synth.normal(w, "x", (w.B, w.T, w.D), 0, variant)
+            cond = synth.cond_vectors(w, t_k, variant=tick)
+            dy = torch.empty((w.B, w.T, w.D), dtype=torch.float32, device=U.DEV)
+            rb.reflex_adarmsnorm(U.to_dev(x, w.dtype), dy, U.to_dev(cond, w.dtype), *dW, eps=1e-6)
+            y_or = orc.adarmsnorm_batched(x, cond, W1, b1, W2, b2, 1e-6)
+            U.check_close(U.to_host(dy), y_or, w.dtype, f"norm tick {tick} step {k}", rel_clause=True)
+            y32 = dy.cpu().numpy()   # the oracle continues from the GPU's fp32 y so errors do not compound across calls
+            q = y32.reshape(w.B, w.T, w.Hq, w.d)
+            kd = np.ascontiguousarray(y32[:, :, :64]).reshape(w.B, w.T, 1, 64)
+            vd = np.ascontiguousarray(y32[:, :, 64:]).reshape(w.B, w.T, 1, 64)
+            out = torch.empty((w.B, w.T, w.Hq, w.d), dtype=torch.float32, device=U.DEV)
+            rb.reflex_partitioned_attention(tw.g, 0, dy.view(w.B, w.T, w.Hq, w.d), U.to_dev(kd, w.dtype), U.to_dev(vd, w.dtype), out)
+            want = tw.o.attention(0, 0, q[0], kd[0], vd[0])
+            U.check_close(U.to_host(out)[0], want, w.dtype, f"attention tick {tick} step {k}")
+            v = synth.normal(w, "v_flow", (w.B, w.T, w.A), 0, variant)
+            rb.reflex_flow_step(x_gpu, U.to_dev(v, w.dtype), None, k, w.K)
+            orc.flow_step(x_or, v, w.K)
+        U.check_close(U.to_host(x_gpu), x_or, w.dtype, f"action chunk tick {tick}")
+    assert evicted_total == 24
+
+
+# ------------------------------------------------------------------------------------------------
+# config 2: one pi0-class layer, batch 1, bf16
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("count", [5, 32, 45])
+def test_cfg2_layer(U, impl, count):
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"]
+    tw = U.Twin(w, head0=[7], poison=True)
+    rb.reflex_cache_set_attention_impl(tw.g, rb.ATTN_SIMT if impl == "simt" else rb.ATTN_AUTO)
+    tw.init_static([0], [w.S])
+    for i in range(count):
+        tw.append([0], 1, i)
+    tw.check_state()
+    for dyn_mask in (0, 1):
+        tw.attention(0, 10 + dyn_mask, dyn_mask=dyn_mask, what=f"cfg2 attention mask={dyn_mask}")
+        tw.attention(0, 10 + dyn_mask, dyn_mask=dyn_mask, partitioned=True, what="cfg2 attention vs partitioned oracle")
+    tw.check_state()   # attention only reads the cached regions (timestep invariance)
+    # AdaRMSNorm over the 10-step schedule and the Euler chain
+    from oracle import reflex_oracle as orc
+    for k in (0, 3, 9):
+        x = synth.norm_input(w, 0, k)
+        cond = synth.cond_vectors(w, orc.flow_time(k, w.K))
+        _norm_case(U, w, x, cond, gate_buf=(k == 3), alias=(k == 9), what=f"cfg2 norm step {k}")
+    x0 = synth.normal(w, "noise", (w.B, w.T, w.A))
+    x_or = x0.astype(np.float64).copy(); x_gpu = torch.from_numpy(x0).to(U.DEV)
+    mirror = torch.empty((w.B, w.T, w.A), dtype=torch.bfloat16, device=U.DEV)
+    for k in range(w.K):
+        v = synth.normal(w, "v_flow", (w.B, w.T, w.A), 0, k)
+        rb.reflex_flow_step(x_gpu, U.to_dev(v, w.dtype), mirror, k, w.K)
+        orc.flow_step(x_or, v, w.K)
+    U.check_close(U.to_host(x_gpu), x_or, synth.DTYPE_F32, "cfg2 action chunk (fp32 master)")
+    assert torch.equal(mirror, x_gpu.to(torch.bfloat16))
+
+
+# ------------------------------------------------------------------------------------------------
+# config 3 shapes: 18 layers, streaming ticks with a new (shorter) prefix, stale rows poisoned
+# ------------------------------------------------------------------------------------------------
+def test_cfg3_stream_ticks(U):
+    w = synth.CONFIGS["cfg3"]
+    tw = U.Twin(w, head0=[30], poison=True)
+    S_sched = {0: 816, 10: 800, 20: 816}
+    for tick in range(0, 34):
+        if tick in S_sched:
+            tw.init_static([0], [S_sched[tick]], variant=tick)
+        tw.append([0], 1, tick)
+        if tick in (0, 1, 9, 10, 11, 31, 32, 33):
+            tw.check_state()
+            for layer in ((0, 17) if tick not in (10, 32) else range(w.L)):
+                tw.attention(layer, tick, what=f"cfg3 tick {tick}")
+
+
+# ------------------------------------------------------------------------------------------------
+# config 4 shapes: 64 streams with random ring offsets and mixed fill levels
+# ------------------------------------------------------------------------------------------------
+def test_cfg4_batched_streams(U):
+    w = synth.CONFIGS["cfg4"].with_(L=3)
+    head0 = synth.ring_head0(w)
+    tw = U.Twin(w, head0=head0, poison=True)
+    tw.init_static(list(range(w.B)), [w.S] * w.B)
+    # 60 streams get >= 32 appends (full rings at different offsets), 4 stay partially filled
+    for i in range(40):
+        ids = [b for b in range(w.B) if not (b in (5, 17, 40, 63) and i >= 3 + b % 7)]
+        tw.append(ids, 1, i)
+    tw.check_state()
+    assert sorted(set(tw.o.count)) != [32]
+    tw.attention(0, 0, streams=[0, 5, 17, 31, 40, 62, 63], what="cfg4 step 0")
+    tw.attention(2, 9, streams=[1, 63], what="cfg4 step 9")
+    from oracle import reflex_oracle as orc
+    x = synth.norm_input(w, 1, 0)
+    _norm_case(U, w, x, synth.cond_vectors(w, 0.7), layer=1, what="cfg4 norm")
+    _norm_case(U, w, x, synth.cond_vectors(w, 0.2), layer=1, gate_buf=True, what="cfg4 norm two-launch")
+
+
+# ------------------------------------------------------------------------------------------------
+# config 5 shapes: long context, outliers in the norm input, t near 0 and 1
+# ------------------------------------------------------------------------------------------------
+def test_cfg5_long_context(U):
+    w = synth.CONFIGS["cfg5"].with_(L=2, B=4)
+    tw = U.Twin(w, head0=synth.ring_head0(w), poison=True)
+    tw.init_static(list(range(w.B)), [w.S, w.S - 100, w.S, 1])
+    for i in range(3):
+        tw.append(list(range(w.B)), 100, i)      # frame-sized appends; wraps the 256-slot ring
+    tw.check_state()
+    tw.attention(1, 0, streams=[0, 1, 3], what="cfg5 attention")
+    for t in (0.0, 1e-4, 1e-3, 1 - 1e-3, 1 - 1e-4, 1.0):
+        x = synth.norm_input(w, 0, int(t * 1000))
+        assert (np.abs(x) > 100).any()
+        _norm_case(U, w, x, synth.cond_vectors(w, t), what=f"cfg5 norm t={t}")
+
+
+# ------------------------------------------------------------------------------------------------
+# edge cases and degenerate shapes
+# ------------------------------------------------------------------------------------------------
+EDGE = [
+    # name, B, L, Hq, Hkv, d, S_max, S, N, T, appends(m list), dtype
+    ("S0_T1_N1", 2, 1, 2, 2, 32, 4, 0, 1, 1, [1, 1], synth.DTYPE_F32),
+    ("gqa4to2_d64", 3, 2, 4, 2, 64, 40, 33, 5, 7, [2, 2, 2], synth.DTYPE_BF16),
+    ("mha_d128", 1, 1, 3, 3, 128, 70, 70, 9, 33, [9, 4], synth.DTYPE_BF16),
+    ("m_equals_N", 2, 1, 8, 1, 256, 100, 64, 16, 17, [16, 16, 3], synth.DTYPE_BF16),
+    ("empty_ring", 1, 1, 8, 1, 256, 130, 129, 8, 50, [], synth.DTYPE_BF16),
+    ("f32_d256", 1, 1, 8, 2, 256, 65, 65, 33, 5, [33, 1], synth.DTYPE_F32),
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+def test_edge_shapes(U, case):
+    name, B, L, Hq, Hkv, d, S_max, S, N, T, appends, dtype = case
+    w = synth.Workload(name, 77, dtype, B=B, L=L, Hq=Hq, Hkv=Hkv, d=d, S=S, S_max=S_max, N=N, T=T, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w, head0=[(3 * b) % N for b in range(B)], T_max=T + 3, poison=True)
+    tw.init_static(list(range(B)), [S] * B)
+    for i, m in enumerate(appends):
+        tw.append(list(range(B)), m, i)
+    tw.check_state()
+    for layer in range(L):
+        for dyn_mask in (0, 1):
+            tw.attention(layer, dyn_mask, dyn_mask=dyn_mask, what=name)
+    if T > 1:
+        tw.attention(0, 5, T=T - 1, what=name + " T<T_max")
+    tw.attention(0, 6, scale=0.05, what=name + " scale override")
+
+
+def test_error_paths_leave_state_unchanged(U):
+    rb = U.rb
+    w = synth.Workload("err", 5, synth.DTYPE_BF16, B=2, L=1, Hq=2, Hkv=1, d=64, S=8, S_max=8, N=4, T=4, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w)
+    z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device=U.DEV)
+    q, kd, out = z(2, 4, 2, 64), z(2, 4, 1, 64), z(2, 4, 2, 64)
+
+    def code(fn, *a, **k):
+        with pytest.raises(rb.ReflexError) as e:
+            fn(*a, **k)
+        return e.value.code
+
+    assert code(rb.reflex_partitioned_attention, tw.g, 0, q, kd, kd, out) == rb.ERR_STATE          # prefix never set
+    tw.init_static([0], [8])
+    assert code(rb.reflex_partitioned_attention, tw.g, 0, q, kd, kd, out) == rb.ERR_STATE          # stream 1 still unset
+    tw.init_static([1], [0])                                                                        # S = 0 after an explicit init is legal
+    rb.reflex_partitioned_attention(tw.g, 0, q, kd, kd, out)
+    assert code(rb.reflex_partitioned_attention, tw.g, 1, q, kd, kd, out) == rb.ERR_INVALID_ARG    # layer out of range
+    assert code(rb.reflex_partitioned_attention, tw.g, 0, z(2, 5, 2, 64), z(2, 5, 1, 64), z(2, 5, 1, 64), z(2, 5, 2, 64)) == rb.ERR_SHAPE
+    assert code(rb.reflex_partitioned_attention, tw.g, 0, q, kd, kd, out, dyn_mask=2) == rb.ERR_INVALID_ARG
+    assert code(rb.reflex_partitioned_attention, tw.g, 0, q.view(-1)[4:4 + 2 * 3 * 2 * 64].view(2, 3, 2, 64), kd[:, :3].contiguous(), kd[:, :3].contiguous(), out) == rb.ERR_ALIGN
+    assert code(rb.reflex_cache_append_sliding, tw.g, [0], z(1, 1, 5, 1, 64), z(1, 1, 5, 1, 64)) == rb.ERR_SHAPE     # m > N
+    assert code(rb.reflex_cache_append_sliding, tw.g, [2], z(1, 1, 1, 1, 64), z(1, 1, 1, 1, 64)) == rb.ERR_INVALID_ARG
+    assert code(rb.reflex_cache_append_sliding, tw.g, [0, 0], z(2, 1, 1, 1, 64), z(2, 1, 1, 1, 64)) == rb.ERR_INVALID_ARG
+    assert code(rb.reflex_cache_init_static, tw.g, [0], z(1, 1, 9, 1, 64), z(1, 1, 9, 1, 64)) == rb.ERR_SHAPE        # S > S_max
+    assert code(rb.reflex_cache_init_static, tw.g, [0], z(1, 1, 4, 1, 64), z(1, 1, 4, 1, 64), S=[5]) == rb.ERR_SHAPE  # S > S_src
+    tw.check_state()                                                                                                   # nothing moved
+    assert code(rb.reflex_cache_set_attention_impl, tw.g, 9) == rb.ERR_INVALID_ARG
+
+
+def test_adarmsnorm_gate_off_is_rmsnorm_and_flow_closed_form(U):
+    """The gate switched off (W2 = 0, b2 = 0) leaves plain weight-free RMSNorm; checked against torch on the GPU
+    tensor's own values as well as the oracle. Euler with constant v lands on x0 - v."""
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"].with_(B=3)
+    x = synth.norm_input(w, 0, 99)
+    cond = synth.cond_vectors(w, 0.5)
+    W1, b1, W2, b2 = synth.gate_weights(w, 0)
+    dx = U.to_dev(x, w.dtype); dy = torch.empty_like(dx)
+    rb.reflex_adarmsnorm(dx, dy, U.to_dev(cond, w.dtype), U.to_dev(W1, w.dtype), U.to_dev(b1, w.dtype),
+                         U.to_dev(np.zeros_like(W2), w.dtype), U.to_dev(b2, w.dtype), eps=1e-6)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x).double(), (w.D,), eps=1e-6).numpy()
+    U.check_close(U.to_host(dy), ref, w.dtype, "gate-off norm", rel_clause=True)
+    x0 = synth.normal(w, "noise", (w.B, w.T, w.A)); v = synth.normal(w, "v_flow", (w.B, w.T, w.A))
+    xg = torch.from_numpy(x0).to(U.DEV)
+    for k in range(w.K):
+        rb.reflex_flow_step(xg, U.to_dev(v, w.dtype), None, k, w.K)
+    assert np.max(np.abs(U.to_host(xg) - (x0.astype(np.float64) - v))) <= 2e-6
+
+
+def test_stale_dynamic_kv_negative_control(U):
+    """A cache that ignored the timestep (dynamic K/V frozen at step 0) is far outside tolerance."""
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"]
+    tw = U.Twin(w)
+    tw.init_static([0], [w.S]); tw.append([0], 8, 0)
+    q = synth.normal(w, "q", (1, w.T, w.Hq, w.d), 0, 1)
+    kd0, vd0 = synth.normal(w, "k_dyn", (1, w.T, 1, w.d), 0, 0), synth.normal(w, "v_dyn", (1, w.T, 1, w.d), 0, 0)
+    kd1, vd1 = synth.normal(w, "k_dyn", (1, w.T, 1, w.d), 0, 1), synth.normal(w, "v_dyn", (1, w.T, 1, w.d), 0, 1)
+    out = torch.empty((1, w.T, w.Hq, w.d), dtype=torch.bfloat16, device=U.DEV)
+    rb.reflex_partitioned_attention(tw.g, 0, U.to_dev(q, w.dtype), U.to_dev(kd0, w.dtype), U.to_dev(vd0, w.dtype), out)
+    right = tw.o.attention(0, 0, q[0], kd1[0], vd1[0])
+    assert np.abs(U.to_host(out)[0] - right).max() > 10 * U.BF16_MAX_ABS
+
+
+@pytest.mark.parametrize("cfg", ["cfg1", "cfg2"])
+def test_10k_tick_stream_stays_finite(U, cfg):
+    """Stability protocol (Sec. 4.4, stability table), raised to 10k ticks: every output of every tick is
+    checked for NaN/Inf on the device (flag word, no host sync); outlier-laden norm inputs as in the long-context stress."""
+    rb = U.rb
+    w = synth.CONFIGS[cfg].with_(outlier_frac=1e-3, outlier_mult=1e3)
+    cache = rb.Cache(w.L, w.B, w.Hq, w.Hkv, w.d, w.S_max, w.N, w.T, w.dtype, device=U.DEV)
+    tdt = rb.torch_dtype(w.dtype)
+    g = torch.Generator(device=U.DEV); g.manual_seed(w.seed)
+    rnd = lambda *s: torch.randn(*s, generator=g, device=U.DEV, dtype=torch.float32).to(tdt)
+    rb.reflex_cache_init_static(cache, [0], rnd(1, w.L, w.S, w.Hkv, w.d), rnd(1, w.L, w.S, w.Hkv, w.d))
+    W1, b1, W2, b2 = [U.to_dev(a, w.dtype) for a in synth.gate_weights(w, 0)]
+    n_var = 7
+    xs = [U.to_dev(synth.norm_input(w, 0, i), w.dtype) for i in range(n_var)]
+    conds = [U.to_dev(synth.cond_vectors(w, 1.0 - k / w.K), w.dtype) for k in range(w.K)]
+    qs, kds, vds, vs = [[rnd(*s) for _ in range(n_var)] for s in ((w.B, w.T, w.Hq, w.d), (w.B, w.T, w.Hkv, w.d), (w.B, w.T, w.Hkv, w.d), (w.B, w.T, w.A))]
+    kn, vn = [rnd(1, w.L, 1, w.Hkv, w.d) for _ in range(n_var)], [rnd(1, w.L, 1, w.Hkv, w.d) for _ in range(n_var)]
+    y = torch.empty_like(xs[0]); out = torch.empty_like(qs[0])
+    xa = torch.empty((w.B, w.T, w.A), dtype=torch.float32, device=U.DEV)
+    bad = torch.zeros((), dtype=torch.int64, device=U.DEV)
+    ticks = 10000
+    steps = w.K
+    for tick in range(ticks):
+        rb.reflex_cache_append_sliding(cache, [0], kn[tick % n_var], vn[tick % n_var])
+        xa.copy_(vs[tick % n_var].float())
+        for k in range(steps):
+            i = (tick + k) % n_var
+            rb.reflex_adarmsnorm(xs[i], y, conds[k], W1, b1, W2, b2)
+            rb.reflex_partitioned_attention(cache, 0, qs[i], kds[i], vds[i], out)
+            rb.reflex_flow_step(xa, vs[i], None, k, w.K)
+            if tick % 10 == 0 or k == steps - 1:   # every tick's final outputs, every step of each 10th tick
+                bad += (~torch.isfinite(y.float())).sum() + (~torch.isfinite(out.float())).sum() + (~torch.isfinite(xa)).sum()
+    assert int(bad.item()) == 0
+    sl, hd, ct, tot = rb.reflex_cache_get_state(cache)
+    assert tot == [ticks] and ct == [w.N] and hd == [ticks % w.N]
