@@ -1,0 +1,308 @@
+#!/usr/bin/env python
+"""Benchmark of the Reflex hot path on B200: denoising steps/s over one batch of synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg4] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path: for each of the L layers AdaRMSNorm then partitioned
+attention, then the Euler update, over all B streams (inputs resident in HBM). Prints ONE JSON line.
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU: the path has no exchange
+step, so there is no data-path collective; the reported time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops", FALLBACK_BF16_TFLOPS)),
+                    "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 1400.0)), "source": "measured"}
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Reads (never sets) SM clock, power and clock-event reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples = []          # (wall time, sm_mhz, reasons bitmask, power W)
+        self.max_mhz = None
+        self._stop_evt = threading.Event()
+        self.ok = False
+
+    def run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+            while not self._stop_evt.is_set():
+                try:
+                    mhz = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+                    try:
+                        reasons = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                    except Exception:
+                        reasons = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                    try:
+                        power = pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0
+                    except Exception:
+                        power = None
+                    self.samples.append((time.time(), mhz, int(reasons), power))
+                except Exception:
+                    pass
+                time.sleep(self.period)
+        except Exception:
+            self.ok = False
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def summary(self, t0: float, t1: float):
+        names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+                 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = "sampled during the timed region"
+        if not inside:
+            inside, note = self.samples, "timed region shorter than the sampling period: samples span warm-up and timed region"
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "note": "NVML unavailable"}
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        powers = [s[3] for s in inside if s[3] is not None]
+        return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.max_mhz,
+                "reasons": [n for bit, n in names.items() if mask & bit], "samples": len(inside),
+                "power_w_max": max(powers) if powers else None, "note": note}
+
+
+def oracle_sample_seconds(w, n_units: int):
+    """Times the CPU oracle, as it stands, on n_units (stream, layer) units of the workload:
+    AdaRMSNorm + attention by definition over the gathered context, plus one Euler update of the batch."""
+    import numpy as np
+
+    from oracle import reflex_oracle as orc
+    from paper_2607_14695_b200 import synth
+
+    B = min(w.B, max(1, n_units))
+    L = (n_units + B - 1) // B
+    wl = w.with_(B=B, L=L)
+    oc = orc.OracleCache(L, B, w.Hkv, w.d, w.S_max, w.N, head0=list(synth.ring_head0(wl)))
+    for b in range(B):
+        oc.init_static(b, synth.normal(wl, "k_static", (L, w.S, w.Hkv, w.d), 0, b), synth.normal(wl, "v_static", (L, w.S, w.Hkv, w.d), 0, b))
+        oc.append_sliding(b, synth.normal(wl, "k_new", (L, w.N, w.Hkv, w.d), 0, b), synth.normal(wl, "v_new", (L, w.N, w.Hkv, w.d), 0, b))
+    x = synth.norm_input(wl, 0, 0); cond = synth.cond_vectors(wl, 1.0)
+    W1, b1, W2, b2 = synth.gate_weights(wl, 0)
+    q = synth.normal(wl, "q", (B, w.T, w.Hq, w.d)); kd = synth.normal(wl, "k_dyn", (B, w.T, w.Hkv, w.d)); vd = synth.normal(wl, "v_dyn", (B, w.T, w.Hkv, w.d))
+    xa = synth.normal(wl, "noise", (B, w.T, w.A)).astype(np.float64); v = synth.normal(wl, "v_flow", (B, w.T, w.A))
+    done = 0
+    t0 = time.perf_counter()
+    for layer in range(L):
+        for b in range(B):
+            if done >= n_units:
+                break
+            orc.adarmsnorm(x[b], cond[b], W1, b1, W2, b2, 1e-6)
+            oc.attention(b, layer, q[b], kd[b], vd[b])
+            done += 1
+    orc.flow_step(xa, v, w.K)
+    return time.perf_counter() - t0, orc.max_threads()
+
+
+def run_reference(args, w):
+    """The reference arm is the CPU oracle (there is no other implementation of the paper's method here):
+    each step is a bounded sample of the workload, scaled to a whole step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    units = w.B * w.L
+    t1, threads = oracle_sample_seconds(w, 1)
+    budget = 100.0 / max(1, args.steps + args.warmup)
+    n = int(max(1, min(units, budget / max(t1, 1e-6))))
+    for _ in range(args.warmup):
+        oracle_sample_seconds(w, n)
+    times = [oracle_sample_seconds(w, n)[0] for _ in range(args.steps)]
+    sec_per_step = statistics.mean(times) * units / n
+    value = 1.0 / sec_per_step
+    sample = f"{n} of {units} (stream, layer) units per step (AdaRMSNorm + attention by definition) + one Euler update, scaled by {units}/{n}"
+    line = {"impl": "reference", "metric": "denoising_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "L": w.L, "S": w.S, "N": w.N, "T": w.T},
+            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg4", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--attn", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2607_14695_b200 import synth
+    w = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_14695_b200 import binding as rb
+    from paper_2607_14695_b200 import build as rbuild
+    from paper_2607_14695_b200.runner import StepRunner
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        rbuild.build()
+    if world > 1:
+        dist.barrier()
+    rb.load()
+
+    impl = {"auto": rb.ATTN_AUTO, "simt": rb.ATTN_SIMT, "tc": rb.ATTN_TC}[args.attn]
+    runner = StepRunner(w, device=f"cuda:{local_rank}", attn_impl=impl, host_inputs=not args.no_e2e)
+    alg = runner.algorithmic()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for k in range(args.warmup):
+        runner.step(k)
+    barrier()
+    # ---- timed region: exactly K steps, device-timed on the launching stream ----
+    launches0 = rb.reflex_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
+    e0.record(stream)
+    for k in range(args.steps):
+        runner.step(k)
+    e1.record(stream)
+    barrier()
+    wall1 = time.time()
+    launches = rb.reflex_kernel_launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    # ---- the same K steps again with events around every attention / norm call (per-kernel durations) ----
+    ev_attn, ev_norm, step_marks = [], [], []
+    for k in range(args.steps):
+        m = torch.cuda.Event(enable_timing=True); m.record(stream); step_marks.append(m)
+        runner.step_timed(k, ev_attn, ev_norm)
+    m = torch.cuda.Event(enable_timing=True); m.record(stream); step_marks.append(m)
+    barrier()
+    clocks = sampler.summary(wall0, wall1)
+    attn_ms = [a.elapsed_time(b) for a, b in ev_attn]
+    norm_ms = [a.elapsed_time(b) for a, b in ev_norm]
+    step_ms = sorted(step_marks[i].elapsed_time(step_marks[i + 1]) for i in range(args.steps))
+    # ---- end to end: inputs from pinned host memory, action chunk back to the host, every step ----
+    e2e = None
+    if not args.no_e2e:
+        for k in range(3):
+            runner.step_from_host(k)
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e = max(3, min(args.steps, 30))
+        h0.record(stream)
+        for k in range(n_e2e):
+            runner.step_from_host(k)
+        h1.record(stream)
+        barrier()
+        e2e_ms = h0.elapsed_time(h1)
+    sampler.stop()
+
+    t = torch.tensor([ms_total, e2e_ms if not args.no_e2e else 0.0], dtype=torch.float64, device=f"cuda:{local_rank}")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_max = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ms_per_step = ms_total / args.steps
+    value = world * args.steps / (ms_total * 1e-3)          # every rank runs its own replica of the batch
+    attn_avg_ms = statistics.mean(attn_ms)
+    norm_avg_ms = statistics.mean(norm_ms)
+    attn_gbs = alg["attn_bytes_per_launch"] / (attn_avg_ms * 1e-3) / 1e9
+    attn_tflops = alg["attn_flops_per_launch"] / (attn_avg_ms * 1e-3) / 1e12
+    line = {
+        "metric": "denoising_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "us_per_step": ms_per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == synth.DTYPE_BF16 else "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: B={w.B} streams x L={w.L} layers, Hq={w.Hq}/Hkv={w.Hkv}, d={w.d}, static S={w.S}, ring N={w.N}, "
+                               f"dynamic T={w.T}, D={w.D}, K={w.K}; one step = L x (AdaRMSNorm + partitioned attention) + Euler update",
+                   "parallelism": "replicas only (independent streams per GPU, no collective)" if world > 1 else "single GPU",
+                   "attention_impl": args.attn, "l2_policy": f"inputs larger than L2: {runner.input_bytes_resident() / 1e6:.0f} MB of cache + per-layer inputs are read per step pair (L2 is 126 MB)",
+                   "bytes_per_step_algorithmic": alg["bytes_per_step"], "flops_per_step": alg["flops_per_step"]},
+        "gpu_launches": int(launches),
+        "step_ms": {"p50": step_ms[len(step_ms) // 2], "p95": step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))], "max": step_ms[-1],
+                    "note": "per-step times from the instrumented pass"},
+        "hbm_gbs_whole_step": alg["bytes_per_step"] / (ms_per_step * 1e-3) / 1e9,
+        "roofline": {"kernel": "partitioned attention", "bound": "hbm", "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": attn_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                     "bytes_per_launch": alg["attn_bytes_per_launch"], "avg_launch_us": attn_avg_ms * 1e3,
+                     "frac_of_nominal_8TBs": attn_gbs / 8000.0,
+                     "tensor": {"achieved_tflops": attn_tflops, "peak_tflops_sustained": peaks["bf16_tflops_sustained"],
+                                "frac": attn_tflops / peaks["bf16_tflops_sustained"]}},
+        "kernels": {"attention_avg_us": attn_avg_ms * 1e3, "adarmsnorm_avg_us": norm_avg_ms * 1e3,
+                    "adarmsnorm_gbs": alg["norm_bytes_per_launch"] / (norm_avg_ms * 1e-3) / 1e9,
+                    "attention_share_of_step": attn_avg_ms * w.L / (statistics.mean(step_ms))},
+        "clocks": clocks,
+    }
+    if not args.no_e2e:
+        line["e2e"] = {"value": world * n_e2e / (e2e_ms_max * 1e-3), "unit": "steps/s", "h2d_bytes_per_step": int(runner.h2d_bytes_per_step),
+                       "d2h_bytes_per_step": int(runner.d2h_bytes_per_step), "steps": n_e2e}
+    if world == 1 and not args.no_cpu_baseline:
+        units = w.B * w.L
+        t1, threads = oracle_sample_seconds(w, 1)
+        n = int(max(1, min(units, args.cpu_seconds / max(t1, 1e-6))))
+        ts, threads = oracle_sample_seconds(w, n)
+        line["cpu_baseline"] = {"value": 1.0 / (ts * units / n), "unit": "steps/s", "cores": threads, "kind": "oracle",
+                                "sample": f"{n} of {units} (stream, layer) units (AdaRMSNorm + attention by definition) + one Euler update, "
+                                          f"{ts:.1f} s of CPU time, scaled by {units}/{n}"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

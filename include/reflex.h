@@ -65,6 +65,8 @@ typedef struct {
 
 const char *reflex_last_error_string(void);
 const char *reflex_version(void);
+/* Kernels launched by this library in this process so far (all entry points, all threads). */
+unsigned long long reflex_kernel_launch_count(void);
 
 /* ---- helpers around the five hot-path calls -------------------------------------------------- */
 

@@ -23,7 +23,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_IMPLEMENTED = -1, -2, -3, -4, -5, -6, -7
 
 EXPORTS = [
-    "reflex_last_error_string", "reflex_version", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
+    "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_init_static", "reflex_cache_append_sliding",
     "reflex_adarmsnorm", "reflex_partitioned_attention", "reflex_flow_step",
@@ -56,6 +56,7 @@ def load():
     dp = ctypes.POINTER(CacheDesc)
     lib.reflex_last_error_string.restype = ctypes.c_char_p
     lib.reflex_version.restype = ctypes.c_char_p
+    lib.reflex_kernel_launch_count.restype = ctypes.c_ulonglong
     lib.reflex_cache_slab_bytes.argtypes = [dp]; lib.reflex_cache_slab_bytes.restype = ctypes.c_size_t
     lib.reflex_workspace_bytes.argtypes = [dp]; lib.reflex_workspace_bytes.restype = ctypes.c_size_t
     lib.reflex_cache_create.argtypes = [dp, vp, vp, vp, i32p, vp, ctypes.POINTER(vp)]
@@ -69,9 +70,7 @@ def load():
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
     for name in EXPORTS:
-        fn = getattr(lib, name)
-        if fn.restype is ctypes.c_int or fn.restype is None:
-            fn.restype = ctypes.c_int
+        getattr(lib, name)  # every declared symbol must resolve
     _lib = lib
     return lib
 
@@ -115,6 +114,10 @@ def dtype_code(t: torch.Tensor) -> int:
 
 def reflex_version() -> str:
     return load().reflex_version().decode()
+
+
+def reflex_kernel_launch_count() -> int:
+    return int(load().reflex_kernel_launch_count())
 
 
 def reflex_cache_slab_bytes(desc: CacheDesc) -> int:

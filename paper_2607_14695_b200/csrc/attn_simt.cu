@@ -224,9 +224,11 @@ static cudaError_t launch_simt_t(const AttnParams &p, cudaStream_t st)
         case 8: attn_simt_kernel<T, 8><<<grid, kSimtWarps * 32, 0, st>>>(p); break;
         default: return cudaErrorInvalidValue;
     }
+    count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || p.nsplit == 1) return e;
     attn_merge_kernel<T><<<dim3(rows, p.B), p.d, 0, st>>>(p);
+    count_launch();
     return cudaGetLastError();
 }
 

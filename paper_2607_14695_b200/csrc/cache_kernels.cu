@@ -24,6 +24,7 @@ cudaError_t launch_state_init(StreamState *state, int64_t *total, uint32_t *stat
                               cudaStream_t st)
 {
     state_init_kernel<<<(B + 127) / 128, 128, 0, st>>>(state, total, status, head0, B, N);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -59,6 +60,7 @@ cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, co
     dim3 grid(chunks, L, n);
     init_static_kernel<<<grid, 256, 0, st>>>((uint4 *)k_slab, (uint4 *)v_slab, (const uint4 *)k_src, (const uint4 *)v_src,
                                              state, batch, src_stream0, L, B, S_max + N, S_src, row_units);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -119,6 +121,7 @@ cudaError_t launch_append_sliding(void *k_slab, void *v_slab, const void *k_src,
     append_sliding_kernel<<<grid, 256, 0, st>>>((uint4 *)k_slab, (uint4 *)v_slab, (const uint4 *)k_src,
                                                 (const uint4 *)v_src, state, total, batch, src_stream0, L, B, S_max, N, m,
                                                 row_units);
+    count_launch();
     return cudaGetLastError();
 }
 

@@ -155,6 +155,7 @@ static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, c
         const int cols = 64;
         dim3 grid((D + cols - 1) / cols, B);
         gate_kernel<T><<<grid, 256, (size_t)(Cd + Hd) * 4, st>>>(cond, W1, b1, W2, b2, gate_buf, D, Cd, Hd, cols);
+        count_launch();
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
@@ -181,6 +182,7 @@ static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, c
         }
         adarmsnorm_kernel<T, false><<<grid, 256, smem, st>>>(x, y, nullptr, nullptr, nullptr, nullptr, nullptr, gate_buf, R, D, Cd, Hd, eps, rows_per_block);
     }
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -219,6 +221,7 @@ cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, fl
         flow_step_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(x, (const __nv_bfloat16 *)v, (__nv_bfloat16 *)x_lowp, n, dt);
     else
         flow_step_kernel<float><<<blocks, 256, 0, st>>>(x, (const float *)v, (float *)x_lowp, n, dt);
+    count_launch();
     return cudaGetLastError();
 }
 

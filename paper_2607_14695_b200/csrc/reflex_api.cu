@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in reflex.h: argument validation, the host mirror of the ring state,
 // kernel selection and launches. No call below allocates device memory.
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -70,6 +71,9 @@ int check_stream_ids(const reflex_cache *c, const int32_t *ids, int n)
 
 namespace reflex {
 
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
 WorkspaceLayout workspace_layout(const reflex_cache_desc &d)
 {
     WorkspaceLayout w;
@@ -96,6 +100,7 @@ extern "C" {
 
 const char *reflex_last_error_string(void) { return g_err; }
 const char *reflex_version(void) { return "reflex-b200 0.1 (sm_100a)"; }
+unsigned long long reflex_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 size_t reflex_cache_slab_bytes(const reflex_cache_desc *d)
 {

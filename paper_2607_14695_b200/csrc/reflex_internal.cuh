@@ -53,6 +53,9 @@ struct AttnParams {
     int dtype;
 };
 
+// Number of kernels this library has launched in this process (every launcher bumps it).
+void count_launch(int n = 1);
+
 // ---- launchers (each returns the cudaError_t of its launch) ----
 cudaError_t launch_state_init(StreamState *state, int64_t *total, uint32_t *status, const int32_t *head0_dev_or_null,
                               int B, int N, cudaStream_t st);

@@ -1,0 +1,149 @@
+"""Drives the hot path the way a serving loop would (product code: CUDA library only, no oracle).
+
+One "denoising step" = for every layer in order: AdaRMSNorm, then partitioned attention; then the
+Euler update of the action chunk. The projections that sit between those calls in the real layer are
+not part of this path, so every (layer, step-variant) has its own seeded inputs resident in HBM:
+all bytes the path must read are really read, and nothing is batched across layers or steps.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as rb
+from . import synth
+
+
+class StepRunner:
+    def __init__(self, w: synth.Workload, device: str = "cuda:0", variants: int = 2, attn_impl: int = rb.ATTN_AUTO,
+                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_two_launch: bool = False):
+        self.w = w
+        self.device = torch.device(device)
+        self.variants = variants
+        self.gate_two_launch = gate_two_launch
+        tdt = rb.torch_dtype(w.dtype)
+        self.tdt = tdt
+        g = torch.Generator(device=self.device)
+        g.manual_seed(1234 + w.seed)
+        self._gen = g
+
+        def rnd(*shape, std=1.0):
+            t = torch.randn(*shape, generator=g, device=self.device, dtype=torch.float32)
+            if std != 1.0:
+                t = t * std
+            return t.to(tdt).contiguous()
+
+        self.rnd = rnd
+        head0 = [int(h) for h in synth.ring_head0(w)]
+        self.cache = rb.Cache(w.L, w.B, w.Hq, w.Hkv, w.d, w.S_max, w.N, w.T, w.dtype, device=device, ring_head0=head0)
+        rb.reflex_cache_set_attention_impl(self.cache, attn_impl)
+        ids = list(range(w.B))
+        # static prefix, a few streams at a time to bound the staging tensors
+        chunk = max(1, min(w.B, 8))
+        for i0 in range(0, w.B, chunk):
+            sub = ids[i0:i0 + chunk]
+            rb.reflex_cache_init_static(self.cache, sub, rnd(len(sub), w.L, w.S, w.Hkv, w.d), rnd(len(sub), w.L, w.S, w.Hkv, w.d))
+        fill = w.N if ring_fill is None else ring_fill
+        left = fill
+        while left > 0:
+            m = min(left, w.N)
+            rb.reflex_cache_append_sliding(self.cache, ids, rnd(w.B, w.L, m, w.Hkv, w.d), rnd(w.B, w.L, m, w.Hkv, w.d))
+            left -= m
+        # per (layer, variant) inputs
+        self.x = [[self._norm_input() for _ in range(variants)] for _ in range(w.L)]
+        self.q = [[rnd(w.B, w.T, w.Hq, w.d) for _ in range(variants)] for _ in range(w.L)]
+        self.kd = [[rnd(w.B, w.T, w.Hkv, w.d) for _ in range(variants)] for _ in range(w.L)]
+        self.vd = [[rnd(w.B, w.T, w.Hkv, w.d) for _ in range(variants)] for _ in range(w.L)]
+        self.vflow = [rnd(w.B, w.T, w.A) for _ in range(variants)]
+        self.W = [[rnd(w.Hd, w.Cd, std=0.02), torch.zeros(w.Hd, dtype=tdt, device=self.device),
+                   rnd(w.D, w.Hd, std=0.02), torch.zeros(w.D, dtype=tdt, device=self.device)] for _ in range(w.L)]
+        self.cond = [torch.from_numpy(synth.cond_vectors(w, 1.0 - k / w.K)).to(self.device).to(tdt).contiguous() for k in range(w.K)]
+        self.y = torch.empty((w.B, w.T, w.D), dtype=tdt, device=self.device)
+        self.out = torch.empty((w.B, w.T, w.Hq, w.d), dtype=tdt, device=self.device)
+        self.gate_buf = torch.empty((w.B, w.D), dtype=torch.float32, device=self.device) if gate_two_launch else None
+        self.xa = torch.randn(w.B, w.T, w.A, generator=g, device=self.device, dtype=torch.float32)
+        self.host = None
+        if host_inputs:
+            self._make_host_copies()
+        torch.cuda.synchronize(self.device)
+
+    def _norm_input(self):
+        w = self.w
+        t = torch.randn(w.B, w.T, w.D, generator=self._gen, device=self.device, dtype=torch.float32)
+        if w.outlier_frac > 0:
+            mask = torch.rand(w.B, w.T, w.D, generator=self._gen, device=self.device) < w.outlier_frac
+            t = torch.where(mask, t * w.outlier_mult, t)
+        return t.to(self.tdt).contiguous()
+
+    # ---- bytes and flops the method must move / compute (per launch and per step) ----
+    def algorithmic(self):
+        w = self.w
+        es = 2 if w.dtype == synth.DTYPE_BF16 else 4
+        kv = (w.S + w.N + w.T) * w.Hkv * w.d * es * 2
+        qo = 2 * w.T * w.Hq * w.d * es
+        attn_bytes = w.B * (kv + qo)
+        norm_bytes = w.B * (2 * w.T * w.D * es + w.Cd * es) + (w.Hd * w.Cd + w.D * w.Hd + w.Hd + w.D) * es
+        flow_bytes = w.B * w.T * w.A * (8 + es)
+        attn_flops = 4.0 * w.B * w.T * w.Hq * (w.S + w.N + w.T) * w.d
+        return {"attn_bytes_per_launch": attn_bytes, "norm_bytes_per_launch": norm_bytes, "flow_bytes_per_launch": flow_bytes,
+                "bytes_per_step": w.L * (attn_bytes + norm_bytes) + flow_bytes, "attn_flops_per_launch": attn_flops,
+                "flops_per_step": w.L * attn_flops}
+
+    def input_bytes_resident(self):
+        n = 0
+        for group in (self.x, self.q, self.kd, self.vd):
+            for per_layer in group:
+                for t in per_layer:
+                    n += t.numel() * t.element_size()
+        n += 2 * self.cache.k_slab.numel() * self.cache.k_slab.element_size()
+        return n
+
+    # ---- the step ----
+    def norm(self, layer: int, k: int, variant: int):
+        W1, b1, W2, b2 = self.W[layer]
+        rb.reflex_adarmsnorm(self.x[layer][variant], self.y, self.cond[k % self.w.K], W1, b1, W2, b2, gate_buf=self.gate_buf)
+
+    def attention(self, layer: int, variant: int):
+        rb.reflex_partitioned_attention(self.cache, layer, self.q[layer][variant], self.kd[layer][variant], self.vd[layer][variant], self.out)
+
+    def flow(self, k: int, variant: int):
+        rb.reflex_flow_step(self.xa, self.vflow[variant], None, k % self.w.K, self.w.K)
+
+    def step(self, k: int):
+        """One denoising step over all layers and streams, inputs already in HBM."""
+        variant = k % self.variants
+        for layer in range(self.w.L):
+            self.norm(layer, k, variant)
+            self.attention(layer, variant)
+        self.flow(k, variant)
+
+    def step_timed(self, k: int, ev_attn, ev_norm):
+        """Same launches as step(), with CUDA events around every attention and norm call."""
+        variant = k % self.variants
+        rec = lambda: (lambda e: (e.record(), e)[1])(torch.cuda.Event(enable_timing=True))
+        for layer in range(self.w.L):
+            a = rec(); self.norm(layer, k, variant); b = rec(); self.attention(layer, variant); c = rec()
+            ev_norm.append((a, b)); ev_attn.append((b, c))
+        self.flow(k, variant)
+
+    # ---- end to end: this step's inputs come from pinned host memory, the action chunk goes back ----
+    def _make_host_copies(self):
+        pin = lambda t: t.cpu().pin_memory()
+        self.host = {name: [[pin(t) for t in per_layer] for per_layer in getattr(self, name)] for name in ("x", "q", "kd", "vd")}
+        self.host["vflow"] = [pin(t) for t in self.vflow]
+        self.host_xa = torch.empty(self.xa.shape, dtype=torch.float32).pin_memory()
+        nb = lambda t: t.numel() * t.element_size()
+        self.h2d_bytes_per_step = sum(nb(self.host[n][l][0]) for n in ("x", "q", "kd", "vd") for l in range(self.w.L)) + nb(self.host["vflow"][0])
+        self.d2h_bytes_per_step = nb(self.host_xa)
+
+    def step_from_host(self, k: int):
+        variant = k % self.variants
+        for layer in range(self.w.L):
+            for name in ("x", "q", "kd", "vd"):
+                getattr(self, name)[layer][variant].copy_(self.host[name][layer][variant], non_blocking=True)
+            self.norm(layer, k, variant)
+            self.attention(layer, variant)
+        self.vflow[variant].copy_(self.host["vflow"][variant], non_blocking=True)
+        self.flow(k, variant)
+        self.host_xa.copy_(self.xa, non_blocking=True)

@@ -266,7 +266,8 @@ def test_stale_dynamic_kv_negative_control(U):
     out = torch.empty((1, w.T, w.Hq, w.d), dtype=torch.bfloat16, device=U.DEV)
     rb.reflex_partitioned_attention(tw.g, 0, U.to_dev(q, w.dtype), U.to_dev(kd0, w.dtype), U.to_dev(vd0, w.dtype), out)
     right = tw.o.attention(0, 0, q[0], kd1[0], vd1[0])
-    assert np.abs(U.to_host(out)[0] - right).max() > 10 * U.BF16_MAX_ABS
+    err = np.abs(U.to_host(out)[0] - right)
+    assert err.max() > 5 * U.BF16_MAX_ABS and err.mean() > 5 * U.BF16_MEAN_ABS
 
 
 @pytest.mark.parametrize("cfg", ["cfg1", "cfg2"])
