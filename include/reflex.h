@@ -102,6 +102,12 @@ int reflex_cache_slot_map(reflex_cache_t *cache, int b, int32_t *slot_of_age);
 
 int reflex_cache_set_attention_impl(reflex_cache_t *cache, int impl);
 
+/* Every device-side wait in the kernels is bounded; a wait that runs out raises a status word in the
+ * workspace instead of hanging the GPU. Reads that word (synchronises `stream`): REFLEX_OK, or
+ * REFLEX_ERR_TIMEOUT with the wait site in the error string. The word stays set until the cache is
+ * created again. */
+int reflex_cache_check_status(reflex_cache_t *cache, void *stream);
+
 /* ---- the five hot-path calls ------------------------------------------------------------------ */
 
 /* Sec. 3.1 "Static Prefix ... computed once and permanently pinned"; timestep invariance of the

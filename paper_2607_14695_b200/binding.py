@@ -25,7 +25,7 @@ ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT
 EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
-    "reflex_cache_set_attention_impl", "reflex_cache_init_static", "reflex_cache_append_sliding",
+    "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
     "reflex_adarmsnorm", "reflex_partitioned_attention", "reflex_flow_step",
 ]
 
@@ -64,6 +64,7 @@ def load():
     lib.reflex_cache_get_state.argtypes = [vp, i32p, i32p, i32p, i64p, vp]
     lib.reflex_cache_slot_map.argtypes = [vp, i, i32p]
     lib.reflex_cache_set_attention_impl.argtypes = [vp, i]
+    lib.reflex_cache_check_status.argtypes = [vp, vp]
     lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_cache_append_sliding.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
@@ -178,6 +179,10 @@ def reflex_cache_slot_map(cache: Cache, b: int):
 
 def reflex_cache_set_attention_impl(cache: Cache, impl: int):
     _check(load().reflex_cache_set_attention_impl(cache.handle, int(impl)))
+
+
+def reflex_cache_check_status(cache: Cache, stream=None):
+    _check(load().reflex_cache_check_status(cache.handle, _stream(stream)))
 
 
 def reflex_cache_init_static(cache: Cache, stream_ids, k_static, v_static, S=None, stream=None):

@@ -227,7 +227,14 @@ static cudaError_t launch_simt_t(const AttnParams &p, cudaStream_t st)
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || p.nsplit == 1) return e;
-    attn_merge_kernel<T><<<dim3(rows, p.B), p.d, 0, st>>>(p);
+    return launch_attention_merge(p, st);
+}
+
+cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st)
+{
+    const int rows = p.T * p.Hq;
+    if (p.dtype == REFLEX_DTYPE_BF16) attn_merge_kernel<__nv_bfloat16><<<dim3(rows, p.B), p.d, 0, st>>>(p);
+    else attn_merge_kernel<float><<<dim3(rows, p.B), p.d, 0, st>>>(p);
     count_launch();
     return cudaGetLastError();
 }

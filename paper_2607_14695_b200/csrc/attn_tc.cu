@@ -1,0 +1,559 @@
+// Partitioned attention (Eq. 1) on the 5th-generation tensor cores: tcgen05.mma with TMEM accumulators,
+// K/V tiles of the three regions staged by TMA straight from where they live (static rows and ring slots
+// of the slab, dynamic tokens from the caller's tensors) -- no gather, no copy.
+//
+// One CTA owns one 128-row query tile of one (stream, KV head): rows are (token, head-in-group) pairs, so
+// all G query heads that share a KV head ride in the same MMA. It walks 64-key tiles with an online
+// softmax:
+//   warp 0        TMA producer (Q once, then K and V tiles through a 2-stage ring each)
+//   warp 1        MMA issuer: S = Q K^T (M128 N64, K-major operands), O += P V (M128 N=d, V is MN-major)
+//   warps 2..5    softmax: S from TMEM, mask, running max / sum, P (bf16) into swizzled shared memory,
+//                 lazy rescale of O in TMEM, final normalisation and store
+// S is double buffered in TMEM and P in shared memory, so Q K^T of tile j+1 overlaps the softmax of tile j.
+// With nsplit > 1 a CTA covers a slice of the key tiles and writes an (m, l, O) partial that the merge
+// kernel of the SIMT path combines.
+//
+// Every wait on an mbarrier is bounded; when one runs out the CTA raises a status word, stops waiting and
+// drains, so a mistake cannot hang the device.
+#include <cuda.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "reflex_internal.cuh"
+#include "sm100_ptx.cuh"
+
+namespace reflex {
+
+using namespace ptx;
+
+constexpr int kBM = 128;        // query rows per CTA
+constexpr int kBN = 64;         // keys per tile
+constexpr int kStages = 2;      // K and V ring depth
+constexpr int kTcThreads = 192;
+constexpr unsigned long long kWaitNs = 1000000000ull;  // every mbarrier wait gives up after ~1 s
+constexpr float kRescaleThreshold = 8.0f;  // in log2 units: O is rescaled only when the max grows by > 2^8
+
+struct TcParams {
+    const StreamState *state;
+    void *out;
+    float *partials;
+    uint32_t *status;
+    int B, L, Hq, Hkv, G, S_max, N, T, layer;
+    int dyn_mask;
+    float scale, scale_log2;
+    int nsplit;
+    int tile_tokens;  // 128 / G
+    int n_qtiles;
+};
+
+template <int HD> struct TcSmem {
+    static constexpr int CH = HD / 64;                  // 64-element (128-byte) chunks along head_dim
+    static constexpr uint32_t Q_BYTES = CH * kBM * 128;
+    static constexpr uint32_t KV_STAGE = CH * kBN * 128;
+    static constexpr uint32_t P_BYTES = kBM * 128;
+    static constexpr uint32_t OFF_Q = 0;
+    static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
+    static constexpr uint32_t OFF_V = OFF_K + kStages * KV_STAGE;
+    static constexpr uint32_t OFF_P = OFF_V + kStages * KV_STAGE;
+    static constexpr uint32_t OFF_BAR = OFF_P + 2 * P_BYTES;
+    static constexpr uint32_t TOTAL = OFF_BAR + 256 + 1024;  // barriers + slack to align the base to 1024 B
+};
+
+// barrier slots (8 bytes each) from OFF_BAR
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_SEMPTY = 11, B_PFULL = 13, B_PVDONE = 15, B_COUNT = 17 };
+
+struct TileRef {
+    int dyn;            // 0: slab map, 1: dynamic-token map
+    int row0;           // first row of the tile in that map's row axis
+    int kind;           // 0 static, 1 ring, 2 dynamic
+    int idx;            // tile index inside its region
+};
+
+struct TileGeom {
+    int S, N, T, count, oldest, ns, nr, nd, row_base, S_max, b;
+    __device__ __forceinline__ TileRef decode(int it) const
+    {
+        TileRef t;
+        if (it < ns) { t.dyn = 0; t.kind = 0; t.idx = it; t.row0 = row_base + it * kBN; }
+        else if (it < ns + nr) { t.dyn = 0; t.kind = 1; t.idx = it - ns; t.row0 = row_base + S_max + t.idx * kBN; }
+        else { t.dyn = 1; t.kind = 2; t.idx = it - ns - nr; t.row0 = b * T + t.idx * kBN; }
+        return t;
+    }
+    // which of the 64 keys of a tile are live (independent of the query row)
+    __device__ __forceinline__ uint64_t tile_mask(const TileRef &t) const
+    {
+        if (t.kind == 1) {
+            if (count >= N && (t.idx + 1) * kBN <= N) return ~0ull;
+            uint64_t m = 0;
+            for (int c = 0; c < kBN; ++c) {
+                const int slot = t.idx * kBN + c;
+                int age = slot - oldest;
+                if (age < 0) age += N;
+                if (slot < N && age < count) m |= (1ull << c);
+            }
+            return m;
+        }
+        const int len = (t.kind == 0) ? S : T;
+        const int valid = len - t.idx * kBN;
+        return valid >= kBN ? ~0ull : ((1ull << valid) - 1ull);
+    }
+};
+
+template <int HD>
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
+               const __grid_constant__ CUtensorMap tm_vd, const TcParams p)
+{
+    using L = TcSmem<HD>;
+    constexpr int CH = L::CH;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColO = 0, kColS = HD;  // O: HD fp32 columns; S: 2 x 64 columns
+    static_assert(HD + 2 * kBN <= 512, "TMEM budget");
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    const uint32_t bar0 = base + L::OFF_BAR;
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * (uint32_t)i; };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::OFF_BAR + 8 * B_COUNT);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qt = blockIdx.x % p.n_qtiles;
+    const int kvh = blockIdx.x / p.n_qtiles;
+    const int b = blockIdx.y;
+    const int split = blockIdx.z;
+    const int t0 = qt * p.tile_tokens;
+
+    TileGeom g;
+    {
+        const StreamState st = p.state[b];
+        g.S = st.static_len > 0 ? st.static_len : 0;
+        g.N = p.N; g.T = p.T; g.count = st.count;
+        g.oldest = (st.head - st.count) % p.N;
+        if (g.oldest < 0) g.oldest += p.N;
+        g.ns = (g.S + kBN - 1) / kBN;
+        g.nr = g.count > 0 ? (p.N + kBN - 1) / kBN : 0;
+        g.nd = (p.T + kBN - 1) / kBN;
+        g.row_base = (p.layer * p.B + b) * (p.S_max + p.N);
+        g.S_max = p.S_max; g.b = b;
+    }
+    const int n_tiles = g.ns + g.nr + g.nd;
+    const int per = (n_tiles + p.nsplit - 1) / p.nsplit;
+    const int it0 = split * per;
+    const int it1 = min(n_tiles, it0 + per);
+    const int n_local = max(0, it1 - it0);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < B_COUNT; ++i) {
+            const bool many = (i == B_SEMPTY || i == B_SEMPTY + 1 || i == B_PFULL || i == B_PFULL + 1);
+            mbar_init(bar(i), many ? 128u : 1u);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd);
+    }
+    if (warp == 1) tmem_alloc(smem_u32((const void *)tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // bounded wait (about one second of wall time): false, and the abort flag raised, when the barrier never flips
+    auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool {
+        if (mbar_try_wait(bar(i), parity)) return true;
+        const unsigned long long t_start = globaltimer_ns();
+        for (uint32_t n = 1;; ++n) {
+            if (mbar_try_wait(bar(i), parity)) return true;
+            if ((n & 255u) == 0u) {
+                if (*abort_flag) return false;
+                if (globaltimer_ns() - t_start > kWaitNs) break;
+            }
+        }
+        *abort_flag = 1u;
+        atomicCAS(p.status, 0u, 0x80000000u | (code << 16) | (blockIdx.x & 0xFFFFu));
+        return false;
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && n_local > 0) {
+            mbar_expect_tx(bar(B_QFULL), L::Q_BYTES);
+            for (int c = 0; c < CH; ++c)
+                tma_load_4d(base + L::OFF_Q + c * (kBM * 128), &tm_q, bar(B_QFULL), c * 64, kvh * p.G, t0, b);
+            bool ok = true;
+            for (int jj = 0; jj < n_local && ok; ++jj) {
+                const int st = jj % kStages;
+                const uint32_t ph = (uint32_t)((jj / kStages) - 1) & 1u;
+                const TileRef tr = g.decode(it0 + jj);
+                if (jj >= kStages) ok = wait(B_KEMPTY + st, ph, 1);
+                if (!ok) break;
+                mbar_expect_tx(bar(B_KFULL + st), L::KV_STAGE);
+                for (int c = 0; c < CH; ++c)
+                    tma_load_3d(base + L::OFF_K + st * L::KV_STAGE + c * (kBN * 128), tr.dyn ? &tm_kd : &tm_k, bar(B_KFULL + st),
+                                c * 64, kvh, tr.row0);
+                if (jj >= kStages) ok = wait(B_VEMPTY + st, ph, 2);
+                if (!ok) break;
+                mbar_expect_tx(bar(B_VFULL + st), L::KV_STAGE);
+                for (int c = 0; c < CH; ++c)
+                    tma_load_3d(base + L::OFF_V + st * L::KV_STAGE + c * (kBN * 128), tr.dyn ? &tm_vd : &tm_v, bar(B_VFULL + st),
+                                c * 64, kvh, tr.row0);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && n_local > 0) {
+            constexpr uint32_t idesc_qk = umma_idesc_bf16(kBM, kBN, false);
+            constexpr uint32_t idesc_pv = umma_idesc_bf16(kBM, HD, true);
+            auto issue_qk = [&](int jj) {
+                const int st = jj % kStages, buf = jj & 1;
+                const uint32_t d_tmem = tmem_base + kColS + buf * kBN;
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t a = base + L::OFF_Q + (kk >> 2) * (kBM * 128) + (kk & 3) * 32;
+                    const uint32_t bb = base + L::OFF_K + st * L::KV_STAGE + (kk >> 2) * (kBN * 128) + (kk & 3) * 32;
+                    umma_ss(d_tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(bar(B_KEMPTY + st));
+                umma_commit(bar(B_SFULL + buf));
+            };
+            bool ok = wait(B_QFULL, 0, 3) && wait(B_KFULL + 0, 0, 4);
+            if (ok) { tc_fence_after(); issue_qk(0); }
+            for (int jj = 0; jj < n_local && ok; ++jj) {
+                if (jj + 1 < n_local) {
+                    const int nj = jj + 1;
+                    ok = wait(B_KFULL + (nj % kStages), (uint32_t)(nj / kStages) & 1u, 5);
+                    if (ok && nj >= 2) ok = wait(B_SEMPTY + (nj & 1), (uint32_t)((nj >> 1) - 1) & 1u, 6);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(nj);
+                }
+                const int st = jj % kStages, buf = jj & 1;
+                ok = wait(B_VFULL + st, (uint32_t)(jj / kStages) & 1u, 7) && wait(B_PFULL + buf, (uint32_t)(jj >> 1) & 1u, 8);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < kBN / 16; ++kk) {
+                    const uint32_t a = base + L::OFF_P + buf * L::P_BYTES + kk * 32;
+                    const uint32_t bb = base + L::OFF_V + st * L::KV_STAGE + kk * (16 * 128);
+                    umma_ss(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, kBN * 128, 1024), idesc_pv,
+                            (jj > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(bar(B_VEMPTY + st));
+                umma_commit(bar(B_PVDONE + buf));
+            }
+        }
+    } else {
+        // ---------------- softmax / correction / epilogue: one query row per thread ----------------
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int t_row = t0 + row / p.G;
+        const int hq = kvh * p.G + row % p.G;
+        const bool row_live = t_row < p.T && row < p.tile_tokens * p.G;
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int jj = 0; jj < n_local && ok; ++jj) {
+            const int buf = jj & 1;
+            const uint32_t ph = (uint32_t)(jj >> 1) & 1u;
+            const TileRef tr = g.decode(it0 + jj);
+            const uint64_t tmask = g.tile_mask(tr);
+            uint64_t rmask = tmask;
+            if (tr.kind == 2 && p.dyn_mask) {
+                const int lim = t_row - tr.idx * kBN;
+                rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
+            }
+            ok = wait(B_SFULL + buf, ph, 9);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t r0[32], r1[32];
+            const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kBN;
+            tmem_ld32(s_addr, r0);
+            tmem_ld32(s_addr + 32, r1);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar(B_SEMPTY + buf));
+            float s[64];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
+            if (rmask != ~0ull) {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) if (!((rmask >> c) & 1ull)) s[c] = -INFINITY;
+            }
+            float mx = s[0];
+#pragma unroll
+            for (int c = 1; c < 64; ++c) mx = fmaxf(mx, s[c]);
+            if (jj == 0) {
+                m_ref = mx;
+            } else {
+                const bool grow = (mx - m_ref) * p.scale_log2 > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, grow)) {
+                    // O (and l) were accumulated against m_ref: bring them to the new reference before this tile's P V
+                    const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
+                    if (grow) m_ref = mx;
+                    l *= alpha;
+                    ok = wait(B_PVDONE + ((jj - 1) & 1), (uint32_t)((jj - 1) >> 1) & 1u, 10);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < HD / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tmem_base + lane_addr + kColO + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
+            float sum = 0.f;
+            uint32_t packed[32];
+#pragma unroll
+            for (int c = 0; c < 64; c += 2) {
+                const float p0 = ex2(fmaf(s[c], p.scale_log2, -mr));
+                const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, -mr));
+                sum += p0 + p1;
+                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                packed[c >> 1] = *reinterpret_cast<uint32_t *>(&h);
+            }
+            l += sum;
+            if (jj >= 2) {
+                ok = wait(B_PVDONE + buf, (uint32_t)((jj >> 1) - 1) & 1u, 11);  // P[buf] was read by the P V of tile jj-2
+                if (!ok) break;
+            }
+            uint8_t *p_row = smem + L::OFF_P + buf * L::P_BYTES + row * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint4 v = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+                *reinterpret_cast<uint4 *>(p_row + ((c ^ (row & 7)) << 4)) = v;
+            }
+            if (tmask != ~0ull) {
+                // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows
+                const int st = jj % kStages;
+                ok = wait(B_VFULL + st, (uint32_t)(jj / kStages) & 1u, 12);
+                if (!ok) break;
+                if (row < kBN && !((tmask >> row) & 1ull)) {
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::KV_STAGE + c * (kBN * 128) + row * 128);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(B_PFULL + buf));
+        }
+        // ---- epilogue ----
+        if (n_local > 0 && ok) {
+            const int last = n_local - 1;
+            ok = wait(B_PVDONE + (last & 1), (uint32_t)(last >> 1) & 1u, 13);
+        }
+        const int rows_total = p.T * p.Hq;
+        if (p.nsplit == 1) {
+            if (n_local > 0 && ok) {
+                tc_fence_after();
+                const float inv = 1.f / l;
+                __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + hq) * HD;
+#pragma unroll 1
+                for (int c = 0; c < HD / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                    tmem_wait_ld();
+                    if (row_live) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 v;
+                            uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * k]) * inv,
+                                                                         __uint_as_float(o[8 * i + 2 * k + 1]) * inv);
+                                vv[k] = *reinterpret_cast<uint32_t *>(&h);
+                            }
+                            *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = v;
+                        }
+                    }
+                }
+            }
+        } else {
+            float *part = p.partials + (((size_t)b * rows_total + (size_t)t_row * p.Hq + hq) * p.nsplit + split) * (HD + 2);
+            if (n_local > 0 && ok) {
+                tc_fence_after();
+                if (row_live) { part[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; part[1] = l; }
+#pragma unroll 1
+                for (int c = 0; c < HD / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                    tmem_wait_ld();
+                    if (row_live) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            *reinterpret_cast<float2 *>(part + 2 + c * 32 + 2 * i) = make_float2(__uint_as_float(o[2 * i]), __uint_as_float(o[2 * i + 1]));
+                    }
+                }
+            } else if (row_live) {
+                part[0] = -INFINITY; part[1] = 0.f;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side: tensor maps and launch
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return (EncodeTiledFn)sym;
+    }();
+    return fn;
+}
+
+// rank-3 map over rows of [rows][Hkv][d] bf16, box = 64 rows x 1 head x 64 elements, 128-byte swizzle
+bool make_kv_map(CUtensorMap *m, const void *ptr, uint64_t rows, int Hkv, int d)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)Hkv, rows};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)Hkv * d * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)kBN};
+    cuuint32_t es[3] = {1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// rank-4 map over q [B][T][Hq][d], box = (64 elements, G heads, 128/G tokens, 1 stream): rows land as (token, head)
+bool make_q_map(CUtensorMap *m, const void *ptr, int B, int T, int Hq, int d, int G)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)Hq, (cuuint64_t)T, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)Hq * d * 2, (cuuint64_t)T * Hq * d * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)G, (cuuint32_t)(kBM / G), 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct MapCache {
+    std::mutex mu;
+    std::map<std::tuple<const void *, int, int, int, int, int>, CUtensorMap> maps;  // (ptr, kind, a, b, c, d)
+    bool get(CUtensorMap *out, const void *ptr, int kind, int a, int b, int c, int d,
+             bool (*make)(CUtensorMap *, const void *, int, int, int, int))
+    {
+        std::lock_guard<std::mutex> lk(mu);
+        auto key = std::make_tuple(ptr, kind, a, b, c, d);
+        auto it = maps.find(key);
+        if (it != maps.end()) { *out = it->second; return true; }
+        if (maps.size() > 8192) maps.clear();
+        CUtensorMap m;
+        if (!make(&m, ptr, a, b, c, d)) return false;
+        maps[key] = m;
+        *out = m;
+        return true;
+    }
+};
+
+MapCache &cache() { static MapCache c; return c; }
+
+bool mk_slab(CUtensorMap *m, const void *ptr, int rows, int Hkv, int d, int) { return make_kv_map(m, ptr, (uint64_t)rows, Hkv, d); }
+bool mk_q(CUtensorMap *m, const void *ptr, int BT /*B<<16|T not used*/, int Hq, int d, int G)
+{
+    return make_q_map(m, ptr, BT >> 16, BT & 0xFFFF, Hq, d, G);
+}
+
+template <int HD>
+cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
+                     const CUtensorMap *mvd, const TcParams &tp, dim3 grid, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcSmem<HD>::TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    attn_tc_kernel<HD><<<grid, kTcThreads, TcSmem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_supported(const AttnParams &p)
+{
+    if (p.dtype != REFLEX_DTYPE_BF16) return false;
+    if (!(p.d == 64 || p.d == 128 || p.d == 256)) return false;
+    const int G = p.Hq / p.Hkv;
+    if (G > kBM || (kBM % G) != 0) return false;
+    if (p.B > 65535 || p.T > 65535) return false;
+    if ((uint64_t)p.L * p.B * (uint64_t)(p.S_max + p.N) > 0x7FFFFFFFull || (uint64_t)p.B * p.T > 0x7FFFFFFFull) return false;
+    return encode_fn() != nullptr;
+}
+
+int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
+{
+    const int G = p.Hq / p.Hkv;
+    const int tile_tokens = kBM / G;
+    const int n_qtiles = (p.T + tile_tokens - 1) / tile_tokens;
+    const int ctas = n_qtiles * p.Hkv * p.B;
+    const int n_tiles = (p.S_max + kBN - 1) / kBN + (p.N + kBN - 1) / kBN + (p.T + kBN - 1) / kBN;
+    if (ctas >= sm_count) return 1;
+    int want = (sm_count + ctas - 1) / ctas;
+    if (want > n_tiles) want = n_tiles;
+    if (want > kMaxSplits) want = kMaxSplits;
+    const size_t per_split = (size_t)p.B * p.T * p.Hq * (p.d + 2) * sizeof(float);
+    if (per_split > 0 && (size_t)want * per_split > partial_bytes) want = (int)(partial_bytes / per_split);
+    return want < 1 ? 1 : want;
+}
+
+cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, cudaStream_t st)
+{
+    const int G = p.Hq / p.Hkv;
+    const int rows_slab = p.L * p.B * (p.S_max + p.N);
+    CUtensorMap mk, mv, mkd, mvd, mq;
+    if (!cache().get(&mk, p.k_slab, 0, rows_slab, p.Hkv, p.d, 0, mk_slab) || !cache().get(&mv, p.v_slab, 0, rows_slab, p.Hkv, p.d, 0, mk_slab) ||
+        !cache().get(&mkd, p.k_dyn, 0, p.B * p.T, p.Hkv, p.d, 0, mk_slab) || !cache().get(&mvd, p.v_dyn, 0, p.B * p.T, p.Hkv, p.d, 0, mk_slab) ||
+        !cache().get(&mq, p.q, 1, (p.B << 16) | p.T, p.Hq, p.d, G, mk_q))
+        return cudaErrorInvalidValue;
+    TcParams tp;
+    tp.state = p.state; tp.out = p.out; tp.partials = p.partials; tp.status = status;
+    tp.B = p.B; tp.L = p.L; tp.Hq = p.Hq; tp.Hkv = p.Hkv; tp.G = G; tp.S_max = p.S_max; tp.N = p.N; tp.T = p.T; tp.layer = p.layer;
+    tp.dyn_mask = p.dyn_mask; tp.scale = p.scale; tp.scale_log2 = p.scale * 1.4426950408889634f;
+    tp.nsplit = p.nsplit;
+    tp.tile_tokens = kBM / G;
+    tp.n_qtiles = (p.T + tp.tile_tokens - 1) / tp.tile_tokens;
+    dim3 grid(tp.n_qtiles * p.Hkv, p.B, p.nsplit);
+    cudaError_t e;
+    switch (p.d) {
+        case 64: e = launch_t<64>(&mq, &mk, &mv, &mkd, &mvd, tp, grid, st); break;
+        case 128: e = launch_t<128>(&mq, &mk, &mv, &mkd, &mvd, tp, grid, st); break;
+        case 256: e = launch_t<256>(&mq, &mk, &mv, &mkd, &mvd, tp, grid, st); break;
+        default: return cudaErrorInvalidValue;
+    }
+    if (e != cudaSuccess || p.nsplit == 1) return e;
+    return launch_attention_merge(p, st);
+}
+
+}  // namespace reflex

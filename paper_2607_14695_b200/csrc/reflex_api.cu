@@ -203,6 +203,20 @@ int reflex_cache_slot_map(reflex_cache_t *c, int b, int32_t *slot_of_age)
     return REFLEX_OK;
 }
 
+int reflex_cache_check_status(reflex_cache_t *c, void *stream)
+{
+    if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");
+    uint32_t word = 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(&word, c->ws + c->lay.status_off, sizeof(word), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "status read-back");
+    if (word != 0u)
+        return fail(REFLEX_ERR_TIMEOUT, "a device-side wait ran out (status 0x%08x: wait site %u, block %u); results of that launch are invalid",
+                    word, (word >> 16) & 0x7FFFu, word & 0xFFFFu);
+    return REFLEX_OK;
+}
+
 int reflex_cache_set_attention_impl(reflex_cache_t *c, int impl)
 {
     if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");
@@ -324,9 +338,17 @@ int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, co
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)d.d);
     p.dtype = d.dtype;
     p.nsplit = 1;
-    if (c->attn_impl == REFLEX_ATTN_TC) return fail(REFLEX_ERR_NOT_IMPLEMENTED, "tensor-core attention is not built for this shape");
-    p.nsplit = simt_choose_splits(p, c->lay.partial_bytes, c->sm_count);
-    cudaError_t e = launch_attention_simt(p, (cudaStream_t)stream);
+    const bool tc_ok = tc_supported(p);
+    if (c->attn_impl == REFLEX_ATTN_TC && !tc_ok)
+        return fail(REFLEX_ERR_NOT_IMPLEMENTED, "tensor-core attention needs bf16, d in {64,128,256} and 128 %% (Hq/Hkv) == 0");
+    cudaError_t e;
+    if (tc_ok && c->attn_impl != REFLEX_ATTN_SIMT) {
+        p.nsplit = tc_choose_splits(p, c->lay.partial_bytes, c->sm_count);
+        e = launch_attention_tc(p, (uint32_t *)(c->ws + c->lay.status_off), (cudaStream_t)stream);
+    } else {
+        p.nsplit = simt_choose_splits(p, c->lay.partial_bytes, c->sm_count);
+        e = launch_attention_simt(p, (cudaStream_t)stream);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");
     return REFLEX_OK;
 }

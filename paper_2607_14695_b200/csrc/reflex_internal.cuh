@@ -71,5 +71,9 @@ cudaError_t launch_adarmsnorm(const void *x, void *y, const void *cond, const vo
 cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, float dt, int dtype, cudaStream_t st);
 cudaError_t launch_attention_simt(const AttnParams &p, cudaStream_t st);
 int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
+cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st);  // combines nsplit (m, l, acc) partials
+bool tc_supported(const AttnParams &p);
+int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
+cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, cudaStream_t st);
 
 }  // namespace reflex

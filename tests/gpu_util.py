@@ -101,6 +101,7 @@ class Twin:
         out = torch.full((w.B, T, w.Hq, w.d), float("nan"), dtype=rb.torch_dtype(w.dtype), device=DEV)
         rb.reflex_partitioned_attention(self.g, layer, to_dev(q, w.dtype), to_dev(kd, w.dtype), to_dev(vd, w.dtype), out,
                                         scale=scale, dyn_mask=dyn_mask)
+        rb.reflex_cache_check_status(self.g)   # no bounded device-side wait ran out
         got = to_host(out)
         assert np.isfinite(got).all(), f"{what}: non-finite output"
         streams = list(range(w.B)) if streams is None else streams

@@ -85,13 +85,13 @@ def test_cfg1_full_trace(U):
 # ------------------------------------------------------------------------------------------------
 # config 2: one pi0-class layer, batch 1, bf16
 # ------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "tc"])
 @pytest.mark.parametrize("count", [5, 32, 45])
 def test_cfg2_layer(U, impl, count):
     rb = U.rb
     w = synth.CONFIGS["cfg2"]
     tw = U.Twin(w, head0=[7], poison=True)
-    rb.reflex_cache_set_attention_impl(tw.g, rb.ATTN_SIMT if impl == "simt" else rb.ATTN_AUTO)
+    rb.reflex_cache_set_attention_impl(tw.g, rb.ATTN_SIMT if impl == "simt" else rb.ATTN_TC)
     tw.init_static([0], [w.S])
     for i in range(count):
         tw.append([0], 1, i)
@@ -184,14 +184,19 @@ EDGE = [
     ("m_equals_N", 2, 1, 8, 1, 256, 100, 64, 16, 17, [16, 16, 3], synth.DTYPE_BF16),
     ("empty_ring", 1, 1, 8, 1, 256, 130, 129, 8, 50, [], synth.DTYPE_BF16),
     ("f32_d256", 1, 1, 8, 2, 256, 65, 65, 33, 5, [33, 1], synth.DTYPE_F32),
+    ("long_dyn_T130", 2, 1, 8, 1, 256, 200, 191, 70, 130, [70, 5], synth.DTYPE_BF16),       # several dynamic and ring tiles
+    ("g16_two_kv", 2, 2, 32, 2, 128, 96, 64, 64, 9, [64], synth.DTYPE_BF16),               # G = 16, exact tile boundaries
+    ("g3_simt_only", 1, 1, 6, 2, 64, 20, 20, 4, 5, [3], synth.DTYPE_BF16),                 # 128 % G != 0: SIMT even on auto
 ]
 
 
+@pytest.mark.parametrize("impl", ["simt", "auto"])
 @pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
-def test_edge_shapes(U, case):
+def test_edge_shapes(U, case, impl):
     name, B, L, Hq, Hkv, d, S_max, S, N, T, appends, dtype = case
     w = synth.Workload(name, 77, dtype, B=B, L=L, Hq=Hq, Hkv=Hkv, d=d, S=S, S_max=S_max, N=N, T=T, D=64, Cd=8, Hd=8, A=4, K=2)
     tw = U.Twin(w, head0=[(3 * b) % N for b in range(B)], T_max=T + 3, poison=True)
+    U.rb.reflex_cache_set_attention_impl(tw.g, U.rb.ATTN_SIMT if impl == "simt" else U.rb.ATTN_AUTO)
     tw.init_static(list(range(B)), [S] * B)
     for i, m in enumerate(appends):
         tw.append(list(range(B)), m, i)
