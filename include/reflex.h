@@ -47,9 +47,11 @@ extern "C" {
 #define REFLEX_DTYPE_F32  1
 
 /* attention kernel selection (reflex_cache_set_attention_impl) */
-#define REFLEX_ATTN_AUTO   0   /* tensor-core kernel when the shape qualifies, else the SIMT kernel */
+#define REFLEX_ATTN_AUTO   0   /* a tensor-core kernel when the shape qualifies, else the SIMT kernel */
 #define REFLEX_ATTN_SIMT   1   /* fp32-FMA split-K kernel, any supported shape and dtype            */
-#define REFLEX_ATTN_TC     2   /* tcgen05 kernel only; REFLEX_ERR_NOT_IMPLEMENTED if it cannot run  */
+#define REFLEX_ATTN_TC     2   /* tcgen05 kernel, one CTA per 128-row query tile, key split when the grid is small;
+                                  REFLEX_ERR_NOT_IMPLEMENTED if the shape does not qualify             */
+#define REFLEX_ATTN_TC2    3   /* tcgen05 cta_group::2 kernel: a CTA pair per 256 query rows (batched serving)  */
 
 typedef struct reflex_cache reflex_cache_t; /* opaque, host-side */
 
@@ -137,9 +139,13 @@ int reflex_cache_append_sliding(reflex_cache_t *cache, const int32_t *stream_ids
  *   x, y     device [B][R][D], may alias
  *   cond     device [B][Cd] dtype, or NULL when gate_buf holds a precomputed gate
  *   W1 [Hd][Cd], b1 [Hd], W2 [D][Hd], b2 [D]  device, dtype (ignored when cond == NULL)
- *   gate_buf device [B][D] fp32 or NULL.  cond != NULL, gate_buf == NULL: one fused launch.
- *            cond != NULL, gate_buf != NULL: the gate is written to gate_buf, then used (two launches).
- *            cond == NULL: gate_buf is an input.
+ *   gate_buf device fp32 or NULL.
+ *            cond != NULL, gate_buf == NULL: one fused launch, every block recomputes its stream's gate
+ *                                            (fine for a single stream, wasteful for a batch).
+ *            cond != NULL, gate_buf != NULL: gate_buf holds B*(D+Hd) floats: the gate [B][D] is written
+ *                                            there, followed by [B][Hd] hidden-layer scratch; three
+ *                                            launches (hidden, gate, rows), weights read once per 16 streams.
+ *            cond == NULL: gate_buf [B][D] is an input (a gate computed earlier, e.g. once per tick).
  * Requirements: D % 8 == 0, Cd % 8 == 0, Hd % 8 == 0, D <= 16384, Cd, Hd <= 4096. */
 int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, const void *b1,
                       const void *W2, const void *b2, float *gate_buf, int B, int R, int D, int Cd,

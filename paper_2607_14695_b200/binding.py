@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libreflex_b200.so")
 
 DTYPE_BF16 = 0
 DTYPE_F32 = 1
-ATTN_AUTO, ATTN_SIMT, ATTN_TC = 0, 1, 2
+ATTN_AUTO, ATTN_SIMT, ATTN_TC, ATTN_TC2 = 0, 1, 2, 3
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_IMPLEMENTED = -1, -2, -3, -4, -5, -6, -7
@@ -203,7 +203,8 @@ def reflex_cache_append_sliding(cache: Cache, stream_ids, k_new, v_new, stream=N
 
 
 def reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6, stream=None):
-    """x, y [B][R][D]; cond [B][Cd] or None (then gate_buf [B][D] fp32 is the precomputed gate)."""
+    """x, y [B][R][D]; cond [B][Cd] or None (then gate_buf [B][D] fp32 is the precomputed gate).
+    With cond given, gate_buf (optional) must hold B*(D+Hd) floats: gate, then hidden-layer scratch."""
     B, R, D = x.shape
     Hd, Cd = (W1.shape if W1 is not None else (0, 0))
     _check(load().reflex_adarmsnorm(_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf),
@@ -224,3 +225,40 @@ def reflex_flow_step(x, v, x_lowp, k, K, stream=None):
     B, T, A = x.shape
     _check(load().reflex_flow_step(_ptr(x), _ptr(v), _ptr(x_lowp), B, T, A, int(k), int(K), dtype_code(v), _stream(stream)))
     return x
+
+
+# ---- prepared calls: arguments marshalled once, then replayed with ~1 us of host overhead per call ----
+
+def stream_handle(stream=None) -> ctypes.c_void_p:
+    """ctypes handle of a torch stream (default: the current one), for the prepared calls below."""
+    return _stream(stream)
+
+
+def _prepared(fn, args):
+    lib = load()
+
+    def call(stream: ctypes.c_void_p):
+        rc = fn(*args, stream)
+        if rc != OK:
+            raise ReflexError(rc, lib.reflex_last_error_string().decode())
+
+    return call
+
+
+def prepare_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6):
+    B, R, D = x.shape
+    Hd, Cd = (W1.shape if W1 is not None else (0, 0))
+    args = (_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), B, R, D, int(Cd), int(Hd),
+            float(eps), dtype_code(x))
+    return _prepared(load().reflex_adarmsnorm, args)
+
+
+def prepare_partitioned_attention(cache: Cache, layer, q, k_dyn, v_dyn, out, scale=0.0, dyn_mask=0):
+    args = (cache.handle, int(layer), _ptr(q), _ptr(k_dyn), _ptr(v_dyn), _ptr(out), int(q.shape[1]), float(scale), int(dyn_mask))
+    return _prepared(load().reflex_partitioned_attention, args)
+
+
+def prepare_flow_step(x, v, x_lowp, k, K):
+    B, T, A = x.shape
+    args = (_ptr(x), _ptr(v), _ptr(x_lowp), B, T, A, int(k), int(K), dtype_code(v))
+    return _prepared(load().reflex_flow_step, args)

@@ -410,6 +410,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+}  // namespace reflex
+
+#include "attn_tc2.cuh"
+
+namespace reflex {
+
 // ------------------------------------------------------------------------------------------------
 // host side: tensor maps and launch
 // ------------------------------------------------------------------------------------------------
@@ -499,6 +505,21 @@ cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtenso
     return cudaGetLastError();
 }
 
+template <int HD>
+cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
+                      const CUtensorMap *mvd, const TcParams &tp, dim3 grid, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Tc2Smem<HD>::TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    attn_tc2_kernel<HD><<<grid, kTcThreads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 bool tc_supported(const AttnParams &p)
@@ -528,7 +549,9 @@ int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
     return want < 1 ? 1 : want;
 }
 
-cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, cudaStream_t st)
+bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 || p.d == 256); }
+
+cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, cudaStream_t st)
 {
     const int G = p.Hq / p.Hkv;
     const int rows_slab = p.L * p.B * (p.S_max + p.N);
@@ -544,8 +567,16 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, cudaStrea
     tp.nsplit = p.nsplit;
     tp.tile_tokens = kBM / G;
     tp.n_qtiles = (p.T + tp.tile_tokens - 1) / tp.tile_tokens;
-    dim3 grid(tp.n_qtiles * p.Hkv, p.B, p.nsplit);
     cudaError_t e;
+    if (two_cta) {
+        // pairs of query tiles; an odd tile count leaves the last pair with one idle half
+        tp.n_qtiles = (tp.n_qtiles + 1) / 2;
+        dim3 grid2(2 * tp.n_qtiles * p.Hkv, p.B, 1);
+        if (p.d == 256) return launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
+        if (p.d == 128) return launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
+        return cudaErrorInvalidValue;
+    }
+    dim3 grid(tp.n_qtiles * p.Hkv, p.B, p.nsplit);
     switch (p.d) {
         case 64: e = launch_t<64>(&mq, &mk, &mv, &mkd, &mvd, tp, grid, st); break;
         case 128: e = launch_t<128>(&mq, &mk, &mv, &mkd, &mvd, tp, grid, st); break;

@@ -1,0 +1,348 @@
+// Partitioned attention (Eq. 1), two-CTA form: a cluster of two CTAs (two SMs) drives one
+// tcgen05.mma.cta_group::2 with M = 256 -- two 128-row query tiles of the same (stream, KV head). The B
+// operand of such an MMA is split between the two CTAs' shared memories, so each CTA stages only HALF of
+// every K tile (64 of its 128 keys) and HALF of every V tile (128 of the head_dim columns): the bytes each
+// SM pulls per key are halved against the one-CTA kernel, which is what lets the loads keep up with the
+// tensor pipe at head_dim 256. Included by attn_tc.cu (shares its tile geometry and tensor maps).
+//
+// Per CTA:  warp 0  TMA producer (own Q tile, own K half, own V half)
+//           warp 1  MMA issuer (leader CTA only): S = Q K^T (M256 N128), O += P V (M256 N=d)
+//           warps 2..5  softmax over this CTA's 128 rows x 128 keys, P into swizzled shared memory,
+//                       lazy rescale of O in TMEM, epilogue
+// Barriers the leader's MMA thread waits on collect both CTAs (TMA completions through cta_group::2 loads,
+// softmax arrivals through shared::cluster arrives); completions fan out with multicast commits.
+#pragma once
+
+namespace reflex {
+
+constexpr int kTc2Keys = 128;  // keys per tile = two 64-key halves, one per CTA of the pair
+
+template <int HD> struct Tc2Smem {
+    static constexpr int CH = HD / 64;
+    static constexpr int VCH = CH / 2;                          // this CTA's 64-column chunks of head_dim
+    static constexpr uint32_t Q_BYTES = CH * 128 * 128;
+    static constexpr uint32_t K_STAGE = CH * 64 * 128;          // 64 keys x head_dim
+    static constexpr uint32_t V_STAGE = VCH * 128 * 128;        // 128 keys x head_dim/2
+    static constexpr uint32_t V_HALF = VCH * 64 * 128;          // bytes one 64-key half contributes
+    static constexpr uint32_t P_BYTES = 2 * 128 * 128;          // 128 rows x 128 keys bf16
+    static constexpr uint32_t OFF_Q = 0;
+    static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
+    static constexpr uint32_t OFF_V = OFF_K + 2 * K_STAGE;
+    static constexpr uint32_t OFF_P = OFF_V + 2 * V_STAGE;
+    static constexpr uint32_t OFF_BAR = OFF_P + P_BYTES;
+    static constexpr uint32_t TOTAL = OFF_BAR + 256 + 1024;
+};
+
+enum { C_QFULL = 0, C_KFULL = 1, C_KEMPTY = 3, C_VLAND = 5, C_VEMPTY = 7, C_SFULL = 9, C_SEMPTY = 11, C_PFULL = 13, C_PVDONE = 14, C_COUNT = 15 };
+
+template <int HD>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTcThreads, 1)
+attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
+                const __grid_constant__ CUtensorMap tm_vd, const TcParams p)
+{
+    using L = Tc2Smem<HD>;
+    constexpr int CH = L::CH, VCH = L::VCH;
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColO = 0, kColS = HD;  // O: HD fp32 columns; S: 2 x 128 columns
+    static_assert(HD + 2 * kTc2Keys <= 512 && VCH >= 1, "TMEM budget / head_dim split");
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    const uint32_t bar0 = base + L::OFF_BAR;
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * (uint32_t)i; };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::OFF_BAR + 8 * C_COUNT);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = (blockIdx.x >> 1) % p.n_qtiles;   // n_qtiles holds the number of tile pairs here
+    const int kvh = (blockIdx.x >> 1) / p.n_qtiles;
+    const int b = blockIdx.y;
+    const int t0 = (2 * pair + (int)rank) * p.tile_tokens;
+
+    TileGeom g;
+    {
+        const StreamState st = p.state[b];
+        g.S = st.static_len > 0 ? st.static_len : 0;
+        g.N = p.N; g.T = p.T; g.count = st.count;
+        g.oldest = (st.head - st.count) % p.N;
+        if (g.oldest < 0) g.oldest += p.N;
+        g.ns = (g.S + kBN - 1) / kBN;
+        g.nr = g.count > 0 ? (p.N + kBN - 1) / kBN : 0;
+        g.nd = (p.T + kBN - 1) / kBN;
+        g.row_base = (p.layer * p.B + b) * (p.S_max + p.N);
+        g.S_max = p.S_max; g.b = b;
+    }
+    const int H = g.ns + g.nr + g.nd;       // 64-key halves
+    const int n_tiles = (H + 1) / 2;        // >= 1: there is always a dynamic half
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C_COUNT; ++i) {
+            const bool both = (i == C_SEMPTY || i == C_SEMPTY + 1 || i == C_PFULL);
+            mbar_init(bar(i), both ? 256u : 1u);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd);
+    }
+    if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();   // both CTAs' barriers are initialised before anything crosses the pair
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto wait_impl = [&](int i, uint32_t parity, uint32_t code, bool cluster_scope) -> bool {
+        auto probe = [&]() { return cluster_scope ? mbar_try_wait_cluster(bar(i), parity) : mbar_try_wait(bar(i), parity); };
+        if (probe()) return true;
+        const unsigned long long t_start = globaltimer_ns();
+        for (uint32_t n = 1;; ++n) {
+            if (probe()) return true;
+            if ((n & 255u) == 0u) {
+                if (*abort_flag) return false;
+                if (globaltimer_ns() - t_start > kWaitNs) break;
+            }
+        }
+        *abort_flag = 1u;
+        atomicCAS(p.status, 0u, 0x80000000u | ((code + 32u) << 16) | (blockIdx.x & 0xFFFFu));
+        return false;
+    };
+    auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool { return wait_impl(i, parity, code, false); };
+    auto wait_cl = [&](int i, uint32_t parity, uint32_t code) -> bool { return wait_impl(i, parity, code, true); };
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs) ----------------
+        if (lane == 0) {
+            if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
+            for (int c = 0; c < CH; ++c)
+                tma2_load_4d(base + L::OFF_Q + c * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, c * 64, kvh * p.G, t0, b);
+            bool ok = true;
+            for (int jj = 0; jj < n_tiles && ok; ++jj) {
+                const int st = jj & 1;
+                const uint32_t ph = (uint32_t)((jj >> 1) - 1) & 1u;
+                const int h0 = 2 * jj, h1 = 2 * jj + 1;
+                const int live = (h0 < H ? 1 : 0) + (h1 < H ? 1 : 0);
+                if (jj >= 2) ok = wait(C_KEMPTY + st, ph, 1);
+                if (!ok) break;
+                if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
+                const int myh = 2 * jj + (int)rank;
+                if (myh < H) {
+                    const TileRef tr = g.decode(myh);
+                    for (int c = 0; c < CH; ++c)
+                        tma2_load_3d(base + L::OFF_K + st * L::K_STAGE + c * (64 * 128), tr.dyn ? &tm_kd : &tm_k,
+                                     bar(C_KFULL + st) & kPeerBitMask, c * 64, kvh, tr.row0);
+                }
+                if (jj >= 2) ok = wait(C_VEMPTY + st, ph, 2);
+                if (!ok) break;
+                mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
+                for (int hh = h0; hh <= h1; ++hh) {
+                    if (hh >= H) break;
+                    const TileRef tr = g.decode(hh);
+                    for (int c = 0; c < VCH; ++c)
+                        tma_load_3d(base + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (hh & 1) * (64 * 128), tr.dyn ? &tm_vd : &tm_v,
+                                    bar(C_VLAND + st), ((int)rank * VCH + c) * 64, kvh, tr.row0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader CTA) ----------------
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc_qk = umma_idesc_bf16(256, kTc2Keys, false);
+            constexpr uint32_t idesc_pv = umma_idesc_bf16(256, HD, true);
+            auto issue_qk = [&](int jj) {
+                const int st = jj & 1, buf = jj & 1;
+                const uint32_t d_tmem = tmem_base + kColS + buf * kTc2Keys;
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t a = base + L::OFF_Q + (kk >> 2) * (128 * 128) + (kk & 3) * 32;
+                    const uint32_t bb = base + L::OFF_K + st * L::K_STAGE + (kk >> 2) * (64 * 128) + (kk & 3) * 32;
+                    umma2_ss(d_tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+                }
+                umma2_commit_mc(bar(C_KEMPTY + st), 3);
+                umma2_commit_mc(bar(C_SFULL + buf), 3);
+            };
+            bool ok = wait_cl(C_QFULL, 0, 3) && wait_cl(C_KFULL + 0, 0, 4);
+            if (ok) { tc_fence_after(); issue_qk(0); }
+            for (int jj = 0; jj < n_tiles && ok; ++jj) {
+                if (jj + 1 < n_tiles) {
+                    const int nj = jj + 1;
+                    ok = wait_cl(C_KFULL + (nj & 1), (uint32_t)(nj >> 1) & 1u, 5);
+                    if (ok && nj >= 2) ok = wait_cl(C_SEMPTY + (nj & 1), (uint32_t)((nj >> 1) - 1) & 1u, 6);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(nj);
+                }
+                const int st = jj & 1;
+                ok = wait_cl(C_PFULL, (uint32_t)jj & 1u, 8);   // both CTAs: P written, V landed and cleaned
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
+                    const uint32_t a = base + L::OFF_P + (kk >> 2) * (128 * 128) + (kk & 3) * 32;
+                    const uint32_t bb = base + L::OFF_V + st * L::V_STAGE + kk * (16 * 128);
+                    umma2_ss(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv,
+                             (jj > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma2_commit_mc(bar(C_VEMPTY + st), 3);
+                umma2_commit_mc(bar(C_PVDONE), 3);
+            }
+        }
+    } else {
+        // ---------------- softmax / correction / epilogue (both CTAs): one query row per thread ----------------
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int t_row = t0 + row / p.G;
+        const int hq = kvh * p.G + row % p.G;
+        const bool row_live = t_row < p.T;
+        const uint32_t leader_pfull = mapa(bar(C_PFULL), 0);
+        float m_ref = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int jj = 0; jj < n_tiles && ok; ++jj) {
+            const int buf = jj & 1, st = jj & 1;
+            uint64_t tmask[2], rmask[2];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int h = 2 * jj + hh;
+                tmask[hh] = 0ull; rmask[hh] = 0ull;
+                if (h < H) {
+                    const TileRef tr = g.decode(h);
+                    tmask[hh] = g.tile_mask(tr);
+                    rmask[hh] = tmask[hh];
+                    if (tr.kind == 2 && p.dyn_mask) {
+                        const int lim = t_row - tr.idx * kBN;
+                        rmask[hh] &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
+                    }
+                }
+            }
+            ok = wait(C_SFULL + buf, (uint32_t)(jj >> 1) & 1u, 9);
+            if (!ok) break;
+            tc_fence_after();
+            float s[128];
+            {
+                const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys;
+                uint32_t r[4][32];
+                tmem_ld32(s_addr, r[0]); tmem_ld32(s_addr + 32, r[1]); tmem_ld32(s_addr + 64, r[2]); tmem_ld32(s_addr + 96, r[3]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) s[q4 * 32 + c] = __uint_as_float(r[q4][c]);
+            }
+            tc_fence_before();
+            mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                if (rmask[hh] != ~0ull) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) if (!((rmask[hh] >> c) & 1ull)) s[hh * 64 + c] = -INFINITY;
+                }
+            }
+            float mx = s[0];
+#pragma unroll
+            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+            bool pv_waited = false;
+            if (jj == 0) {
+                m_ref = mx;
+            } else {
+                const bool grow = (mx - m_ref) * p.scale_log2 > kRescaleThreshold;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
+                    if (grow) m_ref = mx;
+                    l *= alpha;
+                    ok = wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 10);
+                    if (!ok) break;
+                    pv_waited = true;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < HD / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tmem_base + lane_addr + kColO + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
+            float sum = 0.f;
+            uint32_t packed[64];
+#pragma unroll
+            for (int c = 0; c < 128; c += 2) {
+                const float p0 = ex2(fmaf(s[c], p.scale_log2, -mr));
+                const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, -mr));
+                sum += p0 + p1;
+                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
+                packed[c >> 1] = *reinterpret_cast<uint32_t *>(&h);
+            }
+            l += sum;
+            if (jj >= 1 && !pv_waited) {
+                ok = wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 11);  // the single P buffer was read by the P V of tile jj-1
+                if (!ok) break;
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                uint8_t *dst = smem + L::OFF_P + (c >> 3) * (128 * 128) + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+            }
+            // this CTA's V half has landed; dead keys get weight 0 but 0 x (stale NaN/Inf) would poison O: clear their rows
+            ok = wait(C_VLAND + st, (uint32_t)(jj >> 1) & 1u, 12);
+            if (!ok) break;
+            {
+                const uint64_t tm = tmask[row >> 6];
+                if (!((tm >> (row & 63)) & 1ull)) {
+#pragma unroll
+                    for (int c = 0; c < VCH; ++c) {
+                        uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + row * 128);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive_cluster(leader_pfull);
+        }
+        // ---- epilogue ----
+        if (ok) ok = wait(C_PVDONE, (uint32_t)(n_tiles - 1) & 1u, 13);
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l;
+            __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + hq) * HD;
+#pragma unroll 1
+            for (int c = 0; c < HD / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                tmem_wait_ld();
+                if (row_live) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 v;
+                        uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * k]) * inv,
+                                                                     __uint_as_float(o[8 * i + 2 * k + 1]) * inv);
+                            vv[k] = *reinterpret_cast<uint32_t *>(&h);
+                        }
+                        *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = v;
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();   // neither CTA retires while its partner can still touch its shared memory or barriers
+    if (warp == 1) tmem_dealloc2(tmem_base, kTmemCols);
+}
+
+}  // namespace reflex

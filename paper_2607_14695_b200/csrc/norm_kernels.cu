@@ -147,18 +147,172 @@ adarmsnorm_kernel(const T *x, T *y, const T *__restrict__ cond, const T *__restr
     }
 }
 
+
+// ---- three-launch form (gate scratch provided): hidden -> gate -> rows. Weights are read once per
+// ---- group of 8 streams instead of once per block, and every launch spreads over the machine.
+constexpr int kGateStreams = 8;
+
+// dot products of one weight row (global, lane-strided 8-element chunks) with kGateStreams vectors staged in
+// shared memory as fp32 ([kGateStreams][len]); returns the per-stream sums reduced over the warp.
+template <typename T>
+__device__ __forceinline__ void row_dots(const T *__restrict__ w, const float *vec_s, int len, int nb, float (&acc)[kGateStreams])
+{
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int s = 0; s < kGateStreams; ++s) acc[s] = 0.f;
+    for (int e = lane * 8; e < len; e += 256) {
+        float f[8];
+        Vec8<T>::load(w + e, f);
+#pragma unroll
+        for (int s = 0; s < kGateStreams; ++s) {
+            if (s < nb) {
+                const float4 a = *reinterpret_cast<const float4 *>(vec_s + s * len + e);
+                const float4 b = *reinterpret_cast<const float4 *>(vec_s + s * len + e + 4);
+                acc[s] = fmaf(f[0], a.x, acc[s]); acc[s] = fmaf(f[1], a.y, acc[s]); acc[s] = fmaf(f[2], a.z, acc[s]); acc[s] = fmaf(f[3], a.w, acc[s]);
+                acc[s] = fmaf(f[4], b.x, acc[s]); acc[s] = fmaf(f[5], b.y, acc[s]); acc[s] = fmaf(f[6], b.z, acc[s]); acc[s] = fmaf(f[7], b.w, acc[s]);
+            }
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < kGateStreams; ++s) acc[s] = warp_sum(acc[s]);
+}
+
+// grid = (ceil(Hd/8), ceil(B/8)); one warp per hidden unit for 8 streams.
+template <typename T>
+__global__ void __launch_bounds__(256)
+gate_hidden_kernel(const T *__restrict__ cond, const T *__restrict__ W1, const T *__restrict__ b1, float *__restrict__ hid_out,
+                   int B, int Cd, int Hd)
+{
+    extern __shared__ __align__(16) float c_s[];  // [kGateStreams][Cd]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int b0 = blockIdx.y * kGateStreams;
+    const int nb = min(kGateStreams, B - b0);
+    for (int i = threadIdx.x * 8; i < nb * Cd; i += blockDim.x * 8) {
+        float f[8];
+        Vec8<T>::load(cond + (size_t)b0 * Cd + i, f);
+        *reinterpret_cast<float4 *>(c_s + i) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4 *>(c_s + i + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+    __syncthreads();
+    const int j = blockIdx.x * 8 + warp;
+    if (j >= Hd) return;
+    float acc[kGateStreams];
+    row_dots<T>(W1 + (size_t)j * Cd, c_s, Cd, nb, acc);
+    const float bias = to_f<T>(b1[j]);
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kGateStreams; ++s) {
+            if (s < nb) {
+                const float z = acc[s] + bias;
+                hid_out[(size_t)(b0 + s) * Hd + j] = z / (1.f + expf(-z));
+            }
+        }
+    }
+}
+
+// grid = (ceil(D/8), ceil(B/8)); one warp per gate column for 8 streams.
+template <typename T>
+__global__ void __launch_bounds__(256)
+gate_out_kernel(const float *__restrict__ hid, const T *__restrict__ W2, const T *__restrict__ b2, float *__restrict__ gate_buf,
+                int B, int D, int Hd)
+{
+    extern __shared__ __align__(16) float h_s[];  // [kGateStreams][Hd]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int b0 = blockIdx.y * kGateStreams;
+    const int nb = min(kGateStreams, B - b0);
+    for (int i = threadIdx.x * 4; i < nb * Hd; i += blockDim.x * 4)
+        *reinterpret_cast<float4 *>(h_s + i) = *reinterpret_cast<const float4 *>(hid + (size_t)b0 * Hd + i);
+    __syncthreads();
+    const int col = blockIdx.x * 8 + warp;
+    if (col >= D) return;
+    float acc[kGateStreams];
+    row_dots<T>(W2 + (size_t)col * Hd, h_s, Hd, nb, acc);
+    const float bias = to_f<T>(b2[col]);
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kGateStreams; ++s)
+            if (s < nb) gate_buf[(size_t)(b0 + s) * D + col] = 1.f + (acc[s] + bias);
+    }
+}
+
+// One warp per row, the row kept in registers between the statistics pass and the scaling pass
+// (D <= 256 * NCH), so x is read from memory exactly once. grid = ceil(B*R / 8).
+template <typename T, int NCH>
+__global__ void __launch_bounds__(256)
+adarmsnorm_rows_kernel(const T *x, T *y, const float *__restrict__ gate_buf, int rows, int R, int D, float eps)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int row = blockIdx.x * 8 + warp;
+    if (row >= rows) return;
+    const int b = row / R;
+    const T *xr = x + (size_t)row * D;
+    T *yr = y + (size_t)row * D;
+    const float *g = gate_buf + (size_t)b * D;
+    float f[NCH][8];
+    float ss = 0.f;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        const int e = c * 256 + lane * 8;
+        if (e < D) {
+            Vec8<T>::load(xr + e, f[c]);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ss = fmaf(f[c][i], f[c][i], ss);
+        }
+    }
+    ss = warp_sum(ss);
+    const float rinv = 1.f / sqrtf(ss / (float)D + eps);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+        const int e = c * 256 + lane * 8;
+        if (e < D) {
+            const float4 g0 = __ldg(reinterpret_cast<const float4 *>(g + e));
+            const float4 g1 = __ldg(reinterpret_cast<const float4 *>(g + e + 4));
+            float o[8];
+            o[0] = f[c][0] * rinv * g0.x; o[1] = f[c][1] * rinv * g0.y; o[2] = f[c][2] * rinv * g0.z; o[3] = f[c][3] * rinv * g0.w;
+            o[4] = f[c][4] * rinv * g1.x; o[5] = f[c][5] * rinv * g1.y; o[6] = f[c][6] * rinv * g1.z; o[7] = f[c][7] * rinv * g1.w;
+            Vec8<T>::store(yr + e, o);
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B, int R, int D, float eps, cudaStream_t st)
+{
+    const int rows = B * R;
+    const int grid = (rows + 7) / 8;
+    if (D <= 512) adarmsnorm_rows_kernel<T, 2><<<grid, 256, 0, st>>>(x, y, gate_buf, rows, R, D, eps);
+    else if (D <= 1024) adarmsnorm_rows_kernel<T, 4><<<grid, 256, 0, st>>>(x, y, gate_buf, rows, R, D, eps);
+    else if (D <= 2048) adarmsnorm_rows_kernel<T, 8><<<grid, 256, 0, st>>>(x, y, gate_buf, rows, R, D, eps);
+    else return cudaErrorNotSupported;
+    count_launch();
+    return cudaGetLastError();
+}
+
 template <typename T>
 static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, const T *b1, const T *W2, const T *b2,
                                  float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, cudaStream_t st)
 {
-    if (cond && gate_buf) {
+    if (cond && gate_buf && Cd <= 1536 && Hd <= 1536) {
+        // gate_buf = [B][D] gate followed by [B][Hd] hidden-layer scratch
+        float *hid = gate_buf + (size_t)B * D;
+        const int groups = (B + kGateStreams - 1) / kGateStreams;
+        gate_hidden_kernel<T><<<dim3((Hd + 7) / 8, groups), 256, (size_t)kGateStreams * Cd * 4, st>>>(cond, W1, b1, hid, B, Cd, Hd);
+        count_launch();
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        gate_out_kernel<T><<<dim3((D + 7) / 8, groups), 256, (size_t)kGateStreams * Hd * 4, st>>>(hid, W2, b2, gate_buf, B, D, Hd);
+        count_launch();
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    } else if (cond && gate_buf) {
+        // very wide conditioning / hidden layers: per-block gate (shared-memory staging of 16 streams would not fit)
         const int cols = 64;
-        dim3 grid((D + cols - 1) / cols, B);
-        gate_kernel<T><<<grid, 256, (size_t)(Cd + Hd) * 4, st>>>(cond, W1, b1, W2, b2, gate_buf, D, Cd, Hd, cols);
+        gate_kernel<T><<<dim3((D + cols - 1) / cols, B), 256, (size_t)(Cd + Hd) * 4, st>>>(cond, W1, b1, W2, b2, gate_buf, D, Cd, Hd, cols);
         count_launch();
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
+    if (gate_buf && D <= 2048) return launch_rows_t<T>(x, y, gate_buf, B, R, D, eps, st);
     // enough blocks to cover the SMs about twice, at least one row per warp
     int chunks = (296 + B - 1) / B;
     const int max_chunks = (R + 7) / 8;

@@ -220,7 +220,7 @@ int reflex_cache_check_status(reflex_cache_t *c, void *stream)
 int reflex_cache_set_attention_impl(reflex_cache_t *c, int impl)
 {
     if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");
-    if (impl != REFLEX_ATTN_AUTO && impl != REFLEX_ATTN_SIMT && impl != REFLEX_ATTN_TC)
+    if (impl != REFLEX_ATTN_AUTO && impl != REFLEX_ATTN_SIMT && impl != REFLEX_ATTN_TC && impl != REFLEX_ATTN_TC2)
         return fail(REFLEX_ERR_INVALID_ARG, "unknown attention implementation %d", impl);
     c->attn_impl = impl;
     return REFLEX_OK;
@@ -339,15 +339,20 @@ int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, co
     p.dtype = d.dtype;
     p.nsplit = 1;
     const bool tc_ok = tc_supported(p);
-    if (c->attn_impl == REFLEX_ATTN_TC && !tc_ok)
-        return fail(REFLEX_ERR_NOT_IMPLEMENTED, "tensor-core attention needs bf16, d in {64,128,256} and 128 %% (Hq/Hkv) == 0");
+    const bool tc2_ok = tc2_supported(p);
+    if ((c->attn_impl == REFLEX_ATTN_TC && !tc_ok) || (c->attn_impl == REFLEX_ATTN_TC2 && !tc2_ok))
+        return fail(REFLEX_ERR_NOT_IMPLEMENTED, "tensor-core attention needs bf16, 128 %% (Hq/Hkv) == 0 and d in {64,128,256} (two-CTA form: {128,256})");
     cudaError_t e;
-    if (tc_ok && c->attn_impl != REFLEX_ATTN_SIMT) {
-        p.nsplit = tc_choose_splits(p, c->lay.partial_bytes, c->sm_count);
-        e = launch_attention_tc(p, (uint32_t *)(c->ws + c->lay.status_off), (cudaStream_t)stream);
-    } else {
+    uint32_t *status = (uint32_t *)(c->ws + c->lay.status_off);
+    if (c->attn_impl == REFLEX_ATTN_SIMT || !tc_ok) {
         p.nsplit = simt_choose_splits(p, c->lay.partial_bytes, c->sm_count);
         e = launch_attention_simt(p, (cudaStream_t)stream);
+    } else {
+        // enough query tiles to fill the machine: the two-CTA kernel (no key split); otherwise one CTA per tile with a key split
+        p.nsplit = tc_choose_splits(p, c->lay.partial_bytes, c->sm_count);
+        const bool two = c->attn_impl == REFLEX_ATTN_TC2 || (c->attn_impl == REFLEX_ATTN_AUTO && tc2_ok && p.nsplit == 1);
+        if (two) p.nsplit = 1;
+        e = launch_attention_tc(p, status, two, (cudaStream_t)stream);
     }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");
     return REFLEX_OK;

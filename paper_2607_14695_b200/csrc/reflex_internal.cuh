@@ -74,6 +74,7 @@ int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st);  // combines nsplit (m, l, acc) partials
 bool tc_supported(const AttnParams &p);
 int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
-cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, cudaStream_t st);
+bool tc2_supported(const AttnParams &p);
+cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, cudaStream_t st);
 
 }  // namespace reflex

@@ -17,11 +17,10 @@ from . import synth
 
 class StepRunner:
     def __init__(self, w: synth.Workload, device: str = "cuda:0", variants: int = 2, attn_impl: int = rb.ATTN_AUTO,
-                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_two_launch: bool = False):
+                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True):
         self.w = w
         self.device = torch.device(device)
         self.variants = variants
-        self.gate_two_launch = gate_two_launch
         tdt = rb.torch_dtype(w.dtype)
         self.tdt = tdt
         g = torch.Generator(device=self.device)
@@ -61,9 +60,11 @@ class StepRunner:
         self.cond = [torch.from_numpy(synth.cond_vectors(w, 1.0 - k / w.K)).to(self.device).to(tdt).contiguous() for k in range(w.K)]
         self.y = torch.empty((w.B, w.T, w.D), dtype=tdt, device=self.device)
         self.out = torch.empty((w.B, w.T, w.Hq, w.d), dtype=tdt, device=self.device)
-        self.gate_buf = torch.empty((w.B, w.D), dtype=torch.float32, device=self.device) if gate_two_launch else None
+        # gate [B][D] + hidden scratch [B][Hd]: lets AdaRMSNorm read the gate weights once per 16 streams
+        self.gate_buf = torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) if gate_scratch else None
         self.xa = torch.randn(w.B, w.T, w.A, generator=g, device=self.device, dtype=torch.float32)
         self.host = None
+        self._calls = {}
         if host_inputs:
             self._make_host_copies()
         torch.cuda.synchronize(self.device)
@@ -99,24 +100,35 @@ class StepRunner:
         n += 2 * self.cache.k_slab.numel() * self.cache.k_slab.element_size()
         return n
 
-    # ---- the step ----
-    def norm(self, layer: int, k: int, variant: int):
+    # ---- the step (calls are marshalled once and cached: the per-call host cost is ~1 us) ----
+    def _call(self, key, make):
+        c = self._calls.get(key)
+        if c is None:
+            c = self._calls[key] = make()
+        return c
+
+    def norm(self, layer: int, k: int, variant: int, sh=None):
+        kk = k % self.w.K
         W1, b1, W2, b2 = self.W[layer]
-        rb.reflex_adarmsnorm(self.x[layer][variant], self.y, self.cond[k % self.w.K], W1, b1, W2, b2, gate_buf=self.gate_buf)
+        self._call(("n", layer, kk, variant), lambda: rb.prepare_adarmsnorm(
+            self.x[layer][variant], self.y, self.cond[kk], W1, b1, W2, b2, gate_buf=self.gate_buf))(sh or rb.stream_handle())
 
-    def attention(self, layer: int, variant: int):
-        rb.reflex_partitioned_attention(self.cache, layer, self.q[layer][variant], self.kd[layer][variant], self.vd[layer][variant], self.out)
+    def attention(self, layer: int, variant: int, sh=None):
+        self._call(("a", layer, variant), lambda: rb.prepare_partitioned_attention(
+            self.cache, layer, self.q[layer][variant], self.kd[layer][variant], self.vd[layer][variant], self.out))(sh or rb.stream_handle())
 
-    def flow(self, k: int, variant: int):
-        rb.reflex_flow_step(self.xa, self.vflow[variant], None, k % self.w.K, self.w.K)
+    def flow(self, k: int, variant: int, sh=None):
+        kk = k % self.w.K
+        self._call(("f", kk, variant), lambda: rb.prepare_flow_step(self.xa, self.vflow[variant], None, kk, self.w.K))(sh or rb.stream_handle())
 
     def step(self, k: int):
         """One denoising step over all layers and streams, inputs already in HBM."""
         variant = k % self.variants
+        sh = rb.stream_handle()
         for layer in range(self.w.L):
-            self.norm(layer, k, variant)
-            self.attention(layer, variant)
-        self.flow(k, variant)
+            self.norm(layer, k, variant, sh)
+            self.attention(layer, variant, sh)
+        self.flow(k, variant, sh)
 
     def step_timed(self, k: int, ev_attn, ev_norm):
         """Same launches as step(), with CUDA events around every attention and norm call."""

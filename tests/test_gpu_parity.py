@@ -24,16 +24,16 @@ def _norm_case(U, w, x, cond, layer=0, eps=1e-6, gate_buf=False, alias=False, wh
     W1, b1, W2, b2 = synth.gate_weights(w, layer)
     dx = U.to_dev(x, w.dtype)
     dy = dx if alias else torch.full_like(dx, float("nan"))
-    gb = torch.empty((x.shape[0], w.D), dtype=torch.float32, device=U.DEV) if gate_buf else None
+    gb = torch.empty((x.shape[0] * (w.D + w.Hd),), dtype=torch.float32, device=U.DEV) if gate_buf else None
     rb.reflex_adarmsnorm(dx, dy, U.to_dev(cond, w.dtype), U.to_dev(W1, w.dtype), U.to_dev(b1, w.dtype), U.to_dev(W2, w.dtype),
                          U.to_dev(b2, w.dtype), gate_buf=gb, eps=eps)
     want = orc.adarmsnorm_batched(x, cond, W1, b1, W2, b2, eps)
     U.check_close(U.to_host(dy), want, w.dtype, what, rel_clause=True)
     if gate_buf:  # the gate itself, fp32, and the precomputed-gate entry
         _, g0 = orc.adarmsnorm(x[0], cond[0], W1, b1, W2, b2, eps, return_gate=True)
-        assert np.max(np.abs(U.to_host(gb[0]) - g0)) <= 1e-5
+        assert np.max(np.abs(U.to_host(gb[: w.D]) - g0)) <= 1e-5
         dy2 = torch.full_like(dx, float("nan"))
-        rb.reflex_adarmsnorm(U.to_dev(x, w.dtype), dy2, None, None, None, None, None, gate_buf=gb, eps=eps)
+        rb.reflex_adarmsnorm(U.to_dev(x, w.dtype), dy2, None, None, None, None, None, gate_buf=gb[: x.shape[0] * w.D].view(x.shape[0], w.D), eps=eps)
         assert torch.equal(dy2, dy)
     return dy
 
@@ -85,13 +85,13 @@ def test_cfg1_full_trace(U):
 # ------------------------------------------------------------------------------------------------
 # config 2: one pi0-class layer, batch 1, bf16
 # ------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("impl", ["simt", "tc"])
+@pytest.mark.parametrize("impl", ["simt", "tc", "tc2"])
 @pytest.mark.parametrize("count", [5, 32, 45])
 def test_cfg2_layer(U, impl, count):
     rb = U.rb
     w = synth.CONFIGS["cfg2"]
     tw = U.Twin(w, head0=[7], poison=True)
-    rb.reflex_cache_set_attention_impl(tw.g, rb.ATTN_SIMT if impl == "simt" else rb.ATTN_TC)
+    rb.reflex_cache_set_attention_impl(tw.g, {"simt": rb.ATTN_SIMT, "tc": rb.ATTN_TC, "tc2": rb.ATTN_TC2}[impl])
     tw.init_static([0], [w.S])
     for i in range(count):
         tw.append([0], 1, i)
@@ -159,9 +159,11 @@ def test_cfg4_batched_streams(U):
 # ------------------------------------------------------------------------------------------------
 # config 5 shapes: long context, outliers in the norm input, t near 0 and 1
 # ------------------------------------------------------------------------------------------------
-def test_cfg5_long_context(U):
+@pytest.mark.parametrize("impl", ["auto", "tc2"])
+def test_cfg5_long_context(U, impl):
     w = synth.CONFIGS["cfg5"].with_(L=2, B=4)
     tw = U.Twin(w, head0=synth.ring_head0(w), poison=True)
+    U.rb.reflex_cache_set_attention_impl(tw.g, U.rb.ATTN_AUTO if impl == "auto" else U.rb.ATTN_TC2)
     tw.init_static(list(range(w.B)), [w.S, w.S - 100, w.S, 1])
     for i in range(3):
         tw.append(list(range(w.B)), 100, i)      # frame-sized appends; wraps the 256-slot ring
@@ -190,13 +192,21 @@ EDGE = [
 ]
 
 
-@pytest.mark.parametrize("impl", ["simt", "auto"])
+@pytest.mark.parametrize("impl", ["simt", "auto", "tc2"])
 @pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
 def test_edge_shapes(U, case, impl):
     name, B, L, Hq, Hkv, d, S_max, S, N, T, appends, dtype = case
     w = synth.Workload(name, 77, dtype, B=B, L=L, Hq=Hq, Hkv=Hkv, d=d, S=S, S_max=S_max, N=N, T=T, D=64, Cd=8, Hd=8, A=4, K=2)
     tw = U.Twin(w, head0=[(3 * b) % N for b in range(B)], T_max=T + 3, poison=True)
-    U.rb.reflex_cache_set_attention_impl(tw.g, U.rb.ATTN_SIMT if impl == "simt" else U.rb.ATTN_AUTO)
+    U.rb.reflex_cache_set_attention_impl(tw.g, {"simt": U.rb.ATTN_SIMT, "auto": U.rb.ATTN_AUTO, "tc2": U.rb.ATTN_TC2}[impl])
+    if impl == "tc2" and not (dtype == synth.DTYPE_BF16 and d in (128, 256) and 128 % (Hq // Hkv) == 0):
+        tw.init_static(list(range(B)), [S] * B)
+        z = torch.zeros((B, T, Hq, d), dtype=U.rb.torch_dtype(dtype), device=U.DEV)
+        zk = torch.zeros((B, T, Hkv, d), dtype=U.rb.torch_dtype(dtype), device=U.DEV)
+        with pytest.raises(U.rb.ReflexError) as e:       # the two-CTA kernel refuses shapes it cannot run; nothing is launched
+            U.rb.reflex_partitioned_attention(tw.g, 0, z, zk, zk, z)
+        assert e.value.code == U.rb.ERR_NOT_IMPLEMENTED
+        return
     tw.init_static(list(range(B)), [S] * B)
     for i, m in enumerate(appends):
         tw.append(list(range(B)), m, i)
