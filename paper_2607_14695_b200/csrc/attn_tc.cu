@@ -515,7 +515,7 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attn_tc2_kernel<HD><<<grid, kTcThreads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
+    attn_tc2_kernel<HD><<<grid, kTc2Threads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
     count_launch();
     return cudaGetLastError();
 }

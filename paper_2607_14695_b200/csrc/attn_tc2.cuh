@@ -7,15 +7,25 @@
 //
 // Per CTA:  warp 0  TMA producer (own Q tile, own K half, own V half)
 //           warp 1  MMA issuer (leader CTA only): S = Q K^T (M256 N128), O += P V (M256 N=d)
-//           warps 2..5  softmax over this CTA's 128 rows x 128 keys, P into swizzled shared memory,
-//                       lazy rescale of O in TMEM, epilogue
+//           warps 2..9  softmax over this CTA's 128 rows x 128 keys (two threads per row, 64 keys each),
+//                       P into swizzled shared memory, lazy rescale of O in TMEM, epilogue
 // Barriers the leader's MMA thread waits on collect both CTAs (TMA completions through cta_group::2 loads,
 // softmax arrivals through shared::cluster arrives); completions fan out with multicast commits.
 #pragma once
 
 namespace reflex {
 
+// Optional timeline of one CTA pair (debug builds only: -DREFLEX_TRACE): clock64 stamps per role and tile into the
+// (otherwise unused) split-K partial area. Compiled out in the product library.
+#ifdef REFLEX_TRACE
+#define TC2_TRACE(role, tile, ev) do { if (blockIdx.x < 2 && blockIdx.y == 0 && (tile) < 16) \
+    reinterpret_cast<long long *>(p.partials)[((blockIdx.x * 4 + (role)) * 16 + (tile)) * 16 + (ev)] = clock64(); } while (0)
+#else
+#define TC2_TRACE(role, tile, ev) do { } while (0)
+#endif
+
 constexpr int kTc2Keys = 128;  // keys per tile = two 64-key halves, one per CTA of the pair
+constexpr int kTc2Threads = 320;  // producer warp, MMA warp, eight softmax warps
 
 template <int HD> struct Tc2Smem {
     static constexpr int CH = HD / 64;
@@ -30,13 +40,15 @@ template <int HD> struct Tc2Smem {
     static constexpr uint32_t OFF_V = OFF_K + 2 * K_STAGE;
     static constexpr uint32_t OFF_P = OFF_V + 2 * V_STAGE;
     static constexpr uint32_t OFF_BAR = OFF_P + P_BYTES;
-    static constexpr uint32_t TOTAL = OFF_BAR + 256 + 1024;
+    static constexpr uint32_t OFF_XCH = OFF_BAR + 128;              // row-maximum exchange between the two halves
+    static constexpr uint32_t NEED = OFF_XCH + 2 * 2 * 128 * 4;     // bytes used from the 1024-byte aligned base
+    static constexpr uint32_t TOTAL = 232448;                       // the whole opt-in shared memory of an SM (227 KB)
 };
 
 enum { C_QFULL = 0, C_KFULL = 1, C_KEMPTY = 3, C_VLAND = 5, C_VEMPTY = 7, C_SFULL = 9, C_SEMPTY = 11, C_PFULL = 13, C_PVDONE = 14, C_COUNT = 15 };
 
 template <int HD>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTcThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTc2Threads, 1)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
                 const __grid_constant__ CUtensorMap tm_vd, const TcParams p)
@@ -56,6 +68,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::OFF_BAR + 8 * C_COUNT);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
+    if ((base - raw_addr) + L::NEED > L::TOTAL) {
+        // the dynamic shared-memory window starts too far from a 1024-byte boundary to hold the tiles: same for every
+        // CTA of the launch, so all of them leave here, before any barrier, cluster or TMEM state exists
+        if (threadIdx.x == 0) atomicCAS(p.status, 0u, 0x80000000u | (99u << 16));
+        return;
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int pair = (blockIdx.x >> 1) % p.n_qtiles;   // n_qtiles holds the number of tile pairs here
@@ -82,7 +100,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int i = 0; i < C_COUNT; ++i) {
             const bool both = (i == C_SEMPTY || i == C_SEMPTY + 1 || i == C_PFULL);
-            mbar_init(bar(i), both ? 256u : 1u);
+            mbar_init(bar(i), both ? 16u : 1u);   // one arrival per softmax warp of either CTA
         }
         *abort_flag = 0u;
         fence_mbar_init();
@@ -97,7 +115,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
 
     auto wait_impl = [&](int i, uint32_t parity, uint32_t code, bool cluster_scope) -> bool {
-        auto probe = [&]() { return cluster_scope ? mbar_try_wait_cluster(bar(i), parity) : mbar_try_wait(bar(i), parity); };
+        auto probe = [&]() { (void)cluster_scope; return mbar_try_wait(bar(i), parity); };
         if (probe()) return true;
         const unsigned long long t_start = globaltimer_ns();
         for (uint32_t n = 1;; ++n) {
@@ -126,8 +144,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint32_t ph = (uint32_t)((jj >> 1) - 1) & 1u;
                 const int h0 = 2 * jj, h1 = 2 * jj + 1;
                 const int live = (h0 < H ? 1 : 0) + (h1 < H ? 1 : 0);
+                TC2_TRACE(0, jj, 0);
                 if (jj >= 2) ok = wait(C_KEMPTY + st, ph, 1);
                 if (!ok) break;
+                TC2_TRACE(0, jj, 1);
                 if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
                 const int myh = 2 * jj + (int)rank;
                 if (myh < H) {
@@ -138,6 +158,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (jj >= 2) ok = wait(C_VEMPTY + st, ph, 2);
                 if (!ok) break;
+                TC2_TRACE(0, jj, 2);
                 mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
                 for (int hh = h0; hh <= h1; ++hh) {
                     if (hh >= H) break;
@@ -170,15 +191,21 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int jj = 0; jj < n_tiles && ok; ++jj) {
                 if (jj + 1 < n_tiles) {
                     const int nj = jj + 1;
+                    TC2_TRACE(1, nj, 0);
                     ok = wait_cl(C_KFULL + (nj & 1), (uint32_t)(nj >> 1) & 1u, 5);
+                    TC2_TRACE(1, nj, 1);
                     if (ok && nj >= 2) ok = wait_cl(C_SEMPTY + (nj & 1), (uint32_t)((nj >> 1) - 1) & 1u, 6);
                     if (!ok) break;
+                    TC2_TRACE(1, nj, 2);
                     tc_fence_after();
                     issue_qk(nj);
+                    TC2_TRACE(1, nj, 3);
                 }
                 const int st = jj & 1;
+                TC2_TRACE(1, jj, 4);
                 ok = wait_cl(C_PFULL, (uint32_t)jj & 1u, 8);   // both CTAs: P written, V landed and cleaned
                 if (!ok) break;
+                TC2_TRACE(1, jj, 5);
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
@@ -189,136 +216,156 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 umma2_commit_mc(bar(C_VEMPTY + st), 3);
                 umma2_commit_mc(bar(C_PVDONE), 3);
+                TC2_TRACE(1, jj, 6);
             }
         }
     } else {
-        // ---------------- softmax / correction / epilogue (both CTAs): one query row per thread ----------------
-        const int quarter = warp & 3;
+        // ---------------- softmax / correction / epilogue (both CTAs) ----------------
+        // Eight warps: two threads per query row, one per 64-key half of the tile (warps 2..5 take the pair
+        // leader's keys, warps 6..9 the partner's). The halves meet once per tile to agree on the row maximum.
+        const int sw = warp - 2;
+        const int half = sw >> 2;                 // which 64 columns of S / 64-key chunk of P / half of O's columns
+        const int quarter = warp & 3;             // TMEM lane quarter this warp may touch
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int t_row = t0 + row / p.G;
         const int hq = kvh * p.G + row % p.G;
         const bool row_live = t_row < p.T;
         const uint32_t leader_pfull = mapa(bar(C_PFULL), 0);
+        float *exch = reinterpret_cast<float *>(smem + L::OFF_XCH);   // [2 buffers][2 halves][128 rows]
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int jj = 0; jj < n_tiles && ok; ++jj) {
+        // A wait that ran out does not leave this loop: every softmax warp keeps meeting the others at the named
+        // barrier (the remaining waits return at once), so no warp is left behind.
+        for (int jj = 0; jj < n_tiles; ++jj) {
             const int buf = jj & 1, st = jj & 1;
-            uint64_t tmask[2], rmask[2];
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int h = 2 * jj + hh;
-                tmask[hh] = 0ull; rmask[hh] = 0ull;
-                if (h < H) {
-                    const TileRef tr = g.decode(h);
-                    tmask[hh] = g.tile_mask(tr);
-                    rmask[hh] = tmask[hh];
-                    if (tr.kind == 2 && p.dyn_mask) {
-                        const int lim = t_row - tr.idx * kBN;
-                        rmask[hh] &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
-                    }
+            const int h = 2 * jj + half;
+            uint64_t tmask = 0ull, rmask = 0ull;
+            if (h < H) {
+                const TileRef tr = g.decode(h);
+                tmask = g.tile_mask(tr);
+                rmask = tmask;
+                if (tr.kind == 2 && p.dyn_mask) {
+                    const int lim = t_row - tr.idx * kBN;
+                    rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
                 }
             }
-            ok = wait(C_SFULL + buf, (uint32_t)(jj >> 1) & 1u, 9);
-            if (!ok) break;
+#define SM_TRACE(ev) do { if (lane == 0 && quarter == 2) TC2_TRACE(2 + half, jj, ev); } while (0)
+            SM_TRACE(0);
+            ok = ok && wait(C_SFULL + buf, (uint32_t)(jj >> 1) & 1u, 9);
+            SM_TRACE(1);
             tc_fence_after();
-            float s[128];
+            float s[64];
             {
-                const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys;
-                uint32_t r[4][32];
-                tmem_ld32(s_addr, r[0]); tmem_ld32(s_addr + 32, r[1]); tmem_ld32(s_addr + 64, r[2]); tmem_ld32(s_addr + 96, r[3]);
+                const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + half * 64;
+                uint32_t r0[32], r1[32];
+                tmem_ld32(s_addr, r0); tmem_ld32(s_addr + 32, r1);
                 tmem_wait_ld();
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4)
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) s[q4 * 32 + c] = __uint_as_float(r[q4][c]);
+                for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
             }
+            SM_TRACE(2);
             tc_fence_before();
-            mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
+            if (rmask != ~0ull) {
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                if (rmask[hh] != ~0ull) {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) if (!((rmask[hh] >> c) & 1ull)) s[hh * 64 + c] = -INFINITY;
-                }
+                for (int c = 0; c < 64; ++c) if (!((rmask >> c) & 1ull)) s[c] = -INFINITY;
             }
-            float mx = s[0];
+            float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
-            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+            for (int c = 4; c < 64; c += 4) {
+                mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
+                mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+            }
+            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            // meet the thread that holds the other 64 keys of this row
+            SM_TRACE(3);
+            exch[(buf * 2 + half) * 128 + row] = mx;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            SM_TRACE(4);
+            mx = fmaxf(mx, exch[(buf * 2 + (half ^ 1)) * 128 + row]);
             bool pv_waited = false;
             if (jj == 0) {
                 m_ref = mx;
             } else {
                 const bool grow = (mx - m_ref) * p.scale_log2 > kRescaleThreshold;
                 if (__any_sync(0xffffffffu, grow)) {
+                    // O (and l) were accumulated against m_ref: bring them to the new reference before this tile's P V.
+                    // Both threads of a row see the same mx, so they decide alike; each rescales its half of O's columns.
                     const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
                     if (grow) m_ref = mx;
                     l *= alpha;
-                    ok = wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 10);
-                    if (!ok) break;
+                    ok = ok && wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 10);
                     pv_waited = true;
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < HD / 32; ++c) {
+                    for (int c = 0; c < HD / 64; ++c) {
                         uint32_t o[32];
-                        tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                        const uint32_t o_addr = tmem_base + lane_addr + kColO + half * (HD / 2) + c * 32;
+                        tmem_ld32(o_addr, o);
                         tmem_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(tmem_base + lane_addr + kColO + c * 32, o);
+                        tmem_st32(o_addr, o);
                     }
                     tmem_wait_st();
                 }
             }
             const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
-            float sum = 0.f;
-            uint32_t packed[64];
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t packed[32];
 #pragma unroll
-            for (int c = 0; c < 128; c += 2) {
+            for (int c = 0; c < 64; c += 2) {
                 const float p0 = ex2(fmaf(s[c], p.scale_log2, -mr));
                 const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, -mr));
-                sum += p0 + p1;
-                __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                packed[c >> 1] = *reinterpret_cast<uint32_t *>(&h);
+                sum4[(c >> 1) & 3] += p0 + p1;
+                __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+                packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
             }
-            l += sum;
+            l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            SM_TRACE(5);
             if (jj >= 1 && !pv_waited) {
-                ok = wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 11);  // the single P buffer was read by the P V of tile jj-1
-                if (!ok) break;
+                ok = ok && wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 11);  // the single P buffer was read by the P V of tile jj-1
             }
+            SM_TRACE(6);
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                uint8_t *dst = smem + L::OFF_P + (c >> 3) * (128 * 128) + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+            for (int c = 0; c < 8; ++c) {
+                uint8_t *dst = smem + L::OFF_P + half * (128 * 128) + row * 128 + ((c ^ (row & 7)) << 4);
                 *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
             }
+            SM_TRACE(7);
             // this CTA's V half has landed; dead keys get weight 0 but 0 x (stale NaN/Inf) would poison O: clear their rows
-            ok = wait(C_VLAND + st, (uint32_t)(jj >> 1) & 1u, 12);
-            if (!ok) break;
-            {
-                const uint64_t tm = tmask[row >> 6];
-                if (!((tm >> (row & 63)) & 1ull)) {
+            ok = ok && wait(C_VLAND + st, (uint32_t)(jj >> 1) & 1u, 12);
+            SM_TRACE(8);
+            if (row < 64 && !((tmask >> row) & 1ull)) {
 #pragma unroll
-                    for (int c = 0; c < VCH; ++c) {
-                        uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + row * 128);
+                for (int c = 0; c < VCH; ++c) {
+                    uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (half * 64 + row) * 128);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
-                    }
+                    for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
                 }
             }
             fence_proxy_async_smem();
+            SM_TRACE(9);
             tc_fence_before();
-            mbar_arrive_cluster(leader_pfull);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(leader_pfull);
+            SM_TRACE(10);
         }
-        // ---- epilogue ----
+        // ---- epilogue: the two threads of a row add their sums, each stores its half of the head_dim columns ----
         if (ok) ok = wait(C_PVDONE, (uint32_t)(n_tiles - 1) & 1u, 13);
+        exch[(0 * 2 + half) * 128 + row] = l;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        l += exch[(0 * 2 + (half ^ 1)) * 128 + row];
         if (ok) {
             tc_fence_after();
             const float inv = 1.f / l;
-            __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + hq) * HD;
+            __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + hq) * HD + half * (HD / 2);
 #pragma unroll 1
-            for (int c = 0; c < HD / 32; ++c) {
+            for (int c = 0; c < HD / 64; ++c) {
                 uint32_t o[32];
-                tmem_ld32(tmem_base + lane_addr + kColO + c * 32, o);
+                tmem_ld32(tmem_base + lane_addr + kColO + half * (HD / 2) + c * 32, o);
                 tmem_wait_ld();
                 if (row_live) {
 #pragma unroll
@@ -327,9 +374,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * k]) * inv,
-                                                                     __uint_as_float(o[8 * i + 2 * k + 1]) * inv);
-                            vv[k] = *reinterpret_cast<uint32_t *>(&h);
+                            __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * k]) * inv,
+                                                                      __uint_as_float(o[8 * i + 2 * k + 1]) * inv);
+                            vv[k] = *reinterpret_cast<uint32_t *>(&hh);
                         }
                         *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = v;
                     }
