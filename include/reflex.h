@@ -142,9 +142,10 @@ int reflex_cache_append_sliding(reflex_cache_t *cache, const int32_t *stream_ids
  *   gate_buf device fp32 or NULL.
  *            cond != NULL, gate_buf == NULL: one fused launch, every block recomputes its stream's gate
  *                                            (fine for a single stream, wasteful for a batch).
- *            cond != NULL, gate_buf != NULL: gate_buf holds B*(D+Hd) floats: the gate [B][D] is written
- *                                            there, followed by [B][Hd] hidden-layer scratch; three
- *                                            launches (hidden, gate, rows), weights read once per 16 streams.
+ *            cond != NULL, gate_buf != NULL: gate_buf holds B*(D+Hd) floats (the gate [B][D] is written to
+ *                                            the first B*D; the rest is reserved scratch). Two launches:
+ *                                            the gate MLP, weights read once per 8 streams, and the row
+ *                                            kernel, which overlaps it (programmatic dependent launch).
  *            cond == NULL: gate_buf [B][D] is an input (a gate computed earlier, e.g. once per tick).
  * Requirements: D % 8 == 0, Cd % 8 == 0, Hd % 8 == 0, D <= 16384, Cd, Hd <= 4096. */
 int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, const void *b1,

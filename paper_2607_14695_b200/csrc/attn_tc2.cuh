@@ -18,7 +18,7 @@ namespace reflex {
 // Optional timeline of one CTA pair (debug builds only: -DREFLEX_TRACE): clock64 stamps per role and tile into the
 // (otherwise unused) split-K partial area. Compiled out in the product library.
 #ifdef REFLEX_TRACE
-#define TC2_TRACE(role, tile, ev) do { if (blockIdx.x < 2 && blockIdx.y == 0 && (tile) < 16) \
+#define TC2_TRACE(role, tile, ev) do { if (blockIdx.x < 2 && blockIdx.y == 0 && (tile) < 16 && (ev) < 16) \
     reinterpret_cast<long long *>(p.partials)[((blockIdx.x * 4 + (role)) * 16 + (tile)) * 16 + (ev)] = clock64(); } while (0)
 #else
 #define TC2_TRACE(role, tile, ev) do { } while (0)
@@ -75,6 +75,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         return;
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 64) TC2_TRACE(2, 15, 0);
     const uint32_t rank = cluster_ctarank();
     const int pair = (blockIdx.x >> 1) % p.n_qtiles;   // n_qtiles holds the number of tile pairs here
     const int kvh = (blockIdx.x >> 1) / p.n_qtiles;
@@ -113,6 +114,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     cluster_wait();   // both CTAs' barriers are initialised before anything crosses the pair
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 64) TC2_TRACE(2, 15, 1);
 
     auto wait_impl = [&](int i, uint32_t parity, uint32_t code, bool cluster_scope) -> bool {
         auto probe = [&]() { (void)cluster_scope; return mbar_try_wait(bar(i), parity); };
@@ -354,7 +356,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             SM_TRACE(10);
         }
         // ---- epilogue: the two threads of a row add their sums, each stores its half of the head_dim columns ----
+        if (threadIdx.x == 64) TC2_TRACE(2, 15, 2);
         if (ok) ok = wait(C_PVDONE, (uint32_t)(n_tiles - 1) & 1u, 13);
+        if (threadIdx.x == 64) TC2_TRACE(2, 15, 3);
         exch[(0 * 2 + half) * 128 + row] = l;
         asm volatile("bar.sync 1, 256;" ::: "memory");
         l += exch[(0 * 2 + (half ^ 1)) * 128 + row];
@@ -385,11 +389,13 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     }
 
+    if (threadIdx.x == 64) TC2_TRACE(2, 15, 4);
     tc_fence_before();
     __syncthreads();
     cluster_arrive();
     cluster_wait();   // neither CTA retires while its partner can still touch its shared memory or barriers
     if (warp == 1) tmem_dealloc2(tmem_base, kTmemCols);
+    if (threadIdx.x == 64) TC2_TRACE(2, 15, 5);
 }
 
 }  // namespace reflex

@@ -148,98 +148,63 @@ adarmsnorm_kernel(const T *x, T *y, const T *__restrict__ cond, const T *__restr
 }
 
 
-// ---- three-launch form (gate scratch provided): hidden -> gate -> rows. Weights are read once per
-// ---- group of 8 streams instead of once per block, and every launch spreads over the machine.
-constexpr int kGateStreams = 8;
+// ---- gate MLP with scratch (gate_buf given): two small launches, hidden then gate, each ONE round of memory
+// ---- latency: a block stages 8 weight rows and the vectors of up to 32 streams in shared memory, then every thread
+// ---- owns one (weight row, stream) dot product -- no shuffles, no dependent loads.
+constexpr int kGateStreams = 32;   // streams per block
+constexpr int kGateUnits = 8;      // weight rows (hidden units or gate columns) per block
 
-// dot products of one weight row (global, lane-strided 8-element chunks) with kGateStreams vectors staged in
-// shared memory as fp32 ([kGateStreams][len]); returns the per-stream sums reduced over the warp.
-template <typename T>
-__device__ __forceinline__ void row_dots(const T *__restrict__ w, const float *vec_s, int len, int nb, float (&acc)[kGateStreams])
-{
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int s = 0; s < kGateStreams; ++s) acc[s] = 0.f;
-    for (int e = lane * 8; e < len; e += 256) {
-        float f[8];
-        Vec8<T>::load(w + e, f);
-#pragma unroll
-        for (int s = 0; s < kGateStreams; ++s) {
-            if (s < nb) {
-                const float4 a = *reinterpret_cast<const float4 *>(vec_s + s * len + e);
-                const float4 b = *reinterpret_cast<const float4 *>(vec_s + s * len + e + 4);
-                acc[s] = fmaf(f[0], a.x, acc[s]); acc[s] = fmaf(f[1], a.y, acc[s]); acc[s] = fmaf(f[2], a.z, acc[s]); acc[s] = fmaf(f[3], a.w, acc[s]);
-                acc[s] = fmaf(f[4], b.x, acc[s]); acc[s] = fmaf(f[5], b.y, acc[s]); acc[s] = fmaf(f[6], b.z, acc[s]); acc[s] = fmaf(f[7], b.w, acc[s]);
-            }
-        }
-    }
-#pragma unroll
-    for (int s = 0; s < kGateStreams; ++s) acc[s] = warp_sum(acc[s]);
-}
-
-// grid = (ceil(Hd/8), ceil(B/8)); one warp per hidden unit for 8 streams.
-template <typename T>
+// out[s][u0+u] = act(bias[u0+u] + W[u0+u][:] . vec[b0+s][:]);  SILU: hidden layer, else 1 + (.) for the gate.
+// vec is T (conditioning) or float (hidden activations). grid = (ceil(units/8), ceil(B/32)), 256 threads.
+template <typename T, typename VT, bool SILU>
 __global__ void __launch_bounds__(256)
-gate_hidden_kernel(const T *__restrict__ cond, const T *__restrict__ W1, const T *__restrict__ b1, float *__restrict__ hid_out,
-                   int B, int Cd, int Hd)
+gate_layer_kernel(const VT *vec, const T *__restrict__ W, const T *__restrict__ bias, float *out, int B, int len, int units,
+                  int wait_prior)
 {
-    extern __shared__ __align__(16) float c_s[];  // [kGateStreams][Cd]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    extern __shared__ __align__(16) float sm_gl[];
+    const int pitch = len + 4;                   // +4 floats: the 32 stream rows start in different banks
+    float *w_s = sm_gl;                          // [8][len]
+    float *v_s = sm_gl + kGateUnits * len;       // [32][pitch]
     const int b0 = blockIdx.y * kGateStreams;
     const int nb = min(kGateStreams, B - b0);
-    for (int i = threadIdx.x * 8; i < nb * Cd; i += blockDim.x * 8) {
+    const int u0 = blockIdx.x * kGateUnits;
+    const int nu = min(kGateUnits, units - u0);
+    // weight rows do not depend on the preceding launch: fetch them first, then wait for it (programmatic dependent launch)
+    for (int i = threadIdx.x * 8; i < nu * len; i += blockDim.x * 8) {
         float f[8];
-        Vec8<T>::load(cond + (size_t)b0 * Cd + i, f);
-        *reinterpret_cast<float4 *>(c_s + i) = make_float4(f[0], f[1], f[2], f[3]);
-        *reinterpret_cast<float4 *>(c_s + i + 4) = make_float4(f[4], f[5], f[6], f[7]);
+        Vec8<T>::load(W + (size_t)u0 * len + i, f);
+        *reinterpret_cast<float4 *>(w_s + i) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4 *>(w_s + i + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+    if (wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int chunks = len / 8;
+    for (int i = threadIdx.x; i < nb * chunks; i += blockDim.x) {
+        const int s = i / chunks, e = (i % chunks) * 8;
+        float f[8];
+        Vec8<VT>::load(vec + (size_t)(b0 + s) * len + e, f);
+        *reinterpret_cast<float4 *>(v_s + s * pitch + e) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4 *>(v_s + s * pitch + e + 4) = make_float4(f[4], f[5], f[6], f[7]);
     }
     __syncthreads();
-    const int j = blockIdx.x * 8 + warp;
-    if (j >= Hd) return;
-    float acc[kGateStreams];
-    row_dots<T>(W1 + (size_t)j * Cd, c_s, Cd, nb, acc);
-    const float bias = to_f<T>(b1[j]);
-    if (lane == 0) {
-#pragma unroll
-        for (int s = 0; s < kGateStreams; ++s) {
-            if (s < nb) {
-                const float z = acc[s] + bias;
-                hid_out[(size_t)(b0 + s) * Hd + j] = z / (1.f + expf(-z));
-            }
-        }
+    const int u = threadIdx.x >> 5, sidx = threadIdx.x & 31;
+    if (u >= nu || sidx >= nb) return;
+    const float *wr = w_s + u * len, *vr = v_s + sidx * pitch;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int e = 0; e < len; e += 4) {
+        const float4 wv = *reinterpret_cast<const float4 *>(wr + e);
+        const float4 vv = *reinterpret_cast<const float4 *>(vr + e);
+        a0 = fmaf(wv.x, vv.x, a0); a1 = fmaf(wv.y, vv.y, a1); a2 = fmaf(wv.z, vv.z, a2); a3 = fmaf(wv.w, vv.w, a3);
     }
-}
-
-// grid = (ceil(D/8), ceil(B/8)); one warp per gate column for 8 streams.
-template <typename T>
-__global__ void __launch_bounds__(256)
-gate_out_kernel(const float *__restrict__ hid, const T *__restrict__ W2, const T *__restrict__ b2, float *__restrict__ gate_buf,
-                int B, int D, int Hd)
-{
-    extern __shared__ __align__(16) float h_s[];  // [kGateStreams][Hd]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int b0 = blockIdx.y * kGateStreams;
-    const int nb = min(kGateStreams, B - b0);
-    for (int i = threadIdx.x * 4; i < nb * Hd; i += blockDim.x * 4)
-        *reinterpret_cast<float4 *>(h_s + i) = *reinterpret_cast<const float4 *>(hid + (size_t)b0 * Hd + i);
-    __syncthreads();
-    const int col = blockIdx.x * 8 + warp;
-    if (col >= D) return;
-    float acc[kGateStreams];
-    row_dots<T>(W2 + (size_t)col * Hd, h_s, Hd, nb, acc);
-    const float bias = to_f<T>(b2[col]);
-    if (lane == 0) {
-#pragma unroll
-        for (int s = 0; s < kGateStreams; ++s)
-            if (s < nb) gate_buf[(size_t)(b0 + s) * D + col] = 1.f + (acc[s] + bias);
-    }
+    const float z = ((a0 + a1) + (a2 + a3)) + to_f<T>(bias[u0 + u]);
+    out[(size_t)(b0 + sidx) * units + u0 + u] = SILU ? z / (1.f + expf(-z)) : 1.f + z;
 }
 
 // One warp per row, the row kept in registers between the statistics pass and the scaling pass
 // (D <= 256 * NCH), so x is read from memory exactly once. grid = ceil(B*R / 8).
 template <typename T, int NCH>
 __global__ void __launch_bounds__(256)
-adarmsnorm_rows_kernel(const T *x, T *y, const float *__restrict__ gate_buf, int rows, int R, int D, float eps)
+adarmsnorm_rows_kernel(const T *x, T *y, const float *gate_buf, int rows, int R, int D, float eps)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int row = blockIdx.x * 8 + warp;
@@ -261,12 +226,15 @@ adarmsnorm_rows_kernel(const T *x, T *y, const float *__restrict__ gate_buf, int
     }
     ss = warp_sum(ss);
     const float rinv = 1.f / sqrtf(ss / (float)D + eps);
+    // the gate may still be in the making by the preceding launch (programmatic dependent launch): x is already in
+    // registers and the statistics are done, now wait for that grid to finish and its writes to be visible
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
         const int e = c * 256 + lane * 8;
         if (e < D) {
-            const float4 g0 = __ldg(reinterpret_cast<const float4 *>(g + e));
-            const float4 g1 = __ldg(reinterpret_cast<const float4 *>(g + e + 4));
+            const float4 g0 = *reinterpret_cast<const float4 *>(g + e);
+            const float4 g1 = *reinterpret_cast<const float4 *>(g + e + 4);
             float o[8];
             o[0] = f[c][0] * rinv * g0.x; o[1] = f[c][1] * rinv * g0.y; o[2] = f[c][2] * rinv * g0.z; o[3] = f[c][3] * rinv * g0.w;
             o[4] = f[c][4] * rinv * g1.x; o[5] = f[c][5] * rinv * g1.y; o[6] = f[c][6] * rinv * g1.z; o[7] = f[c][7] * rinv * g1.w;
@@ -276,34 +244,64 @@ adarmsnorm_rows_kernel(const T *x, T *y, const float *__restrict__ gate_buf, int
 }
 
 template <typename T>
-static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B, int R, int D, float eps, cudaStream_t st)
+static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B, int R, int D, float eps, bool after_gate, cudaStream_t st)
 {
     const int rows = B * R;
-    const int grid = (rows + 7) / 8;
-    if (D <= 512) adarmsnorm_rows_kernel<T, 2><<<grid, 256, 0, st>>>(x, y, gate_buf, rows, R, D, eps);
-    else if (D <= 1024) adarmsnorm_rows_kernel<T, 4><<<grid, 256, 0, st>>>(x, y, gate_buf, rows, R, D, eps);
-    else if (D <= 2048) adarmsnorm_rows_kernel<T, 8><<<grid, 256, 0, st>>>(x, y, gate_buf, rows, R, D, eps);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((rows + 7) / 8);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_gate ? 1 : 0;   // overlap with the gate kernel launched just before on the same stream
+    cudaError_t e;
+    if (D <= 512) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 2>, x, y, gate_buf, rows, R, D, eps);
+    else if (D <= 1024) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 4>, x, y, gate_buf, rows, R, D, eps);
+    else if (D <= 2048) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 8>, x, y, gate_buf, rows, R, D, eps);
     else return cudaErrorNotSupported;
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 template <typename T>
 static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, const T *b1, const T *W2, const T *b2,
                                  float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, cudaStream_t st)
 {
-    if (cond && gate_buf && Cd <= 1536 && Hd <= 1536) {
-        // gate_buf = [B][D] gate followed by [B][Hd] hidden-layer scratch
+    bool after_gate = false;
+    const size_t smem_h = (size_t)(kGateUnits * Cd + kGateStreams * (Cd + 4)) * 4;
+    const size_t smem_g = (size_t)(kGateUnits * Hd + kGateStreams * (Hd + 4)) * 4;
+    if (cond && gate_buf && smem_h <= 160 * 1024 && smem_g <= 160 * 1024) {
+        // gate_buf = [B][D] gate followed by [B][Hd] hidden activations
         float *hid = gate_buf + (size_t)B * D;
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(gate_layer_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(gate_layer_kernel<T, float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+            if (e != cudaSuccess) return e;
+            attr_set = true;
+        }
         const int groups = (B + kGateStreams - 1) / kGateStreams;
-        gate_hidden_kernel<T><<<dim3((Hd + 7) / 8, groups), 256, (size_t)kGateStreams * Cd * 4, st>>>(cond, W1, b1, hid, B, Cd, Hd);
+        gate_layer_kernel<T, T, true><<<dim3((Hd + kGateUnits - 1) / kGateUnits, groups), 256, smem_h, st>>>(cond, W1, b1, hid, B, Cd, Hd, 0);
         count_launch();
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
-        gate_out_kernel<T><<<dim3((D + 7) / 8, groups), 256, (size_t)kGateStreams * Hd * 4, st>>>(hid, W2, b2, gate_buf, B, D, Hd);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((D + kGateUnits - 1) / kGateUnits, groups);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = smem_g;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, gate_layer_kernel<T, float, false>, (const float *)hid, W2, b2, gate_buf, B, Hd, D, 1);
         count_launch();
-        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
+        after_gate = true;
     } else if (cond && gate_buf) {
         // very wide conditioning / hidden layers: per-block gate (shared-memory staging of 16 streams would not fit)
         const int cols = 64;
@@ -312,7 +310,7 @@ static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, c
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    if (gate_buf && D <= 2048) return launch_rows_t<T>(x, y, gate_buf, B, R, D, eps, st);
+    if (gate_buf && D <= 2048) return launch_rows_t<T>(x, y, gate_buf, B, R, D, eps, after_gate, st);
     // enough blocks to cover the SMs about twice, at least one row per warp
     int chunks = (296 + B - 1) / B;
     const int max_chunks = (R + 7) / 8;
