@@ -507,7 +507,7 @@ cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtenso
 
 template <int HD>
 cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
-                      const CUtensorMap *mvd, const TcParams &tp, dim3 grid, cudaStream_t st)
+                      const CUtensorMap *mvd, const CUtensorMap *mo, const TcParams &tp, dim3 grid, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -515,7 +515,7 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attn_tc2_kernel<HD><<<grid, kTc2Threads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
+    attn_tc2_kernel<HD><<<grid, kTc2Threads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, *mo, tp);
     count_launch();
     return cudaGetLastError();
 }
@@ -551,7 +551,7 @@ int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
 
 bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 || p.d == 256); }
 
-cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, cudaStream_t st)
+cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st)
 {
     const int G = p.Hq / p.Hkv;
     const int rows_slab = p.L * p.B * (p.S_max + p.N);
@@ -569,11 +569,18 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     tp.n_qtiles = (p.T + tp.tile_tokens - 1) / tp.tile_tokens;
     cudaError_t e;
     if (two_cta) {
-        // pairs of query tiles; an odd tile count leaves the last pair with one idle half
+        // persistent grid: one cluster (two CTAs) per SM pair walks the (stream, KV head, tile pair) units;
+        // an odd tile count leaves the last pair of a stream with one idle half
+        CUtensorMap mo;
+        if (!cache().get(&mo, p.out, 1, (p.B << 16) | p.T, p.Hq, p.d, G, mk_q)) return cudaErrorInvalidValue;
         tp.n_qtiles = (tp.n_qtiles + 1) / 2;
-        dim3 grid2(2 * tp.n_qtiles * p.Hkv, p.B, 1);
-        if (p.d == 256) return launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
-        if (p.d == 128) return launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
+        const int units = tp.n_qtiles * p.Hkv * p.B;
+        int clusters = sm_count / 2;
+        if (clusters > units) clusters = units;
+        if (clusters < 1) clusters = 1;
+        dim3 grid2(2 * clusters, 1, 1);
+        if (p.d == 256) return launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
+        if (p.d == 128) return launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
         return cudaErrorInvalidValue;
     }
     dim3 grid(tp.n_qtiles * p.Hkv, p.B, p.nsplit);

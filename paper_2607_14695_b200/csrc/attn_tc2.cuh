@@ -1,30 +1,37 @@
-// Partitioned attention (Eq. 1), two-CTA form: a cluster of two CTAs (two SMs) drives one
-// tcgen05.mma.cta_group::2 with M = 256 -- two 128-row query tiles of the same (stream, KV head). The B
-// operand of such an MMA is split between the two CTAs' shared memories, so each CTA stages only HALF of
-// every K tile (64 of its 128 keys) and HALF of every V tile (128 of the head_dim columns): the bytes each
-// SM pulls per key are halved against the one-CTA kernel, which is what lets the loads keep up with the
-// tensor pipe at head_dim 256. Included by attn_tc.cu (shares its tile geometry and tensor maps).
+// Partitioned attention (Eq. 1), two-CTA persistent form, for batched serving.
 //
-// Per CTA:  warp 0  TMA producer (own Q tile, own K half, own V half)
-//           warp 1  MMA issuer (leader CTA only): S = Q K^T (M256 N128), O += P V (M256 N=d)
-//           warps 2..9  softmax over this CTA's 128 rows x 128 keys (two threads per row, 64 keys each),
-//                       P into swizzled shared memory, lazy rescale of O in TMEM, epilogue
+// A cluster of two CTAs (two SMs) drives tcgen05.mma.cta_group::2 with M = 256: two 128-row query tiles of
+// the same (stream, KV head). The B operand of such an MMA is split between the two CTAs' shared memories,
+// so each CTA stages only HALF of every K tile (64 of its 128 keys) and HALF of every V tile (128 of the
+// head_dim columns): the bytes each SM pulls per key are halved against the one-CTA kernel, which is what
+// lets the loads keep up with the tensor pipe at head_dim 256.
+//
+// The grid is persistent: one cluster per SM pair walks a list of work units (stream, KV head, tile pair).
+// Barrier, TMEM and cluster set-up is paid once, and the tail of a unit (last P V, normalisation, store of O)
+// overlaps the head of the next one (its Q / K / V loads and first Q K^T).
+//
+// Per CTA:  warp 0      TMA producer (own Q tile, own K half, own V half)
+//           warp 1      MMA issuer (leader CTA only): S = Q K^T (M256 N128), O += P V (M256 N=d)
+//           warps 2..9  softmax over this CTA's 128 rows x 128 keys: two threads per row (64 keys each),
+//                       P (bf16) into swizzled shared memory, lazy rescale of O in TMEM, and the epilogue:
+//                       O / l staged through shared memory and written with TMA stores
 // Barriers the leader's MMA thread waits on collect both CTAs (TMA completions through cta_group::2 loads,
 // softmax arrivals through shared::cluster arrives); completions fan out with multicast commits.
+// Included by attn_tc.cu (shares its tile geometry and tensor maps).
 #pragma once
 
 namespace reflex {
 
-// Optional timeline of one CTA pair (debug builds only: -DREFLEX_TRACE): clock64 stamps per role and tile into the
-// (otherwise unused) split-K partial area. Compiled out in the product library.
+// Optional timeline of the first cluster (debug builds only: -DREFLEX_TRACE): clock64 stamps into the (otherwise
+// unused) split-K partial area. Compiled out of the product library.
 #ifdef REFLEX_TRACE
-#define TC2_TRACE(role, tile, ev) do { if (blockIdx.x < 2 && blockIdx.y == 0 && (tile) < 16 && (ev) < 16) \
-    reinterpret_cast<long long *>(p.partials)[((blockIdx.x * 4 + (role)) * 16 + (tile)) * 16 + (ev)] = clock64(); } while (0)
+#define TC2_TRACE(role, slot, ev) do { if (blockIdx.x < 2 && (slot) < 16 && (ev) < 16) \
+    reinterpret_cast<long long *>(p.partials)[((blockIdx.x * 4 + (role)) * 16 + (slot)) * 16 + (ev)] = clock64(); } while (0)
 #else
-#define TC2_TRACE(role, tile, ev) do { } while (0)
+#define TC2_TRACE(role, slot, ev) do { } while (0)
 #endif
 
-constexpr int kTc2Keys = 128;  // keys per tile = two 64-key halves, one per CTA of the pair
+constexpr int kTc2Keys = 128;     // keys per tile = two 64-key halves, one per CTA of the pair
 constexpr int kTc2Threads = 320;  // producer warp, MMA warp, eight softmax warps
 
 template <int HD> struct Tc2Smem {
@@ -34,30 +41,39 @@ template <int HD> struct Tc2Smem {
     static constexpr uint32_t K_STAGE = CH * 64 * 128;          // 64 keys x head_dim
     static constexpr uint32_t V_STAGE = VCH * 128 * 128;        // 128 keys x head_dim/2
     static constexpr uint32_t V_HALF = VCH * 64 * 128;          // bytes one 64-key half contributes
-    static constexpr uint32_t P_BYTES = 2 * 128 * 128;          // 128 rows x 128 keys bf16
+    static constexpr uint32_t P_BYTES = 2 * 128 * 128;          // 128 rows x 128 keys bf16; also the staging area of the epilogue
     static constexpr uint32_t OFF_Q = 0;
     static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
     static constexpr uint32_t OFF_V = OFF_K + 2 * K_STAGE;
     static constexpr uint32_t OFF_P = OFF_V + 2 * V_STAGE;
     static constexpr uint32_t OFF_BAR = OFF_P + P_BYTES;
-    static constexpr uint32_t OFF_XCH = OFF_BAR + 128;              // row-maximum exchange between the two halves
+    static constexpr uint32_t OFF_XCH = OFF_BAR + 192;              // row max / row sum exchange between the two halves
     static constexpr uint32_t NEED = OFF_XCH + 2 * 2 * 128 * 4;     // bytes used from the 1024-byte aligned base
     static constexpr uint32_t TOTAL = 232448;                       // the whole opt-in shared memory of an SM (227 KB)
 };
 
-enum { C_QFULL = 0, C_KFULL = 1, C_KEMPTY = 3, C_VLAND = 5, C_VEMPTY = 7, C_SFULL = 9, C_SEMPTY = 11, C_PFULL = 13, C_PVDONE = 14, C_COUNT = 15 };
+enum { C_QFULL = 0, C_QEMPTY = 1, C_KFULL = 2, C_KEMPTY = 4, C_VLAND = 6, C_VEMPTY = 8, C_SFULL = 10, C_SEMPTY = 12,
+       C_PFULL = 14, C_PVDONE = 15, C_OFREE = 16, C_COUNT = 17 };
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
 
 template <int HD>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTc2Threads, 1)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
-                const __grid_constant__ CUtensorMap tm_vd, const TcParams p)
+                const __grid_constant__ CUtensorMap tm_vd, const __grid_constant__ CUtensorMap tm_o, const TcParams p)
 {
     using L = Tc2Smem<HD>;
     constexpr int CH = L::CH, VCH = L::VCH;
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColO = 0, kColS = HD;  // O: HD fp32 columns; S: 2 x 128 columns
     static_assert(HD + 2 * kTc2Keys <= 512 && VCH >= 1, "TMEM budget / head_dim split");
+    static_assert(8 * C_COUNT + 8 <= 192, "barrier area");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -77,14 +93,20 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 64) TC2_TRACE(2, 15, 0);
     const uint32_t rank = cluster_ctarank();
-    const int pair = (blockIdx.x >> 1) % p.n_qtiles;   // n_qtiles holds the number of tile pairs here
-    const int kvh = (blockIdx.x >> 1) / p.n_qtiles;
-    const int b = blockIdx.y;
-    const int t0 = (2 * pair + (int)rank) * p.tile_tokens;
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    const int n_pairs = p.n_qtiles;                    // tile pairs per (stream, KV head)
+    const int n_units = p.B * p.Hkv * n_pairs;
 
-    TileGeom g;
-    {
-        const StreamState st = p.state[b];
+    // geometry of one work unit
+    struct Unit { int b, kvh, t0, H, n_tiles; TileGeom g; };
+    auto load_unit = [&](int u) -> Unit {
+        Unit w;
+        const int pair = u % n_pairs;
+        w.kvh = (u / n_pairs) % p.Hkv;
+        w.b = u / (n_pairs * p.Hkv);
+        w.t0 = (2 * pair + (int)rank) * p.tile_tokens;
+        const StreamState st = p.state[w.b];
+        TileGeom &g = w.g;
         g.S = st.static_len > 0 ? st.static_len : 0;
         g.N = p.N; g.T = p.T; g.count = st.count;
         g.oldest = (st.head - st.count) % p.N;
@@ -92,20 +114,21 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         g.ns = (g.S + kBN - 1) / kBN;
         g.nr = g.count > 0 ? (p.N + kBN - 1) / kBN : 0;
         g.nd = (p.T + kBN - 1) / kBN;
-        g.row_base = (p.layer * p.B + b) * (p.S_max + p.N);
-        g.S_max = p.S_max; g.b = b;
-    }
-    const int H = g.ns + g.nr + g.nd;       // 64-key halves
-    const int n_tiles = (H + 1) / 2;        // >= 1: there is always a dynamic half
+        g.row_base = (p.layer * p.B + w.b) * (p.S_max + p.N);
+        g.S_max = p.S_max; g.b = w.b;
+        w.H = g.ns + g.nr + g.nd;          // 64-key halves
+        w.n_tiles = (w.H + 1) / 2;         // >= 1: there is always a dynamic half
+        return w;
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C_COUNT; ++i) {
-            const bool both = (i == C_SEMPTY || i == C_SEMPTY + 1 || i == C_PFULL);
-            mbar_init(bar(i), both ? 16u : 1u);   // one arrival per softmax warp of either CTA
+            const bool both = (i == C_SEMPTY || i == C_SEMPTY + 1 || i == C_PFULL || i == C_OFREE);
+            mbar_init(bar(i), both ? 16u : 1u);   // "both": one arrival per softmax warp of either CTA
         }
         *abort_flag = 0u;
         fence_mbar_init();
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd);
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd); prefetch_tmap(&tm_o);
     }
     if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), kTmemCols);
     tc_fence_before();
@@ -116,12 +139,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 64) TC2_TRACE(2, 15, 1);
 
-    auto wait_impl = [&](int i, uint32_t parity, uint32_t code, bool cluster_scope) -> bool {
-        auto probe = [&]() { (void)cluster_scope; return mbar_try_wait(bar(i), parity); };
-        if (probe()) return true;
+    auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool {
+        if (mbar_try_wait(bar(i), parity)) return true;
         const unsigned long long t_start = globaltimer_ns();
         for (uint32_t n = 1;; ++n) {
-            if (probe()) return true;
+            if (mbar_try_wait(bar(i), parity)) return true;
             if ((n & 255u) == 0u) {
                 if (*abort_flag) return false;
                 if (globaltimer_ns() - t_start > kWaitNs) break;
@@ -131,44 +153,49 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         atomicCAS(p.status, 0u, 0x80000000u | ((code + 32u) << 16) | (blockIdx.x & 0xFFFFu));
         return false;
     };
-    auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool { return wait_impl(i, parity, code, false); };
-    auto wait_cl = [&](int i, uint32_t parity, uint32_t code) -> bool { return wait_impl(i, parity, code, true); };
 
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
-            if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
-            for (int c = 0; c < CH; ++c)
-                tma2_load_4d(base + L::OFF_Q + c * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, c * 64, kvh * p.G, t0, b);
             bool ok = true;
-            for (int jj = 0; jj < n_tiles && ok; ++jj) {
-                const int st = jj & 1;
-                const uint32_t ph = (uint32_t)((jj >> 1) - 1) & 1u;
-                const int h0 = 2 * jj, h1 = 2 * jj + 1;
-                const int live = (h0 < H ? 1 : 0) + (h1 < H ? 1 : 0);
-                TC2_TRACE(0, jj, 0);
-                if (jj >= 2) ok = wait(C_KEMPTY + st, ph, 1);
-                if (!ok) break;
-                TC2_TRACE(0, jj, 1);
-                if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
-                const int myh = 2 * jj + (int)rank;
-                if (myh < H) {
-                    const TileRef tr = g.decode(myh);
-                    for (int c = 0; c < CH; ++c)
-                        tma2_load_3d(base + L::OFF_K + st * L::K_STAGE + c * (64 * 128), tr.dyn ? &tm_kd : &tm_k,
-                                     bar(C_KFULL + st) & kPeerBitMask, c * 64, kvh, tr.row0);
+            int gt = 0, ui = 0;
+            for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
+                const Unit w = load_unit(u);
+                for (int jj = 0; jj < w.n_tiles && ok; ++jj) {
+                    const int gi = gt + jj, st = gi & 1;
+                    const uint32_t ph = (uint32_t)((gi >> 1) - 1) & 1u;
+                    const int h0 = 2 * jj, h1 = 2 * jj + 1;
+                    const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
+                    if (gi >= 2) ok = wait(C_KEMPTY + st, ph, 1);
+                    if (!ok) break;
+                    if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
+                    const int myh = 2 * jj + (int)rank;
+                    if (myh < w.H) {
+                        const TileRef tr = w.g.decode(myh);
+                        for (int c = 0; c < CH; ++c)
+                            tma2_load_3d(base + L::OFF_K + st * L::K_STAGE + c * (64 * 128), tr.dyn ? &tm_kd : &tm_k,
+                                         bar(C_KFULL + st) & kPeerBitMask, c * 64, w.kvh, tr.row0);
+                    }
+                    if (jj == 0) {
+                        // this unit's Q tile, once the last Q K^T of the previous unit has drained the buffer
+                        if (ui >= 1) ok = wait(C_QEMPTY, (uint32_t)(ui - 1) & 1u, 14);
+                        if (!ok) break;
+                        if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
+                        for (int c = 0; c < CH; ++c)
+                            tma2_load_4d(base + L::OFF_Q + c * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, c * 64, w.kvh * p.G, w.t0, w.b);
+                    }
+                    if (gi >= 2) ok = wait(C_VEMPTY + st, ph, 2);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
+                    for (int hh = h0; hh <= h1; ++hh) {
+                        if (hh >= w.H) break;
+                        const TileRef tr = w.g.decode(hh);
+                        for (int c = 0; c < VCH; ++c)
+                            tma_load_3d(base + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (hh & 1) * (64 * 128), tr.dyn ? &tm_vd : &tm_v,
+                                        bar(C_VLAND + st), ((int)rank * VCH + c) * 64, w.kvh, tr.row0);
+                    }
                 }
-                if (jj >= 2) ok = wait(C_VEMPTY + st, ph, 2);
-                if (!ok) break;
-                TC2_TRACE(0, jj, 2);
-                mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
-                for (int hh = h0; hh <= h1; ++hh) {
-                    if (hh >= H) break;
-                    const TileRef tr = g.decode(hh);
-                    for (int c = 0; c < VCH; ++c)
-                        tma_load_3d(base + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (hh & 1) * (64 * 128), tr.dyn ? &tm_vd : &tm_v,
-                                    bar(C_VLAND + st), ((int)rank * VCH + c) * 64, kvh, tr.row0);
-                }
+                gt += w.n_tiles;
             }
         }
     } else if (warp == 1) {
@@ -176,8 +203,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(256, kTc2Keys, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(256, HD, true);
-            auto issue_qk = [&](int jj) {
-                const int st = jj & 1, buf = jj & 1;
+            auto issue_qk = [&](int gi, bool last_of_unit) {
+                const int st = gi & 1, buf = gi & 1;
                 const uint32_t d_tmem = tmem_base + kColS + buf * kTc2Keys;
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
@@ -187,209 +214,239 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 umma2_commit_mc(bar(C_KEMPTY + st), 3);
                 umma2_commit_mc(bar(C_SFULL + buf), 3);
+                if (last_of_unit) umma2_commit_mc(bar(C_QEMPTY), 3);   // Q has been read for the last time
             };
-            bool ok = wait_cl(C_QFULL, 0, 3) && wait_cl(C_KFULL + 0, 0, 4);
-            if (ok) { tc_fence_after(); issue_qk(0); }
-            for (int jj = 0; jj < n_tiles && ok; ++jj) {
-                if (jj + 1 < n_tiles) {
-                    const int nj = jj + 1;
-                    TC2_TRACE(1, nj, 0);
-                    ok = wait_cl(C_KFULL + (nj & 1), (uint32_t)(nj >> 1) & 1u, 5);
-                    TC2_TRACE(1, nj, 1);
-                    if (ok && nj >= 2) ok = wait_cl(C_SEMPTY + (nj & 1), (uint32_t)((nj >> 1) - 1) & 1u, 6);
-                    if (!ok) break;
-                    TC2_TRACE(1, nj, 2);
-                    tc_fence_after();
-                    issue_qk(nj);
-                    TC2_TRACE(1, nj, 3);
-                }
-                const int st = jj & 1;
-                TC2_TRACE(1, jj, 4);
-                ok = wait_cl(C_PFULL, (uint32_t)jj & 1u, 8);   // both CTAs: P written, V landed and cleaned
-                if (!ok) break;
-                TC2_TRACE(1, jj, 5);
+            // wait for the K tile and the S buffer of global tile gi, then issue its Q K^T
+            auto qk_when_ready = [&](int gi, bool last_of_unit) -> bool {
+                bool ok2 = wait(C_KFULL + (gi & 1), (uint32_t)(gi >> 1) & 1u, 5);
+                if (ok2 && gi >= 2) ok2 = wait(C_SEMPTY + (gi & 1), (uint32_t)((gi >> 1) - 1) & 1u, 6);
+                if (!ok2) return false;
                 tc_fence_after();
+                issue_qk(gi, last_of_unit);
+                return true;
+            };
+            bool ok = true;
+            int gt = 0, ui = 0;
+            for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
+                const Unit w = load_unit(u);
+                ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk_when_ready(gt, w.n_tiles == 1);
+                for (int jj = 0; jj < w.n_tiles && ok; ++jj) {
+                    const int gi = gt + jj;
+                    if (jj + 1 < w.n_tiles) {
+                        ok = qk_when_ready(gi + 1, jj + 2 == w.n_tiles);
+                        if (!ok) break;
+                    }
+                    const int st = gi & 1;
+                    ok = wait(C_PFULL, (uint32_t)gi & 1u, 8);   // both CTAs: P written, V landed and cleaned
+                    if (ok && jj == 0 && ui >= 1) ok = wait(C_OFREE, (uint32_t)(ui - 1) & 1u, 15);   // previous O has been read out
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
-                    const uint32_t a = base + L::OFF_P + (kk >> 2) * (128 * 128) + (kk & 3) * 32;
-                    const uint32_t bb = base + L::OFF_V + st * L::V_STAGE + kk * (16 * 128);
-                    umma2_ss(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv,
-                             (jj > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
+                        const uint32_t a = base + L::OFF_P + (kk >> 2) * (128 * 128) + (kk & 3) * 32;
+                        const uint32_t bb = base + L::OFF_V + st * L::V_STAGE + kk * (16 * 128);
+                        umma2_ss(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv,
+                                 (jj > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma2_commit_mc(bar(C_VEMPTY + st), 3);
+                    umma2_commit_mc(bar(C_PVDONE), 3);
                 }
-                umma2_commit_mc(bar(C_VEMPTY + st), 3);
-                umma2_commit_mc(bar(C_PVDONE), 3);
-                TC2_TRACE(1, jj, 6);
+                gt += w.n_tiles;
             }
         }
     } else {
         // ---------------- softmax / correction / epilogue (both CTAs) ----------------
         // Eight warps: two threads per query row, one per 64-key half of the tile (warps 2..5 take the pair
         // leader's keys, warps 6..9 the partner's). The halves meet once per tile to agree on the row maximum.
+        // A wait that ran out never leaves these loops: every softmax warp keeps meeting the others at the named
+        // barrier (the remaining waits return at once), so no warp is left behind.
         const int sw = warp - 2;
         const int half = sw >> 2;                 // which 64 columns of S / 64-key chunk of P / half of O's columns
         const int quarter = warp & 3;             // TMEM lane quarter this warp may touch
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        const int t_row = t0 + row / p.G;
-        const int hq = kvh * p.G + row % p.G;
-        const bool row_live = t_row < p.T;
         const uint32_t leader_pfull = mapa(bar(C_PFULL), 0);
+        const uint32_t leader_ofree = mapa(bar(C_OFREE), 0);
         float *exch = reinterpret_cast<float *>(smem + L::OFF_XCH);   // [2 buffers][2 halves][128 rows]
-        float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        // A wait that ran out does not leave this loop: every softmax warp keeps meeting the others at the named
-        // barrier (the remaining waits return at once), so no warp is left behind.
-        for (int jj = 0; jj < n_tiles; ++jj) {
-            const int buf = jj & 1, st = jj & 1;
-            const int h = 2 * jj + half;
-            uint64_t tmask = 0ull, rmask = 0ull;
-            if (h < H) {
-                const TileRef tr = g.decode(h);
-                tmask = g.tile_mask(tr);
-                rmask = tmask;
-                if (tr.kind == 2 && p.dyn_mask) {
-                    const int lim = t_row - tr.idx * kBN;
-                    rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
-                }
-            }
-#define SM_TRACE(ev) do { if (lane == 0 && quarter == 2) TC2_TRACE(2 + half, jj, ev); } while (0)
-            SM_TRACE(0);
-            ok = ok && wait(C_SFULL + buf, (uint32_t)(jj >> 1) & 1u, 9);
-            SM_TRACE(1);
-            tc_fence_after();
-            float s[64];
-            {
-                const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + half * 64;
-                uint32_t r0[32], r1[32];
-                tmem_ld32(s_addr, r0); tmem_ld32(s_addr + 32, r1);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
-            }
-            SM_TRACE(2);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
-            if (rmask != ~0ull) {
-#pragma unroll
-                for (int c = 0; c < 64; ++c) if (!((rmask >> c) & 1ull)) s[c] = -INFINITY;
-            }
-            float mx4[4] = {s[0], s[1], s[2], s[3]};
-#pragma unroll
-            for (int c = 4; c < 64; c += 4) {
-                mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
-                mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
-            }
-            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            // meet the thread that holds the other 64 keys of this row
-            SM_TRACE(3);
-            exch[(buf * 2 + half) * 128 + row] = mx;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            SM_TRACE(4);
-            mx = fmaxf(mx, exch[(buf * 2 + (half ^ 1)) * 128 + row]);
-            bool pv_waited = false;
-            if (jj == 0) {
-                m_ref = mx;
-            } else {
-                const bool grow = (mx - m_ref) * p.scale_log2 > kRescaleThreshold;
-                if (__any_sync(0xffffffffu, grow)) {
-                    // O (and l) were accumulated against m_ref: bring them to the new reference before this tile's P V.
-                    // Both threads of a row see the same mx, so they decide alike; each rescales its half of O's columns.
-                    const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
-                    if (grow) m_ref = mx;
-                    l *= alpha;
-                    ok = ok && wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 10);
-                    pv_waited = true;
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int c = 0; c < HD / 64; ++c) {
-                        uint32_t o[32];
-                        const uint32_t o_addr = tmem_base + lane_addr + kColO + half * (HD / 2) + c * 32;
-                        tmem_ld32(o_addr, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(o_addr, o);
+        int gt = 0;
+        [[maybe_unused]] int ui_s = 0;
+        for (int u = cluster_id; u < n_units; u += n_clusters, ++ui_s) {
+            const Unit w = load_unit(u);
+            const int t_row = w.t0 + row / p.G;
+            if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 0);
+            float m_ref = -INFINITY, l = 0.f;
+            for (int jj = 0; jj < w.n_tiles; ++jj) {
+                const int gi = gt + jj, buf = gi & 1, st = gi & 1;
+                const int h = 2 * jj + half;
+                uint64_t tmask = 0ull, rmask = 0ull;
+                if (h < w.H) {
+                    const TileRef tr = w.g.decode(h);
+                    tmask = w.g.tile_mask(tr);
+                    rmask = tmask;
+                    if (tr.kind == 2 && p.dyn_mask) {
+                        const int lim = t_row - tr.idx * kBN;
+                        rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
                     }
-                    tmem_wait_st();
                 }
-            }
-            const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t packed[32];
+                ok = ok && wait(C_SFULL + buf, (uint32_t)(gi >> 1) & 1u, 9);
+                if (threadIdx.x == 64 && jj == 0) TC2_TRACE(2, ui_s, 1);
+                tc_fence_after();
+                float s[64];
+                {
+                    const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + half * 64;
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32(s_addr, r0); tmem_ld32(s_addr + 32, r1);
+                    tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-                const float p0 = ex2(fmaf(s[c], p.scale_log2, -mr));
-                const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, -mr));
-                sum4[(c >> 1) & 3] += p0 + p1;
-                __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
-                packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
-            }
-            l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-            SM_TRACE(5);
-            if (jj >= 1 && !pv_waited) {
-                ok = ok && wait(C_PVDONE, (uint32_t)(jj - 1) & 1u, 11);  // the single P buffer was read by the P V of tile jj-1
-            }
-            SM_TRACE(6);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                uint8_t *dst = smem + L::OFF_P + half * (128 * 128) + row * 128 + ((c ^ (row & 7)) << 4);
-                *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
-            }
-            SM_TRACE(7);
-            // this CTA's V half has landed; dead keys get weight 0 but 0 x (stale NaN/Inf) would poison O: clear their rows
-            ok = ok && wait(C_VLAND + st, (uint32_t)(jj >> 1) & 1u, 12);
-            SM_TRACE(8);
-            if (row < 64 && !((tmask >> row) & 1ull)) {
-#pragma unroll
-                for (int c = 0; c < VCH; ++c) {
-                    uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (half * 64 + row) * 128);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
+                    for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
                 }
-            }
-            fence_proxy_async_smem();
-            SM_TRACE(9);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(leader_pfull);
-            SM_TRACE(10);
-        }
-        // ---- epilogue: the two threads of a row add their sums, each stores its half of the head_dim columns ----
-        if (threadIdx.x == 64) TC2_TRACE(2, 15, 2);
-        if (ok) ok = wait(C_PVDONE, (uint32_t)(n_tiles - 1) & 1u, 13);
-        if (threadIdx.x == 64) TC2_TRACE(2, 15, 3);
-        exch[(0 * 2 + half) * 128 + row] = l;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        l += exch[(0 * 2 + (half ^ 1)) * 128 + row];
-        if (ok) {
-            tc_fence_after();
-            const float inv = 1.f / l;
-            __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + hq) * HD + half * (HD / 2);
-#pragma unroll 1
-            for (int c = 0; c < HD / 64; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tmem_base + lane_addr + kColO + half * (HD / 2) + c * 32, o);
-                tmem_wait_ld();
-                if (row_live) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
+                if (tmask != ~0ull) {
+                    // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows as soon
+                    // as this CTA's V half has landed (long before the P V that reads them)
+                    ok = ok && wait(C_VLAND + st, (uint32_t)(gi >> 1) & 1u, 12);
+                    if (row < 64 && !((tmask >> row) & 1ull)) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 v;
-                        uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+                        for (int c = 0; c < VCH; ++c) {
+                            uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (half * 64 + row) * 128);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * k]) * inv,
-                                                                      __uint_as_float(o[8 * i + 2 * k + 1]) * inv);
-                            vv[k] = *reinterpret_cast<uint32_t *>(&hh);
+                            for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
                         }
-                        *reinterpret_cast<uint4 *>(orow + c * 32 + i * 8) = v;
                     }
                 }
+                if (rmask != ~0ull) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) if (!((rmask >> c) & 1ull)) s[c] = -INFINITY;
+                }
+                float mx4[4] = {s[0], s[1], s[2], s[3]};
+#pragma unroll
+                for (int c = 4; c < 64; c += 4) {
+                    mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
+                    mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+                }
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                // meet the thread that holds the other 64 keys of this row (thread 64 first makes sure that the TMA stores of
+                // the previous unit have read the staging area, which is the P buffer every thread writes after this barrier)
+                exch[(buf * 2 + half) * 128 + row] = mx;
+                if (jj == 0 && threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                mx = fmaxf(mx, exch[(buf * 2 + (half ^ 1)) * 128 + row]);
+                bool pv_waited = false;
+                if (jj == 0) {
+                    m_ref = mx;
+                } else {
+                    const bool grow = (mx - m_ref) * p.scale_log2 > kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        // O (and l) were accumulated against m_ref: bring them to the new reference before this tile's P V.
+                        // Both threads of a row see the same mx, so they decide alike; each rescales its half of O's columns.
+                        const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
+                        if (grow) m_ref = mx;
+                        l *= alpha;
+                        ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 10);
+                        pv_waited = true;
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c = 0; c < HD / 64; ++c) {
+                            uint32_t o[32];
+                            const uint32_t o_addr = tmem_base + lane_addr + kColO + half * (HD / 2) + c * 32;
+                            tmem_ld32(o_addr, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(o_addr, o);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t packed[32];
+#pragma unroll
+                for (int c = 0; c < 64; c += 2) {
+                    const float p0 = ex2(fmaf(s[c], p.scale_log2, -mr));
+                    const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, -mr));
+                    sum4[(c >> 1) & 3] += p0 + p1;
+                    __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+                    packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
+                }
+                l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                if (gi >= 1 && !pv_waited)
+                    ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 11);  // the single P buffer was read by the previous P V
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint8_t *dst = smem + L::OFF_P + half * (128 * 128) + row * 128 + ((c ^ (row & 7)) << 4);
+                    *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+                }
+                // the arrive below also tells the leader that this CTA's V half is in place
+                if (tmask == ~0ull) ok = ok && wait(C_VLAND + st, (uint32_t)(gi >> 1) & 1u, 12);
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(leader_pfull);
             }
+            gt += w.n_tiles;
+            // ---- epilogue of the unit ----
+            // The two threads of a row add their sums; each thread normalises its half of the head_dim columns, 64 at a
+            // time, into the (now idle) P buffer laid out like a Q tile, and one thread hands the tile to TMA stores.
+            if (threadIdx.x == 64) { TC2_TRACE(2, 15, 2); TC2_TRACE(2, ui_s, 2); }
+            const int g_last = gt - 1;
+            ok = ok && wait(C_PVDONE, (uint32_t)g_last & 1u, 13);
+            if (threadIdx.x == 64) { TC2_TRACE(2, 15, 3); TC2_TRACE(2, ui_s, 3); }
+            const int xb = (g_last + 1) & 1;
+            exch[(xb * 2 + half) * 128 + row] = l;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            l += exch[(xb * 2 + (half ^ 1)) * 128 + row];
+            const float inv = 1.f / l;
+            tc_fence_after();
+            const bool store_unit = w.t0 < p.T;   // an idle partner tile (odd tile count) has nothing to write
+#pragma unroll 1
+            for (int rnd = 0; rnd < HD / 128; ++rnd) {
+                uint32_t o0[32], o1[32];
+                const uint32_t o_addr = tmem_base + lane_addr + kColO + half * (HD / 2) + rnd * 64;
+                tmem_ld32(o_addr, o0); tmem_ld32(o_addr + 32, o1);
+                tmem_wait_ld();
+                if (rnd == HD / 128 - 1) {
+                    // all of O is in registers: the next unit's first P V may overwrite the accumulator
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(leader_ofree);
+                }
+                uint8_t *srow = smem + L::OFF_P + half * (128 * 128) + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t *src = (c < 4) ? (o0 + 8 * c) : (o1 + 8 * (c - 4));
+                    uint4 v;
+                    uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(src[2 * k]) * inv, __uint_as_float(src[2 * k + 1]) * inv);
+                        vv[k] = *reinterpret_cast<uint32_t *>(&hh);
+                    }
+                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (threadIdx.x == 64) {
+                    if (store_unit) {
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh)
+                            tma_store_4d(&tm_o, base + L::OFF_P + hh * (128 * 128), hh * (HD / 2) + rnd * 64, w.kvh * p.G, w.t0, w.b);
+                    }
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    // before the staging area is rewritten the store must have read it: at once between rounds, but after
+                    // the last round only when the next unit is about to write P (see the top of the tile loop)
+                    if (rnd + 1 < HD / 128) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                }
+                if (rnd + 1 < HD / 128) asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+            if (threadIdx.x == 64) { TC2_TRACE(2, 15, 4); TC2_TRACE(2, ui_s, 4); }
         }
+        if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores of this CTA are complete
     }
 
-    if (threadIdx.x == 64) TC2_TRACE(2, 15, 4);
     tc_fence_before();
     __syncthreads();
     cluster_arrive();

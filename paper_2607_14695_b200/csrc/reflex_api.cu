@@ -352,7 +352,7 @@ int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, co
         p.nsplit = tc_choose_splits(p, c->lay.partial_bytes, c->sm_count);
         const bool two = c->attn_impl == REFLEX_ATTN_TC2 || (c->attn_impl == REFLEX_ATTN_AUTO && tc2_ok && p.nsplit == 1);
         if (two) p.nsplit = 1;
-        e = launch_attention_tc(p, status, two, (cudaStream_t)stream);
+        e = launch_attention_tc(p, status, two, c->sm_count, (cudaStream_t)stream);
     }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");
     return REFLEX_OK;

@@ -75,6 +75,6 @@ cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st);  // co
 bool tc_supported(const AttnParams &p);
 int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 bool tc2_supported(const AttnParams &p);
-cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, cudaStream_t st);
+cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st);
 
 }  // namespace reflex
