@@ -152,6 +152,25 @@ int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, 
                       const void *W2, const void *b2, float *gate_buf, int B, int R, int D, int Cd,
                       int Hd, float eps, int dtype, void *stream);
 
+/* No counterpart in the paper: a convenience for callers that cannot hand the library any scratch memory.
+ * Same result as reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf, ...) with a gate_buf, but the gate
+ * and hidden-layer scratch lives in an array built into the library image (96 Ki floats = 384 KiB of device
+ * memory on every GPU that loads the library, held until the process exits), so nothing is allocated: not by
+ * this call, not by the caller. Meant for code that must not call cudaMalloc where it runs -- a control loop
+ * with a latency bound (an allocation can synchronise the whole device), a plug-in inside a host program that
+ * owns all device memory through its own pool, a callback that may not block -- and that has no spare buffer
+ * of its own to lend.
+ *   Limit: B*(D+Hd) <= 98304 floats and D <= 2048 (e.g. 64 streams x (1024 + 256)); larger shapes return
+ *   REFLEX_ERR_SHAPE and must use reflex_adarmsnorm with a caller-provided gate_buf.
+ *   The first call on each device looks up the array's device address (with that device current); make that
+ *   first call outside any stream capture.
+ *   All calls on a device share the one array and it keeps the previous call's contents (every value that is read
+ *   is rewritten first, nothing needs clearing): two calls that overlap on the GPU, e.g. on different streams, race.
+ *   x, y, cond, W1, b1, W2, b2, B, R, D, Cd, Hd, eps, dtype, stream: as in reflex_adarmsnorm; cond is required. */
+int reflex_adarmsnorm_noalloc(const void *x, void *y, const void *cond, const void *W1, const void *b1,
+                              const void *W2, const void *b2, int B, int R, int D, int Cd, int Hd, float eps,
+                              int dtype, void *stream);
+
 /* Eq. 1 / App. A Prop. 1: for every stream b, KV head j and its G*T query rows,
  *   out = softmax(scale * Q [K_pin; K_slide; K_dyn]^T) [V_pin; V_slide; V_dyn]
  * over static rows [0, static_len[b]), the live ring slots (physical order; softmax does not depend

@@ -26,7 +26,7 @@ EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
-    "reflex_adarmsnorm", "reflex_partitioned_attention", "reflex_flow_step",
+    "reflex_adarmsnorm", "reflex_adarmsnorm_noalloc", "reflex_partitioned_attention", "reflex_flow_step",
 ]
 
 
@@ -68,6 +68,7 @@ def load():
     lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_cache_append_sliding.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+    lib.reflex_adarmsnorm_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
     for name in EXPORTS:
@@ -209,6 +210,16 @@ def reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6, strea
     Hd, Cd = (W1.shape if W1 is not None else (0, 0))
     _check(load().reflex_adarmsnorm(_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf),
                                     B, R, D, int(Cd), int(Hd), float(eps), dtype_code(x), _stream(stream)))
+    return y
+
+
+def reflex_adarmsnorm_noalloc(x, y, cond, W1, b1, W2, b2, eps=1e-6, stream=None):
+    """AdaRMSNorm for callers that have no scratch buffer to lend: the gate scratch is an array inside the library
+    (B*(D+Hd) <= 98304 floats). Calls on one device share that array, so calls that overlap on the GPU race."""
+    B, R, D = x.shape
+    Hd, Cd = W1.shape
+    _check(load().reflex_adarmsnorm_noalloc(_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2),
+                                            B, R, D, int(Cd), int(Hd), float(eps), dtype_code(x), _stream(stream)))
     return y
 
 

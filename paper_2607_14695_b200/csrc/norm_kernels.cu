@@ -378,3 +378,50 @@ cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, fl
 }
 
 }  // namespace reflex
+
+// ------------------------------------------------------------------------------------------------
+// Entry point that needs no scratch from the caller (see reflex.h). Lives in this file because host code
+// may only name the array below through cudaGetSymbolAddress, and that lookup has to sit beside the definition.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kNoAllocFloats = 96 * 1024;   // 384 KiB per GPU that loads the library, held until the process exits
+static __device__ __align__(256) float g_noalloc_gate[kNoAllocFloats];
+
+constexpr int kMaxDevices = 64;
+float *g_noalloc_ptr[kMaxDevices] = {};        // device address of the array, per device, resolved on first use
+
+}  // namespace
+
+extern "C" int reflex_adarmsnorm_noalloc(const void *x, void *y, const void *cond, const void *W1, const void *b1,
+                                         const void *W2, const void *b2, int B, int R, int D, int Cd, int Hd, float eps,
+                                         int dtype, void *stream)
+{
+    // same argument checks as reflex_adarmsnorm with cond given, plus the size limit of the built-in scratch
+    if (B < 1 || R < 1 || D < 8 || D % 8 != 0 || D > 2048 || Hd < 8 || Hd % 8 != 0 || Cd < 8 || Cd % 8 != 0 || Cd > 4096 || Hd > 4096)
+        return reflex::api_fail(REFLEX_ERR_SHAPE, "reflex_adarmsnorm_noalloc: need B, R >= 1, D a multiple of 8 in [8, 2048], Cd and Hd multiples of 8 in [8, 4096]");
+    if ((size_t)B * (size_t)(D + Hd) > kNoAllocFloats)
+        return reflex::api_fail(REFLEX_ERR_SHAPE, "reflex_adarmsnorm_noalloc: B*(D+Hd) = %zu floats exceeds the built-in scratch of %zu floats; "
+                                "use reflex_adarmsnorm with a caller-provided gate_buf", (size_t)B * (size_t)(D + Hd), kNoAllocFloats);
+    if (!x || !y || !cond || !W1 || !b1 || !W2 || !b2) return reflex::api_fail(REFLEX_ERR_INVALID_ARG, "reflex_adarmsnorm_noalloc: NULL argument");
+    if (dtype != REFLEX_DTYPE_BF16 && dtype != REFLEX_DTYPE_F32) return reflex::api_fail(REFLEX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (!(eps >= 0.f)) return reflex::api_fail(REFLEX_ERR_INVALID_ARG, "eps must be >= 0");
+    const void *ptrs[7] = {x, y, cond, W1, b1, W2, b2};
+    for (const void *q : ptrs)
+        if (reinterpret_cast<uintptr_t>(q) & 15u) return reflex::api_fail(REFLEX_ERR_ALIGN, "reflex_adarmsnorm_noalloc: pointer not 16-byte aligned");
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return reflex::api_fail(REFLEX_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return reflex::api_fail(REFLEX_ERR_INVALID_ARG, "device ordinal %d not supported", dev);
+    if (!g_noalloc_ptr[dev]) {
+        // First call on this device: turn the symbol into a device address. In host code `g_noalloc_gate` is only a
+        // stand-in for the symbol, never an address a kernel could use.
+        float *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_noalloc_gate);
+        if (e != cudaSuccess || !ptr) return reflex::api_fail(REFLEX_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        g_noalloc_ptr[dev] = ptr;
+    }
+    e = reflex::launch_adarmsnorm(x, y, cond, W1, b1, W2, b2, g_noalloc_ptr[dev], B, R, D, Cd, Hd, eps, dtype, (cudaStream_t)stream);
+    if (e != cudaSuccess) return reflex::api_fail(REFLEX_ERR_CUDA, "adarmsnorm launch: %s", cudaGetErrorString(e));
+    return REFLEX_OK;
+}

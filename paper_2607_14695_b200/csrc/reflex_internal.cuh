@@ -53,6 +53,9 @@ struct AttnParams {
     int dtype;
 };
 
+// Records a failure for reflex_last_error_string() and returns `code` (printf-style message).
+int api_fail(int code, const char *fmt, ...);
+
 // Number of kernels this library has launched in this process (every launcher bumps it).
 void count_launch(int n = 1);
 
