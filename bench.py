@@ -159,7 +159,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg4", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
-    ap.add_argument("--attn", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--attn", default="auto", choices=["auto", "simt", "tc", "tc2"])
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
@@ -194,61 +195,104 @@ def main():
         dist.barrier()
     rb.load()
 
-    impl = {"auto": rb.ATTN_AUTO, "simt": rb.ATTN_SIMT, "tc": rb.ATTN_TC}[args.attn]
+    impl = {"auto": rb.ATTN_AUTO, "simt": rb.ATTN_SIMT, "tc": rb.ATTN_TC, "tc2": rb.ATTN_TC2}[args.attn]
     runner = StepRunner(w, device=f"cuda:{local_rank}", attn_impl=impl, host_inputs=not args.no_e2e)
     alg = runner.algorithmic()
     stream = torch.cuda.current_stream()
+    use_graph = not args.no_graph
+    if use_graph:
+        runner.capture_steps()
+    do_step = runner.step_graph if use_graph else runner.step
+    l2_flush = None
+    if runner.input_bytes_resident() < 4 * 126e6:
+        l2_flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=f"cuda:{local_rank}")   # small workload: flush L2 between steps
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    def timed_steps(n, step_fn):
+        """n steps; device time by CUDA events on the launching stream. With an L2 flush between steps each step is
+        bracketed by its own pair of events so the flush stays outside the timed region."""
+        if l2_flush is None:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for k in range(n):
+                step_fn(k)
+            b.record(stream)
+            barrier()
+            return a.elapsed_time(b), None
+        evs = []
+        for k in range(n):
+            l2_flush.fill_(k & 0xFF)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); step_fn(k); b.record(stream)
+            evs.append((a, b))
+        barrier()
+        per = [a.elapsed_time(b) for a, b in evs]
+        return sum(per), per
+
     sampler = ClockSampler(local_rank)
     sampler.start()
     for k in range(args.warmup):
-        runner.step(k)
+        do_step(k)
     barrier()
-    # ---- timed region: exactly K steps, device-timed on the launching stream ----
+    # ---- timed region: exactly K steps ----
     launches0 = rb.reflex_kernel_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
-    e0.record(stream)
-    for k in range(args.steps):
-        runner.step(k)
-    e1.record(stream)
-    barrier()
+    ms_total, per_step = timed_steps(args.steps, do_step)
     wall1 = time.time()
-    launches = rb.reflex_kernel_launch_count() - launches0
-    ms_total = e0.elapsed_time(e1)
-    # ---- the same K steps again with events around every attention / norm call (per-kernel durations) ----
-    ev_attn, ev_norm, step_marks = [], [], []
-    for k in range(args.steps):
-        m = torch.cuda.Event(enable_timing=True); m.record(stream); step_marks.append(m)
-        runner.step_timed(k, ev_attn, ev_norm)
-    m = torch.cuda.Event(enable_timing=True); m.record(stream); step_marks.append(m)
-    barrier()
+    launches = (args.steps * runner.kernels_per_step) if use_graph else (rb.reflex_kernel_launch_count() - launches0)
     clocks = sampler.summary(wall0, wall1)
-    attn_ms = [a.elapsed_time(b) for a, b in ev_attn]
-    norm_ms = [a.elapsed_time(b) for a, b in ev_norm]
-    step_ms = sorted(step_marks[i].elapsed_time(step_marks[i + 1]) for i in range(args.steps))
+    # ---- per-kernel durations: graphs that hold only the attention (resp. AdaRMSNorm) launches of one step, replayed
+    # ---- back to back; and per-step times of the whole step ----
+    reps = max(3, min(args.steps, 20))
+
+    def avg_launch_ms(fn_variant, calls_per_graph):
+        graphs = [runner.capture(lambda v=v: fn_variant(v))[0] for v in range(runner.variants)]
+        for g in graphs:
+            g.replay()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(reps):
+            graphs[i % len(graphs)].replay()
+        b.record(stream)
+        barrier()
+        return a.elapsed_time(b) / (reps * calls_per_graph)
+
+    sh = rb.stream_handle
+    attn_avg_ms = avg_launch_ms(lambda v: [runner.attention(l, v, sh()) for l in range(w.L)], w.L)
+    norm_avg_ms = avg_launch_ms(lambda v: [runner.norm(l, v, v, sh()) for l in range(w.L)], w.L)
+    step_marks = []
+    for k in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); do_step(k); b.record(stream)
+        step_marks.append((a, b))
+    barrier()
+    step_ms = sorted(a.elapsed_time(b) for a, b in step_marks) if per_step is None else sorted(per_step)
     # ---- end to end: inputs from pinned host memory, action chunk back to the host, every step ----
-    e2e = None
+    e2e_ms = 0.0
+    n_e2e = max(3, min(args.steps, 30))
     if not args.no_e2e:
+        def e2e_step(k):
+            runner.copy_inputs_from_host(k)
+            do_step(k)
+            runner.copy_result_to_host()
         for k in range(3):
-            runner.step_from_host(k)
+            e2e_step(k)
         barrier()
         h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n_e2e = max(3, min(args.steps, 30))
         h0.record(stream)
         for k in range(n_e2e):
-            runner.step_from_host(k)
+            e2e_step(k)
         h1.record(stream)
         barrier()
         e2e_ms = h0.elapsed_time(h1)
     sampler.stop()
 
-    t = torch.tensor([ms_total, e2e_ms if not args.no_e2e else 0.0], dtype=torch.float64, device=f"cuda:{local_rank}")
+    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=f"cuda:{local_rank}")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms_total, e2e_ms_max = float(t[0]), float(t[1])
@@ -260,8 +304,6 @@ def main():
     peaks = measured_peaks()
     ms_per_step = ms_total / args.steps
     value = world * args.steps / (ms_total * 1e-3)          # every rank runs its own replica of the batch
-    attn_avg_ms = statistics.mean(attn_ms)
-    norm_avg_ms = statistics.mean(norm_ms)
     attn_gbs = alg["attn_bytes_per_launch"] / (attn_avg_ms * 1e-3) / 1e9
     attn_tflops = alg["attn_flops_per_launch"] / (attn_avg_ms * 1e-3) / 1e12
     line = {
@@ -271,15 +313,18 @@ def main():
         "config": {"workload": f"{w.name}: B={w.B} streams x L={w.L} layers, Hq={w.Hq}/Hkv={w.Hkv}, d={w.d}, static S={w.S}, ring N={w.N}, "
                                f"dynamic T={w.T}, D={w.D}, K={w.K}; one step = L x (AdaRMSNorm + partitioned attention) + Euler update",
                    "parallelism": "replicas only (independent streams per GPU, no collective)" if world > 1 else "single GPU",
-                   "attention_impl": args.attn, "l2_policy": f"inputs larger than L2: {runner.input_bytes_resident() / 1e6:.0f} MB of cache + per-layer inputs are read per step pair (L2 is 126 MB)",
+                   "attention_impl": args.attn, "launch": "CUDA graph replay, one graph per step" if use_graph else "direct launches",
+                   "l2_policy": (f"inputs larger than L2: {runner.input_bytes_resident() / 1e6:.0f} MB of cache + per-layer inputs are read per step pair (L2 is 126 MB)"
+                                 if l2_flush is None else "L2 flushed (256 MB write) before every timed step; each step timed by its own event pair"),
                    "bytes_per_step_algorithmic": alg["bytes_per_step"], "flops_per_step": alg["flops_per_step"]},
         "gpu_launches": int(launches),
         "step_ms": {"p50": step_ms[len(step_ms) // 2], "p95": step_ms[min(len(step_ms) - 1, int(0.95 * len(step_ms)))], "max": step_ms[-1],
-                    "note": "per-step times from the instrumented pass"},
+                    "note": "per-step event pairs"},
         "hbm_gbs_whole_step": alg["bytes_per_step"] / (ms_per_step * 1e-3) / 1e9,
         "roofline": {"kernel": "partitioned attention", "bound": "hbm", "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": attn_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
                      "bytes_per_launch": alg["attn_bytes_per_launch"], "avg_launch_us": attn_avg_ms * 1e3,
+                     "how": "average over graph replays that hold only the L attention launches of a step, CUDA events on the launching stream",
                      "frac_of_nominal_8TBs": attn_gbs / 8000.0,
                      "tensor": {"achieved_tflops": attn_tflops, "peak_tflops_sustained": peaks["bf16_tflops_sustained"],
                                 "frac": attn_tflops / peaks["bf16_tflops_sustained"]}},

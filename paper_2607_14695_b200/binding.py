@@ -26,7 +26,7 @@ EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
-    "reflex_adarmsnorm", "reflex_adarmsnorm_noalloc", "reflex_partitioned_attention", "reflex_flow_step",
+    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_partitioned_attention", "reflex_flow_step",
 ]
 
 
@@ -68,6 +68,7 @@ def load():
     lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_cache_append_sliding.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+    lib.reflex_adarmsnorm_gate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     lib.reflex_adarmsnorm_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
@@ -213,6 +214,15 @@ def reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6, strea
     return y
 
 
+def reflex_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, D, stream=None):
+    """gate_buf[:B*D] <- 1 + W2 SiLU(W1 c + b1) + b2 (fp32); gate_buf holds B*(D+Hd) floats."""
+    B, Cd = cond.shape
+    Hd = W1.shape[0]
+    _check(load().reflex_adarmsnorm_gate(_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), B, int(D), int(Cd), int(Hd),
+                                         dtype_code(cond), _stream(stream)))
+    return gate_buf
+
+
 def reflex_adarmsnorm_noalloc(x, y, cond, W1, b1, W2, b2, eps=1e-6, stream=None):
     """AdaRMSNorm for callers that have no scratch buffer to lend: the gate scratch is an array inside the library
     (B*(D+Hd) <= 98304 floats). Calls on one device share that array, so calls that overlap on the GPU race."""
@@ -262,6 +272,12 @@ def prepare_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6):
     args = (_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), B, R, D, int(Cd), int(Hd),
             float(eps), dtype_code(x))
     return _prepared(load().reflex_adarmsnorm, args)
+
+
+def prepare_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, D):
+    B, Cd = cond.shape
+    args = (_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), B, int(D), int(Cd), int(W1.shape[0]), dtype_code(cond))
+    return _prepared(load().reflex_adarmsnorm_gate, args)
 
 
 def prepare_partitioned_attention(cache: Cache, layer, q, k_dyn, v_dyn, out, scale=0.0, dyn_mask=0):

@@ -266,40 +266,55 @@ static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B,
     return e;
 }
 
+static bool gate_scratch_fits(int Cd, int Hd)
+{
+    const size_t smem_h = (size_t)(kGateUnits * Cd + kGateStreams * (Cd + 4)) * 4;
+    const size_t smem_g = (size_t)(kGateUnits * Hd + kGateStreams * (Hd + 4)) * 4;
+    return smem_h <= 160 * 1024 && smem_g <= 160 * 1024;
+}
+
+// gamma(c) = 1 + W2 SiLU(W1 c + b1) + b2 for B streams into gate_buf[B][D]; hidden activations go to gate_buf + B*D.
+template <typename T>
+static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const T *W2, const T *b2, float *gate_buf, int B, int D,
+                                 int Cd, int Hd, cudaStream_t st)
+{
+    const size_t smem_h = (size_t)(kGateUnits * Cd + kGateStreams * (Cd + 4)) * 4;
+    const size_t smem_g = (size_t)(kGateUnits * Hd + kGateStreams * (Hd + 4)) * 4;
+    float *hid = gate_buf + (size_t)B * D;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(gate_layer_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gate_layer_kernel<T, float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int groups = (B + kGateStreams - 1) / kGateStreams;
+    gate_layer_kernel<T, T, true><<<dim3((Hd + kGateUnits - 1) / kGateUnits, groups), 256, smem_h, st>>>(cond, W1, b1, hid, B, Cd, Hd, 0);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((D + kGateUnits - 1) / kGateUnits, groups);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = smem_g;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, gate_layer_kernel<T, float, false>, (const float *)hid, W2, b2, gate_buf, B, Hd, D, 1);
+    count_launch();
+    return e;
+}
+
 template <typename T>
 static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, const T *b1, const T *W2, const T *b2,
                                  float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, cudaStream_t st)
 {
     bool after_gate = false;
-    const size_t smem_h = (size_t)(kGateUnits * Cd + kGateStreams * (Cd + 4)) * 4;
-    const size_t smem_g = (size_t)(kGateUnits * Hd + kGateStreams * (Hd + 4)) * 4;
-    if (cond && gate_buf && smem_h <= 160 * 1024 && smem_g <= 160 * 1024) {
-        // gate_buf = [B][D] gate followed by [B][Hd] hidden activations
-        float *hid = gate_buf + (size_t)B * D;
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaError_t e = cudaFuncSetAttribute(gate_layer_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(gate_layer_kernel<T, float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-            if (e != cudaSuccess) return e;
-            attr_set = true;
-        }
-        const int groups = (B + kGateStreams - 1) / kGateStreams;
-        gate_layer_kernel<T, T, true><<<dim3((Hd + kGateUnits - 1) / kGateUnits, groups), 256, smem_h, st>>>(cond, W1, b1, hid, B, Cd, Hd, 0);
-        count_launch();
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((D + kGateUnits - 1) / kGateUnits, groups);
-        cfg.blockDim = dim3(256);
-        cfg.dynamicSmemBytes = smem_g;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, gate_layer_kernel<T, float, false>, (const float *)hid, W2, b2, gate_buf, B, Hd, D, 1);
-        count_launch();
+    if (cond && gate_buf && gate_scratch_fits(Cd, Hd)) {
+        cudaError_t e = launch_gate_t<T>(cond, W1, b1, W2, b2, gate_buf, B, D, Cd, Hd, st);
         if (e != cudaSuccess) return e;
         after_gate = true;
     } else if (cond && gate_buf) {
@@ -362,6 +377,17 @@ __global__ void flow_step_kernel(float *__restrict__ x, const T *__restrict__ v,
             else x_lowp[i] = nx;
         }
     }
+}
+
+cudaError_t launch_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf,
+                                   int B, int D, int Cd, int Hd, int dtype, cudaStream_t st)
+{
+    if (!gate_scratch_fits(Cd, Hd)) return cudaErrorNotSupported;
+    if (dtype == REFLEX_DTYPE_BF16)
+        return launch_gate_t<__nv_bfloat16>((const __nv_bfloat16 *)cond, (const __nv_bfloat16 *)W1, (const __nv_bfloat16 *)b1,
+                                            (const __nv_bfloat16 *)W2, (const __nv_bfloat16 *)b2, gate_buf, B, D, Cd, Hd, st);
+    return launch_gate_t<float>((const float *)cond, (const float *)W1, (const float *)b1, (const float *)W2, (const float *)b2,
+                                gate_buf, B, D, Cd, Hd, st);
 }
 
 cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, float dt, int dtype, cudaStream_t st)

@@ -17,7 +17,7 @@ from . import synth
 
 class StepRunner:
     def __init__(self, w: synth.Workload, device: str = "cuda:0", variants: int = 2, attn_impl: int = rb.ATTN_AUTO,
-                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True):
+                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, overlap_gate: bool = True):
         self.w = w
         self.device = torch.device(device)
         self.variants = variants
@@ -62,6 +62,13 @@ class StepRunner:
         self.out = torch.empty((w.B, w.T, w.Hq, w.d), dtype=tdt, device=self.device)
         # gate [B][D] + hidden scratch [B][Hd]: lets AdaRMSNorm read the gate weights once per 16 streams
         self.gate_buf = torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) if gate_scratch else None
+        # The gate of Eq. 2 depends on c = [emb(t_k), s_t] only, not on the layer's input: with overlap_gate the gate of layer
+        # l+1 is computed on a second stream while layer l's attention runs (two buffers, by layer parity), and the
+        # row kernel of layer l+1 then takes it as a ready gate. Same launches, same order of dependent work.
+        self.overlap_gate = overlap_gate and gate_scratch
+        if self.overlap_gate:
+            self.gate_bufs = [torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) for _ in range(2)]
+            self.side = torch.cuda.Stream(device=self.device)
         self.xa = torch.randn(w.B, w.T, w.A, generator=g, device=self.device, dtype=torch.float32)
         self.host = None
         self._calls = {}
@@ -121,14 +128,63 @@ class StepRunner:
         kk = k % self.w.K
         self._call(("f", kk, variant), lambda: rb.prepare_flow_step(self.xa, self.vflow[variant], None, kk, self.w.K))(sh or rb.stream_handle())
 
+    def gate(self, layer: int, k: int, sh):
+        kk = k % self.w.K
+        W1, b1, W2, b2 = self.W[layer]
+        self._call(("g", layer, kk), lambda: rb.prepare_adarmsnorm_gate(self.cond[kk], W1, b1, W2, b2, self.gate_bufs[layer & 1], self.w.D))(sh)
+
+    def rows(self, layer: int, variant: int, sh):
+        w = self.w
+        self._call(("r", layer, variant), lambda: rb.prepare_adarmsnorm(
+            self.x[layer][variant], self.y, None, None, None, None, None, gate_buf=self.gate_bufs[layer & 1][: w.B * w.D].view(w.B, w.D)))(sh)
+
     def step(self, k: int):
         """One denoising step over all layers and streams, inputs already in HBM."""
         variant = k % self.variants
-        sh = rb.stream_handle()
+        main = torch.cuda.current_stream()
+        sh = rb.stream_handle(main)
+        if not self.overlap_gate:
+            for layer in range(self.w.L):
+                self.norm(layer, k, variant, sh)
+                self.attention(layer, variant, sh)
+            self.flow(k, variant, sh)
+            return
+        side_h = rb.stream_handle(self.side)
+        self.gate(0, k, sh)
         for layer in range(self.w.L):
-            self.norm(layer, k, variant, sh)
+            self.rows(layer, variant, sh)
+            if layer + 1 < self.w.L:
+                self.side.wait_stream(main)          # the next gate may start once this layer's rows are queued
+                self.gate(layer + 1, k, side_h)
             self.attention(layer, variant, sh)
+            if layer + 1 < self.w.L:
+                main.wait_stream(self.side)          # ... and must be complete before the next layer's rows
         self.flow(k, variant, sh)
+
+    # ---- CUDA graphs: the launch-bound inner loop is captured once and replayed (host cost per step: one launch) ----
+    def capture(self, fn):
+        """Capture the library calls made by fn() into a CUDA graph; returns (graph, number of kernels in it)."""
+        fn()                                   # warm-up outside capture (first-call set-up, lazy module loading)
+        torch.cuda.synchronize(self.device)
+        g = torch.cuda.CUDAGraph()
+        n0 = rb.reflex_kernel_launch_count()
+        with torch.cuda.graph(g):
+            fn()
+        return g, rb.reflex_kernel_launch_count() - n0
+
+    def capture_steps(self):
+        """One graph per distinct step (conditioning index x input variant)."""
+        import math
+        period = self.w.K * self.variants // math.gcd(self.w.K, self.variants)
+        self.step_graphs, self.kernels_per_step = [], 0
+        for k in range(period):
+            g, n = self.capture(lambda k=k: self.step(k))
+            self.step_graphs.append(g)
+            self.kernels_per_step = n
+        return self.step_graphs
+
+    def step_graph(self, k: int):
+        self.step_graphs[k % len(self.step_graphs)].replay()
 
     def step_timed(self, k: int, ev_attn, ev_norm):
         """Same launches as step(), with CUDA events around every attention and norm call."""
@@ -149,13 +205,13 @@ class StepRunner:
         self.h2d_bytes_per_step = sum(nb(self.host[n][l][0]) for n in ("x", "q", "kd", "vd") for l in range(self.w.L)) + nb(self.host["vflow"][0])
         self.d2h_bytes_per_step = nb(self.host_xa)
 
-    def step_from_host(self, k: int):
+    def copy_inputs_from_host(self, k: int):
+        """This step's inputs (every layer's x, Q, K_dyn, V_dyn and the velocity) from pinned host memory."""
         variant = k % self.variants
         for layer in range(self.w.L):
             for name in ("x", "q", "kd", "vd"):
                 getattr(self, name)[layer][variant].copy_(self.host[name][layer][variant], non_blocking=True)
-            self.norm(layer, k, variant)
-            self.attention(layer, variant)
         self.vflow[variant].copy_(self.host["vflow"][variant], non_blocking=True)
-        self.flow(k, variant)
+
+    def copy_result_to_host(self):
         self.host_xa.copy_(self.xa, non_blocking=True)
