@@ -22,6 +22,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture (profiles/)
+NCU_TRAFFIC_BYTES = {("cfg4", "auto"): 76.3e6, ("cfg4", "tc2"): 76.3e6}
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -292,10 +294,8 @@ def main():
         e2e_ms = h0.elapsed_time(h1)
     sampler.stop()
 
-    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=f"cuda:{local_rank}")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms_max = float(t[0]), float(t[1])
+    from paper_2607_14695_b200 import multi
+    ms_total, e2e_ms_max = multi.max_over_ranks([ms_total, e2e_ms], device=f"cuda:{local_rank}")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -303,7 +303,7 @@ def main():
 
     peaks = measured_peaks()
     ms_per_step = ms_total / args.steps
-    value = world * args.steps / (ms_total * 1e-3)          # every rank runs its own replica of the batch
+    value = multi.replica_throughput(args.steps, world, ms_total)     # every rank runs its own replica of the batch
     attn_gbs = alg["attn_bytes_per_launch"] / (attn_avg_ms * 1e-3) / 1e9
     attn_tflops = alg["attn_flops_per_launch"] / (attn_avg_ms * 1e-3) / 1e12
     line = {
@@ -322,7 +322,8 @@ def main():
                     "note": "per-step event pairs"},
         "hbm_gbs_whole_step": alg["bytes_per_step"] / (ms_per_step * 1e-3) / 1e9,
         "roofline": {"kernel": "partitioned attention", "bound": "hbm", "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": attn_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                     "frac": attn_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.attn)), "traffic_source": "profiles/attn_tc2_cfg4_ncu_full.md (dram read + write of one launch)",
                      "bytes_per_launch": alg["attn_bytes_per_launch"], "avg_launch_us": attn_avg_ms * 1e3,
                      "how": "average over graph replays that hold only the L attention launches of a step, CUDA events on the launching stream",
                      "frac_of_nominal_8TBs": attn_gbs / 8000.0,
@@ -334,7 +335,7 @@ def main():
         "clocks": clocks,
     }
     if not args.no_e2e:
-        line["e2e"] = {"value": world * n_e2e / (e2e_ms_max * 1e-3), "unit": "steps/s", "h2d_bytes_per_step": int(runner.h2d_bytes_per_step),
+        line["e2e"] = {"value": multi.replica_throughput(n_e2e, world, e2e_ms_max), "unit": "steps/s", "h2d_bytes_per_step": int(runner.h2d_bytes_per_step),
                        "d2h_bytes_per_step": int(runner.d2h_bytes_per_step), "steps": n_e2e}
     if world == 1 and not args.no_cpu_baseline:
         units = w.B * w.L

@@ -66,7 +66,7 @@ class StepRunner:
         # l+1 is computed on a second stream while layer l's attention runs (two buffers, by layer parity), and the
         # row kernel of layer l+1 then takes it as a ready gate. Same launches, same order of dependent work.
         self.overlap_gate = overlap_gate and gate_scratch
-        if self.overlap_gate:
+        if gate_scratch:
             self.gate_bufs = [torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) for _ in range(2)]
             self.side = torch.cuda.Stream(device=self.device)
         self.xa = torch.randn(w.B, w.T, w.A, generator=g, device=self.device, dtype=torch.float32)
