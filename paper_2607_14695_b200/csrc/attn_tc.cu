@@ -81,25 +81,41 @@ struct TileGeom {
         else { t.dyn = 1; t.kind = 2; t.idx = it - ns - nr; t.row0 = b * T + t.idx * kBN; }
         return t;
     }
+    // bits [lo, hi) of a 64-bit word (0 <= lo, hi <= 64)
+    static __device__ __forceinline__ uint64_t bit_range(int lo, int hi)
+    {
+        lo = max(lo, 0); hi = min(hi, 64);
+        if (hi <= lo) return 0ull;
+        const uint64_t upto_hi = (hi >= 64) ? ~0ull : ((1ull << hi) - 1ull);
+        return upto_hi & ~((1ull << lo) - 1ull);
+    }
     // which of the 64 keys of a tile are live (independent of the query row)
     __device__ __forceinline__ uint64_t tile_mask(const TileRef &t) const
     {
+        const int base = t.idx * kBN;
         if (t.kind == 1) {
-            if (count >= N && (t.idx + 1) * kBN <= N) return ~0ull;
-            uint64_t m = 0;
-            for (int c = 0; c < kBN; ++c) {
-                const int slot = t.idx * kBN + c;
-                int age = slot - oldest;
-                if (age < 0) age += N;
-                if (slot < N && age < count) m |= (1ull << c);
-            }
+            // live ring slots are the circular run of `count` slots that starts at `oldest`
+            const int c = min(count, N);
+            const int end = oldest + c;                       // may pass N: the run wraps
+            uint64_t m = bit_range(oldest - base, min(end, N) - base);
+            if (end > N) m |= bit_range(0 - base, end - N - base);
             return m;
         }
         const int len = (t.kind == 0) ? S : T;
-        const int valid = len - t.idx * kBN;
-        return valid >= kBN ? ~0ull : ((1ull << valid) - 1ull);
+        return bit_range(0, len - base);
     }
 };
+
+// s[c] = -inf for every key c of a 64-key half that `mask` marks dead (constant bit tests, two selects per word)
+__device__ __forceinline__ void apply_key_mask(float (&s)[64], uint64_t mask)
+{
+    const uint32_t lo = (uint32_t)mask, hi = (uint32_t)(mask >> 32);
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+        if (!(lo & (1u << c))) s[c] = -INFINITY;
+        if (!(hi & (1u << c))) s[32 + c] = -INFINITY;
+    }
+}
 
 template <int HD>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -280,10 +296,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             float s[64];
 #pragma unroll
             for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
-            if (rmask != ~0ull) {
-#pragma unroll
-                for (int c = 0; c < 64; ++c) if (!((rmask >> c) & 1ull)) s[c] = -INFINITY;
-            }
+            if (rmask != ~0ull) apply_key_mask(s, rmask);
             float mx = s[0];
 #pragma unroll
             for (int c = 1; c < 64; ++c) mx = fmaxf(mx, s[c]);

@@ -225,18 +225,23 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 issue_qk(gi, last_of_unit);
                 return true;
             };
+            // Q K^T of tile jj+1 is issued before waiting for P(jj): S is double buffered in TMEM, so the tensor pipe works
+            // on the next tile's logits while the softmax threads finish this tile. (Issuing Q K^T two tiles ahead, or in
+            // whichever order inputs arrive, was measured and is slower: with two K stages the extra Q K^T lands in front
+            // of a P V that the softmax threads are waiting for.)
             bool ok = true;
             int gt = 0, ui = 0;
             for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
                 const Unit w = load_unit(u);
-                ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk_when_ready(gt, w.n_tiles == 1);
-                for (int jj = 0; jj < w.n_tiles && ok; ++jj) {
+                const int n = w.n_tiles;
+                ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk_when_ready(gt, n == 1);
+                for (int jj = 0; jj < n && ok; ++jj) {
                     const int gi = gt + jj;
-                    if (jj + 1 < w.n_tiles) {
-                        ok = qk_when_ready(gi + 1, jj + 2 == w.n_tiles);
+                    const int st = gi & 1;
+                    if (jj + 1 < n) {
+                        ok = qk_when_ready(gi + 1, jj + 2 == n);
                         if (!ok) break;
                     }
-                    const int st = gi & 1;
                     ok = wait(C_PFULL, (uint32_t)gi & 1u, 8);   // both CTAs: P written, V landed and cleaned
                     if (ok && jj == 0 && ui >= 1) ok = wait(C_OFREE, (uint32_t)(ui - 1) & 1u, 15);   // previous O has been read out
                     if (!ok) break;
@@ -251,7 +256,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     umma2_commit_mc(bar(C_VEMPTY + st), 3);
                     umma2_commit_mc(bar(C_PVDONE), 3);
                 }
-                gt += w.n_tiles;
+                gt += n;
             }
         }
     } else {
@@ -289,7 +294,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
                     }
                 }
+#define SM_EV(ev) do { if (threadIdx.x == 64 && ui_s == 0) TC2_TRACE(3, jj, ev); } while (0)
+                SM_EV(0);
                 ok = ok && wait(C_SFULL + buf, (uint32_t)(gi >> 1) & 1u, 9);
+                SM_EV(1);
                 if (threadIdx.x == 64 && jj == 0) TC2_TRACE(2, ui_s, 1);
                 tc_fence_after();
                 float s[64];
@@ -301,6 +309,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
                 }
+                SM_EV(2);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
@@ -317,10 +326,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
-                if (rmask != ~0ull) {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) if (!((rmask >> c) & 1ull)) s[c] = -INFINITY;
-                }
+                if (rmask != ~0ull) apply_key_mask(s, rmask);
                 float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
                 for (int c = 4; c < 64; c += 4) {
@@ -330,9 +336,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // meet the thread that holds the other 64 keys of this row (thread 64 first makes sure that the TMA stores of
                 // the previous unit have read the staging area, which is the P buffer every thread writes after this barrier)
+                SM_EV(3);
                 exch[(buf * 2 + half) * 128 + row] = mx;
                 if (jj == 0 && threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 asm volatile("bar.sync 1, 256;" ::: "memory");
+                SM_EV(4);
                 mx = fmaxf(mx, exch[(buf * 2 + (half ^ 1)) * 128 + row]);
                 bool pv_waited = false;
                 if (jj == 0) {
@@ -366,26 +374,35 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 uint32_t packed[32];
 #pragma unroll
                 for (int c = 0; c < 64; c += 2) {
-                    const float p0 = ex2(fmaf(s[c], p.scale_log2, -mr));
-                    const float p1 = ex2(fmaf(s[c + 1], p.scale_log2, -mr));
+                    // P = 2^(s*scale*log2e - m). One pair in four takes the FMA-pipe exponential so the MUFU unit and the
+                    // FMA pipe share the load.
+                    const float x0 = fmaf(s[c], p.scale_log2, -mr), x1 = fmaf(s[c + 1], p.scale_log2, -mr);
+                    const bool on_fma = ((c >> 1) & 3) == 3;
+                    const float p0 = on_fma ? ex2_fma(x0) : ex2(x0);
+                    const float p1 = on_fma ? ex2_fma(x1) : ex2(x1);
                     sum4[(c >> 1) & 3] += p0 + p1;
                     __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
                 }
                 l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                SM_EV(5);
                 if (gi >= 1 && !pv_waited)
                     ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 11);  // the single P buffer was read by the previous P V
+                SM_EV(6);
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     uint8_t *dst = smem + L::OFF_P + half * (128 * 128) + row * 128 + ((c ^ (row & 7)) << 4);
                     *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
                 }
+                SM_EV(7);
                 // the arrive below also tells the leader that this CTA's V half is in place
                 if (tmask == ~0ull) ok = ok && wait(C_VLAND + st, (uint32_t)(gi >> 1) & 1u, 12);
+                SM_EV(8);
                 fence_proxy_async_smem();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(leader_pfull);
+                SM_EV(9);
             }
             gt += w.n_tiles;
             // ---- epilogue of the unit ----

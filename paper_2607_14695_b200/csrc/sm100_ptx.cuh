@@ -134,6 +134,22 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
     return t;
 }
 
+// 2^x on the FMA pipe (no MUFU): round x to the nearest integer with the 1.5*2^23 trick, a cubic for 2^f on
+// f in [-0.5, 0.5] (max relative error 7.7e-5, far below the bf16 rounding of P), and the integer part added into
+// the exponent field. Used for a fraction of the softmax exponentials so that the MUFU unit (16 results per clock
+// per SM) is not the only path they take. Arguments below -125 give exactly 0.
+__device__ __forceinline__ float ex2_fma(float x)
+{
+    const float xc = fmaxf(x, -125.f);
+    const float t = xc + 12582912.f;                // 1.5 * 2^23: the low mantissa bits of t hold round(xc)
+    const float f = xc - (t - 12582912.f);
+    float pl = fmaf(f, 0.05508868f, 0.24260405f);
+    pl = fmaf(f, pl, 0.69327623f);
+    pl = fmaf(f, pl, 0.99992895f);
+    const float r = __int_as_float(__float_as_int(pl) + (__float_as_int(t) << 23));
+    return x < -125.f ? 0.f : r;                    // masked keys (x = -inf) get weight exactly 0
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
