@@ -183,6 +183,32 @@ class StepRunner:
             self.kernels_per_step = n
         return self.step_graphs
 
+    # ---- one control tick of the stream: ring append, fresh noise, K denoising steps ----
+    def tick(self):
+        w = self.w
+        sh = rb.stream_handle()
+        if not hasattr(self, "_tick_src"):
+            self._tick_src = (self.rnd(w.B, w.L, w.m, w.Hkv, w.d), self.rnd(w.B, w.L, w.m, w.Hkv, w.d),
+                              torch.randn(w.B, w.T, w.A, generator=self._gen, device=self.device, dtype=torch.float32))
+            self._ids = list(range(w.B))
+        kn, vn, noise = self._tick_src
+        rb.reflex_cache_append_sliding(self.cache, self._ids, kn, vn)      # O(m) in-place append in every layer
+        self.xa.copy_(noise)                                               # x ~ N(0, I) at t = 1
+        for k in range(w.K):
+            self.step(k)
+
+    def capture_tick(self):
+        self.tick_graph, self.kernels_per_tick = self.capture(self.tick)
+        return self.tick_graph
+
+    def refresh_static(self, S: int):
+        """A new observation: rewrite the static prefix of every stream (S tokens), as happens every few ticks."""
+        w = self.w
+        if not hasattr(self, "_static_src"):
+            self._static_src = (self.rnd(w.B, w.L, w.S_max, w.Hkv, w.d), self.rnd(w.B, w.L, w.S_max, w.Hkv, w.d))
+        ks, vs = self._static_src
+        rb.reflex_cache_init_static(self.cache, list(range(w.B)), ks, vs, S=[S] * w.B)
+
     def step_graph(self, k: int):
         self.step_graphs[k % len(self.step_graphs)].replay()
 
