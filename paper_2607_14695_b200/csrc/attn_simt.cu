@@ -165,37 +165,67 @@ attn_simt_kernel(AttnParams p)
         T *o = (T *)p.out + (((size_t)b * p.T + t) * p.Hq + h) * d;
         RowIO<T, DPL>::store(o + lane * DPL, acc);
     } else {
-        float *part = p.partials + (((size_t)b * rows + r) * p.nsplit + split) * (d + 2);
-        if (lane == 0) { part[0] = m; part[1] = l; }
+        const size_t slot = partial_slot(b, rows, r, p.nsplit, split);
+        float *po = partial_o(p.partials, slot, d), *pml = partial_ml(p.partials, (size_t)p.B * rows * p.nsplit, slot, d);
+        if (lane == 0) { pml[0] = m; pml[1] = l; }
 #pragma unroll
-        for (int i = 0; i < DPL; ++i) part[2 + lane * DPL + i] = acc[i];
+        for (int i = 0; i < DPL; ++i) po[lane * DPL + i] = acc[i];
     }
 }
 
-// grid = (T*Hq, B), block = d threads: merge of split partials, m* = max m_s, l = sum l_s e^{m_s-m*},
-// o = sum acc_s e^{m_s-m*} / l.
-template <typename T>
-__global__ void attn_merge_kernel(AttnParams p)
+// Merge of split partials: m* = max m_s, l = sum l_s e^{m_s-m*}, o = sum acc_s e^{m_s-m*} / l. One warp per query row
+// (lane s fetches slice s's (m, l); every lane owns d/32 output columns), 8 rows per block, all loads independent.
+template <typename T, int DPL>
+__global__ void __launch_bounds__(256)
+attn_merge_kernel(AttnParams p)
 {
-    const int d = p.d;
-    const int r = blockIdx.x, b = blockIdx.y, e = threadIdx.x;
+    constexpr int d = DPL * 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rows = p.T * p.Hq;
-    const float *part = p.partials + ((size_t)b * rows + r) * p.nsplit * (d + 2);
-    float mstar = -INFINITY;
-    for (int s = 0; s < p.nsplit; ++s) mstar = fmaxf(mstar, part[(size_t)s * (d + 2)]);
-    float l = 0.f, o = 0.f;
-    for (int s = 0; s < p.nsplit; ++s) {
-        const float ms = part[(size_t)s * (d + 2)];
-        if (ms == -INFINITY) continue;
-        const float w = expf(ms - mstar);
-        l = fmaf(part[(size_t)s * (d + 2) + 1], w, l);
-        o = fmaf(part[(size_t)s * (d + 2) + 2 + e], w, o);
+    const int gr = blockIdx.x * 8 + warp;      // row over all streams
+    if (gr >= p.B * rows) return;
+    const int b = gr / rows, r = gr % rows;
+    const size_t n_slots = (size_t)p.B * rows * p.nsplit;
+    const size_t slot0 = partial_slot(b, rows, r, p.nsplit, 0);
+    float ms = -INFINITY, ls = 0.f;
+    if (lane < p.nsplit) {
+        const float2 ml = *reinterpret_cast<const float2 *>(partial_ml(p.partials, n_slots, slot0 + lane, d));
+        ms = ml.x; ls = ml.y;
     }
+    float mstar = ms;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
+    const float w = (ms == -INFINITY) ? 0.f : expf(ms - mstar);
+    float l = ls * w;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    float acc[DPL];
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+    for (int s = 0; s < p.nsplit; ++s) {
+        const float ws = __shfl_sync(0xffffffffu, w, s);
+        if (ws == 0.f) continue;               // an empty slice: its O row was never written
+        const float *po = partial_o(p.partials, slot0 + s, d) + lane * DPL;
+        float f[DPL];
+        if constexpr (DPL % 4 == 0) {
+#pragma unroll
+            for (int i = 0; i < DPL; i += 4) {
+                const float4 v = *reinterpret_cast<const float4 *>(po + i);
+                f[i] = v.x; f[i + 1] = v.y; f[i + 2] = v.z; f[i + 3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) f[i] = po[i];
+        }
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] = fmaf(f[i], ws, acc[i]);
+    }
+    const float inv = 1.f / l;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] *= inv;
     const int t = r / p.Hq, h = r % p.Hq;
     T *out = (T *)p.out + (((size_t)b * p.T + t) * p.Hq + h) * d;
-    const float val = o / l;
-    if constexpr (sizeof(T) == 2) out[e] = __float2bfloat16_rn(val);
-    else out[e] = val;
+    RowIO<T, DPL>::store(out + lane * DPL, acc);
 }
 
 int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
@@ -230,13 +260,25 @@ static cudaError_t launch_simt_t(const AttnParams &p, cudaStream_t st)
     return launch_attention_merge(p, st);
 }
 
-cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st)
+template <typename T>
+static cudaError_t launch_merge_t(const AttnParams &p, cudaStream_t st)
 {
-    const int rows = p.T * p.Hq;
-    if (p.dtype == REFLEX_DTYPE_BF16) attn_merge_kernel<__nv_bfloat16><<<dim3(rows, p.B), p.d, 0, st>>>(p);
-    else attn_merge_kernel<float><<<dim3(rows, p.B), p.d, 0, st>>>(p);
+    const int grid = (p.B * p.T * p.Hq + 7) / 8;
+    switch (p.d / 32) {
+        case 1: attn_merge_kernel<T, 1><<<grid, 256, 0, st>>>(p); break;
+        case 2: attn_merge_kernel<T, 2><<<grid, 256, 0, st>>>(p); break;
+        case 4: attn_merge_kernel<T, 4><<<grid, 256, 0, st>>>(p); break;
+        case 8: attn_merge_kernel<T, 8><<<grid, 256, 0, st>>>(p); break;
+        default: return cudaErrorInvalidValue;
+    }
     count_launch();
     return cudaGetLastError();
+}
+
+cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st)
+{
+    if (p.dtype == REFLEX_DTYPE_BF16) return launch_merge_t<__nv_bfloat16>(p, st);
+    return launch_merge_t<float>(p, st);
 }
 
 cudaError_t launch_attention_simt(const AttnParams &p, cudaStream_t st)

@@ -397,10 +397,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 }
             }
         } else {
-            float *part = p.partials + (((size_t)b * rows_total + (size_t)t_row * p.Hq + hq) * p.nsplit + split) * (HD + 2);
+            const size_t slot = partial_slot(b, rows_total, t_row * p.Hq + hq, p.nsplit, split);
+            float *po = partial_o(p.partials, slot, HD);
+            float *pml = partial_ml(p.partials, (size_t)p.B * rows_total * p.nsplit, slot, HD);
             if (n_local > 0 && ok) {
                 tc_fence_after();
-                if (row_live) { part[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; part[1] = l; }
+                if (row_live) { pml[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; pml[1] = l; }
 #pragma unroll 1
                 for (int c = 0; c < HD / 32; ++c) {
                     uint32_t o[32];
@@ -408,12 +410,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     tmem_wait_ld();
                     if (row_live) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            *reinterpret_cast<float2 *>(part + 2 + c * 32 + 2 * i) = make_float2(__uint_as_float(o[2 * i]), __uint_as_float(o[2 * i + 1]));
+                        for (int i = 0; i < 8; ++i)
+                            *reinterpret_cast<float4 *>(po + c * 32 + 4 * i) = make_float4(__uint_as_float(o[4 * i]), __uint_as_float(o[4 * i + 1]),
+                                                                                           __uint_as_float(o[4 * i + 2]), __uint_as_float(o[4 * i + 3]));
                     }
                 }
             } else if (row_live) {
-                part[0] = -INFINITY; part[1] = 0.f;
+                pml[0] = -INFINITY; pml[1] = 0.f;
             }
         }
     }
@@ -564,6 +567,28 @@ int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
 
 bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 || p.d == 256); }
 
+// Key split of the two-CTA kernel: as many slices as it takes to give every cluster (SM pair) a unit, at least four
+// 128-key tiles per slice so that a unit's head and tail stay amortised. Returns 0 when even that leaves most of the
+// machine idle (then the one-CTA kernel with its finer split is the better fit).
+int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
+{
+    const int G = p.Hq / p.Hkv;
+    const int tile_tokens = kBM / G;
+    const int n_pairs = ((p.T + tile_tokens - 1) / tile_tokens + 1) / 2;
+    const int units = n_pairs * p.Hkv * p.B;
+    const int clusters = sm_count / 2;
+    if (units >= clusters) return 1;
+    const int halves = (p.S_max + kBN - 1) / kBN + (p.N + kBN - 1) / kBN + (p.T + kBN - 1) / kBN;
+    const int tiles = (halves + 1) / 2;
+    int want = clusters / units;
+    if (want > tiles / 4) want = tiles / 4;
+    if (want > kMaxSplits) want = kMaxSplits;
+    const size_t per_split = (size_t)p.B * p.T * p.Hq * (p.d + 2) * sizeof(float);
+    if (per_split > 0 && (size_t)want * per_split > partial_bytes) want = (int)(partial_bytes / per_split);
+    if (want < 1) want = 1;
+    return (units * want * 10 >= clusters * 6) ? want : 0;
+}
+
 cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st)
 {
     const int G = p.Hq / p.Hkv;
@@ -587,14 +612,16 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
         CUtensorMap mo;
         if (!cache().get(&mo, p.out, 1, (p.B << 16) | p.T, p.Hq, p.d, G, mk_q)) return cudaErrorInvalidValue;
         tp.n_qtiles = (tp.n_qtiles + 1) / 2;
-        const int units = tp.n_qtiles * p.Hkv * p.B;
+        const int units = tp.n_qtiles * p.Hkv * p.B * p.nsplit;
         int clusters = sm_count / 2;
         if (clusters > units) clusters = units;
         if (clusters < 1) clusters = 1;
         dim3 grid2(2 * clusters, 1, 1);
-        if (p.d == 256) return launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
-        if (p.d == 128) return launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
-        return cudaErrorInvalidValue;
+        if (p.d == 256) e = launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
+        else if (p.d == 128) e = launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
+        else return cudaErrorInvalidValue;
+        if (e != cudaSuccess || p.nsplit == 1) return e;
+        return launch_attention_merge(p, st);
     }
     dim3 grid(tp.n_qtiles * p.Hkv, p.B, p.nsplit);
     switch (p.d) {

@@ -95,15 +95,17 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t rank = cluster_ctarank();
     const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
     const int n_pairs = p.n_qtiles;                    // tile pairs per (stream, KV head)
-    const int n_units = p.B * p.Hkv * n_pairs;
+    const int n_units = p.B * p.Hkv * n_pairs * p.nsplit;   // with nsplit > 1 a unit covers a slice of the key tiles
 
     // geometry of one work unit
-    struct Unit { int b, kvh, t0, H, n_tiles; TileGeom g; };
+    struct Unit { int b, kvh, t0, H, n_tiles, tile0, split; TileGeom g; };
     auto load_unit = [&](int u) -> Unit {
         Unit w;
-        const int pair = u % n_pairs;
-        w.kvh = (u / n_pairs) % p.Hkv;
-        w.b = u / (n_pairs * p.Hkv);
+        w.split = u % p.nsplit;
+        const int uu = u / p.nsplit;
+        const int pair = uu % n_pairs;
+        w.kvh = (uu / n_pairs) % p.Hkv;
+        w.b = uu / (n_pairs * p.Hkv);
         w.t0 = (2 * pair + (int)rank) * p.tile_tokens;
         const StreamState st = p.state[w.b];
         TileGeom &g = w.g;
@@ -117,7 +119,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         g.row_base = (p.layer * p.B + w.b) * (p.S_max + p.N);
         g.S_max = p.S_max; g.b = w.b;
         w.H = g.ns + g.nr + g.nd;          // 64-key halves
-        w.n_tiles = (w.H + 1) / 2;         // >= 1: there is always a dynamic half
+        const int all_tiles = (w.H + 1) / 2;   // >= 1: there is always a dynamic half
+        const int per = (all_tiles + p.nsplit - 1) / p.nsplit;
+        w.tile0 = w.split * per;               // this unit's slice of the key tiles (may be empty for the last splits)
+        w.n_tiles = max(0, min(all_tiles, w.tile0 + per) - w.tile0);
         return w;
     };
 
@@ -161,15 +166,16 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             int gt = 0, ui = 0;
             for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
                 const Unit w = load_unit(u);
+                if (w.n_tiles == 0) { --ui; continue; }   // an empty key slice: every role skips it the same way
                 for (int jj = 0; jj < w.n_tiles && ok; ++jj) {
                     const int gi = gt + jj, st = gi & 1;
                     const uint32_t ph = (uint32_t)((gi >> 1) - 1) & 1u;
-                    const int h0 = 2 * jj, h1 = 2 * jj + 1;
+                    const int h0 = 2 * (w.tile0 + jj), h1 = h0 + 1;
                     const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
                     if (gi >= 2) ok = wait(C_KEMPTY + st, ph, 1);
                     if (!ok) break;
                     if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
-                    const int myh = 2 * jj + (int)rank;
+                    const int myh = h0 + (int)rank;
                     if (myh < w.H) {
                         const TileRef tr = w.g.decode(myh);
                         for (int c = 0; c < CH; ++c)
@@ -234,6 +240,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
                 const Unit w = load_unit(u);
                 const int n = w.n_tiles;
+                if (n == 0) { --ui; continue; }
                 ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk_when_ready(gt, n == 1);
                 for (int jj = 0; jj < n && ok; ++jj) {
                     const int gi = gt + jj;
@@ -280,10 +287,19 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const Unit w = load_unit(u);
             const int t_row = w.t0 + row / p.G;
             if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 0);
+            const int rows_total = p.T * p.Hq;
+            const size_t n_slots = (size_t)p.B * rows_total * p.nsplit;
+            float *pml = nullptr;    // this row's (m, l) slot when the keys are split over several units
+            if (p.nsplit > 1 && t_row < p.T)
+                pml = partial_ml(p.partials, n_slots, partial_slot(w.b, rows_total, t_row * p.Hq + w.kvh * p.G + row % p.G, p.nsplit, w.split), HD);
+            if (w.n_tiles == 0) {
+                if (pml && half == 0) { pml[0] = -INFINITY; pml[1] = 0.f; }   // an empty key slice contributes nothing
+                continue;
+            }
             float m_ref = -INFINITY, l = 0.f;
             for (int jj = 0; jj < w.n_tiles; ++jj) {
                 const int gi = gt + jj, buf = gi & 1, st = gi & 1;
-                const int h = 2 * jj + half;
+                const int h = 2 * (w.tile0 + jj) + half;
                 uint64_t tmask = 0ull, rmask = 0ull;
                 if (h < w.H) {
                     const TileRef tr = w.g.decode(h);
@@ -416,8 +432,45 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             exch[(xb * 2 + half) * 128 + row] = l;
             asm volatile("bar.sync 1, 256;" ::: "memory");
             l += exch[(xb * 2 + (half ^ 1)) * 128 + row];
-            const float inv = 1.f / l;
             tc_fence_after();
+            if (p.nsplit > 1) {
+                // key-split unit: leave (m, l, unnormalised O) for the merge kernel; m in natural-log units like the other
+                // kernels. O goes out 32 columns per thread at a time through the idle P buffer (fp32, swizzled 128-byte
+                // rows), so that the global stores are whole 128-byte row segments instead of one scattered row per lane.
+                if (pml && half == 0) { pml[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; pml[1] = l; }
+#pragma unroll 1
+                for (int sub = 0; sub < HD / 64; ++sub) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem_base + lane_addr + kColO + half * (HD / 2) + sub * 32, o);
+                    tmem_wait_ld();
+                    if (sub == HD / 64 - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(leader_ofree);
+                    }
+                    uint8_t *srow = smem + L::OFF_P + half * (128 * 128) + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    const int tid = threadIdx.x - 64;
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int idx = it * 256 + tid;
+                        const int hh = idx >> 10, rr = (idx >> 3) & 127, cc = idx & 7;
+                        const int tt = w.t0 + rr / p.G;
+                        if (tt < p.T) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(smem + L::OFF_P + hh * (128 * 128) + rr * 128 + ((cc ^ (rr & 7)) << 4));
+                            float *dst = partial_o(p.partials, partial_slot(w.b, rows_total, tt * p.Hq + w.kvh * p.G + rr % p.G, p.nsplit, w.split), HD) +
+                                         hh * (HD / 2) + sub * 32 + cc * 4;
+                            *reinterpret_cast<uint4 *>(dst) = v;
+                        }
+                    }
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                }
+                continue;
+            }
+            const float inv = 1.f / l;
             const bool store_unit = w.t0 < p.T;   // an idle partner tile (odd tile count) has nothing to write
 #pragma unroll 1
             for (int rnd = 0; rnd < HD / 128; ++rnd) {

@@ -94,7 +94,7 @@ WorkspaceLayout workspace_layout(const reflex_cache_desc &d)
     const size_t rows = (size_t)d.T_max * d.Hq;
     const size_t blocks = ((rows + 3) / 4) * (size_t)d.B;
     size_t splits = (8 * 148 + blocks - 1) / blocks;
-    if (splits < 1) splits = 1;
+    if (splits < 2) splits = 2;     // the batched two-CTA kernel may split the keys when streams alone do not fill the SM pairs
     if (splits > (size_t)kMaxSplits) splits = kMaxSplits;
     w.partial_off = off;
     w.partial_bytes = align_up(splits * (size_t)d.B * rows * (size_t)(d.d + 2) * sizeof(float), 256);
@@ -373,10 +373,11 @@ int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, co
         p.nsplit = simt_choose_splits(p, c->lay.partial_bytes, c->sm_count);
         e = launch_attention_simt(p, (cudaStream_t)stream);
     } else {
-        // enough query tiles to fill the machine: the two-CTA kernel (no key split); otherwise one CTA per tile with a key split
-        p.nsplit = tc_choose_splits(p, c->lay.partial_bytes, c->sm_count);
-        const bool two = c->attn_impl == REFLEX_ATTN_TC2 || (c->attn_impl == REFLEX_ATTN_AUTO && tc2_ok && p.nsplit == 1);
-        if (two) p.nsplit = 1;
+        // Batched shapes take the two-CTA kernel (with a key split when the streams alone do not fill the SM pairs);
+        // a single stream or a few take one CTA per query tile with a finer key split.
+        const int split2 = tc2_ok ? tc2_choose_splits(p, c->lay.partial_bytes, c->sm_count) : 0;
+        const bool two = c->attn_impl == REFLEX_ATTN_TC2 || (c->attn_impl == REFLEX_ATTN_AUTO && split2 >= 1);
+        p.nsplit = two ? (split2 >= 1 ? split2 : 1) : tc_choose_splits(p, c->lay.partial_bytes, c->sm_count);
         e = launch_attention_tc(p, status, two, c->sm_count, (cudaStream_t)stream);
     }
     if (e != cudaSuccess) return cuda_fail(e, "attention launch");

@@ -53,6 +53,12 @@ struct AttnParams {
     int dtype;
 };
 
+// Split-K partials in the workspace: for n = B * rows * nsplit (row, split) slots, first n rows of d floats with the
+// unnormalised O (16-byte aligned), then n (m, l) pairs (m in natural-log units; m = -inf, l = 0 for an empty slice).
+__host__ __device__ inline size_t partial_slot(int b, int rows, int r, int nsplit, int s) { return ((size_t)b * rows + r) * nsplit + s; }
+__host__ __device__ inline float *partial_o(float *base, size_t slot, int d) { return base + slot * (size_t)d; }
+__host__ __device__ inline float *partial_ml(float *base, size_t n_slots, size_t slot, int d) { return base + n_slots * (size_t)d + slot * 2; }
+
 // Records a failure for reflex_last_error_string() and returns `code` (printf-style message).
 int api_fail(int code, const char *fmt, ...);
 
@@ -80,6 +86,7 @@ cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st);  // co
 bool tc_supported(const AttnParams &p);
 int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 bool tc2_supported(const AttnParams &p);
+int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st);
 
 }  // namespace reflex
