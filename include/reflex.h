@@ -152,14 +152,16 @@ int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, 
                       const void *W2, const void *b2, float *gate_buf, int B, int R, int D, int Cd,
                       int Hd, float eps, int dtype, void *stream);
 
-/* Eq. 2, the part that does not depend on x: gamma(c) = 1 + W2 SiLU(W1 c + b1) + b2 for every stream, fp32, into
- * gate_buf. c = [emb(t_k), s_t] is known before the layer's input exists, so a caller may run this on a second stream
- * while the previous layer is still busy and then call reflex_adarmsnorm with cond == NULL and this gate.
- *   cond [B][Cd], W1 [Hd][Cd], b1 [Hd], W2 [D][Hd], b2 [D]   device, dtype
- *   gate_buf  device fp32, B*(D+Hd) floats: gate [B][D] first, the rest is scratch for the hidden activations
- * Requirements: D % 8 == 0, Cd and Hd multiples of 8 in [8, 1024]. */
+/* Eq. 2, the part that does not depend on x: gamma_l(c) = 1 + W2_l SiLU(W1_l c + b1_l) + b2_l for every stream and
+ * for L layers at once (the layers' parameters stacked along a leading axis), fp32, into gate_buf.
+ * c = [emb(t_k), s_t] is fixed for a whole denoising step and known before any layer's input exists, so the gates of
+ * all layers of the step can be produced by one call (two launches whatever L is) ahead of the layer loop; each
+ * layer then calls reflex_adarmsnorm with cond == NULL and its slice gate_buf + l*B*D. L = 1 is the single-layer case.
+ *   cond [B][Cd]; W1 [L][Hd][Cd], b1 [L][Hd], W2 [L][D][Hd], b2 [L][D]   device, dtype
+ *   gate_buf  device fp32, L*B*(D+Hd) floats: gates [L][B][D] first, then scratch for the hidden activations
+ * Requirements: D % 8 == 0, Cd and Hd multiples of 8 in [8, 1024], 1 <= L <= 65535. */
 int reflex_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2,
-                           float *gate_buf, int B, int D, int Cd, int Hd, int dtype, void *stream);
+                           float *gate_buf, int L, int B, int D, int Cd, int Hd, int dtype, void *stream);
 
 /* No counterpart in the paper: a convenience for callers that cannot hand the library any scratch memory.
  * Same result as reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf, ...) with a gate_buf, but the gate

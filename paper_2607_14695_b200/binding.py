@@ -68,7 +68,7 @@ def load():
     lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_cache_append_sliding.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
-    lib.reflex_adarmsnorm_gate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    lib.reflex_adarmsnorm_gate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, vp]
     lib.reflex_adarmsnorm_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
@@ -214,11 +214,18 @@ def reflex_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6, strea
     return y
 
 
-def reflex_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, D, stream=None):
-    """gate_buf[:B*D] <- 1 + W2 SiLU(W1 c + b1) + b2 (fp32); gate_buf holds B*(D+Hd) floats."""
+def _gate_dims(cond, W1, W2):
+    """(L, B, D, Cd, Hd) from cond [B][Cd] and W1 [Hd][Cd] or stacked [L][Hd][Cd], W2 [D][Hd] or [L][D][Hd]."""
     B, Cd = cond.shape
-    Hd = W1.shape[0]
-    _check(load().reflex_adarmsnorm_gate(_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), B, int(D), int(Cd), int(Hd),
+    L = W1.shape[0] if W1.dim() == 3 else 1
+    return L, B, int(W2.shape[-2]), int(Cd), int(W1.shape[-2])
+
+
+def reflex_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, stream=None):
+    """gate_buf[:L*B*D] <- 1 + W2_l SiLU(W1_l c + b1_l) + b2_l (fp32) for the L stacked layers; gate_buf holds
+    L*B*(D+Hd) floats."""
+    L, B, D, Cd, Hd = _gate_dims(cond, W1, W2)
+    _check(load().reflex_adarmsnorm_gate(_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), L, B, D, Cd, Hd,
                                          dtype_code(cond), _stream(stream)))
     return gate_buf
 
@@ -274,9 +281,9 @@ def prepare_adarmsnorm(x, y, cond, W1, b1, W2, b2, gate_buf=None, eps=1e-6):
     return _prepared(load().reflex_adarmsnorm, args)
 
 
-def prepare_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, D):
-    B, Cd = cond.shape
-    args = (_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), B, int(D), int(Cd), int(W1.shape[0]), dtype_code(cond))
+def prepare_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf):
+    L, B, D, Cd, Hd = _gate_dims(cond, W1, W2)
+    args = (_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), L, B, D, Cd, Hd, dtype_code(cond))
     return _prepared(load().reflex_adarmsnorm_gate, args)
 
 

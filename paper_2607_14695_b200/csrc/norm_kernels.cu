@@ -159,16 +159,23 @@ constexpr int kGateUnits = 8;      // weight rows (hidden units or gate columns)
 template <typename T, typename VT, bool SILU>
 __global__ void __launch_bounds__(256)
 gate_layer_kernel(const VT *vec, const T *__restrict__ W, const T *__restrict__ bias, float *out, int B, int len, int units,
-                  int wait_prior)
+                  int wait_prior, size_t vec_lstride, size_t out_lstride, int upb)
 {
+    // upb = weight rows per block (a multiple of 8): the staged stream vectors are reused by upb/8 passes of 8 rows
+    // blockIdx.z = layer: weights and biases of the layers are stacked ([L][units][len], [L][units]); the input vectors
+    // are shared by the layers (conditioning, stride 0) or per layer (hidden activations)
+    vec += (size_t)blockIdx.z * vec_lstride;
+    W += (size_t)blockIdx.z * units * len;
+    bias += (size_t)blockIdx.z * units;
+    out += (size_t)blockIdx.z * out_lstride;
     extern __shared__ __align__(16) float sm_gl[];
     const int pitch = len + 4;                   // +4 floats: the 32 stream rows start in different banks
-    float *w_s = sm_gl;                          // [8][len]
-    float *v_s = sm_gl + kGateUnits * len;       // [32][pitch]
+    float *w_s = sm_gl;                          // [upb][len]
+    float *v_s = sm_gl + upb * len;              // [32][pitch]
     const int b0 = blockIdx.y * kGateStreams;
     const int nb = min(kGateStreams, B - b0);
-    const int u0 = blockIdx.x * kGateUnits;
-    const int nu = min(kGateUnits, units - u0);
+    const int u0 = blockIdx.x * upb;
+    const int nu = min(upb, units - u0);
     // weight rows do not depend on the preceding launch: fetch them first, then wait for it (programmatic dependent launch)
     for (int i = threadIdx.x * 8; i < nu * len; i += blockDim.x * 8) {
         float f[8];
@@ -187,17 +194,94 @@ gate_layer_kernel(const VT *vec, const T *__restrict__ W, const T *__restrict__ 
         *reinterpret_cast<float4 *>(v_s + s * pitch + e + 4) = make_float4(f[4], f[5], f[6], f[7]);
     }
     __syncthreads();
-    const int u = threadIdx.x >> 5, sidx = threadIdx.x & 31;
-    if (u >= nu || sidx >= nb) return;
-    const float *wr = w_s + u * len, *vr = v_s + sidx * pitch;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int e = 0; e < len; e += 4) {
-        const float4 wv = *reinterpret_cast<const float4 *>(wr + e);
-        const float4 vv = *reinterpret_cast<const float4 *>(vr + e);
-        a0 = fmaf(wv.x, vv.x, a0); a1 = fmaf(wv.y, vv.y, a1); a2 = fmaf(wv.z, vv.z, a2); a3 = fmaf(wv.w, vv.w, a3);
+    const int sidx = threadIdx.x & 31;
+    if (sidx >= nb) return;
+    const float *vr = v_s + sidx * pitch;
+    for (int u = threadIdx.x >> 5; u < nu; u += kGateUnits) {
+        const float *wr = w_s + u * len;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int e = 0; e < len; e += 4) {
+            const float4 wv = *reinterpret_cast<const float4 *>(wr + e);
+            const float4 vv = *reinterpret_cast<const float4 *>(vr + e);
+            a0 = fmaf(wv.x, vv.x, a0); a1 = fmaf(wv.y, vv.y, a1); a2 = fmaf(wv.z, vv.z, a2); a3 = fmaf(wv.w, vv.w, a3);
+        }
+        const float z = ((a0 + a1) + (a2 + a3)) + to_f<T>(bias[u0 + u]);
+        out[(size_t)(b0 + sidx) * units + u0 + u] = SILU ? z / (1.f + expf(-z)) : 1.f + z;
     }
-    const float z = ((a0 + a1) + (a2 + a3)) + to_f<T>(bias[u0 + u]);
-    out[(size_t)(b0 + sidx) * units + u0 + u] = SILU ? z / (1.f + expf(-z)) : 1.f + z;
+}
+
+// Register-tiled form of one gate layer, used when many layers are evaluated by one call (blockIdx.z = layer): a block
+// owns 64 weight rows and up to 32 streams and each thread accumulates a 2 (rows) x 4 (streams) tile, so one 16-byte
+// shared-memory load feeds up to eight FMAs instead of two. Every dot product is summed in the same order as in
+// gate_layer_kernel (four interleaved partial sums), so the two kernels give identical bits.
+constexpr int kTileUnits = 64;
+template <typename T, typename VT, bool SILU>
+__global__ void __launch_bounds__(256)
+gate_layer_tiled_kernel(const VT *vec, const T *__restrict__ W, const T *__restrict__ bias, float *out, int B, int len, int units,
+                        int wait_prior, size_t vec_lstride, size_t out_lstride)
+{
+    vec += (size_t)blockIdx.z * vec_lstride;
+    W += (size_t)blockIdx.z * units * len;
+    bias += (size_t)blockIdx.z * units;
+    out += (size_t)blockIdx.z * out_lstride;
+    extern __shared__ __align__(16) float sm_gt[];
+    const int pitch = len + 4;
+    float *w_s = sm_gt;                              // [64][pitch]
+    float *v_s = sm_gt + kTileUnits * pitch;         // [32][pitch]
+    const int b0 = blockIdx.y * kGateStreams;
+    const int nb = min(kGateStreams, B - b0);
+    const int u0 = blockIdx.x * kTileUnits;
+    const int nu = min(kTileUnits, units - u0);
+    const int chunks = len / 8;
+    for (int i = threadIdx.x; i < kTileUnits * chunks; i += blockDim.x) {
+        const int u = i / chunks, e = (i % chunks) * 8;
+        float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (u < nu) Vec8<T>::load(W + (size_t)(u0 + u) * len + e, f);
+        *reinterpret_cast<float4 *>(w_s + u * pitch + e) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4 *>(w_s + u * pitch + e + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+    if (wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (int i = threadIdx.x; i < kGateStreams * chunks; i += blockDim.x) {
+        const int sx = i / chunks, e = (i % chunks) * 8;
+        float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (sx < nb) Vec8<VT>::load(vec + (size_t)(b0 + sx) * len + e, f);
+        *reinterpret_cast<float4 *>(v_s + sx * pitch + e) = make_float4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<float4 *>(v_s + sx * pitch + e + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+    __syncthreads();
+    const int sg = threadIdx.x & 7, up = threadIdx.x >> 3;   // streams sg, sg+8, sg+16, sg+24 (bank-conflict free), weight rows up*2, up*2+1
+    const float *w0 = w_s + (up * 2) * pitch, *w1 = w0 + pitch;
+    const float *v0 = v_s + sg * pitch;
+    float4 acc[2][4];
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int e = 0; e < len; e += 4) {
+        const float4 a = *reinterpret_cast<const float4 *>(w0 + e), c = *reinterpret_cast<const float4 *>(w1 + e);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float4 v = *reinterpret_cast<const float4 *>(v0 + j * 8 * pitch + e);
+            acc[0][j].x = fmaf(a.x, v.x, acc[0][j].x); acc[0][j].y = fmaf(a.y, v.y, acc[0][j].y);
+            acc[0][j].z = fmaf(a.z, v.z, acc[0][j].z); acc[0][j].w = fmaf(a.w, v.w, acc[0][j].w);
+            acc[1][j].x = fmaf(c.x, v.x, acc[1][j].x); acc[1][j].y = fmaf(c.y, v.y, acc[1][j].y);
+            acc[1][j].z = fmaf(c.z, v.z, acc[1][j].z); acc[1][j].w = fmaf(c.w, v.w, acc[1][j].w);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int u = up * 2 + i;
+        if (u >= nu) continue;
+        const float bi = to_f<T>(bias[u0 + u]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int sx = sg + 8 * j;
+            if (sx >= nb) continue;
+            const float z = ((acc[i][j].x + acc[i][j].y) + (acc[i][j].z + acc[i][j].w)) + bi;
+            out[(size_t)(b0 + sx) * units + u0 + u] = SILU ? z / (1.f + expf(-z)) : 1.f + z;
+        }
+    }
 }
 
 // One warp per row, the row kept in registers between the statistics pass and the scaling pass
@@ -268,19 +352,23 @@ static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B,
 
 static bool gate_scratch_fits(int Cd, int Hd)
 {
-    const size_t smem_h = (size_t)(kGateUnits * Cd + kGateStreams * (Cd + 4)) * 4;
-    const size_t smem_g = (size_t)(kGateUnits * Hd + kGateStreams * (Hd + 4)) * 4;
+    const size_t smem_h = (size_t)(32 * Cd + kGateStreams * (Cd + 4)) * 4;
+    const size_t smem_g = (size_t)(32 * Hd + kGateStreams * (Hd + 4)) * 4;
     return smem_h <= 160 * 1024 && smem_g <= 160 * 1024;
 }
 
-// gamma(c) = 1 + W2 SiLU(W1 c + b1) + b2 for B streams into gate_buf[B][D]; hidden activations go to gate_buf + B*D.
+// gamma_l(c) = 1 + W2_l SiLU(W1_l c + b1_l) + b2_l for L layers (stacked weights) and B streams: gates into
+// gate_buf[L][B][D], hidden activations into gate_buf + L*B*D ([L][B][Hd]). Two launches whatever L is.
 template <typename T>
-static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const T *W2, const T *b2, float *gate_buf, int B, int D,
-                                 int Cd, int Hd, cudaStream_t st)
+static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const T *W2, const T *b2, float *gate_buf, int L, int B,
+                                 int D, int Cd, int Hd, cudaStream_t st)
 {
-    const size_t smem_h = (size_t)(kGateUnits * Cd + kGateStreams * (Cd + 4)) * 4;
-    const size_t smem_g = (size_t)(kGateUnits * Hd + kGateStreams * (Hd + 4)) * 4;
-    float *hid = gate_buf + (size_t)B * D;
+    // one layer: 8 weight rows per block (more blocks, lower latency); many layers: 32 rows per block, so the staged
+    // stream vectors are fetched four times less often
+    const int upb = L > 1 ? 32 : kGateUnits;
+    const size_t smem_h = (size_t)(upb * Cd + kGateStreams * (Cd + 4)) * 4;
+    const size_t smem_g = (size_t)(upb * Hd + kGateStreams * (Hd + 4)) * 4;
+    float *hid = gate_buf + (size_t)L * B * D;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(gate_layer_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
@@ -289,12 +377,43 @@ static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const 
         attr_set = true;
     }
     const int groups = (B + kGateStreams - 1) / kGateStreams;
-    gate_layer_kernel<T, T, true><<<dim3((Hd + kGateUnits - 1) / kGateUnits, groups), 256, smem_h, st>>>(cond, W1, b1, hid, B, Cd, Hd, 0);
+    const size_t tiled_h = (size_t)(kTileUnits + kGateStreams) * (Cd + 4) * 4, tiled_g = (size_t)(kTileUnits + kGateStreams) * (Hd + 4) * 4;
+    if (L > 1 && tiled_h <= 200 * 1024 && tiled_g <= 200 * 1024) {
+        // many layers in one call: throughput of the whole batch matters more than the latency of one small grid
+        static bool tiled_attr_set = false;
+        if (!tiled_attr_set) {
+            cudaError_t e = cudaFuncSetAttribute(gate_layer_tiled_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(gate_layer_tiled_kernel<T, float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            tiled_attr_set = true;
+        }
+        gate_layer_tiled_kernel<T, T, true><<<dim3((Hd + kTileUnits - 1) / kTileUnits, groups, L), 256, tiled_h, st>>>(
+            cond, W1, b1, hid, B, Cd, Hd, 0, (size_t)0, (size_t)B * Hd);
+        count_launch();
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((D + kTileUnits - 1) / kTileUnits, groups, L);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = tiled_g;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, gate_layer_tiled_kernel<T, float, false>, (const float *)hid, W2, b2, gate_buf, B, Hd, D, 1,
+                               (size_t)B * Hd, (size_t)B * D);
+        count_launch();
+        return e;
+    }
+    gate_layer_kernel<T, T, true><<<dim3((Hd + upb - 1) / upb, groups, L), 256, smem_h, st>>>(
+        cond, W1, b1, hid, B, Cd, Hd, 0, (size_t)0, (size_t)B * Hd, upb);
     count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((D + kGateUnits - 1) / kGateUnits, groups);
+    cfg.gridDim = dim3((D + upb - 1) / upb, groups, L);
     cfg.blockDim = dim3(256);
     cfg.dynamicSmemBytes = smem_g;
     cfg.stream = st;
@@ -303,7 +422,8 @@ static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, gate_layer_kernel<T, float, false>, (const float *)hid, W2, b2, gate_buf, B, Hd, D, 1);
+    e = cudaLaunchKernelEx(&cfg, gate_layer_kernel<T, float, false>, (const float *)hid, W2, b2, gate_buf, B, Hd, D, 1,
+                           (size_t)B * Hd, (size_t)B * D, upb);
     count_launch();
     return e;
 }
@@ -314,7 +434,7 @@ static cudaError_t launch_norm_t(const T *x, T *y, const T *cond, const T *W1, c
 {
     bool after_gate = false;
     if (cond && gate_buf && gate_scratch_fits(Cd, Hd)) {
-        cudaError_t e = launch_gate_t<T>(cond, W1, b1, W2, b2, gate_buf, B, D, Cd, Hd, st);
+        cudaError_t e = launch_gate_t<T>(cond, W1, b1, W2, b2, gate_buf, 1, B, D, Cd, Hd, st);
         if (e != cudaSuccess) return e;
         after_gate = true;
     } else if (cond && gate_buf) {
@@ -380,14 +500,14 @@ __global__ void flow_step_kernel(float *__restrict__ x, const T *__restrict__ v,
 }
 
 cudaError_t launch_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf,
-                                   int B, int D, int Cd, int Hd, int dtype, cudaStream_t st)
+                                   int L, int B, int D, int Cd, int Hd, int dtype, cudaStream_t st)
 {
     if (!gate_scratch_fits(Cd, Hd)) return cudaErrorNotSupported;
     if (dtype == REFLEX_DTYPE_BF16)
         return launch_gate_t<__nv_bfloat16>((const __nv_bfloat16 *)cond, (const __nv_bfloat16 *)W1, (const __nv_bfloat16 *)b1,
-                                            (const __nv_bfloat16 *)W2, (const __nv_bfloat16 *)b2, gate_buf, B, D, Cd, Hd, st);
+                                            (const __nv_bfloat16 *)W2, (const __nv_bfloat16 *)b2, gate_buf, L, B, D, Cd, Hd, st);
     return launch_gate_t<float>((const float *)cond, (const float *)W1, (const float *)b1, (const float *)W2, (const float *)b2,
-                                gate_buf, B, D, Cd, Hd, st);
+                                gate_buf, L, B, D, Cd, Hd, st);
 }
 
 cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, float dt, int dtype, cudaStream_t st)

@@ -324,8 +324,9 @@ int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, 
 }
 
 int reflex_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf,
-                           int B, int D, int Cd, int Hd, int dtype, void *stream)
+                           int L, int B, int D, int Cd, int Hd, int dtype, void *stream)
 {
+    if (L < 1 || L > 65535) return fail(REFLEX_ERR_SHAPE, "L=%d must be in [1, 65535]", L);
     if (dtype != REFLEX_DTYPE_BF16 && dtype != REFLEX_DTYPE_F32) return fail(REFLEX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (!cond || !W1 || !b1 || !W2 || !b2 || !gate_buf) return fail(REFLEX_ERR_INVALID_ARG, "NULL argument");
     if (B < 1) return fail(REFLEX_ERR_SHAPE, "B=%d must be >= 1", B);
@@ -334,7 +335,7 @@ int reflex_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, con
         return fail(REFLEX_ERR_SHAPE, "Cd=%d, Hd=%d must be multiples of 8 in [8, 1024]", Cd, Hd);
     if (!aligned16(cond) || !aligned16(W1) || !aligned16(W2) || !aligned16(b1) || !aligned16(b2) || !aligned16(gate_buf))
         return fail(REFLEX_ERR_ALIGN, "cond / W1 / b1 / W2 / b2 / gate_buf not 16-byte aligned");
-    cudaError_t e = launch_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, B, D, Cd, Hd, dtype, (cudaStream_t)stream);
+    cudaError_t e = launch_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf, L, B, D, Cd, Hd, dtype, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "adarmsnorm gate launch");
     return REFLEX_OK;
 }

@@ -78,7 +78,7 @@ cudaError_t launch_adarmsnorm(const void *x, void *y, const void *cond, const vo
                               const void *b2, float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, int dtype,
                               cudaStream_t st);
 cudaError_t launch_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf,
-                                   int B, int D, int Cd, int Hd, int dtype, cudaStream_t st);
+                                   int L, int B, int D, int Cd, int Hd, int dtype, cudaStream_t st);
 cudaError_t launch_flow_step(float *x, const void *v, void *x_lowp, size_t n, float dt, int dtype, cudaStream_t st);
 cudaError_t launch_attention_simt(const AttnParams &p, cudaStream_t st);
 int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);

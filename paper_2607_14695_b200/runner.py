@@ -17,7 +17,7 @@ from . import synth
 
 class StepRunner:
     def __init__(self, w: synth.Workload, device: str = "cuda:0", variants: int = 2, attn_impl: int = rb.ATTN_AUTO,
-                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, overlap_gate: bool = True):
+                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, gate_mode: str = "step"):
         self.w = w
         self.device = torch.device(device)
         self.variants = variants
@@ -55,18 +55,23 @@ class StepRunner:
         self.kd = [[rnd(w.B, w.T, w.Hkv, w.d) for _ in range(variants)] for _ in range(w.L)]
         self.vd = [[rnd(w.B, w.T, w.Hkv, w.d) for _ in range(variants)] for _ in range(w.L)]
         self.vflow = [rnd(w.B, w.T, w.A) for _ in range(variants)]
-        self.W = [[rnd(w.Hd, w.Cd, std=0.02), torch.zeros(w.Hd, dtype=tdt, device=self.device),
-                   rnd(w.D, w.Hd, std=0.02), torch.zeros(w.D, dtype=tdt, device=self.device)] for _ in range(w.L)]
+        # gate-MLP parameters of all layers, stacked along a leading layer axis (self.W[l] are views of layer l)
+        self.W1s, self.b1s = rnd(w.L, w.Hd, w.Cd, std=0.02), torch.zeros(w.L, w.Hd, dtype=tdt, device=self.device)
+        self.W2s, self.b2s = rnd(w.L, w.D, w.Hd, std=0.02), torch.zeros(w.L, w.D, dtype=tdt, device=self.device)
+        self.W = [[self.W1s[l], self.b1s[l], self.W2s[l], self.b2s[l]] for l in range(w.L)]
         self.cond = [torch.from_numpy(synth.cond_vectors(w, 1.0 - k / w.K)).to(self.device).to(tdt).contiguous() for k in range(w.K)]
         self.y = torch.empty((w.B, w.T, w.D), dtype=tdt, device=self.device)
         self.out = torch.empty((w.B, w.T, w.Hq, w.d), dtype=tdt, device=self.device)
         # gate [B][D] + hidden scratch [B][Hd]: lets AdaRMSNorm read the gate weights once per 16 streams
         self.gate_buf = torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) if gate_scratch else None
-        # The gate of Eq. 2 depends on c = [emb(t_k), s_t] only, not on the layer's input: with overlap_gate the gate of layer
-        # l+1 is computed on a second stream while layer l's attention runs (two buffers, by layer parity), and the
-        # row kernel of layer l+1 then takes it as a ready gate. Same launches, same order of dependent work.
-        self.overlap_gate = overlap_gate and gate_scratch
+        # The gate of Eq. 2 depends on c = [emb(t_k), s_t] only, not on any layer's input. gate_mode:
+        #   "step"    (default) one call at the start of the step computes the gates of all L layers (two launches), every
+        #             layer's row kernel then takes its slice as a ready gate;
+        #   "overlap" the gate of layer l+1 is computed on a second stream while layer l's attention runs;
+        #   "inline"  each layer's reflex_adarmsnorm call computes its own gate (three launches per layer).
+        self.gate_mode = gate_mode if gate_scratch else "inline"
         if gate_scratch:
+            self.gate_all = torch.empty((w.L * w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device)
             self.gate_bufs = [torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) for _ in range(2)]
             self.side = torch.cuda.Stream(device=self.device)
         self.xa = torch.randn(w.B, w.T, w.A, generator=g, device=self.device, dtype=torch.float32)
@@ -131,34 +136,45 @@ class StepRunner:
     def gate(self, layer: int, k: int, sh):
         kk = k % self.w.K
         W1, b1, W2, b2 = self.W[layer]
-        self._call(("g", layer, kk), lambda: rb.prepare_adarmsnorm_gate(self.cond[kk], W1, b1, W2, b2, self.gate_bufs[layer & 1], self.w.D))(sh)
+        self._call(("g", layer, kk), lambda: rb.prepare_adarmsnorm_gate(self.cond[kk], W1, b1, W2, b2, self.gate_bufs[layer & 1]))(sh)
 
-    def rows(self, layer: int, variant: int, sh):
+    def gates_of_step(self, k: int, sh):
+        """gamma_l(c_k) for all layers of this step in one call."""
+        kk = k % self.w.K
+        self._call(("G", kk), lambda: rb.prepare_adarmsnorm_gate(self.cond[kk], self.W1s, self.b1s, self.W2s, self.b2s, self.gate_all))(sh)
+
+    def rows(self, layer: int, variant: int, sh, from_step_gates: bool = False):
         w = self.w
-        self._call(("r", layer, variant), lambda: rb.prepare_adarmsnorm(
-            self.x[layer][variant], self.y, None, None, None, None, None, gate_buf=self.gate_bufs[layer & 1][: w.B * w.D].view(w.B, w.D)))(sh)
+        n = w.B * w.D
+        gate = self.gate_all[layer * n:(layer + 1) * n] if from_step_gates else self.gate_bufs[layer & 1][:n]
+        self._call(("r", layer, variant, from_step_gates), lambda: rb.prepare_adarmsnorm(
+            self.x[layer][variant], self.y, None, None, None, None, None, gate_buf=gate.view(w.B, w.D)))(sh)
 
     def step(self, k: int):
         """One denoising step over all layers and streams, inputs already in HBM."""
         variant = k % self.variants
         main = torch.cuda.current_stream()
         sh = rb.stream_handle(main)
-        if not self.overlap_gate:
+        if self.gate_mode == "step":
+            self.gates_of_step(k, sh)
+            for layer in range(self.w.L):
+                self.rows(layer, variant, sh, True)
+                self.attention(layer, variant, sh)
+        elif self.gate_mode == "overlap":
+            side_h = rb.stream_handle(self.side)
+            self.gate(0, k, sh)
+            for layer in range(self.w.L):
+                self.rows(layer, variant, sh)
+                if layer + 1 < self.w.L:
+                    self.side.wait_stream(main)          # the next gate may start once this layer's rows are queued
+                    self.gate(layer + 1, k, side_h)
+                self.attention(layer, variant, sh)
+                if layer + 1 < self.w.L:
+                    main.wait_stream(self.side)          # ... and must be complete before the next layer's rows
+        else:
             for layer in range(self.w.L):
                 self.norm(layer, k, variant, sh)
                 self.attention(layer, variant, sh)
-            self.flow(k, variant, sh)
-            return
-        side_h = rb.stream_handle(self.side)
-        self.gate(0, k, sh)
-        for layer in range(self.w.L):
-            self.rows(layer, variant, sh)
-            if layer + 1 < self.w.L:
-                self.side.wait_stream(main)          # the next gate may start once this layer's rows are queued
-                self.gate(layer + 1, k, side_h)
-            self.attention(layer, variant, sh)
-            if layer + 1 < self.w.L:
-                main.wait_stream(self.side)          # ... and must be complete before the next layer's rows
         self.flow(k, variant, sh)
 
     # ---- CUDA graphs: the launch-bound inner loop is captured once and replayed (host cost per step: one launch) ----

@@ -320,3 +320,33 @@ def test_10k_tick_stream_stays_finite(U, cfg):
     assert int(bad.item()) == 0
     sl, hd, ct, tot = rb.reflex_cache_get_state(cache)
     assert tot == [ticks] and ct == [w.N] and hd == [ticks % w.N]
+
+
+def test_gate_for_all_layers_matches_per_layer_calls_and_oracle(U):
+    """reflex_adarmsnorm_gate with L stacked layers == L single-layer calls (bitwise) == the oracle's gamma."""
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"].with_(B=5, L=3)
+    cond = synth.cond_vectors(w, 0.4)
+    Ws = [synth.gate_weights(w, l, std=0.05) for l in range(w.L)]
+    stack = lambda i: U.to_dev(np.stack([Ws[l][i] for l in range(w.L)]), w.dtype)
+    W1s, b1s, W2s, b2s = stack(0), stack(1), stack(2), stack(3)
+    dcond = U.to_dev(cond, w.dtype)
+    all_buf = torch.full((w.L * w.B * (w.D + w.Hd),), float("nan"), dtype=torch.float32, device=U.DEV)
+    rb.reflex_adarmsnorm_gate(dcond, W1s, b1s, W2s, b2s, all_buf)
+    x = synth.norm_input(w, 0, 0)
+    for l in range(w.L):
+        one = torch.full((w.B * (w.D + w.Hd),), float("nan"), dtype=torch.float32, device=U.DEV)
+        rb.reflex_adarmsnorm_gate(dcond, W1s[l], b1s[l], W2s[l], b2s[l], one)
+        g_all = all_buf[l * w.B * w.D:(l + 1) * w.B * w.D]
+        assert torch.equal(g_all, one[: w.B * w.D])
+        for b in (0, 4):
+            _, g = orc.adarmsnorm(x[b], cond[b], *Ws[l], 1e-6, return_gate=True)
+            assert np.max(np.abs(U.to_host(g_all.view(w.B, w.D)[b]) - g)) <= 1e-5
+        # a layer's rows with its slice of the step's gates == the all-in-one call
+        dx = U.to_dev(x, w.dtype)
+        y1, y2 = torch.empty_like(dx), torch.empty_like(dx)
+        rb.reflex_adarmsnorm(dx, y1, None, None, None, None, None, gate_buf=g_all.view(w.B, w.D))
+        rb.reflex_adarmsnorm(dx, y2, dcond, W1s[l], b1s[l], W2s[l], b2s[l], gate_buf=one)
+        assert torch.equal(y1, y2)
+        U.check_close(U.to_host(y1), orc.adarmsnorm_batched(x, cond, *Ws[l], 1e-6), w.dtype, f"rows with step gates, layer {l}", rel_clause=True)
