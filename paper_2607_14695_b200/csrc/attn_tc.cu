@@ -523,7 +523,7 @@ cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtenso
 
 template <int HD>
 cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
-                      const CUtensorMap *mvd, const CUtensorMap *mo, const TcParams &tp, dim3 grid, cudaStream_t st)
+                      const CUtensorMap *mvd, const TcParams &tp, dim3 grid, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -531,7 +531,7 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attn_tc2_kernel<HD><<<grid, kTc2Threads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, *mo, tp);
+    attn_tc2_kernel<HD><<<grid, kTc2Threads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
     count_launch();
     return cudaGetLastError();
 }
@@ -609,16 +609,14 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     if (two_cta) {
         // persistent grid: one cluster (two CTAs) per SM pair walks the (stream, KV head, tile pair) units;
         // an odd tile count leaves the last pair of a stream with one idle half
-        CUtensorMap mo;
-        if (!cache().get(&mo, p.out, 1, (p.B << 16) | p.T, p.Hq, p.d, G, mk_q)) return cudaErrorInvalidValue;
         tp.n_qtiles = (tp.n_qtiles + 1) / 2;
         const int units = tp.n_qtiles * p.Hkv * p.B * p.nsplit;
         int clusters = sm_count / 2;
         if (clusters > units) clusters = units;
         if (clusters < 1) clusters = 1;
         dim3 grid2(2 * clusters, 1, 1);
-        if (p.d == 256) e = launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
-        else if (p.d == 128) e = launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
+        if (p.d == 256) e = launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
+        else if (p.d == 128) e = launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
         else return cudaErrorInvalidValue;
         if (e != cudaSuccess || p.nsplit == 1) return e;
         return launch_attention_merge(p, st);

@@ -12,9 +12,13 @@
 //
 // Per CTA:  warp 0      TMA producer (own Q tile, own K half, own V half)
 //           warp 1      MMA issuer (leader CTA only): S = Q K^T (M256 N128), O += P V (M256 N=d)
-//           warps 2..9  softmax over this CTA's 128 rows x 128 keys: two threads per row (64 keys each),
-//                       P (bf16) into swizzled shared memory, lazy rescale of O in TMEM, and the epilogue:
-//                       O / l staged through shared memory and written with TMA stores
+//           warps 2..   softmax over this CTA's 128 rows x 128 keys: NP threads per row (128 / NP keys each),
+//                       P (bf16) written back into tensor memory over the logits it came from, lazy rescale
+//                       of O in tensor memory, and the epilogue: O / l straight from registers to global memory
+// P never touches shared memory: P V takes its A operand from tensor memory. With head_dim 256 the Q K^T
+// MMAs alone read shared memory at its full bandwidth (a 4 KB slice of Q plus 4 KB of K per 64-cycle
+// instruction), so every byte of shared-memory traffic that is not an operand read or a TMA fill stretches
+// the tensor pipe; the 32 KB a P buffer would take pays for a third V stage instead.
 // Barriers the leader's MMA thread waits on collect both CTAs (TMA completions through cta_group::2 loads,
 // softmax arrivals through shared::cluster arrives); completions fan out with multicast commits.
 // Included by attn_tc.cu (shares its tile geometry and tensor maps).
@@ -32,48 +36,82 @@ namespace reflex {
 #endif
 
 constexpr int kTc2Keys = 128;     // keys per tile = two 64-key halves, one per CTA of the pair
-constexpr int kTc2Threads = 320;  // producer warp, MMA warp, eight softmax warps
+#ifndef REFLEX_TC2_NP
+#define REFLEX_TC2_NP 2
+#endif
+constexpr int kTc2Parts = REFLEX_TC2_NP;            // softmax threads per query row (2 or 4)
+constexpr int kTc2Threads = 64 + 128 * kTc2Parts;   // producer warp, MMA warp, 4 * kTc2Parts softmax warps
+static_assert(kTc2Parts == 2 || kTc2Parts == 4, "softmax threads per row");
+
+// Round a float up to the next bf16 value, as raw upper 16 bits (the softmax threads of a row exchange their
+// maxima in this form: any common reference >= the true maximum serves, and 16 bits keep the exchange area small).
+__device__ __forceinline__ uint32_t bf16_bits_round_up(float x)
+{
+    uint32_t u = __float_as_uint(x);
+    if (!(u >> 31) && (u & 0xFFFFu)) u += 0x10000u;   // positive: towards +inf; negative: truncation already rounds up
+    return u >> 16;
+}
+
+// s[c] = -inf for every key c < K of a slice that `mask` marks dead
+template <int K>
+__device__ __forceinline__ void apply_slice_mask(float (&s)[K], uint64_t mask)
+{
+    const uint32_t lo = (uint32_t)mask, hi = (uint32_t)(mask >> 32);
+#pragma unroll
+    for (int c = 0; c < K; ++c) {
+        const uint32_t w = c < 32 ? lo : hi;
+        if (!(w & (1u << (c & 31)))) s[c] = -INFINITY;
+    }
+}
 
 template <int HD> struct Tc2Smem {
     static constexpr int CH = HD / 64;
     static constexpr int VCH = CH / 2;                          // this CTA's 64-column chunks of head_dim
+    static constexpr int NKS = (HD == 256) ? 2 : 4;             // K stages
+    static constexpr int NVS = (HD == 256) ? 3 : 4;             // V stages (P lives in tensor memory, which pays for the third)
     static constexpr uint32_t Q_BYTES = CH * 128 * 128;
     static constexpr uint32_t K_STAGE = CH * 64 * 128;          // 64 keys x head_dim
     static constexpr uint32_t V_STAGE = VCH * 128 * 128;        // 128 keys x head_dim/2
     static constexpr uint32_t V_HALF = VCH * 64 * 128;          // bytes one 64-key half contributes
-    static constexpr uint32_t P_BYTES = 2 * 128 * 128;          // 128 rows x 128 keys bf16; also the staging area of the epilogue
     static constexpr uint32_t OFF_Q = 0;
     static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
-    static constexpr uint32_t OFF_V = OFF_K + 2 * K_STAGE;
-    static constexpr uint32_t OFF_P = OFF_V + 2 * V_STAGE;
-    static constexpr uint32_t OFF_BAR = OFF_P + P_BYTES;
-    static constexpr uint32_t OFF_XCH = OFF_BAR + 192;              // row max / row sum exchange between the two halves
-    static constexpr uint32_t NEED = OFF_XCH + 2 * 2 * 128 * 4;     // bytes used from the 1024-byte aligned base
-    static constexpr uint32_t TOTAL = 232448;                       // the whole opt-in shared memory of an SM (227 KB)
+    static constexpr uint32_t OFF_V = OFF_K + NKS * K_STAGE;
+    static constexpr uint32_t OFF_BAR = OFF_V + NVS * V_STAGE;
+    static constexpr uint32_t BAR_BYTES = 256;
+    static constexpr uint32_t OFF_XMAX = OFF_BAR + BAR_BYTES;                   // row maxima: 2 buffers x 128 rows x NP 16-bit values
+    static constexpr uint32_t XMAX_BYTES = 2 * 128 * kTc2Parts * 2;
+    static constexpr uint32_t XSUM_BYTES = kTc2Parts * 128 * 4;                 // row sums: NP x 128 rows fp32
+    static constexpr uint32_t TOTAL = 232448;                                   // the whole opt-in shared memory of an SM (227 KB)
+    // the sums get an area of their own when it fits, else they reuse the maxima's (with two more barriers per unit)
+    static constexpr bool XSUM_OWN = OFF_XMAX + XMAX_BYTES + XSUM_BYTES <= TOTAL;
+    static constexpr uint32_t OFF_XSUM = XSUM_OWN ? OFF_XMAX + XMAX_BYTES : OFF_XMAX;
+    static constexpr uint32_t NEED = XSUM_OWN ? OFF_XSUM + XSUM_BYTES
+                                              : OFF_XMAX + (XMAX_BYTES > XSUM_BYTES ? XMAX_BYTES : XSUM_BYTES);   // from the 1024-byte aligned base
+    static_assert(NEED <= TOTAL, "shared memory budget");
+    // mbarrier indices
+    static constexpr int C_QFULL = 0, C_QEMPTY = 1, C_KFULL = 2, C_KEMPTY = C_KFULL + NKS, C_VLAND = C_KEMPTY + NKS,
+                         C_VEMPTY = C_VLAND + NVS, C_SFULL = C_VEMPTY + NVS, C_PFULL = C_SFULL + 2, C_PVDONE = C_PFULL + 1,
+                         C_OFREE = C_PVDONE + 1, C_COUNT = C_OFREE + 1;
+    static_assert(8 * C_COUNT + 8 <= BAR_BYTES, "barrier area");
 };
 
-enum { C_QFULL = 0, C_QEMPTY = 1, C_KFULL = 2, C_KEMPTY = 4, C_VLAND = 6, C_VEMPTY = 8, C_SFULL = 10, C_SEMPTY = 12,
-       C_PFULL = 14, C_PVDONE = 15, C_OFREE = 16, C_COUNT = 17 };
-
-__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3)
-{
-    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
-
+// (18 warps are five on at least one of the four schedulers, whose 16 K registers then allow 96 per thread)
 template <int HD>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTc2Threads, 1)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
-                const __grid_constant__ CUtensorMap tm_vd, const __grid_constant__ CUtensorMap tm_o, const TcParams p)
+                const __grid_constant__ CUtensorMap tm_vd, const TcParams p)
 {
     using L = Tc2Smem<HD>;
-    constexpr int CH = L::CH, VCH = L::VCH;
+    constexpr int CH = L::CH, VCH = L::VCH, NKS = L::NKS, NVS = L::NVS;
+    constexpr int C_QFULL = L::C_QFULL, C_QEMPTY = L::C_QEMPTY, C_KFULL = L::C_KFULL, C_KEMPTY = L::C_KEMPTY, C_VLAND = L::C_VLAND,
+                  C_VEMPTY = L::C_VEMPTY, C_SFULL = L::C_SFULL, C_PFULL = L::C_PFULL, C_PVDONE = L::C_PVDONE, C_OFREE = L::C_OFREE,
+                  C_COUNT = L::C_COUNT;
     constexpr uint32_t kTmemCols = 512;
-    constexpr uint32_t kColO = 0, kColS = HD;  // O: HD fp32 columns; S: 2 x 128 columns
+    // O: HD fp32 columns. S: 2 x 128 fp32 columns; P(j) (bf16, two keys per column) overwrites the first 64 columns of
+    // S(j)'s buffer once every thread of the row has taken its logits out, and is the A operand of P V from there.
+    constexpr uint32_t kColO = 0, kColS = HD;
     static_assert(HD + 2 * kTc2Keys <= 512 && VCH >= 1, "TMEM budget / head_dim split");
-    static_assert(8 * C_COUNT + 8 <= 192, "barrier area");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -128,12 +166,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C_COUNT; ++i) {
-            const bool both = (i == C_SEMPTY || i == C_SEMPTY + 1 || i == C_PFULL || i == C_OFREE);
-            mbar_init(bar(i), both ? 16u : 1u);   // "both": one arrival per softmax warp of either CTA
+            const bool both = (i == C_PFULL || i == C_OFREE);
+            mbar_init(bar(i), both ? (uint32_t)(8 * kTc2Parts) : 1u);   // "both": one arrival per softmax warp of either CTA
         }
         *abort_flag = 0u;
         fence_mbar_init();
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd); prefetch_tmap(&tm_o);
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd);
     }
     if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), kTmemCols);
     tc_fence_before();
@@ -162,46 +200,81 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
-            bool ok = true;
-            int gt = 0, ui = 0;
-            for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
-                const Unit w = load_unit(u);
-                if (w.n_tiles == 0) { --ui; continue; }   // an empty key slice: every role skips it the same way
-                for (int jj = 0; jj < w.n_tiles && ok; ++jj) {
-                    const int gi = gt + jj, st = gi & 1;
-                    const uint32_t ph = (uint32_t)((gi >> 1) - 1) & 1u;
-                    const int h0 = 2 * (w.tile0 + jj), h1 = h0 + 1;
-                    const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
-                    if (gi >= 2) ok = wait(C_KEMPTY + st, ph, 1);
-                    if (!ok) break;
-                    if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
-                    const int myh = h0 + (int)rank;
-                    if (myh < w.H) {
-                        const TileRef tr = w.g.decode(myh);
-                        for (int c = 0; c < CH; ++c)
-                            tma2_load_3d(base + L::OFF_K + st * L::K_STAGE + c * (64 * 128), tr.dyn ? &tm_kd : &tm_k,
-                                         bar(C_KFULL + st) & kPeerBitMask, c * 64, w.kvh, tr.row0);
-                    }
-                    if (jj == 0) {
-                        // this unit's Q tile, once the last Q K^T of the previous unit has drained the buffer
-                        if (ui >= 1) ok = wait(C_QEMPTY, (uint32_t)(ui - 1) & 1u, 14);
-                        if (!ok) break;
-                        if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
-                        for (int c = 0; c < CH; ++c)
-                            tma2_load_4d(base + L::OFF_Q + c * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, c * 64, w.kvh * p.G, w.t0, w.b);
-                    }
-                    if (gi >= 2) ok = wait(C_VEMPTY + st, ph, 2);
-                    if (!ok) break;
-                    mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
-                    for (int hh = h0; hh <= h1; ++hh) {
-                        if (hh >= w.H) break;
-                        const TileRef tr = w.g.decode(hh);
-                        for (int c = 0; c < VCH; ++c)
-                            tma_load_3d(base + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (hh & 1) * (64 * 128), tr.dyn ? &tm_vd : &tm_v,
-                                        bar(C_VLAND + st), ((int)rank * VCH + c) * 64, w.kvh, tr.row0);
-                    }
+            // The loads are issued in the order in which the tensor pipe frees their stages. The MMA thread issues
+            // Q K^T(j+1) before P V(j), so the K stage of tile j+1 (freed by Q K^T(j-1)) comes free before the V stage
+            // of tile j (freed by P V(j-2)): a K cursor runs one tile ahead of a V cursor through the same list of
+            // units, and neither load waits behind a stage that frees later than its own.
+            struct Cursor { int u, ui, jj, g; bool valid; Unit w; };
+            auto settle = [&](Cursor &c) {   // first unit at or after c.u with a non-empty key slice
+                c.valid = false;
+                for (; c.u < n_units; c.u += n_clusters) {
+                    c.w = load_unit(c.u);
+                    if (c.w.n_tiles > 0) { c.valid = true; c.jj = 0; return; }
                 }
-                gt += w.n_tiles;
+            };
+            auto advance = [&](Cursor &c) {
+                ++c.g;
+                if (++c.jj == c.w.n_tiles) { c.u += n_clusters; ++c.ui; settle(c); }
+            };
+            bool ok = true;
+            auto issue_k = [&](const Cursor &c) {
+                const Unit &w = c.w;
+                const int gi = c.g, st = gi % NKS;
+                const uint32_t ph = (uint32_t)(gi / NKS - 1) & 1u;
+                const int h0 = 2 * (w.tile0 + c.jj), h1 = h0 + 1;
+                const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
+                if (c.ui == 0) TC2_TRACE(0, c.jj, 0);
+                if (gi >= NKS) ok = wait(C_KEMPTY + st, ph, 1);
+                if (!ok) return;
+                if (c.ui == 0) TC2_TRACE(0, c.jj, 1);
+                if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
+                const int myh = h0 + (int)rank;
+                if (myh < w.H) {
+                    const TileRef tr = w.g.decode(myh);
+                    for (int ch = 0; ch < CH; ++ch)
+                        tma2_load_3d(base + L::OFF_K + st * L::K_STAGE + ch * (64 * 128), tr.dyn ? &tm_kd : &tm_k,
+                                     bar(C_KFULL + st) & kPeerBitMask, ch * 64, w.kvh, tr.row0);
+                }
+                if (c.jj == 0) {
+                    // this unit's Q tile, once the last Q K^T of the previous unit has drained the buffer
+                    if (c.ui >= 1) ok = wait(C_QEMPTY, (uint32_t)(c.ui - 1) & 1u, 14);
+                    if (!ok) return;
+                    if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
+                    for (int ch = 0; ch < CH; ++ch)
+                        tma2_load_4d(base + L::OFF_Q + ch * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, ch * 64, w.kvh * p.G, w.t0, w.b);
+                }
+            };
+            auto issue_v = [&](const Cursor &c) {
+                const Unit &w = c.w;
+                const int gi = c.g, st = gi % NVS;
+                const uint32_t ph = (uint32_t)(gi / NVS - 1) & 1u;
+                const int h0 = 2 * (w.tile0 + c.jj), h1 = h0 + 1;
+                const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
+                if (gi >= NVS) ok = wait(C_VEMPTY + st, ph, 2);
+                if (!ok) return;
+                if (c.ui == 0) TC2_TRACE(0, c.jj, 2);
+                mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
+                for (int hh = h0; hh <= h1; ++hh) {
+                    if (hh >= w.H) break;
+                    const TileRef tr = w.g.decode(hh);
+                    for (int ch = 0; ch < VCH; ++ch)
+                        tma_load_3d(base + L::OFF_V + st * L::V_STAGE + ch * (128 * 128) + (hh & 1) * (64 * 128), tr.dyn ? &tm_vd : &tm_v,
+                                    bar(C_VLAND + st), ((int)rank * VCH + ch) * 64, w.kvh, tr.row0);
+                }
+            };
+            Cursor ck, cv;
+            ck.u = cluster_id; ck.ui = 0; ck.jj = 0; ck.g = 0;
+            settle(ck);
+            cv = ck;
+            if (ck.valid) { issue_k(ck); advance(ck); }
+            while (cv.valid && ok) {
+                if (ck.valid) {
+                    issue_k(ck);
+                    if (!ok) break;
+                    advance(ck);
+                }
+                issue_v(cv);
+                advance(cv);
             }
         }
     } else if (warp == 1) {
@@ -210,7 +283,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             constexpr uint32_t idesc_qk = umma_idesc_bf16(256, kTc2Keys, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(256, HD, true);
             auto issue_qk = [&](int gi, bool last_of_unit) {
-                const int st = gi & 1, buf = gi & 1;
+                const int st = gi % NKS, buf = gi & 1;
                 const uint32_t d_tmem = tmem_base + kColS + buf * kTc2Keys;
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
@@ -222,19 +295,16 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 umma2_commit_mc(bar(C_SFULL + buf), 3);
                 if (last_of_unit) umma2_commit_mc(bar(C_QEMPTY), 3);   // Q has been read for the last time
             };
-            // wait for the K tile and the S buffer of global tile gi, then issue its Q K^T
+            // wait for the K tile of global tile gi, then issue its Q K^T. Its S buffer needs no wait of its own: the buffer
+            // last held P(gi-2), read by P V(gi-2), which this thread issued earlier and the tensor pipe runs in order.
             auto qk_when_ready = [&](int gi, bool last_of_unit) -> bool {
-                bool ok2 = wait(C_KFULL + (gi & 1), (uint32_t)(gi >> 1) & 1u, 5);
-                if (ok2 && gi >= 2) ok2 = wait(C_SEMPTY + (gi & 1), (uint32_t)((gi >> 1) - 1) & 1u, 6);
-                if (!ok2) return false;
+                if (!wait(C_KFULL + gi % NKS, (uint32_t)(gi / NKS) & 1u, 5)) return false;
                 tc_fence_after();
                 issue_qk(gi, last_of_unit);
                 return true;
             };
             // Q K^T of tile jj+1 is issued before waiting for P(jj): S is double buffered in TMEM, so the tensor pipe works
-            // on the next tile's logits while the softmax threads finish this tile. (Issuing Q K^T two tiles ahead, or in
-            // whichever order inputs arrive, was measured and is slower: with two K stages the extra Q K^T lands in front
-            // of a P V that the softmax threads are waiting for.)
+            // on the next tile's logits while the softmax threads finish this tile.
             bool ok = true;
             int gt = 0, ui = 0;
             for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
@@ -244,42 +314,51 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk_when_ready(gt, n == 1);
                 for (int jj = 0; jj < n && ok; ++jj) {
                     const int gi = gt + jj;
-                    const int st = gi & 1;
+                    const int st = gi % NVS;
+                    if (ui == 0) TC2_TRACE(1, jj, 0);
                     if (jj + 1 < n) {
                         ok = qk_when_ready(gi + 1, jj + 2 == n);
                         if (!ok) break;
                     }
+                    if (ui == 0) TC2_TRACE(1, jj, 1);
                     ok = wait(C_PFULL, (uint32_t)gi & 1u, 8);   // both CTAs: P written, V landed and cleaned
+                    if (ui == 0) TC2_TRACE(1, jj, 2);
                     if (ok && jj == 0 && ui >= 1) ok = wait(C_OFREE, (uint32_t)(ui - 1) & 1u, 15);   // previous O has been read out
                     if (!ok) break;
                     tc_fence_after();
+                    const uint32_t p_tmem = tmem_base + kColS + (gi & 1) * kTc2Keys;
 #pragma unroll
                     for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
-                        const uint32_t a = base + L::OFF_P + (kk >> 2) * (128 * 128) + (kk & 3) * 32;
                         const uint32_t bb = base + L::OFF_V + st * L::V_STAGE + kk * (16 * 128);
-                        umma2_ss(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv,
-                                 (jj > 0 || kk > 0) ? 1u : 0u);
+                        umma2_ts(tmem_base + kColO, p_tmem + kk * 8, umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
                     }
                     umma2_commit_mc(bar(C_VEMPTY + st), 3);
                     umma2_commit_mc(bar(C_PVDONE), 3);
+                    if (ui == 0) TC2_TRACE(1, jj, 3);
                 }
                 gt += n;
             }
         }
     } else {
         // ---------------- softmax / correction / epilogue (both CTAs) ----------------
-        // Eight warps: two threads per query row, one per 64-key half of the tile (warps 2..5 take the pair
-        // leader's keys, warps 6..9 the partner's). The halves meet once per tile to agree on the row maximum.
-        // A wait that ran out never leaves these loops: every softmax warp keeps meeting the others at the named
-        // barrier (the remaining waits return at once), so no warp is left behind.
+        // 4 * NP warps: NP threads per query row, one per KT-key slice of the 128-key tile (slice `part`; a warp's TMEM
+        // lane quarter fixes which 32 rows it serves). The threads of a row meet once per tile to agree on the row
+        // maximum. A wait that ran out never leaves these loops: every softmax warp keeps meeting the others at the
+        // named barrier (the remaining waits return at once), so no warp is left behind.
+        constexpr int NP = kTc2Parts, KT = kTc2Keys / NP, SMT = 128 * NP;
+        constexpr uint64_t kSliceFull = (KT == 64) ? ~0ull : ((1ull << (KT & 63)) - 1ull);
         const int sw = warp - 2;
-        const int half = sw >> 2;                 // which 64 columns of S / 64-key chunk of P / half of O's columns
+        const int part = sw >> 2;                 // which KT-key slice of the tile
+        const int half = (part * KT) >> 6;        // the 64-key half (one CTA's K rows) that slice lies in
+        const int koff = (part * KT) & 63;        // first key of the slice inside its half
         const int quarter = warp & 3;             // TMEM lane quarter this warp may touch
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const uint32_t leader_pfull = mapa(bar(C_PFULL), 0);
         const uint32_t leader_ofree = mapa(bar(C_OFREE), 0);
-        float *exch = reinterpret_cast<float *>(smem + L::OFF_XCH);   // [2 buffers][2 halves][128 rows]
+        uint16_t *xmax = reinterpret_cast<uint16_t *>(smem + L::OFF_XMAX);   // [2 buffers][128 rows][NP], bf16 bit patterns
+        float *xsum = reinterpret_cast<float *>(smem + L::OFF_XSUM);         // [NP][128 rows]
+        __nv_bfloat16 *out_bf = reinterpret_cast<__nv_bfloat16 *>(p.out);
         bool ok = true;
         int gt = 0;
         [[maybe_unused]] int ui_s = 0;
@@ -293,14 +372,15 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (p.nsplit > 1 && t_row < p.T)
                 pml = partial_ml(p.partials, n_slots, partial_slot(w.b, rows_total, t_row * p.Hq + w.kvh * p.G + row % p.G, p.nsplit, w.split), HD);
             if (w.n_tiles == 0) {
-                if (pml && half == 0) { pml[0] = -INFINITY; pml[1] = 0.f; }   // an empty key slice contributes nothing
+                if (pml && part == 0) { pml[0] = -INFINITY; pml[1] = 0.f; }   // an empty key slice contributes nothing
                 continue;
             }
             float m_ref = -INFINITY, l = 0.f;
             for (int jj = 0; jj < w.n_tiles; ++jj) {
-                const int gi = gt + jj, buf = gi & 1, st = gi & 1;
+                const int gi = gt + jj, buf = gi & 1, st = gi % NVS;
+                const uint32_t vph = (uint32_t)(gi / NVS) & 1u;
                 const int h = 2 * (w.tile0 + jj) + half;
-                uint64_t tmask = 0ull, rmask = 0ull;
+                uint64_t tmask = 0ull, rmask = 0ull;   // liveness of the 64 keys of this half: for every row / for this row
                 if (h < w.H) {
                     const TileRef tr = w.g.decode(h);
                     tmask = w.g.tile_mask(tr);
@@ -310,30 +390,29 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
                     }
                 }
+                const uint64_t smask = (rmask >> koff) & kSliceFull;   // this thread's KT keys
 #define SM_EV(ev) do { if (threadIdx.x == 64 && ui_s == 0) TC2_TRACE(3, jj, ev); } while (0)
                 SM_EV(0);
                 ok = ok && wait(C_SFULL + buf, (uint32_t)(gi >> 1) & 1u, 9);
                 SM_EV(1);
                 if (threadIdx.x == 64 && jj == 0) TC2_TRACE(2, ui_s, 1);
                 tc_fence_after();
-                float s[64];
+                float s[KT];
                 {
-                    const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + half * 64;
-                    uint32_t r0[32], r1[32];
-                    tmem_ld32(s_addr, r0); tmem_ld32(s_addr + 32, r1);
+                    const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + part * KT;
+                    uint32_t r[KT];
+#pragma unroll
+                    for (int q = 0; q < KT / 32; ++q) tmem_ld32(s_addr + 32 * q, *reinterpret_cast<uint32_t(*)[32]>(r + 32 * q));
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(r0[c]); s[32 + c] = __uint_as_float(r1[c]); }
+                    for (int c = 0; c < KT; ++c) s[c] = __uint_as_float(r[c]);
                 }
                 SM_EV(2);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(mapa(bar(C_SEMPTY + buf), 0));
                 if (tmask != ~0ull) {
                     // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows as soon
                     // as this CTA's V half has landed (long before the P V that reads them)
-                    ok = ok && wait(C_VLAND + st, (uint32_t)(gi >> 1) & 1u, 12);
-                    if (row < 64 && !((tmask >> row) & 1ull)) {
+                    ok = ok && wait(C_VLAND + st, vph, 12);
+                    if (koff == 0 && row < 64 && !((tmask >> row) & 1ull)) {
 #pragma unroll
                         for (int c = 0; c < VCH; ++c) {
                             uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (half * 64 + row) * 128);
@@ -342,40 +421,43 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
-                if (rmask != ~0ull) apply_key_mask(s, rmask);
+                if (smask != kSliceFull) apply_slice_mask<KT>(s, smask);
                 float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
-                for (int c = 4; c < 64; c += 4) {
+                for (int c = 4; c < KT; c += 4) {
                     mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
                     mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
                 }
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                // meet the thread that holds the other 64 keys of this row (thread 64 first makes sure that the TMA stores of
-                // the previous unit have read the staging area, which is the P buffer every thread writes after this barrier)
+                // meet the threads that hold the other keys of this row: every one of them publishes its maximum rounded up
+                // to bf16 and takes the largest of the NP published values, so all agree. Past this barrier every thread of the
+                // row has its logits in registers, so P may overwrite them in tensor memory.
                 SM_EV(3);
-                exch[(buf * 2 + half) * 128 + row] = mx;
-                if (jj == 0 && threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                xmax[(buf * 128 + row) * NP + part] = (uint16_t)bf16_bits_round_up(mx);
+                asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
                 SM_EV(4);
-                mx = fmaxf(mx, exch[(buf * 2 + (half ^ 1)) * 128 + row]);
-                bool pv_waited = false;
+                {
+                    const uint16_t *xr = xmax + (buf * 128 + row) * NP;
+                    mx = -INFINITY;
+#pragma unroll
+                    for (int q = 0; q < NP; ++q) mx = fmaxf(mx, __uint_as_float((uint32_t)xr[q] << 16));
+                }
                 if (jj == 0) {
                     m_ref = mx;
                 } else {
                     const bool grow = (mx - m_ref) * p.scale_log2 > kRescaleThreshold;
                     if (__any_sync(0xffffffffu, grow)) {
                         // O (and l) were accumulated against m_ref: bring them to the new reference before this tile's P V.
-                        // Both threads of a row see the same mx, so they decide alike; each rescales its half of O's columns.
+                        // All threads of a row see the same mx, so they decide alike; each rescales its share of O's columns.
                         const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
                         if (grow) m_ref = mx;
                         l *= alpha;
                         ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 10);
-                        pv_waited = true;
                         tc_fence_after();
 #pragma unroll 1
-                        for (int c = 0; c < HD / 64; ++c) {
+                        for (int c = 0; c < HD / NP / 32; ++c) {
                             uint32_t o[32];
-                            const uint32_t o_addr = tmem_base + lane_addr + kColO + half * (HD / 2) + c * 32;
+                            const uint32_t o_addr = tmem_base + lane_addr + kColO + part * (HD / NP) + c * 32;
                             tmem_ld32(o_addr, o);
                             tmem_wait_ld();
 #pragma unroll
@@ -387,9 +469,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
                 float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t packed[32];
+                uint32_t packed[KT / 2];
 #pragma unroll
-                for (int c = 0; c < 64; c += 2) {
+                for (int c = 0; c < KT; c += 2) {
                     // P = 2^(s*scale*log2e - m). One pair in four takes the FMA-pipe exponential so the MUFU unit and the
                     // FMA pipe share the load.
                     const float x0 = fmaf(s[c], p.scale_log2, -mr), x1 = fmaf(s[c + 1], p.scale_log2, -mr);
@@ -402,19 +484,24 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
                 SM_EV(5);
-                if (gi >= 1 && !pv_waited)
-                    ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 11);  // the single P buffer was read by the previous P V
-                SM_EV(6);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint8_t *dst = smem + L::OFF_P + half * (128 * 128) + row * 128 + ((c ^ (row & 7)) << 4);
-                    *reinterpret_cast<uint4 *>(dst) = make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+                // P goes into the first 64 columns of S's buffer (two keys per column): the A operand of this tile's P V.
+                // (No wait for an earlier P V: the one that read this buffer, two tiles back, was issued before the Q K^T
+                // that produced the logits just consumed.)
+                {
+                    const uint32_t p_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + part * (KT / 2);
+                    if constexpr (KT == 64) tmem_st32(p_addr, *reinterpret_cast<const uint32_t(*)[32]>(packed));
+                    else tmem_st16(p_addr, *reinterpret_cast<const uint32_t(*)[16]>(packed));
+                    tmem_wait_st();
                 }
                 SM_EV(7);
+                // Every phase of the P V barrier is observed, one per tile, although nothing here depends on the previous
+                // P V any more: a parity wait tells "this phase" from "the next" only for a waiter that never falls two
+                // phases behind, and the waits that do matter (rescaling O, reading O out) come at irregular times.
+                if (gi >= 1) ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 11);
                 // the arrive below also tells the leader that this CTA's V half is in place
-                if (tmask == ~0ull) ok = ok && wait(C_VLAND + st, (uint32_t)(gi >> 1) & 1u, 12);
+                if (tmask == ~0ull) ok = ok && wait(C_VLAND + st, vph, 12);
                 SM_EV(8);
-                fence_proxy_async_smem();
+                fence_proxy_async_smem();   // V rows cleared above are read by the tensor pipe
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(leader_pfull);
@@ -422,99 +509,69 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             gt += w.n_tiles;
             // ---- epilogue of the unit ----
-            // The two threads of a row add their sums; each thread normalises its half of the head_dim columns, 64 at a
-            // time, into the (now idle) P buffer laid out like a Q tile, and one thread hands the tile to TMA stores.
+            // The threads of a row add their sums; each thread takes its share of the head_dim columns out of tensor
+            // memory, 32 at a time, and stores its row segment straight to global memory in 32-byte pieces (whole sectors).
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 2); TC2_TRACE(2, ui_s, 2); }
             const int g_last = gt - 1;
             ok = ok && wait(C_PVDONE, (uint32_t)g_last & 1u, 13);
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 3); TC2_TRACE(2, ui_s, 3); }
-            const int xb = (g_last + 1) & 1;
-            exch[(xb * 2 + half) * 128 + row] = l;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            l += exch[(xb * 2 + (half ^ 1)) * 128 + row];
+            if constexpr (!L::XSUM_OWN) asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // the maxima of the last tile have been read
+            xsum[part * 128 + row] = l;
+            asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
+#pragma unroll
+            for (int q = 1; q < NP; ++q) l += xsum[((part + q) % NP) * 128 + row];
+            if constexpr (!L::XSUM_OWN) asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // ... and the sums, before new maxima land there
             tc_fence_after();
+            const bool row_live = t_row < p.T;
+            const int hq = w.kvh * p.G + row % p.G;
+            constexpr int EC = HD / NP;            // this thread's columns of O
             if (p.nsplit > 1) {
-                // key-split unit: leave (m, l, unnormalised O) for the merge kernel; m in natural-log units like the other
-                // kernels. O goes out 32 columns per thread at a time through the idle P buffer (fp32, swizzled 128-byte
-                // rows), so that the global stores are whole 128-byte row segments instead of one scattered row per lane.
-                if (pml && half == 0) { pml[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; pml[1] = l; }
+                // key-split unit: leave (m, l, unnormalised O) for the merge kernel; m in natural-log units like the other kernels
+                if (pml && part == 0) { pml[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; pml[1] = l; }
+                float *po = row_live ? partial_o(p.partials, partial_slot(w.b, rows_total, t_row * p.Hq + hq, p.nsplit, w.split), HD) + part * EC : nullptr;
 #pragma unroll 1
-                for (int sub = 0; sub < HD / 64; ++sub) {
+                for (int c = 0; c < EC / 32; ++c) {
                     uint32_t o[32];
-                    tmem_ld32(tmem_base + lane_addr + kColO + half * (HD / 2) + sub * 32, o);
+                    tmem_ld32(tmem_base + lane_addr + kColO + part * EC + c * 32, o);
                     tmem_wait_ld();
-                    if (sub == HD / 64 - 1) {
+                    if (c == EC / 32 - 1) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(leader_ofree);
                     }
-                    uint8_t *srow = smem + L::OFF_P + half * (128 * 128) + row * 128;
+                    if (row_live) {
 #pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
-                    const int tid = threadIdx.x - 64;
-#pragma unroll
-                    for (int it = 0; it < 8; ++it) {
-                        const int idx = it * 256 + tid;
-                        const int hh = idx >> 10, rr = (idx >> 3) & 127, cc = idx & 7;
-                        const int tt = w.t0 + rr / p.G;
-                        if (tt < p.T) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(smem + L::OFF_P + hh * (128 * 128) + rr * 128 + ((cc ^ (rr & 7)) << 4));
-                            float *dst = partial_o(p.partials, partial_slot(w.b, rows_total, tt * p.Hq + w.kvh * p.G + rr % p.G, p.nsplit, w.split), HD) +
-                                         hh * (HD / 2) + sub * 32 + cc * 4;
-                            *reinterpret_cast<uint4 *>(dst) = v;
-                        }
+                        for (int i = 0; i < 4; ++i) st_global_v8(po + c * 32 + 8 * i, *reinterpret_cast<const uint32_t(*)[8]>(o + 8 * i));
                     }
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
                 }
                 continue;
             }
             const float inv = 1.f / l;
-            const bool store_unit = w.t0 < p.T;   // an idle partner tile (odd tile count) has nothing to write
+            __nv_bfloat16 *orow = row_live ? out_bf + (((size_t)w.b * p.T + t_row) * p.Hq + hq) * HD + part * EC : nullptr;
 #pragma unroll 1
-            for (int rnd = 0; rnd < HD / 128; ++rnd) {
-                uint32_t o0[32], o1[32];
-                const uint32_t o_addr = tmem_base + lane_addr + kColO + half * (HD / 2) + rnd * 64;
-                tmem_ld32(o_addr, o0); tmem_ld32(o_addr + 32, o1);
+            for (int c = 0; c < EC / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem_base + lane_addr + kColO + part * EC + c * 32, o);
                 tmem_wait_ld();
-                if (rnd == HD / 128 - 1) {
+                if (c == EC / 32 - 1) {
                     // all of O is in registers: the next unit's first P V may overwrite the accumulator
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(leader_ofree);
                 }
-                uint8_t *srow = smem + L::OFF_P + half * (128 * 128) + row * 128;
+                uint32_t pk[16];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t *src = (c < 4) ? (o0 + 8 * c) : (o1 + 8 * (c - 4));
-                    uint4 v;
-                    uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(src[2 * k]) * inv, __uint_as_float(src[2 * k + 1]) * inv);
-                        vv[k] = *reinterpret_cast<uint32_t *>(&hh);
-                    }
-                    *reinterpret_cast<uint4 *>(srow + ((c ^ (row & 7)) << 4)) = v;
+                for (int k = 0; k < 16; ++k) {
+                    __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[2 * k]) * inv, __uint_as_float(o[2 * k + 1]) * inv);
+                    pk[k] = *reinterpret_cast<uint32_t *>(&hh);
                 }
-                fence_proxy_async_smem();
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (threadIdx.x == 64) {
-                    if (store_unit) {
-#pragma unroll
-                        for (int hh = 0; hh < 2; ++hh)
-                            tma_store_4d(&tm_o, base + L::OFF_P + hh * (128 * 128), hh * (HD / 2) + rnd * 64, w.kvh * p.G, w.t0, w.b);
-                    }
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    // before the staging area is rewritten the store must have read it: at once between rounds, but after
-                    // the last round only when the next unit is about to write P (see the top of the tile loop)
-                    if (rnd + 1 < HD / 128) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (row_live) {
+                    st_global_v8(orow + c * 32, *reinterpret_cast<const uint32_t(*)[8]>(pk));
+                    st_global_v8(orow + c * 32 + 16, *reinterpret_cast<const uint32_t(*)[8]>(pk + 8));
                 }
-                if (rnd + 1 < HD / 128) asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 4); TC2_TRACE(2, ui_s, 4); }
         }
-        if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores of this CTA are complete
     }
 
     tc_fence_before();
