@@ -90,8 +90,8 @@ template <int HD> struct Tc2Smem {
     static_assert(NEED <= TOTAL, "shared memory budget");
     // mbarrier indices
     static constexpr int C_QFULL = 0, C_QEMPTY = 1, C_KFULL = 2, C_KEMPTY = C_KFULL + NKS, C_VLAND = C_KEMPTY + NKS,
-                         C_VEMPTY = C_VLAND + NVS, C_SFULL = C_VEMPTY + NVS, C_PFULL = C_SFULL + 2, C_PVDONE = C_PFULL + 1,
-                         C_OFREE = C_PVDONE + 1, C_COUNT = C_OFREE + 1;
+                         C_VEMPTY = C_VLAND + NVS, C_SFULL = C_VEMPTY + NVS, C_PFULL = C_SFULL + 2, C_PVDONE = C_PFULL + 2,
+                         C_OFREE = C_PVDONE + 2, C_COUNT = C_OFREE + 1;   // P V completion: one barrier per S/P buffer
     static_assert(8 * C_COUNT + 8 <= BAR_BYTES, "barrier area");
 };
 
@@ -166,7 +166,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C_COUNT; ++i) {
-            const bool both = (i == C_PFULL || i == C_OFREE);
+            const bool both = (i == C_PFULL || i == C_PFULL + 1 || i == C_OFREE);
             mbar_init(bar(i), both ? (uint32_t)(8 * kTc2Parts) : 1u);   // "both": one arrival per softmax warp of either CTA
         }
         *abort_flag = 0u;
@@ -279,11 +279,20 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA) ----------------
+        // Q K^T of tile j+1 is issued before waiting for P(j): S is double buffered in TMEM, so the tensor pipe works on the
+        // next tile's logits while the softmax threads finish this tile. S(j+2) overwrites the buffer that held P(j); the MMAs
+        // of one thread run in issue order, and Q K^T(j+2) is issued after P V(j), so the pipe itself keeps that hazard away.
+        // (Two issuing threads in two warps, one per kind of MMA with the hazard made explicit by a completion barrier, were
+        // measured 3 % slower: Q K^T(j+2) then starts a P V latency later. This thread shares its scheduler with two softmax
+        // warps and is short of issue slots whenever they run dense arithmetic; a stand-alone issue loop beside pure-FMA
+        // warps took 600 cycles per MMA instead of 65.)
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(256, kTc2Keys, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(256, HD, true);
-            auto issue_qk = [&](int gi, bool last_of_unit) {
+            auto qk = [&](int gi, bool last) -> bool {
                 const int st = gi % NKS, buf = gi & 1;
+                if (!wait(C_KFULL + st, (uint32_t)(gi / NKS) & 1u, 5)) return false;
+                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + kColS + buf * kTc2Keys;
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
@@ -293,48 +302,31 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 umma2_commit_mc(bar(C_KEMPTY + st), 3);
                 umma2_commit_mc(bar(C_SFULL + buf), 3);
-                if (last_of_unit) umma2_commit_mc(bar(C_QEMPTY), 3);   // Q has been read for the last time
-            };
-            // wait for the K tile of global tile gi, then issue its Q K^T. Its S buffer needs no wait of its own: the buffer
-            // last held P(gi-2), read by P V(gi-2), which this thread issued earlier and the tensor pipe runs in order.
-            auto qk_when_ready = [&](int gi, bool last_of_unit) -> bool {
-                if (!wait(C_KFULL + gi % NKS, (uint32_t)(gi / NKS) & 1u, 5)) return false;
-                tc_fence_after();
-                issue_qk(gi, last_of_unit);
+                if (last) umma2_commit_mc(bar(C_QEMPTY), 3);
                 return true;
             };
-            // Q K^T of tile jj+1 is issued before waiting for P(jj): S is double buffered in TMEM, so the tensor pipe works
-            // on the next tile's logits while the softmax threads finish this tile.
             bool ok = true;
             int gt = 0, ui = 0;
             for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
                 const Unit w = load_unit(u);
                 const int n = w.n_tiles;
                 if (n == 0) { --ui; continue; }
-                ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk_when_ready(gt, n == 1);
+                ok = wait(C_QFULL, (uint32_t)ui & 1u, 3) && qk(gt, n == 1);
                 for (int jj = 0; jj < n && ok; ++jj) {
-                    const int gi = gt + jj;
-                    const int st = gi % NVS;
-                    if (ui == 0) TC2_TRACE(1, jj, 0);
-                    if (jj + 1 < n) {
-                        ok = qk_when_ready(gi + 1, jj + 2 == n);
-                        if (!ok) break;
-                    }
-                    if (ui == 0) TC2_TRACE(1, jj, 1);
-                    ok = wait(C_PFULL, (uint32_t)gi & 1u, 8);   // both CTAs: P written, V landed and cleaned
-                    if (ui == 0) TC2_TRACE(1, jj, 2);
-                    if (ok && jj == 0 && ui >= 1) ok = wait(C_OFREE, (uint32_t)(ui - 1) & 1u, 15);   // previous O has been read out
+                    const int gi = gt + jj, st = gi % NVS, buf = gi & 1;
+                    if (jj + 1 < n) { ok = qk(gi + 1, jj + 2 == n); if (!ok) break; }
+                    ok = wait(C_PFULL + buf, (uint32_t)(gi >> 1) & 1u, 8);
+                    if (ok && jj == 0 && ui >= 1) ok = wait(C_OFREE, (uint32_t)(ui - 1) & 1u, 15);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t p_tmem = tmem_base + kColS + (gi & 1) * kTc2Keys;
+                    const uint32_t p_tmem = tmem_base + kColS + buf * kTc2Keys;
 #pragma unroll
                     for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
                         const uint32_t bb = base + L::OFF_V + st * L::V_STAGE + kk * (16 * 128);
                         umma2_ts(tmem_base + kColO, p_tmem + kk * 8, umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
                     }
                     umma2_commit_mc(bar(C_VEMPTY + st), 3);
-                    umma2_commit_mc(bar(C_PVDONE), 3);
-                    if (ui == 0) TC2_TRACE(1, jj, 3);
+                    umma2_commit_mc(bar(C_PVDONE + buf), 3);
                 }
                 gt += n;
             }
@@ -354,7 +346,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int quarter = warp & 3;             // TMEM lane quarter this warp may touch
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        const uint32_t leader_pfull = mapa(bar(C_PFULL), 0);
+        const uint32_t leader_pfull[2] = {mapa(bar(C_PFULL), 0), mapa(bar(C_PFULL + 1), 0)};
         const uint32_t leader_ofree = mapa(bar(C_OFREE), 0);
         uint16_t *xmax = reinterpret_cast<uint16_t *>(smem + L::OFF_XMAX);   // [2 buffers][128 rows][NP], bf16 bit patterns
         float *xsum = reinterpret_cast<float *>(smem + L::OFF_XSUM);         // [NP][128 rows]
@@ -422,11 +414,17 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 if (smask != kSliceFull) apply_slice_mask<KT>(s, smask);
+                // three-input maxima: half the instructions of a two-input chain (the single MMA-issuing thread shares its
+                // scheduler with two of these warps, and every issue slot they do not take is one it can have)
                 float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
-                for (int c = 4; c < KT; c += 4) {
-                    mx4[0] = fmaxf(mx4[0], s[c]); mx4[1] = fmaxf(mx4[1], s[c + 1]);
-                    mx4[2] = fmaxf(mx4[2], s[c + 2]); mx4[3] = fmaxf(mx4[3], s[c + 3]);
+                for (int c = 4; c + 7 < KT; c += 8) {
+                    mx4[0] = max3_f32(mx4[0], s[c], s[c + 1]); mx4[1] = max3_f32(mx4[1], s[c + 2], s[c + 3]);
+                    mx4[2] = max3_f32(mx4[2], s[c + 4], s[c + 5]); mx4[3] = max3_f32(mx4[3], s[c + 6], s[c + 7]);
+                }
+                static_assert((KT - 4) % 8 == 4 || (KT - 4) % 8 == 0, "tail of the maximum loop");
+                if constexpr ((KT - 4) % 8 == 4) {
+                    mx4[0] = max3_f32(mx4[0], s[KT - 4], s[KT - 3]); mx4[1] = max3_f32(mx4[1], s[KT - 2], s[KT - 1]);
                 }
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // meet the threads that hold the other keys of this row: every one of them publishes its maximum rounded up
@@ -452,7 +450,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         const float alpha = grow ? ex2((m_ref - mx) * p.scale_log2) : 1.f;
                         if (grow) m_ref = mx;
                         l *= alpha;
-                        ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 10);
+                        ok = ok && wait(C_PVDONE + ((gi - 1) & 1), (uint32_t)((gi - 1) >> 1) & 1u, 10);
                         tc_fence_after();
 #pragma unroll 1
                         for (int c = 0; c < HD / NP / 32; ++c) {
@@ -468,21 +466,27 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
-                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                // P = 2^(s*scale*log2e - m), two keys per instruction wherever the hardware has a packed form (the scaling FMA
+                // and the running sums); the exponentials themselves all go to the MUFU unit. Emulating a share of them on the
+                // FMA pipe shortens this loop in isolation but fills the issue slots the MMA thread needs: measured slower.
+                SM_EV(6);
+                const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(-mr, -mr);
+                uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
                 uint32_t packed[KT / 2];
 #pragma unroll
                 for (int c = 0; c < KT; c += 2) {
-                    // P = 2^(s*scale*log2e - m). One pair in four takes the FMA-pipe exponential so the MUFU unit and the
-                    // FMA pipe share the load.
-                    const float x0 = fmaf(s[c], p.scale_log2, -mr), x1 = fmaf(s[c + 1], p.scale_log2, -mr);
-                    const bool on_fma = ((c >> 1) & 3) == 3;
-                    const float p0 = on_fma ? ex2_fma(x0) : ex2(x0);
-                    const float p1 = on_fma ? ex2_fma(x1) : ex2(x1);
-                    sum4[(c >> 1) & 3] += p0 + p1;
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(s[c], s[c + 1]), sc2, nm2), x0, x1);
+                    const float p0 = ex2(x0), p1 = ex2(x1);
+                    sum2[(c >> 1) & 3] = add_f32x2(sum2[(c >> 1) & 3], pack_f32x2(p0, p1));
                     __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
                 }
-                l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                {
+                    float a, b;
+                    unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), a, b);
+                    l += a + b;
+                }
                 SM_EV(5);
                 // P goes into the first 64 columns of S's buffer (two keys per column): the A operand of this tile's P V.
                 // (No wait for an earlier P V: the one that read this buffer, two tiles back, was issued before the Q K^T
@@ -494,17 +498,18 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tmem_wait_st();
                 }
                 SM_EV(7);
-                // Every phase of the P V barrier is observed, one per tile, although nothing here depends on the previous
-                // P V any more: a parity wait tells "this phase" from "the next" only for a waiter that never falls two
-                // phases behind, and the waits that do matter (rescaling O, reading O out) come at irregular times.
-                if (gi >= 1) ok = ok && wait(C_PVDONE, (uint32_t)(gi - 1) & 1u, 11);
+                // (The waits on a P V barrier, one barrier per S/P buffer, come at irregular times: before rescaling O and before
+                // reading O out. Their parity test stays unambiguous because S(g) exists only after P V(g-2) completed, so the
+                // barrier of tile g-1 has finished the phase of tile g-3 and cannot have passed that of tile g+1.)
                 // the arrive below also tells the leader that this CTA's V half is in place
                 if (tmask == ~0ull) ok = ok && wait(C_VLAND + st, vph, 12);
                 SM_EV(8);
                 fence_proxy_async_smem();   // V rows cleared above are read by the tensor pipe
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(leader_pfull);
+                // (one barrier per S/P buffer: the two CTAs' softmax warps are not synchronised with each other, and on a single
+                // barrier a CTA one tile ahead would complete this tile's phase with its arrivals for the next)
+                if (lane == 0) mbar_arrive_cluster(leader_pfull[buf]);
                 SM_EV(9);
             }
             gt += w.n_tiles;
@@ -513,7 +518,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // memory, 32 at a time, and stores its row segment straight to global memory in 32-byte pieces (whole sectors).
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 2); TC2_TRACE(2, ui_s, 2); }
             const int g_last = gt - 1;
-            ok = ok && wait(C_PVDONE, (uint32_t)g_last & 1u, 13);
+            ok = ok && wait(C_PVDONE + (g_last & 1), (uint32_t)(g_last >> 1) & 1u, 13);
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 3); TC2_TRACE(2, ui_s, 3); }
             if constexpr (!L::XSUM_OWN) asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // the maxima of the last tile have been read
             xsum[part * 128 + row] = l;
@@ -522,6 +527,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int q = 1; q < NP; ++q) l += xsum[((part + q) % NP) * 128 + row];
             if constexpr (!L::XSUM_OWN) asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // ... and the sums, before new maxima land there
             tc_fence_after();
+            if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 5);
             const bool row_live = t_row < p.T;
             const int hq = w.kvh * p.G + row % p.G;
             constexpr int EC = HD / NP;            // this thread's columns of O
@@ -565,10 +571,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[2 * k]) * inv, __uint_as_float(o[2 * k + 1]) * inv);
                     pk[k] = *reinterpret_cast<uint32_t *>(&hh);
                 }
+                if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 6 + 2 * c);
                 if (row_live) {
                     st_global_v8(orow + c * 32, *reinterpret_cast<const uint32_t(*)[8]>(pk));
                     st_global_v8(orow + c * 32 + 16, *reinterpret_cast<const uint32_t(*)[8]>(pk + 8));
                 }
+                if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 7 + 2 * c);
             }
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 4); TC2_TRACE(2, ui_s, 4); }
         }
