@@ -289,16 +289,21 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(256, kTc2Keys, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(256, HD, true);
+            const uint64_t qdesc0 = umma_desc_sw128(base + L::OFF_Q, 16, 1024), kdesc0 = umma_desc_sw128(base + L::OFF_K, 16, 1024);
+            const uint64_t vdesc0 = umma_desc_sw128(base + L::OFF_V, 128 * 128, 1024);
             auto qk = [&](int gi, bool last) -> bool {
                 const int st = gi % NKS, buf = gi & 1;
                 if (!wait(C_KFULL + st, (uint32_t)(gi / NKS) & 1u, 5)) return false;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + kColS + buf * kTc2Keys;
+                uint64_t qd = qdesc0, kd = kdesc0;
+                umma_desc_advance(kd, (uint32_t)st * L::K_STAGE);
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t a = base + L::OFF_Q + (kk >> 2) * (128 * 128) + (kk & 3) * 32;
-                    const uint32_t bb = base + L::OFF_K + st * L::K_STAGE + (kk >> 2) * (64 * 128) + (kk & 3) * 32;
-                    umma2_ss(d_tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+                    umma2_ss(d_tmem, qd, kd, idesc_qk, kk > 0 ? 1u : 0u);
+                    // next 16 columns of head_dim: 32 bytes on inside a 64-column chunk, else on to the next chunk
+                    umma_desc_advance(qd, (kk & 3) == 3 ? 128 * 128 - 96 : 32);
+                    umma_desc_advance(kd, (kk & 3) == 3 ? 64 * 128 - 96 : 32);
                 }
                 umma2_commit_mc(bar(C_KEMPTY + st), 3);
                 umma2_commit_mc(bar(C_SFULL + buf), 3);
@@ -320,10 +325,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t p_tmem = tmem_base + kColS + buf * kTc2Keys;
+                    uint64_t vd = vdesc0;
+                    umma_desc_advance(vd, (uint32_t)st * L::V_STAGE);
 #pragma unroll
                     for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
-                        const uint32_t bb = base + L::OFF_V + st * L::V_STAGE + kk * (16 * 128);
-                        umma2_ts(tmem_base + kColO, p_tmem + kk * 8, umma_desc_sw128(bb, 128 * 128, 1024), idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
+                        umma2_ts(tmem_base + kColO, p_tmem + kk * 8, vd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
+                        umma_desc_advance(vd, 16 * 128);   // the next 16 keys
                     }
                     umma2_commit_mc(bar(C_VEMPTY + st), 3);
                     umma2_commit_mc(bar(C_PVDONE + buf), 3);
@@ -402,7 +409,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 SM_EV(2);
                 if (tmask != ~0ull) {
                     // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows as soon
-                    // as this CTA's V half has landed (long before the P V that reads them)
+                    // as this CTA's V half has landed. (Doing it at the end of the tile, where every thread waits for V anyway,
+                    // puts the clearing stores and their proxy fence in front of the P-ready arrival: measured slower.)
                     ok = ok && wait(C_VLAND + st, vph, 12);
                     if (koff == 0 && row < 64 && !((tmask >> row) & 1ull)) {
 #pragma unroll

@@ -87,6 +87,17 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
     return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
+// Moves the start address of a shared-memory descriptor by `bytes` (a multiple of 16 that keeps the address inside the
+// 256 KB the 14-bit field covers): one 32-bit add on the low word, in place. The thread that issues MMAs competes for issue
+// slots with the warps doing the arithmetic, so each instruction between two MMAs counts.
+__device__ __forceinline__ void umma_desc_advance(uint64_t &desc, uint32_t bytes)
+{
+    asm("{\n\t.reg .b32 lo, hi;\n\t"
+        "mov.b64 {lo, hi}, %0;\n\t"
+        "add.u32 lo, lo, %1;\n\t"
+        "mov.b64 %0, {lo, hi};\n\t}"
+        : "+l"(desc) : "r"(bytes >> 4));
+}
 // Instruction descriptor: D fp32, A/B bf16, optional MN-major B.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool b_mn_major)
 {
