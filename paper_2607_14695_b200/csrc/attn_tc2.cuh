@@ -286,7 +286,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // measured 3 % slower: Q K^T(j+2) then starts a P V latency later. This thread shares its scheduler with two softmax
         // warps and is short of issue slots whenever they run dense arithmetic; a stand-alone issue loop beside pure-FMA
         // warps took 600 cycles per MMA instead of 65.)
-        if (lane == 0 && rank == 0) {
+        // The whole warp runs these loops converged and one elected lane issues (see umma2_ss_elect).
+        if (rank == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(256, kTc2Keys, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(256, HD, true);
             const uint64_t qdesc0 = umma_desc_sw128(base + L::OFF_Q, 16, 1024), kdesc0 = umma_desc_sw128(base + L::OFF_K, 16, 1024);
@@ -300,14 +301,14 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 umma_desc_advance(kd, (uint32_t)st * L::K_STAGE);
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
-                    umma2_ss(d_tmem, qd, kd, idesc_qk, kk > 0 ? 1u : 0u);
+                    umma2_ss_elect(d_tmem, qd, kd, idesc_qk, kk > 0 ? 1u : 0u);
                     // next 16 columns of head_dim: 32 bytes on inside a 64-column chunk, else on to the next chunk
                     umma_desc_advance(qd, (kk & 3) == 3 ? 128 * 128 - 96 : 32);
                     umma_desc_advance(kd, (kk & 3) == 3 ? 64 * 128 - 96 : 32);
                 }
-                umma2_commit_mc(bar(C_KEMPTY + st), 3);
-                umma2_commit_mc(bar(C_SFULL + buf), 3);
-                if (last) umma2_commit_mc(bar(C_QEMPTY), 3);
+                umma2_commit_mc_elect(bar(C_KEMPTY + st), 3);
+                umma2_commit_mc_elect(bar(C_SFULL + buf), 3);
+                if (last) umma2_commit_mc_elect(bar(C_QEMPTY), 3);
                 return true;
             };
             bool ok = true;
@@ -329,11 +330,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     umma_desc_advance(vd, (uint32_t)st * L::V_STAGE);
 #pragma unroll
                     for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
-                        umma2_ts(tmem_base + kColO, p_tmem + kk * 8, vd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
+                        umma2_ts_elect(tmem_base + kColO, p_tmem + kk * 8, vd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
                         umma_desc_advance(vd, 16 * 128);   // the next 16 keys
                     }
-                    umma2_commit_mc(bar(C_VEMPTY + st), 3);
-                    umma2_commit_mc(bar(C_PVDONE + buf), 3);
+                    umma2_commit_mc_elect(bar(C_VEMPTY + st), 3);
+                    umma2_commit_mc_elect(bar(C_PVDONE + buf), 3);
                 }
                 gt += n;
             }
