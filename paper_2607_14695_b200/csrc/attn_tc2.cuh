@@ -200,10 +200,13 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
-            // The loads are issued in the order in which the tensor pipe frees their stages. The MMA thread issues
-            // Q K^T(j+1) before P V(j), so the K stage of tile j+1 (freed by Q K^T(j-1)) comes free before the V stage
-            // of tile j (freed by P V(j-2)): a K cursor runs one tile ahead of a V cursor through the same list of
-            // units, and neither load waits behind a stage that frees later than its own.
+            // The loads are issued in the order in which the tensor pipe frees their stages. The MMA warp issues
+            // Q K^T(j+1) before P V(j), so the completions come as QK(0) QK(1) PV(0) QK(2) PV(1) ...: K(g) may go once
+            // QK(g - NKS) is done (position 2(g-NKS)-1 in that sequence), V(g) once PV(g - NVS) is done (position
+            // 2(g-NVS)+2). A K cursor therefore runs kLead = NKS - NVS + 1 tiles ahead of a V cursor through the same
+            // list of units, and neither load waits behind a stage that frees later than its own.
+            constexpr int kLead = NKS - NVS + 1;
+            static_assert(kLead == 0 || kLead == 1, "order of K and V loads");
             struct Cursor { int u, ui, jj, g; bool valid; Unit w; };
             auto settle = [&](Cursor &c) {   // first unit at or after c.u with a non-empty key slice
                 c.valid = false;
@@ -266,7 +269,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ck.u = cluster_id; ck.ui = 0; ck.jj = 0; ck.g = 0;
             settle(ck);
             cv = ck;
-            if (ck.valid) { issue_k(ck); advance(ck); }
+            if (kLead == 1 && ck.valid) { issue_k(ck); advance(ck); }
             while (cv.valid && ok) {
                 if (ck.valid) {
                     issue_k(ck);
