@@ -531,9 +531,21 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attn_tc2_kernel<HD><<<grid, kTc2Threads, Tc2Smem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
+    // programmatic stream serialisation: the grid may be scheduled while the preceding kernel drains; it waits
+    // (griddepcontrol.wait) before it touches global memory
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kTc2Threads);
+    cfg.dynamicSmemBytes = Tc2Smem<HD>::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc2_kernel<HD>, *mq, *mk, *mv, *mkd, *mvd, tp);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace

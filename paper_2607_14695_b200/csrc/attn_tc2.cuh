@@ -181,6 +181,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 64) TC2_TRACE(2, 15, 1);
+    // Programmatic dependent launch: this grid may have been scheduled while the kernel ahead of it on the stream was still
+    // running (its set-up above touches no global memory); from here on everything that kernel wrote is visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool {
         if (mbar_try_wait(bar(i), parity)) return true;
@@ -489,7 +492,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int c = 0; c < KT; c += 2) {
                     float x0, x1;
                     unpack_f32x2(fma_f32x2(pack_f32x2(s[c], s[c + 1]), sc2, nm2), x0, x1);
+#ifdef DBG_NOEXP
+                    const float p0 = x0 * 1e-3f, p1 = x1 * 1e-3f;
+#else
                     const float p0 = ex2(x0), p1 = ex2(x1);
+#endif
                     sum2[(c >> 1) & 3] = add_f32x2(sum2[(c >> 1) & 3], pack_f32x2(p0, p1));
                     __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
@@ -526,6 +533,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             gt += w.n_tiles;
             // ---- epilogue of the unit ----
+            // (before this cluster's last epilogue: let the next kernel on the stream be scheduled; it waits for this grid's end)
+            if (threadIdx.x == 64 && u + n_clusters >= n_units) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             // The threads of a row add their sums; each thread takes its share of the head_dim columns out of tensor
             // memory, 32 at a time, and stores its row segment straight to global memory in 32-byte pieces (whole sectors).
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 2); TC2_TRACE(2, ui_s, 2); }

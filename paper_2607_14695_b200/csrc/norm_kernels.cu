@@ -288,8 +288,14 @@ gate_layer_tiled_kernel(const VT *vec, const T *__restrict__ W, const T *__restr
 // (D <= 256 * NCH), so x is read from memory exactly once. grid = ceil(B*R / 8).
 template <typename T, int NCH>
 __global__ void __launch_bounds__(256)
-adarmsnorm_rows_kernel(const T *x, T *y, const float *gate_buf, int rows, int R, int D, float eps)
+adarmsnorm_rows_kernel(const T *x, T *y, const float *gate_buf, int rows, int R, int D, float eps, int wait_first)
 {
+    // Programmatic dependent launch, both ways. This grid may have been scheduled before the kernel launched ahead of it on
+    // the stream has finished: unless that kernel is the library's own gate kernel (which does not write x: wait_first = 0)
+    // nothing is read before it is known to be complete. And the kernel launched after this one may be scheduled as soon as
+    // every block of this grid has started; it waits the same way before it touches memory.
+    if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int row = blockIdx.x * 8 + warp;
     if (row >= rows) return;
@@ -298,12 +304,17 @@ adarmsnorm_rows_kernel(const T *x, T *y, const float *gate_buf, int rows, int R,
     T *yr = y + (size_t)row * D;
     const float *g = gate_buf + (size_t)b * D;
     float f[NCH][8];
+    float4 gg[NCH][2];
     float ss = 0.f;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
         const int e = c * 256 + lane * 8;
         if (e < D) {
             Vec8<T>::load(xr + e, f[c]);
+            if (wait_first) {   // the gate is final already: fetch it in the same round trip as the row
+                gg[c][0] = *reinterpret_cast<const float4 *>(g + e);
+                gg[c][1] = *reinterpret_cast<const float4 *>(g + e + 4);
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) ss = fmaf(f[c][i], f[c][i], ss);
         }
@@ -312,13 +323,13 @@ adarmsnorm_rows_kernel(const T *x, T *y, const float *gate_buf, int rows, int R,
     const float rinv = 1.f / sqrtf(ss / (float)D + eps);
     // the gate may still be in the making by the preceding launch (programmatic dependent launch): x is already in
     // registers and the statistics are done, now wait for that grid to finish and its writes to be visible
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
         const int e = c * 256 + lane * 8;
         if (e < D) {
-            const float4 g0 = *reinterpret_cast<const float4 *>(g + e);
-            const float4 g1 = *reinterpret_cast<const float4 *>(g + e + 4);
+            const float4 g0 = wait_first ? gg[c][0] : *reinterpret_cast<const float4 *>(g + e);
+            const float4 g1 = wait_first ? gg[c][1] : *reinterpret_cast<const float4 *>(g + e + 4);
             float o[8];
             o[0] = f[c][0] * rinv * g0.x; o[1] = f[c][1] * rinv * g0.y; o[2] = f[c][2] * rinv * g0.z; o[3] = f[c][3] * rinv * g0.w;
             o[4] = f[c][4] * rinv * g1.x; o[5] = f[c][5] * rinv * g1.y; o[6] = f[c][6] * rinv * g1.z; o[7] = f[c][7] * rinv * g1.w;
@@ -329,6 +340,8 @@ adarmsnorm_rows_kernel(const T *x, T *y, const float *gate_buf, int rows, int R,
 
 template <typename T>
 static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B, int R, int D, float eps, bool after_gate, cudaStream_t st)
+// after_gate: the kernel launched just before on this stream is the gate kernel of the same call (it may still be running
+// while the rows are read and their statistics taken); otherwise the grid waits for whatever precedes it before reading.
 {
     const int rows = B * R;
     cudaLaunchConfig_t cfg = {};
@@ -340,11 +353,12 @@ static cudaError_t launch_rows_t(const T *x, T *y, const float *gate_buf, int B,
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = after_gate ? 1 : 0;   // overlap with the gate kernel launched just before on the same stream
+    cfg.numAttrs = 1;
+    const int wait_first = after_gate ? 0 : 1;
     cudaError_t e;
-    if (D <= 512) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 2>, x, y, gate_buf, rows, R, D, eps);
-    else if (D <= 1024) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 4>, x, y, gate_buf, rows, R, D, eps);
-    else if (D <= 2048) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 8>, x, y, gate_buf, rows, R, D, eps);
+    if (D <= 512) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 2>, x, y, gate_buf, rows, R, D, eps, wait_first);
+    else if (D <= 1024) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 4>, x, y, gate_buf, rows, R, D, eps, wait_first);
+    else if (D <= 2048) e = cudaLaunchKernelEx(&cfg, adarmsnorm_rows_kernel<T, 8>, x, y, gate_buf, rows, R, D, eps, wait_first);
     else return cudaErrorNotSupported;
     count_launch();
     return e;
