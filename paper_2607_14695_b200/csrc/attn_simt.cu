@@ -180,6 +180,9 @@ __global__ void __launch_bounds__(256)
 attn_merge_kernel(AttnParams p)
 {
     constexpr int d = DPL * 32;
+    // launched with programmatic stream serialisation: wait for the attention kernel ahead of it before reading its partials
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rows = p.T * p.Hq;
     const int gr = blockIdx.x * 8 + warp;      // row over all streams
@@ -263,16 +266,25 @@ static cudaError_t launch_simt_t(const AttnParams &p, cudaStream_t st)
 template <typename T>
 static cudaError_t launch_merge_t(const AttnParams &p, cudaStream_t st)
 {
-    const int grid = (p.B * p.T * p.Hq + 7) / 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.B * p.T * p.Hq + 7) / 8);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e;
     switch (p.d / 32) {
-        case 1: attn_merge_kernel<T, 1><<<grid, 256, 0, st>>>(p); break;
-        case 2: attn_merge_kernel<T, 2><<<grid, 256, 0, st>>>(p); break;
-        case 4: attn_merge_kernel<T, 4><<<grid, 256, 0, st>>>(p); break;
-        case 8: attn_merge_kernel<T, 8><<<grid, 256, 0, st>>>(p); break;
+        case 1: e = cudaLaunchKernelEx(&cfg, attn_merge_kernel<T, 1>, p); break;
+        case 2: e = cudaLaunchKernelEx(&cfg, attn_merge_kernel<T, 2>, p); break;
+        case 4: e = cudaLaunchKernelEx(&cfg, attn_merge_kernel<T, 4>, p); break;
+        case 8: e = cudaLaunchKernelEx(&cfg, attn_merge_kernel<T, 8>, p); break;
         default: return cudaErrorInvalidValue;
     }
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st)

@@ -138,6 +138,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L::OFF_BAR + 8 * B_COUNT);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
+    // programmatic dependent launch: scheduled, perhaps, before the kernel ahead on the stream has finished; nothing is read
+    // before it has. The kernel after this one may be scheduled once every CTA here has started (it waits the same way).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x % p.n_qtiles;
     const int kvh = blockIdx.x / p.n_qtiles;
@@ -516,9 +520,19 @@ cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtenso
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attn_tc_kernel<HD><<<grid, kTcThreads, TcSmem<HD>::TOTAL, st>>>(*mq, *mk, *mv, *mkd, *mvd, tp);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = TcSmem<HD>::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<HD>, *mq, *mk, *mv, *mkd, *mvd, tp);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 template <int HD>
