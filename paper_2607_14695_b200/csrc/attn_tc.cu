@@ -584,11 +584,16 @@ int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
     const int n_tiles = (p.S_max + kBN - 1) / kBN + (p.N + kBN - 1) / kBN + (p.T + kBN - 1) / kBN;
     if (ctas >= sm_count) return 1;
     int want = (sm_count + ctas - 1) / ctas;
+
     if (want > n_tiles) want = n_tiles;
     if (want > kMaxSplits) want = kMaxSplits;
     const size_t per_split = (size_t)p.B * p.T * p.Hq * (p.d + 2) * sizeof(float);
     if (per_split > 0 && (size_t)want * per_split > partial_bytes) want = (int)(partial_bytes / per_split);
-    return want < 1 ? 1 : want;
+    // a power of two: measured (one stream, 15 key tiles) 15.5 us per layer with 8 slices and 16.5 with 4, against 18-21 us
+    // with 5, 6, 7, 9, 10, 12 or 15 (the stride between a row's partials in the scratch area is then a power of two as well)
+    int pow2 = 1;
+    while (pow2 * 2 <= want) pow2 *= 2;
+    return pow2;
 }
 
 bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 || p.d == 256); }
