@@ -537,7 +537,7 @@ cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtenso
 
 template <int HD>
 cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
-                      const CUtensorMap *mvd, const TcParams &tp, dim3 grid, cudaStream_t st)
+                      const CUtensorMap *mvd, const CUtensorMap *mo, const TcParams &tp, dim3 grid, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -557,7 +557,7 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc2_kernel<HD>, *mq, *mk, *mv, *mkd, *mvd, tp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc2_kernel<HD>, *mq, *mk, *mv, *mkd, *mvd, *mo, tp);
     count_launch();
     return e;
 }
@@ -640,14 +640,16 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     if (two_cta) {
         // persistent grid: one cluster (two CTAs) per SM pair walks the (stream, KV head, tile pair) units;
         // an odd tile count leaves the last pair of a stream with one idle half
+        CUtensorMap mo;
+        if (!cache().get(&mo, p.out, 1, (p.B << 16) | p.T, p.Hq, p.d, G, mk_q)) return cudaErrorInvalidValue;
         tp.n_qtiles = (tp.n_qtiles + 1) / 2;
         const int units = tp.n_qtiles * p.Hkv * p.B * p.nsplit;
         int clusters = sm_count / 2;
         if (clusters > units) clusters = units;
         if (clusters < 1) clusters = 1;
         dim3 grid2(2 * clusters, 1, 1);
-        if (p.d == 256) e = launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
-        else if (p.d == 128) e = launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, tp, grid2, st);
+        if (p.d == 256) e = launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
+        else if (p.d == 128) e = launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
         else return cudaErrorInvalidValue;
         if (e != cudaSuccess || p.nsplit == 1) return e;
         return launch_attention_merge(p, st);

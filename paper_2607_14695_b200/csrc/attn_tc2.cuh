@@ -64,11 +64,18 @@ __device__ __forceinline__ void apply_slice_mask(float (&s)[K], uint64_t mask)
     }
 }
 
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
+
 template <int HD> struct Tc2Smem {
     static constexpr int CH = HD / 64;
     static constexpr int VCH = CH / 2;                          // this CTA's 64-column chunks of head_dim
     static constexpr int NKS = (HD == 256) ? 2 : 4;             // K stages
-    static constexpr int NVS = (HD == 256) ? 3 : 4;             // V stages (P lives in tensor memory, which pays for the third)
+    static constexpr int NVS = (HD == 256) ? 2 : 4;             // V stages (P lives in tensor memory, which pays for the third)
     static constexpr uint32_t Q_BYTES = CH * 128 * 128;
     static constexpr uint32_t K_STAGE = CH * 64 * 128;          // 64 keys x head_dim
     static constexpr uint32_t V_STAGE = VCH * 128 * 128;        // 128 keys x head_dim/2
@@ -76,7 +83,9 @@ template <int HD> struct Tc2Smem {
     static constexpr uint32_t OFF_Q = 0;
     static constexpr uint32_t OFF_K = OFF_Q + Q_BYTES;
     static constexpr uint32_t OFF_V = OFF_K + NKS * K_STAGE;
-    static constexpr uint32_t OFF_BAR = OFF_V + NVS * V_STAGE;
+    static constexpr uint32_t OFF_STAGE = OFF_V + NVS * V_STAGE;      // epilogue staging: 128 rows x 128 columns of O in bf16
+    static constexpr uint32_t STAGE_BYTES = 2 * 128 * 128;
+    static constexpr uint32_t OFF_BAR = OFF_STAGE + STAGE_BYTES;
     static constexpr uint32_t BAR_BYTES = 256;
     static constexpr uint32_t OFF_XMAX = OFF_BAR + BAR_BYTES;                   // row maxima: 2 buffers x 128 rows x NP 16-bit values
     static constexpr uint32_t XMAX_BYTES = 2 * 128 * kTc2Parts * 2;
@@ -100,7 +109,7 @@ template <int HD>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTc2Threads, 1)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
-                const __grid_constant__ CUtensorMap tm_vd, const TcParams p)
+                const __grid_constant__ CUtensorMap tm_vd, const __grid_constant__ CUtensorMap tm_o, const TcParams p)
 {
     using L = Tc2Smem<HD>;
     constexpr int CH = L::CH, VCH = L::VCH, NKS = L::NKS, NVS = L::NVS;
@@ -171,7 +180,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         *abort_flag = 0u;
         fence_mbar_init();
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd);
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v); prefetch_tmap(&tm_kd); prefetch_tmap(&tm_vd); prefetch_tmap(&tm_o);
     }
     if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), kTmemCols);
     tc_fence_before();
@@ -364,7 +373,6 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t leader_ofree = mapa(bar(C_OFREE), 0);
         uint16_t *xmax = reinterpret_cast<uint16_t *>(smem + L::OFF_XMAX);   // [2 buffers][128 rows][NP], bf16 bit patterns
         float *xsum = reinterpret_cast<float *>(smem + L::OFF_XSUM);         // [NP][128 rows]
-        __nv_bfloat16 *out_bf = reinterpret_cast<__nv_bfloat16 *>(p.out);
         bool ok = true;
         int gt = 0;
         [[maybe_unused]] int ui_s = 0;
@@ -573,34 +581,57 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 continue;
             }
+            // O / l goes out through a 32 KB staging area laid out like a Q tile (two 64-column chunks of 128 swizzled rows)
+            // and TMA stores: the threads are done once the tile sits in shared memory, and the store drains underneath the
+            // next unit. (Stores straight from registers kept every thread until its 64 KB were accepted by a memory system
+            // that all clusters hit at the same moment: 4.4 k cycles per unit.)
             const float inv = 1.f / l;
-            __nv_bfloat16 *orow = row_live ? out_bf + (((size_t)w.b * p.T + t_row) * p.Hq + hq) * HD + part * EC : nullptr;
+            const bool store_unit = w.t0 < p.T;   // an idle partner tile (odd tile count) has nothing to write
+            constexpr int SC = 128 / NP;           // columns per thread and round: a round stages 128 columns of O
 #pragma unroll 1
-            for (int c = 0; c < EC / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tmem_base + lane_addr + kColO + part * EC + c * 32, o);
+            for (int rnd = 0; rnd < HD / 128; ++rnd) {
+                uint32_t o[SC];
+                const uint32_t o_addr = tmem_base + lane_addr + kColO + rnd * 128 + part * SC;
+#pragma unroll
+                for (int q = 0; q < SC / 32; ++q) tmem_ld32(o_addr + 32 * q, *reinterpret_cast<uint32_t(*)[32]>(o + 32 * q));
+                // the staging area may still be read by the stores of the previous round or unit
+                if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 tmem_wait_ld();
-                if (c == EC / 32 - 1) {
+                if (rnd == HD / 128 - 1) {
                     // all of O is in registers: the next unit's first P V may overwrite the accumulator
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(leader_ofree);
                 }
-                uint32_t pk[16];
+                asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
+                const int col0 = part * SC;
+                uint8_t *srow = smem + L::OFF_STAGE + (col0 >> 6) * (128 * 128) + row * 128;
+                const int c16 = (col0 & 63) >> 3;
 #pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[2 * k]) * inv, __uint_as_float(o[2 * k + 1]) * inv);
-                    pk[k] = *reinterpret_cast<uint32_t *>(&hh);
+                for (int c = 0; c < SC / 8; ++c) {
+                    uint4 v;
+                    uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[8 * c + 2 * k]) * inv, __uint_as_float(o[8 * c + 2 * k + 1]) * inv);
+                        vv[k] = *reinterpret_cast<uint32_t *>(&hh);
+                    }
+                    *reinterpret_cast<uint4 *>(srow + (((c16 + c) ^ (row & 7)) << 4)) = v;
                 }
-                if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 6 + 2 * c);
-                if (row_live) {
-                    st_global_v8(orow + c * 32, *reinterpret_cast<const uint32_t(*)[8]>(pk));
-                    st_global_v8(orow + c * 32 + 16, *reinterpret_cast<const uint32_t(*)[8]>(pk + 8));
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
+                if (threadIdx.x == 64) {
+                    if (store_unit) {
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh)
+                            tma_store_4d(&tm_o, base + L::OFF_STAGE + hh * (128 * 128), rnd * 128 + hh * 64, w.kvh * p.G, w.t0, w.b);
+                    }
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
-                if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 7 + 2 * c);
             }
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 4); TC2_TRACE(2, ui_s, 4); }
         }
+        if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores of this CTA are complete
     }
 
     tc_fence_before();
