@@ -39,6 +39,10 @@ constexpr int kTc2Keys = 128;     // keys per tile = two 64-key halves, one per 
 #ifndef REFLEX_TC2_NP
 #define REFLEX_TC2_NP 2
 #endif
+#ifndef REFLEX_TC2_POLY
+#define REFLEX_TC2_POLY 2
+#endif
+constexpr int kTc2PolyEighths = REFLEX_TC2_POLY;   // of every 8 key pairs, how many take their exponentials on the FMA pipe
 constexpr int kTc2Parts = REFLEX_TC2_NP;            // softmax threads per query row (2 or 4)
 constexpr int kTc2Threads = 64 + 128 * kTc2Parts;   // producer warp, MMA warp, 4 * kTc2Parts softmax warps
 static_assert(kTc2Parts == 2 || kTc2Parts == 4, "softmax threads per row");
@@ -489,22 +493,21 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 const float mr = (m_ref == -INFINITY) ? 0.f : m_ref * p.scale_log2;
-                // P = 2^(s*scale*log2e - m), two keys per instruction wherever the hardware has a packed form (the scaling FMA
-                // and the running sums); the exponentials themselves all go to the MUFU unit. Emulating a share of them on the
-                // FMA pipe shortens this loop in isolation but fills the issue slots the MMA thread needs: measured slower.
+                // P = 2^(s*scale*log2e - m), two keys per instruction wherever the hardware has a packed form (the scaling FMA,
+                // the running sums, the polynomial). A quarter of the key pairs take a cubic on the FMA pipe, the rest the MUFU
+                // unit (4 results per clock and scheduler): measured 2/8 35.4 us, 0/8 35.6, 3/8 35.9, 4/8 36.4 per launch.
                 SM_EV(6);
                 const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(-mr, -mr);
+                const Ex2PolyConsts pk = ex2_poly_consts();
                 uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
                 uint32_t packed[KT / 2];
 #pragma unroll
                 for (int c = 0; c < KT; c += 2) {
                     float x0, x1;
                     unpack_f32x2(fma_f32x2(pack_f32x2(s[c], s[c + 1]), sc2, nm2), x0, x1);
-#ifdef DBG_NOEXP
-                    const float p0 = x0 * 1e-3f, p1 = x1 * 1e-3f;
-#else
-                    const float p0 = ex2(x0), p1 = ex2(x1);
-#endif
+                    float p0, p1;
+                    if (((c >> 1) & 7) < kTc2PolyEighths) ex2_poly_f32x2(x0, x1, pk, p0, p1);
+                    else { p0 = ex2(x0); p1 = ex2(x1); }
                     sum2[(c >> 1) & 3] = add_f32x2(sum2[(c >> 1) & 3], pack_f32x2(p0, p1));
                     __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     packed[c >> 1] = *reinterpret_cast<uint32_t *>(&hh);
@@ -513,6 +516,17 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     float a, b;
                     unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), a, b);
                     l += a + b;
+                }
+                if (kTc2PolyEighths > 0 && smask != kSliceFull) {
+                    // the polynomial gives a masked key 2^-125 instead of 0 (nothing for the sum, but P must be exactly 0
+                    // there): clear those halves of the packed words
+#pragma unroll
+                    for (int c = 0; c < KT; c += 2) {
+                        if (((c >> 1) & 7) < kTc2PolyEighths) {
+                            const uint32_t two = (uint32_t)(smask >> c) & 3u;
+                            packed[c >> 1] &= ((two & 1u) ? 0x0000FFFFu : 0u) | ((two & 2u) ? 0xFFFF0000u : 0u);
+                        }
+                    }
                 }
                 SM_EV(5);
                 // P goes into the first 64 columns of S's buffer (two keys per column): the A operand of this tile's P V.

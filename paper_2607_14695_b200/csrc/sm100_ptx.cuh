@@ -193,6 +193,33 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
 __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ float max3_f32(float a, float b, float c) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c)); return d; }
 
+// 2^x for a packed pair on the FMA pipe (same scheme as ex2_fma, the arithmetic in f32x2 instructions): arguments are
+// clamped at -125, so anything below gives 2^-125 (2.4e-38) instead of 0; the caller zeroes what must be exactly 0.
+struct Ex2PolyConsts { uint64_t magic, neg_magic, neg_one, c3, c2, c1, c0; };
+__device__ __forceinline__ Ex2PolyConsts ex2_poly_consts()
+{
+    Ex2PolyConsts k;
+    k.magic = pack_f32x2(12582912.f, 12582912.f); k.neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+    k.neg_one = pack_f32x2(-1.f, -1.f);
+    k.c3 = pack_f32x2(0.05508868f, 0.05508868f); k.c2 = pack_f32x2(0.24260405f, 0.24260405f);
+    k.c1 = pack_f32x2(0.69327623f, 0.69327623f); k.c0 = pack_f32x2(0.99992895f, 0.99992895f);
+    return k;
+}
+__device__ __forceinline__ void ex2_poly_f32x2(float x0, float x1, const Ex2PolyConsts &k, float &p0, float &p1)
+{
+    const uint64_t xc = pack_f32x2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t t = add_f32x2(xc, k.magic);                       // low mantissa bits of each half: round(x)
+    const uint64_t f = fma_f32x2(add_f32x2(t, k.neg_magic), k.neg_one, xc);   // x - round(x) in [-0.5, 0.5]
+    uint64_t pl = fma_f32x2(f, k.c3, k.c2);
+    pl = fma_f32x2(f, pl, k.c1);
+    pl = fma_f32x2(f, pl, k.c0);
+    float t0, t1, q0, q1;
+    unpack_f32x2(t, t0, t1);
+    unpack_f32x2(pl, q0, q1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
