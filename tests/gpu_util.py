@@ -92,10 +92,12 @@ class Twin:
             assert np.array_equal(ks[:, b, w.S_max:][:, live], self.o.k_ring[:, b, live])
             assert np.array_equal(vs[:, b, w.S_max:][:, live], self.o.v_ring[:, b, live])
 
-    def attention(self, layer, variant, dyn_mask=0, T=None, streams=None, scale=0.0, what="attention", partitioned=False):
+    def attention(self, layer, variant, dyn_mask=0, T=None, streams=None, scale=0.0, what="attention", partitioned=False, q_scale=1.0, rel_clause=False):
         w = self.w
         T = w.T if T is None else T
         q = synth.normal(w, "q", (w.B, T, w.Hq, w.d), layer, variant)
+        if q_scale != 1.0:   # wider logits (the same rounding to the storage dtype on both sides)
+            q = synth.round_storage(q * np.float32(q_scale), w.dtype)
         kd = synth.normal(w, "k_dyn", (w.B, T, w.Hkv, w.d), layer, variant)
         vd = synth.normal(w, "v_dyn", (w.B, T, w.Hkv, w.d), layer, variant)
         out = torch.full((w.B, T, w.Hq, w.d), float("nan"), dtype=rb.torch_dtype(w.dtype), device=DEV)
@@ -108,5 +110,5 @@ class Twin:
         res = []
         for b in streams:
             want = self.o.attention(b, layer, q[b], kd[b], vd[b], dyn_mask, None if scale <= 0 else scale, partitioned=partitioned)
-            res.append(check_close(got[b], want, w.dtype, f"{what} stream {b} layer {layer}"))
+            res.append(check_close(got[b], want, w.dtype, f"{what} stream {b} layer {layer}", rel_clause=rel_clause))
         return res

@@ -219,6 +219,37 @@ def test_edge_shapes(U, case, impl):
     tw.attention(0, 6, scale=0.05, what=name + " scale override")
 
 
+@pytest.mark.parametrize("impl", ["tc", "tc2"])
+def test_wide_logits_exercise_the_lazy_rescale(U, impl):
+    """Queries scaled up so that row maxima keep growing by more than 2^8 from tile to tile: O and l are rescaled in
+    tensor memory over and over, with and without the causal mask over the dynamic tokens. With logits this wide a row's
+    output is close to single V rows (|v| up to 4.5), where the bf16 spacing of the output itself passes 2e-2: the bf16
+    output-spacing allowance applies."""
+    w = synth.Workload("wide", 31, synth.DTYPE_BF16, B=3, L=1, Hq=8, Hkv=1, d=256, S=700, S_max=704, N=40, T=50, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w, head0=[5, 0, 39], poison=True)
+    U.rb.reflex_cache_set_attention_impl(tw.g, {"tc": U.rb.ATTN_TC, "tc2": U.rb.ATTN_TC2}[impl])
+    tw.init_static(list(range(w.B)), [700, 650, 1])
+    for i in range(3):
+        tw.append(list(range(w.B)), 17, i)
+    for q_scale in (6.0, 20.0):
+        tw.attention(0, 1, dyn_mask=0, q_scale=q_scale, rel_clause=True, what=f"wide logits x{q_scale} {impl}")
+        tw.attention(0, 2, dyn_mask=1, q_scale=q_scale, rel_clause=True, what=f"wide logits x{q_scale} causal {impl}")
+
+
+def test_two_cta_kernel_many_units_head_dim_128(U):
+    """More work units than SM pairs at head_dim 128 (four K and four V stages), two KV heads, several key tiles per unit:
+    the persistent loop crosses unit boundaries with every stage and buffer rotation."""
+    w = synth.Workload("units128", 32, synth.DTYPE_BF16, B=42, L=1, Hq=8, Hkv=2, d=128, S=300, S_max=320, N=48, T=20, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w, head0=[(7 * b) % w.N for b in range(w.B)], poison=True)
+    U.rb.reflex_cache_set_attention_impl(tw.g, U.rb.ATTN_TC2)
+    tw.init_static(list(range(w.B)), [300 - (b % 5) * 31 for b in range(w.B)])
+    for i in range(4):
+        tw.append([b for b in range(w.B) if not (b % 9 == 4 and i >= 2)], 16, i)
+    tw.check_state()
+    tw.attention(0, 0, dyn_mask=0, what="units128")
+    tw.attention(0, 1, dyn_mask=1, streams=[0, 4, 13, 41], what="units128 causal")
+
+
 def test_error_paths_leave_state_unchanged(U):
     rb = U.rb
     w = synth.Workload("err", 5, synth.DTYPE_BF16, B=2, L=1, Hq=2, Hkv=1, d=64, S=8, S_max=8, N=4, T=4, D=64, Cd=8, Hd=8, A=4, K=2)
