@@ -564,6 +564,21 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
 
 }  // namespace
 
+// rank-2 map over a row-major bf16 matrix [rows][inner], box = box_rows x 64 elements, 128-byte swizzle (cached like the others)
+bool tensor_map_2d_bf16(CUtensorMap *out, const void *ptr, int inner, int rows, int box_rows)
+{
+    return cache().get(out, ptr, 3, inner, rows, box_rows, 0, [](CUtensorMap *m, const void *p_, int inner_, int rows_, int box_rows_, int) -> bool {
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return false;
+        cuuint64_t dims[2] = {(cuuint64_t)inner_, (cuuint64_t)rows_};
+        cuuint64_t strides[1] = {(cuuint64_t)inner_ * 2};
+        cuuint32_t box[2] = {64, (cuuint32_t)box_rows_};
+        cuuint32_t es[2] = {1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(p_), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
+}
+
 bool tc_supported(const AttnParams &p)
 {
     if (p.dtype != REFLEX_DTYPE_BF16) return false;

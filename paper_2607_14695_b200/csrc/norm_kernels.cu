@@ -390,6 +390,14 @@ static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const 
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    if constexpr (sizeof(T) == 2) {
+        // bf16: both layers on the tensor cores, whatever L is (one call for L layers and L calls give the same bits); the
+        // FMA kernels below remain for fp32 and for widths the tensor-core kernel does not take
+        if (gate_tc_supported(B, D, Cd, Hd)) {
+            cudaError_t e = launch_gate_tc(cond, W1, b1, W2, b2, gate_buf, L, B, D, Cd, Hd, st);
+            if (e != cudaErrorInvalidValue) return e;   // invalid value: no tensor maps from this driver, fall through
+        }
+    }
     const int groups = (B + kGateStreams - 1) / kGateStreams;
     const size_t tiled_h = (size_t)(kTileUnits + kGateStreams) * (Cd + 4) * 4, tiled_g = (size_t)(kTileUnits + kGateStreams) * (Hd + 4) * 4;
     if (L > 1 && tiled_h <= 200 * 1024 && tiled_g <= 200 * 1024) {

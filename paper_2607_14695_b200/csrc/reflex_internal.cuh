@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cuda.h>
+
 #include "reflex.h"
 
 namespace reflex {
@@ -84,9 +86,14 @@ cudaError_t launch_attention_simt(const AttnParams &p, cudaStream_t st);
 int simt_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 cudaError_t launch_attention_merge(const AttnParams &p, cudaStream_t st);  // combines nsplit (m, l, acc) partials
 bool tc_supported(const AttnParams &p);
+bool tensor_map_2d_bf16(CUtensorMap *out, const void *ptr, int inner, int rows, int box_rows);
 int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 bool tc2_supported(const AttnParams &p);
 int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count);
 cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st);
+// gate MLP of AdaRMSNorm on tcgen05 (bf16): false when the shapes or the driver do not allow it (the caller falls back)
+bool gate_tc_supported(int B, int D, int Cd, int Hd);
+cudaError_t launch_gate_tc(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf, int L, int B,
+                           int D, int Cd, int Hd, cudaStream_t st);
 
 }  // namespace reflex
