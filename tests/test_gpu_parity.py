@@ -250,6 +250,20 @@ def test_two_cta_kernel_many_units_head_dim_128(U):
     tw.attention(0, 1, dyn_mask=1, streams=[0, 4, 13, 41], what="units128 causal")
 
 
+@pytest.mark.parametrize("T", [25, 100])
+def test_frame_granular_window(U, T):
+    """The ablation shapes of the paper's context-window study: a sliding window of 10 frames x 256 tokens fed one frame
+    (m = 256) per tick, action chunks of 25 and 100 tokens. The ring wraps several times at different offsets per stream."""
+    w = synth.Workload("frames", 41, synth.DTYPE_BF16, B=3, L=1, Hq=8, Hkv=1, d=256, S=300, S_max=320, N=2560, T=T, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w, head0=[0, 1000, 2559], poison=True)
+    tw.init_static(list(range(w.B)), [300, 257, 64])
+    for i in range(13):                      # 13 frames into a 10-frame window; stream 2 joins late and stays partly filled
+        tw.append([b for b in range(w.B) if not (b == 2 and i < 6)], 256, i)
+        if i in (2, 9, 12):
+            tw.check_state()
+            tw.attention(0, i, dyn_mask=i & 1, what=f"frames tick {i}")
+
+
 def test_error_paths_leave_state_unchanged(U):
     rb = U.rb
     w = synth.Workload("err", 5, synth.DTYPE_BF16, B=2, L=1, Hq=2, Hkv=1, d=64, S=8, S_max=8, N=4, T=4, D=64, Cd=8, Hd=8, A=4, K=2)
