@@ -46,6 +46,7 @@ struct TcParams {
     int nsplit;
     int tile_tokens;  // 128 / G
     int n_qtiles;
+    int cluster_merge;  // one-CTA kernel: the nsplit key slices of a query tile form a cluster and merge through shared memory
 };
 
 template <int HD> struct TcSmem {
@@ -198,6 +199,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         atomicCAS(p.status, 0u, 0x80000000u | (code << 16) | (blockIdx.x & 0xFFFFu));
         return false;
     };
+
+    // what a softmax thread carries into the in-cluster merge (cluster_merge): its row's maximum (log2 units) and sum
+    float fin_m = -INFINITY, fin_l = 0.f;
+    bool fin_ok = true;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -400,6 +405,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                     }
                 }
             }
+        } else if (p.cluster_merge) {
+            fin_ok = ok;
+            if (n_local > 0 && ok) { fin_m = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale_log2; fin_l = l; }
         } else {
             const size_t slot = partial_slot(b, rows_total, t_row * p.Hq + hq, p.nsplit, split);
             float *po = partial_o(p.partials, slot, HD);
@@ -423,6 +431,92 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 pml[0] = -INFINITY; pml[1] = 0.f;
             }
         }
+    }
+
+    if (p.nsplit > 1 && p.cluster_merge) {
+        // ---- merge of the key slices inside the cluster (one CTA per slice, all of the same query tile) ----
+        // 1. every softmax thread publishes its row's (m, l); 2. with everybody's (m, l) it scales its own O row to the
+        // common maximum and stages it in shared memory (the Q / K / V buffers are idle now), column-major in 16-byte
+        // units so that rows (lanes) are contiguous; 3. CTA s adds up columns [s, s+1) * head_dim / nsplit of all slices
+        // through distributed shared memory, divides by the common sum and writes them. Three cluster barriers: after
+        // 1, after 2, and before anybody leaves (a peer may still be reading this CTA's staging area).
+        const int ns = p.nsplit;
+        const uint32_t my_rank = cluster_ctarank();
+        float2 *ml_own = reinterpret_cast<float2 *>(smem + L::OFF_P);                  // [128 rows]
+        float4 *stage = reinterpret_cast<float4 *>(smem + L::OFF_Q);                   // [HD / 4][128 rows]
+        const int row_m = (warp & 3) * 32 + lane;
+        if (warp >= 2) ml_own[row_m] = make_float2(fin_m, fin_l);
+        cluster_arrive();
+        cluster_wait();
+        float w_own = 0.f, l_all = 0.f;
+        uint32_t live_peers = 0u;
+        if (warp >= 2) {
+            float mstar = -INFINITY;
+            float pm[8], pl[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                pm[q] = -INFINITY; pl[q] = 0.f;
+                if (q < ns) {
+                    const uint32_t a = mapa(smem_u32(ml_own + row_m), (uint32_t)q);
+                    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(pm[q]), "=f"(pl[q]) : "r"(a) : "memory");
+                }
+                mstar = fmaxf(mstar, pm[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const float wq = (pm[q] == -INFINITY) ? 0.f : ex2(pm[q] - mstar);
+                l_all = fmaf(pl[q], wq, l_all);
+                if (pl[q] * wq > 0.f) live_peers |= 1u << q;
+                if (q == (int)my_rank) w_own = wq;
+            }
+            if (fin_l > 0.f && fin_ok) {
+                tc_fence_after();
+                const uint32_t lane_addr_m = (uint32_t)((warp & 3) * 32) << 16;
+#pragma unroll 1
+                for (int c = 0; c < HD / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem_base + lane_addr_m + kColO + c * 32, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        stage[(c * 8 + i) * 128 + row_m] = make_float4(__uint_as_float(o[4 * i]) * w_own, __uint_as_float(o[4 * i + 1]) * w_own,
+                                                                       __uint_as_float(o[4 * i + 2]) * w_own, __uint_as_float(o[4 * i + 3]) * w_own);
+                }
+            }
+        }
+        cluster_arrive();
+        cluster_wait();
+        if (warp >= 2) {
+            const int t_row_m = t0 + row_m / p.G;
+            const int c4_per = HD / 4 / ns, c4_0 = (int)my_rank * c4_per;           // this CTA's columns, in float4 units
+            if (t_row_m < p.T && l_all > 0.f) {
+                const float inv = 1.f / l_all;
+                __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row_m) * p.Hq + kvh * p.G + row_m % p.G) * HD + c4_0 * 4;
+#pragma unroll 1
+                for (int c4 = 0; c4 < c4_per; c4 += 2) {                            // 8 columns = one 16-byte store at a time
+                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    for (int q = 0; q < ns; ++q) {
+                        if (!((live_peers >> q) & 1u)) continue;
+                        const uint32_t a = mapa(smem_u32(stage + (c4_0 + c4) * 128 + row_m), (uint32_t)q);
+                        float4 v0, v1;
+                        asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v0.x), "=f"(v0.y), "=f"(v0.z), "=f"(v0.w) : "r"(a) : "memory");
+                        asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v1.x), "=f"(v1.y), "=f"(v1.z), "=f"(v1.w) : "r"(a + 128 * 16) : "memory");
+                        acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+                        acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+                    }
+                    uint4 v;
+                    uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
+                        vv[k] = *reinterpret_cast<uint32_t *>(&h);
+                    }
+                    *reinterpret_cast<uint4 *>(orow + c4 * 4) = v;
+                }
+            }
+        }
+        cluster_arrive();
+        cluster_wait();
     }
 
     tc_fence_before();
@@ -525,11 +619,13 @@ cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtenso
     cfg.blockDim = dim3(kTcThreads);
     cfg.dynamicSmemBytes = TcSmem<HD>::TOTAL;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // the key slices of a query tile merge inside a cluster
+    attr[1].val.clusterDim.x = 1; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = (unsigned)tp.nsplit;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = tp.cluster_merge ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel<HD>, *mq, *mk, *mv, *mkd, *mvd, tp);
     count_launch();
     return e;
@@ -651,6 +747,7 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     tp.nsplit = p.nsplit;
     tp.tile_tokens = kBM / G;
     tp.n_qtiles = (p.T + tp.tile_tokens - 1) / tp.tile_tokens;
+    tp.cluster_merge = (!two_cta && p.nsplit > 1 && p.nsplit <= 8 && (p.d / 4) % (2 * p.nsplit) == 0) ? 1 : 0;
     cudaError_t e;
     if (two_cta) {
         // persistent grid: one cluster (two CTAs) per SM pair walks the (stream, KV head, tile pair) units;
@@ -676,7 +773,7 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
         case 256: e = launch_t<256>(&mq, &mk, &mv, &mkd, &mvd, tp, grid, st); break;
         default: return cudaErrorInvalidValue;
     }
-    if (e != cudaSuccess || p.nsplit == 1) return e;
+    if (e != cudaSuccess || p.nsplit == 1 || tp.cluster_merge) return e;
     return launch_attention_merge(p, st);
 }
 
