@@ -231,7 +231,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0 && n_local > 0) {
+        // (the whole warp runs the loop converged, one elected lane issues: see umma_ss_elect)
+        if (n_local > 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kBM, kBN, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(kBM, HD, true);
             auto issue_qk = [&](int jj) {
@@ -241,10 +242,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t a = base + L::OFF_Q + (kk >> 2) * (kBM * 128) + (kk & 3) * 32;
                     const uint32_t bb = base + L::OFF_K + st * L::KV_STAGE + (kk >> 2) * (kBN * 128) + (kk & 3) * 32;
-                    umma_ss(d_tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
+                    umma_ss_elect(d_tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, 16, 1024), idesc_qk, kk > 0 ? 1u : 0u);
                 }
-                umma_commit(bar(B_KEMPTY + st));
-                umma_commit(bar(B_SFULL + buf));
+                umma_commit_elect(bar(B_KEMPTY + st));
+                umma_commit_elect(bar(B_SFULL + buf));
             };
             bool ok = wait(B_QFULL, 0, 3) && wait(B_KFULL + 0, 0, 4);
             if (ok) { tc_fence_after(); issue_qk(0); }
@@ -265,11 +266,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 for (int kk = 0; kk < kBN / 16; ++kk) {
                     const uint32_t a = base + L::OFF_P + buf * L::P_BYTES + kk * 32;
                     const uint32_t bb = base + L::OFF_V + st * L::KV_STAGE + kk * (16 * 128);
-                    umma_ss(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, kBN * 128, 1024), idesc_pv,
+                    umma_ss_elect(tmem_base + kColO, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(bb, kBN * 128, 1024), idesc_pv,
                             (jj > 0 || kk > 0) ? 1u : 0u);
                 }
-                umma_commit(bar(B_VEMPTY + st));
-                umma_commit(bar(B_PVDONE + buf));
+                umma_commit_elect(bar(B_VEMPTY + st));
+                umma_commit_elect(bar(B_PVDONE + buf));
             }
         }
     } else {
