@@ -394,12 +394,15 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 continue;
             }
             float m_ref = -INFINITY, l = 0.f;
+            const int full_halves = w.g.S / kBN;      // 64-key halves that lie entirely inside the static prefix
             for (int jj = 0; jj < w.n_tiles; ++jj) {
                 const int gi = gt + jj, buf = gi & 1, st = gi % NVS;
                 const uint32_t vph = (uint32_t)(gi / NVS) & 1u;
                 const int h = 2 * (w.tile0 + jj) + half;
                 uint64_t tmask = 0ull, rmask = 0ull;   // liveness of the 64 keys of this half: for every row / for this row
-                if (h < w.H) {
+                if (h < full_halves) {
+                    tmask = rmask = ~0ull;             // inside the static prefix, before its last (partial) half: the common case
+                } else if (h < w.H) {
                     const TileRef tr = w.g.decode(h);
                     tmask = w.g.tile_mask(tr);
                     rmask = tmask;
