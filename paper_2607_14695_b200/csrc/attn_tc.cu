@@ -710,26 +710,33 @@ int tc_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
 
 bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 || p.d == 256); }
 
-// Key split of the two-CTA kernel: as many slices as it takes to give every cluster (SM pair) a unit, at least four
-// 128-key tiles per slice so that a unit's head and tail stay amortised. Returns 0 when even that leaves most of the
-// machine idle (then the one-CTA kernel with its finer split is the better fit).
+// Key split of the two-CTA kernel: 1, 2, 4 or 8 slices, whichever a small cost model makes cheapest. A unit (tile pair
+// of one stream and KV head) walks its 128-key tiles at about 1.3 us each, units run in waves of one per SM pair, and
+// splitting costs a fixed 3 us (merge launch) plus the fp32 partials' round trip through memory. Measured at the
+// 898-key shape: 1 stream 14.4 us with 8 slices; 2 streams 15.4 with 4; 4 streams 17.5 with 4; 8 to 32 streams 19.5 to
+// 21.7 unsplit (split in two: 21.6 to 40); at 4466 keys and 16 streams 41 us split in two, 51 unsplit, 47 in four.
 int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
 {
     const int G = p.Hq / p.Hkv;
     const int tile_tokens = kBM / G;
     const int n_pairs = ((p.T + tile_tokens - 1) / tile_tokens + 1) / 2;
     const int units = n_pairs * p.Hkv * p.B;
-    const int clusters = sm_count / 2;
+    const int clusters = sm_count / 2 > 0 ? sm_count / 2 : 1;
     if (units >= clusters) return 1;
     const int halves = (p.S_max + kBN - 1) / kBN + (p.N + kBN - 1) / kBN + (p.T + kBN - 1) / kBN;
     const int tiles = (halves + 1) / 2;
-    int want = clusters / units;
-    if (want > tiles / 4) want = tiles / 4;
-    if (want > kMaxSplits) want = kMaxSplits;
-    const size_t per_split = (size_t)p.B * p.T * p.Hq * (p.d + 2) * sizeof(float);
-    if (per_split > 0 && (size_t)want * per_split > partial_bytes) want = (int)(partial_bytes / per_split);
-    if (want < 1) want = 1;
-    return (units * want * 10 >= clusters * 6) ? want : 0;
+    const double per_split_bytes = (double)p.B * p.T * p.Hq * (p.d + 2) * sizeof(float);
+    int best = 1;
+    double best_us = 1e30;
+    for (int ns = 1; ns <= 8; ns *= 2) {
+        if (ns > tiles) break;
+        if (ns > 1 && per_split_bytes * ns > (double)partial_bytes) break;
+        const int waves = (units * ns + clusters - 1) / clusters;
+        const double loop_us = 1.3 * waves * ((tiles + ns - 1) / ns);
+        const double split_us = ns > 1 ? 3.0 + 2.0 * per_split_bytes * ns / 3.4e6 : 0.0;
+        if (loop_us + split_us < best_us - 0.05) { best_us = loop_us + split_us; best = ns; }
+    }
+    return best;
 }
 
 cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st)
