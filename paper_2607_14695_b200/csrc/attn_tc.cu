@@ -446,6 +446,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         float2 *ml_own = reinterpret_cast<float2 *>(smem + L::OFF_P);                  // [128 rows]
         float4 *stage = reinterpret_cast<float4 *>(smem + L::OFF_Q);                   // [HD / 4][128 rows]
         const int row_m = (warp & 3) * 32 + lane;
+        // (the cluster barriers are warp-aligned instructions: the lanes of the producer warp that idled while lane 0 ran the
+        // loads must not reach them before lane 0 does, so the CTA meets here first)
+        __syncthreads();
         if (warp >= 2) ml_own[row_m] = make_float2(fin_m, fin_l);
         cluster_arrive();
         cluster_wait();
@@ -470,18 +473,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 if (pl[q] * wq > 0.f) live_peers |= 1u << q;
                 if (q == (int)my_rank) w_own = wq;
             }
-            if (fin_l > 0.f && fin_ok) {
+            {
+                // (the tensor-memory loads are warp-wide: every lane takes part, whatever its own row's weight; a row without
+                // weight in this slice, or a slice without tiles whose accumulator was never written, stages nothing)
                 tc_fence_after();
                 const uint32_t lane_addr_m = (uint32_t)((warp & 3) * 32) << 16;
+                const bool mine = fin_l > 0.f && w_own > 0.f && fin_ok;
 #pragma unroll 1
                 for (int c = 0; c < HD / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tmem_base + lane_addr_m + kColO + c * 32, o);
                     tmem_wait_ld();
+                    if (mine) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        stage[(c * 8 + i) * 128 + row_m] = make_float4(__uint_as_float(o[4 * i]) * w_own, __uint_as_float(o[4 * i + 1]) * w_own,
-                                                                       __uint_as_float(o[4 * i + 2]) * w_own, __uint_as_float(o[4 * i + 3]) * w_own);
+                        for (int i = 0; i < 8; ++i)
+                            stage[(c * 8 + i) * 128 + row_m] = make_float4(__uint_as_float(o[4 * i]) * w_own, __uint_as_float(o[4 * i + 1]) * w_own,
+                                                                           __uint_as_float(o[4 * i + 2]) * w_own, __uint_as_float(o[4 * i + 3]) * w_own);
+                    }
                 }
             }
         }
@@ -649,14 +657,46 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
     cfg.blockDim = dim3(kTc2Threads);
     cfg.dynamicSmemBytes = Tc2Smem<HD>::TOTAL;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // a pair of CTAs, or all the pairs that merge their key slices
+    attr[1].val.clusterDim.x = 2u * (unsigned)(tp.cluster_merge ? tp.nsplit : 1); attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc2_kernel<HD>, *mq, *mk, *mv, *mkd, *mvd, *mo, tp);
     count_launch();
     return e;
+}
+
+// how many clusters of `cluster_ctas` CTAs of the two-CTA kernel the device holds at once (asked once per shape; clusters
+// of 8 fit only once or twice per GPC, far fewer than SMs / 8)
+template <int HD>
+int tc2_active_clusters_t(int cluster_ctas)
+{
+    static int cached[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    if (cluster_ctas < 2 || cluster_ctas > 8) return 0;
+    if (cached[cluster_ctas] != 0) return cached[cluster_ctas] > 0 ? cached[cluster_ctas] : 0;
+    int n = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cluster_ctas * 64u);
+    cfg.blockDim = dim3(kTc2Threads);
+    cfg.dynamicSmemBytes = Tc2Smem<HD>::TOTAL;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster_ctas; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Tc2Smem<HD>::TOTAL);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveClusters(&n, attn_tc2_kernel<HD>, &cfg);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+    cached[cluster_ctas] = n > 0 ? n : -1;
+    return n > 0 ? n : 0;
+}
+
+int tc2_active_clusters(int d, int cluster_ctas)
+{
+    return d == 256 ? tc2_active_clusters_t<256>(cluster_ctas) : d == 128 ? tc2_active_clusters_t<128>(cluster_ctas) : 0;
 }
 
 }  // namespace
@@ -715,6 +755,35 @@ bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 
 // splitting costs a fixed 3 us (merge launch) plus the fp32 partials' round trip through memory. Measured at the
 // 898-key shape: 1 stream 14.4 us with 8 slices; 2 streams 15.4 with 4; 4 streams 17.5 with 4; 8 to 32 streams 19.5 to
 // 21.7 unsplit (split in two: 21.6 to 40); at 4466 keys and 16 streams 41 us split in two, 51 unsplit, 47 in four.
+// The nsplit pairs that share a tile pair can merge inside one cluster (no partials, no merge launch) when the cluster stays
+// within the portable size of 8 CTAs, all clusters are resident at once with exactly one unit each, and a thread's share of
+// the columns is whole 16-byte stores. Measured against the split with partials: 4466 keys, 16 streams 41.2 -> 35.6 us
+// (two slices); 898 keys, 4 streams 18.5 -> 16.5 (four slices); one stream 15.5 merged in four against 14.4 with eight
+// slices and the merge kernel, and 2 streams 16.5 merged in four against 15.9 with partials. The model therefore charges
+// the in-cluster merge 5.5 us (three cluster barriers and the staged reduction keep every CTA of the cluster that long)
+// and uses it only where the partials' round trip would cost more.
+static constexpr double kTc2MergedUs = 5.5;
+static double tc2_partials_us(const AttnParams &p, int nsplit)   // merge launch + fp32 partials written and read back
+{
+    const double per_split_bytes = (double)p.B * p.T * p.Hq * (p.d + 2) * sizeof(float);
+    return 3.0 + 2.0 * per_split_bytes * nsplit / 3.4e6;
+}
+static bool tc2_cluster_merge_ok(const AttnParams &p, int nsplit, int sm_count)
+{
+    if (nsplit != 2 && nsplit != 4) return false;
+    const int G = p.Hq / p.Hkv;
+    const int tile_tokens = kBM / G;
+    const int n_pairs = ((p.T + tile_tokens - 1) / tile_tokens + 1) / 2;
+    const int base_units = n_pairs * p.Hkv * p.B;
+    if (base_units * nsplit * 2 > sm_count) return false;
+    // all clusters resident at once (a second wave would wait for whole clusters). Clusters of 8 get a margin: 16 of them,
+    // the most the device reports, measured 20.4 us where 12 took 17.5 and the unsplit kernel 19.5.
+    const int active = tc2_active_clusters(p.d, 2 * nsplit);
+    if (base_units > (nsplit == 4 ? active - active / 4 : active)) return false;
+    if (tc2_partials_us(p, nsplit) <= kTc2MergedUs) return false;
+    return (p.d / 4 / nsplit / kTc2Parts) % 2 == 0 && p.d / 4 / nsplit / kTc2Parts >= 2;
+}
+
 int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
 {
     const int G = p.Hq / p.Hkv;
@@ -730,10 +799,11 @@ int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
     double best_us = 1e30;
     for (int ns = 1; ns <= 8; ns *= 2) {
         if (ns > tiles) break;
-        if (ns > 1 && per_split_bytes * ns > (double)partial_bytes) break;
-        const int waves = (units * ns + clusters - 1) / clusters;
+        const bool merged = ns > 1 && tc2_cluster_merge_ok(p, ns, sm_count);
+        if (ns > 1 && !merged && per_split_bytes * ns > (double)partial_bytes) break;
+        const int waves = merged ? 1 : (units * ns + clusters - 1) / clusters;
         const double loop_us = 1.3 * waves * ((tiles + ns - 1) / ns);
-        const double split_us = ns > 1 ? 3.0 + 2.0 * per_split_bytes * ns / 3.4e6 : 0.0;
+        const double split_us = ns == 1 ? 0.0 : (merged ? kTc2MergedUs : tc2_partials_us(p, ns));
         if (loop_us + split_us < best_us - 0.05) { best_us = loop_us + split_us; best = ns; }
     }
     return best;
@@ -755,7 +825,8 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     tp.nsplit = p.nsplit;
     tp.tile_tokens = kBM / G;
     tp.n_qtiles = (p.T + tp.tile_tokens - 1) / tp.tile_tokens;
-    tp.cluster_merge = (!two_cta && p.nsplit > 1 && p.nsplit <= 8 && (p.d / 4) % (2 * p.nsplit) == 0) ? 1 : 0;
+    tp.cluster_merge = two_cta ? (tc2_cluster_merge_ok(p, p.nsplit, sm_count) ? 1 : 0)
+                               : ((p.nsplit > 1 && p.nsplit <= 8 && (p.d / 4) % (2 * p.nsplit) == 0) ? 1 : 0);
     cudaError_t e;
     if (two_cta) {
         // persistent grid: one cluster (two CTAs) per SM pair walks the (stream, KV head, tile pair) units;
@@ -767,11 +838,11 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
         int clusters = sm_count / 2;
         if (clusters > units) clusters = units;
         if (clusters < 1) clusters = 1;
-        dim3 grid2(2 * clusters, 1, 1);
+        dim3 grid2(2 * clusters, 1, 1);                      // with cluster_merge: units pairs = units / nsplit clusters of 2 * nsplit CTAs
         if (p.d == 256) e = launch2_t<256>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
         else if (p.d == 128) e = launch2_t<128>(&mq, &mk, &mv, &mkd, &mvd, &mo, tp, grid2, st);
         else return cudaErrorInvalidValue;
-        if (e != cudaSuccess || p.nsplit == 1) return e;
+        if (e != cudaSuccess || p.nsplit == 1 || tp.cluster_merge) return e;
         return launch_attention_merge(p, st);
     }
     dim3 grid(tp.n_qtiles * p.Hkv, p.B, p.nsplit);

@@ -110,7 +110,7 @@ template <int HD> struct Tc2Smem {
 
 // (18 warps are five on at least one of the four schedulers, whose 16 K registers then allow 96 per thread)
 template <int HD>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTc2Threads, 1)
+__global__ void __launch_bounds__(kTc2Threads, 1)   // launched as clusters of 2 CTAs, or of 2 * nsplit (cluster_merge)
 attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_kd,
                 const __grid_constant__ CUtensorMap tm_vd, const __grid_constant__ CUtensorMap tm_o, const TcParams p)
@@ -143,10 +143,20 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 64) TC2_TRACE(2, 15, 0);
-    const uint32_t rank = cluster_ctarank();
-    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    // A pair of CTAs (cluster ranks 2k, 2k+1) drives the cta_group::2 MMAs. Normally the cluster is one pair and walks a
+    // list of units; with cluster_merge the cluster holds the nsplit pairs that share one query tile pair, each taking a
+    // slice of the keys, and merges their (m, l, O) through distributed shared memory at the end (one unit per cluster).
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t rank = crank & 1u, lead = crank & ~1u;      // rank inside the pair; cluster rank of the pair's leader
+    const uint16_t pair_mask = (uint16_t)(3u << lead);         // both CTAs of this pair, for multicast commits
+    const int pairs_per_cluster = p.cluster_merge ? p.nsplit : 1;
+    const int cluster_id = blockIdx.x / (2 * pairs_per_cluster);
+    const int n_clusters = gridDim.x / (2 * pairs_per_cluster);
     const int n_pairs = p.n_qtiles;                    // tile pairs per (stream, KV head)
     const int n_units = p.B * p.Hkv * n_pairs * p.nsplit;   // with nsplit > 1 a unit covers a slice of the key tiles
+    // this pair's first unit and the stride to its next one
+    const int u_start = p.cluster_merge ? cluster_id * p.nsplit + (int)(crank >> 1) : cluster_id;
+    const int u_stride = p.cluster_merge ? n_units : n_clusters;
 
     // geometry of one work unit
     struct Unit { int b, kvh, t0, H, n_tiles, tile0, split; TileGeom g; };
@@ -213,6 +223,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         return false;
     };
 
+    // what a softmax thread carries into the in-cluster merge: its row's reference maximum (log2 units) and sum
+    float fin_m = -INFINITY, fin_l = 0.f;
+    bool fin_ok = true;
+
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
@@ -226,14 +240,14 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             struct Cursor { int u, ui, jj, g; bool valid; Unit w; };
             auto settle = [&](Cursor &c) {   // first unit at or after c.u with a non-empty key slice
                 c.valid = false;
-                for (; c.u < n_units; c.u += n_clusters) {
+                for (; c.u < n_units; c.u += u_stride) {
                     c.w = load_unit(c.u);
                     if (c.w.n_tiles > 0) { c.valid = true; c.jj = 0; return; }
                 }
             };
             auto advance = [&](Cursor &c) {
                 ++c.g;
-                if (++c.jj == c.w.n_tiles) { c.u += n_clusters; ++c.ui; settle(c); }
+                if (++c.jj == c.w.n_tiles) { c.u += u_stride; ++c.ui; settle(c); }
             };
             bool ok = true;
             auto issue_k = [&](const Cursor &c) {
@@ -282,7 +296,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             };
             Cursor ck, cv;
-            ck.u = cluster_id; ck.ui = 0; ck.jj = 0; ck.g = 0;
+            ck.u = u_start; ck.ui = 0; ck.jj = 0; ck.g = 0;
             settle(ck);
             cv = ck;
             if (kLead == 1 && ck.valid) { issue_k(ck); advance(ck); }
@@ -325,14 +339,14 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     umma_desc_advance(qd, (kk & 3) == 3 ? 128 * 128 - 96 : 32);
                     umma_desc_advance(kd, (kk & 3) == 3 ? 64 * 128 - 96 : 32);
                 }
-                umma2_commit_mc_elect(bar(C_KEMPTY + st), 3);
-                umma2_commit_mc_elect(bar(C_SFULL + buf), 3);
-                if (last) umma2_commit_mc_elect(bar(C_QEMPTY), 3);
+                umma2_commit_mc_elect(bar(C_KEMPTY + st), pair_mask);
+                umma2_commit_mc_elect(bar(C_SFULL + buf), pair_mask);
+                if (last) umma2_commit_mc_elect(bar(C_QEMPTY), pair_mask);
                 return true;
             };
             bool ok = true;
             int gt = 0, ui = 0;
-            for (int u = cluster_id; u < n_units && ok; u += n_clusters, ++ui) {
+            for (int u = u_start; u < n_units && ok; u += u_stride, ++ui) {
                 const Unit w = load_unit(u);
                 const int n = w.n_tiles;
                 if (n == 0) { --ui; continue; }
@@ -352,8 +366,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         umma2_ts_elect(tmem_base + kColO, p_tmem + kk * 8, vd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
                         umma_desc_advance(vd, 16 * 128);   // the next 16 keys
                     }
-                    umma2_commit_mc_elect(bar(C_VEMPTY + st), 3);
-                    umma2_commit_mc_elect(bar(C_PVDONE + buf), 3);
+                    umma2_commit_mc_elect(bar(C_VEMPTY + st), pair_mask);
+                    umma2_commit_mc_elect(bar(C_PVDONE + buf), pair_mask);
                 }
                 gt += n;
             }
@@ -373,21 +387,21 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int quarter = warp & 3;             // TMEM lane quarter this warp may touch
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        const uint32_t leader_pfull[2] = {mapa(bar(C_PFULL), 0), mapa(bar(C_PFULL + 1), 0)};
-        const uint32_t leader_ofree = mapa(bar(C_OFREE), 0);
+        const uint32_t leader_pfull[2] = {mapa(bar(C_PFULL), lead), mapa(bar(C_PFULL + 1), lead)};
+        const uint32_t leader_ofree = mapa(bar(C_OFREE), lead);
         uint16_t *xmax = reinterpret_cast<uint16_t *>(smem + L::OFF_XMAX);   // [2 buffers][128 rows][NP], bf16 bit patterns
         float *xsum = reinterpret_cast<float *>(smem + L::OFF_XSUM);         // [NP][128 rows]
         bool ok = true;
         int gt = 0;
         [[maybe_unused]] int ui_s = 0;
-        for (int u = cluster_id; u < n_units; u += n_clusters, ++ui_s) {
+        for (int u = u_start; u < n_units; u += u_stride, ++ui_s) {
             const Unit w = load_unit(u);
             const int t_row = w.t0 + row / p.G;
             if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 0);
             const int rows_total = p.T * p.Hq;
             const size_t n_slots = (size_t)p.B * rows_total * p.nsplit;
             float *pml = nullptr;    // this row's (m, l) slot when the keys are split over several units
-            if (p.nsplit > 1 && t_row < p.T)
+            if (p.nsplit > 1 && !p.cluster_merge && t_row < p.T)   // (merged inside the cluster: no partials exist)
                 pml = partial_ml(p.partials, n_slots, partial_slot(w.b, rows_total, t_row * p.Hq + w.kvh * p.G + row % p.G, p.nsplit, w.split), HD);
             if (w.n_tiles == 0) {
                 if (pml && part == 0) { pml[0] = -INFINITY; pml[1] = 0.f; }   // an empty key slice contributes nothing
@@ -559,7 +573,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             gt += w.n_tiles;
             // ---- epilogue of the unit ----
             // (before this cluster's last epilogue: let the next kernel on the stream be scheduled; it waits for this grid's end)
-            if (threadIdx.x == 64 && u + n_clusters >= n_units) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            if (threadIdx.x == 64 && u + u_stride >= n_units) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             // The threads of a row add their sums; each thread takes its share of the head_dim columns out of tensor
             // memory, 32 at a time, and stores its row segment straight to global memory in 32-byte pieces (whole sectors).
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 2); TC2_TRACE(2, ui_s, 2); }
@@ -577,6 +591,13 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const bool row_live = t_row < p.T;
             const int hq = w.kvh * p.G + row % p.G;
             constexpr int EC = HD / NP;            // this thread's columns of O
+            if (p.cluster_merge) {
+                // the slices of this tile pair meet in the merge phase at the end of the kernel (this pair has no other unit)
+                fin_m = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale_log2;
+                fin_l = l;
+                fin_ok = ok;
+                continue;
+            }
             if (p.nsplit > 1) {
                 // key-split unit: leave (m, l, unnormalised O) for the merge kernel; m in natural-log units like the other kernels
                 if (pml && part == 0) { pml[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; pml[1] = l; }
@@ -649,6 +670,112 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 4); TC2_TRACE(2, ui_s, 4); }
         }
         if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores of this CTA are complete
+    }
+
+    if (p.cluster_merge) {
+        // ---- merge of the key slices inside the cluster ----
+        // Pair q of the cluster holds slice q of the keys for the same 256 query rows; CTAs of equal rank inside their pairs
+        // hold the same 128 rows. 1. every row's (m, l) is published; 2. with all slices' (m, l) each thread scales its
+        // share of its O row to the common maximum and stages it in shared memory (Q and K buffers, idle now), column-major
+        // in 16-byte units; 3. pair q adds up columns [q, q+1) * head_dim / nsplit of all slices through distributed shared
+        // memory, divides by the common sum and writes bf16. A cluster barrier after 1 and after 2; the one at the end of
+        // the kernel keeps every CTA alive while a peer may still read its staging area.
+        constexpr int NP = kTc2Parts;
+        const int ns = p.nsplit;
+        const int sw = warp - 2, part = sw >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        float2 *ml_own = reinterpret_cast<float2 *>(smem + L::OFF_STAGE);      // [128 rows]
+        float4 *stage = reinterpret_cast<float4 *>(smem + L::OFF_Q);           // [HD / 4][128 rows]
+        static_assert(L::OFF_K == L::OFF_Q + L::Q_BYTES && L::Q_BYTES + L::NKS * L::K_STAGE >= (uint32_t)HD * 128 * 4, "staging area of the merge");
+        // (the cluster barriers are warp-aligned instructions: the lanes of the producer warp that idled while lane 0 ran the
+        // loads must not reach them before lane 0 does, so the CTA meets here first)
+        __syncthreads();
+        if (warp >= 2 && part == 0) ml_own[row] = make_float2(fin_m, fin_l);
+        cluster_arrive();
+        cluster_wait();
+        float wgt[8], l_all = 0.f;
+        if (warp >= 2) {
+            float pm[8], mstar = -INFINITY;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                pm[q] = -INFINITY; wgt[q] = 0.f;
+                if (q < ns) {
+                    float lq;
+                    const uint32_t a = mapa(smem_u32(ml_own + row), (uint32_t)(2 * q) + rank);
+                    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(pm[q]), "=f"(lq) : "r"(a) : "memory");
+                    wgt[q] = lq;                                   // the sum for now
+                    if (!(lq > 0.f)) pm[q] = -INFINITY;            // a slice that saw nothing live has no say
+                    mstar = fmaxf(mstar, pm[q]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const float e = (pm[q] == -INFINITY) ? 0.f : ex2(pm[q] - mstar);
+                l_all = fmaf(wgt[q], e, l_all);
+                wgt[q] = e;
+            }
+            float w_own = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (q == (int)(crank >> 1)) w_own = wgt[q];
+            {
+                // (the tensor-memory loads are warp-wide: every lane takes part, whatever its own row's weight; a row without
+                // weight in this slice, or a slice without tiles whose accumulator was never written, stages nothing)
+                tc_fence_after();
+                const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+                constexpr int EC = HD / NP;
+                const bool mine = w_own > 0.f && fin_ok;
+#pragma unroll 1
+                for (int c = 0; c < EC / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tmem_base + lane_addr + kColO + part * EC + c * 32, o);
+                    tmem_wait_ld();
+                    if (mine) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            stage[((part * EC + c * 32) / 4 + i) * 128 + row] =
+                                make_float4(__uint_as_float(o[4 * i]) * w_own, __uint_as_float(o[4 * i + 1]) * w_own,
+                                            __uint_as_float(o[4 * i + 2]) * w_own, __uint_as_float(o[4 * i + 3]) * w_own);
+                    }
+                }
+            }
+        }
+        cluster_arrive();
+        cluster_wait();
+        if (warp >= 2 && fin_ok) {
+            // this pair's columns [crank/2 * HD/ns, +HD/ns), split between the NP threads of the row
+            const int uu = u_start / p.nsplit, pair = uu % n_pairs, kvh = (uu / n_pairs) % p.Hkv, b = uu / (n_pairs * p.Hkv);
+            const int t_row = (2 * pair + (int)rank) * p.tile_tokens + row / p.G;
+            const int c4_thread = HD / 4 / ns / NP;                                    // float4 columns per thread
+            const int c4_0 = (int)(crank >> 1) * (HD / 4 / ns) + part * c4_thread;
+            if (t_row < p.T && l_all > 0.f) {
+                const float inv = 1.f / l_all;
+                __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + kvh * p.G + row % p.G) * HD + c4_0 * 4;
+#pragma unroll 1
+                for (int c4 = 0; c4 < c4_thread; c4 += 2) {                          // 8 columns = one 16-byte store at a time
+                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (q < ns && wgt[q] > 0.f) {
+                            const uint32_t a = mapa(smem_u32(stage + (c4_0 + c4) * 128 + row), (uint32_t)(2 * q) + rank);
+                            float4 v0, v1;
+                            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v0.x), "=f"(v0.y), "=f"(v0.z), "=f"(v0.w) : "r"(a) : "memory");
+                            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v1.x), "=f"(v1.y), "=f"(v1.z), "=f"(v1.w) : "r"(a + 128 * 16) : "memory");
+                            acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+                            acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+                        }
+                    }
+                    uint4 v;
+                    uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
+                        vv[k] = *reinterpret_cast<uint32_t *>(&h);
+                    }
+                    *reinterpret_cast<uint4 *>(orow + c4 * 4) = v;
+                }
+            }
+        }
     }
 
     tc_fence_before();

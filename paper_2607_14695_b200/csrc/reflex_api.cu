@@ -95,6 +95,13 @@ WorkspaceLayout workspace_layout(const reflex_cache_desc &d)
     const size_t blocks = ((rows + 3) / 4) * (size_t)d.B;
     size_t splits = (8 * 148 + blocks - 1) / blocks;
     if (splits < 2) splits = 2;     // the batched two-CTA kernel may split the keys when streams alone do not fill the SM pairs
+    if (d.Hkv > 0 && d.Hq % d.Hkv == 0 && d.Hq / d.Hkv <= 128) {
+        // ... up to one unit per SM pair: (stream, KV head, pair of query tiles) units times key slices
+        const size_t tile_tokens = 128 / (size_t)(d.Hq / d.Hkv);
+        const size_t units = (((size_t)d.T_max + tile_tokens - 1) / tile_tokens + 1) / 2 * (size_t)d.Hkv * (size_t)d.B;
+        const size_t fill = units > 0 ? 74 / units : 0;
+        if (fill > splits) splits = fill;
+    }
     if (splits > (size_t)kMaxSplits) splits = kMaxSplits;
     w.partial_off = off;
     w.partial_bytes = align_up(splits * (size_t)d.B * rows * (size_t)(d.d + 2) * sizeof(float), 256);

@@ -105,7 +105,10 @@ class Twin:
                                         scale=scale, dyn_mask=dyn_mask)
         rb.reflex_cache_check_status(self.g)   # no bounded device-side wait ran out
         got = to_host(out)
-        assert np.isfinite(got).all(), f"{what}: non-finite output"
+        if not np.isfinite(got).all():
+            bad = np.argwhere(~np.isfinite(got))
+            raise AssertionError(f"{what}: non-finite output, {len(bad)} elements; streams {np.unique(bad[:, 0])[:8]}, tokens {np.unique(bad[:, 1])[:12]}, "
+                                 f"heads {np.unique(bad[:, 2])}, columns {np.unique(bad[:, 3])[:6]}..{bad[:, 3].max()} ({len(np.unique(bad[:, 3]))})")
         streams = list(range(w.B)) if streams is None else streams
         res = []
         for b in streams:
