@@ -184,6 +184,38 @@ int reflex_oracle_adarmsnorm(const float *x, const float *c, const float *W1, co
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Adaptive norm followed by the packed projection (Sec. 3.3 "System Optimizations": the query,
+ * key and value projections as one matrix W_QKV = [W_Q; W_K; W_V]; Sec. 4 "Operator Fusion
+ * Impact": the adaptive norm combined with the linear layer after it). By definition
+ *   y = AdaRMSNorm(x; gamma)   (Eq. 2, y kept in double: the fused form never materialises it)
+ *   out[r][n] = sum_i y[r][i] * Wp[n][i]
+ *   x [R][D]  gamma [D] (from reflex_oracle_adarmsnorm)  Wp [Nout][D] (row n = output feature n)
+ *   -> out [R][Nout]; the caller slices the columns into Q, K and V.
+ * ------------------------------------------------------------------------------------------ */
+int reflex_oracle_adarmsnorm_linear(const float *x, const double *gamma, const float *Wp, int R, int D,
+                                    int Nout, double eps, double *out)
+{
+    double *y = (double *)malloc(sizeof(double) * (size_t)R * (size_t)D);
+    if (!y) return -1;
+    for (int r = 0; r < R; ++r) {
+        const float *xr = x + (size_t)r * D;
+        double ss = 0.0;
+        for (int i = 0; i < D; ++i) ss += (double)xr[i] * (double)xr[i];
+        const double rms = sqrt(ss / (double)D + eps);
+        for (int i = 0; i < D; ++i) y[(size_t)r * D + i] = (double)xr[i] / rms * gamma[i];
+    }
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < R; ++r)
+        for (int n = 0; n < Nout; ++n) {
+            double acc = 0.0;
+            for (int i = 0; i < D; ++i) acc += y[(size_t)r * D + i] * (double)Wp[(size_t)n * D + i];
+            out[(size_t)r * Nout + n] = acc;
+        }
+    free(y);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Flow-matching update (Sec. 2.1 "ODE integration", Sec. 3.2 x ~ N(0,I) at t = 1, Appendix C
  * "Flow matching steps 10"): forward Euler with K uniform steps from t = 1 to t = 0,
  *   x <- x + dt * v,  dt = -1/K.

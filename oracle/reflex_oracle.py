@@ -54,6 +54,8 @@ def lib():
         _lib.reflex_oracle_attention_part.restype = i
         _lib.reflex_oracle_adarmsnorm.argtypes = [fp, fp, fp, fp, fp, fp, i, i, i, i, d, dp, dp]
         _lib.reflex_oracle_adarmsnorm.restype = i
+        _lib.reflex_oracle_adarmsnorm_linear.argtypes = [fp, dp, fp, i, i, i, d, dp]
+        _lib.reflex_oracle_adarmsnorm_linear.restype = i
         _lib.reflex_oracle_flow_step.argtypes = [dp, fp, ctypes.c_long, i]
         _lib.reflex_oracle_flow_step.restype = None
         _lib.reflex_oracle_flow_time.argtypes = [i, i]
@@ -124,6 +126,22 @@ def adarmsnorm(x, c, W1, b1, W2, b2, eps=1e-6, return_gate=False):
 def adarmsnorm_batched(x, cond, W1, b1, W2, b2, eps=1e-6):
     """x [B][R][D], cond [B][Cd]: one gate per stream."""
     return np.stack([adarmsnorm(x[b], cond[b], W1, b1, W2, b2, eps) for b in range(x.shape[0])])
+
+
+def adarmsnorm_qkv(x, c, W1, b1, W2, b2, Wqkv, Hq, Hkv, d, eps=1e-6):
+    """Eq. 2 followed by the packed projection W_QKV = [W_Q; W_K; W_V] for one stream:
+    x [R][D], Wqkv [(Hq + 2 Hkv) d][D] -> q [R][Hq][d], k [R][Hkv][d], v [R][Hkv][d], all f64."""
+    _, g = adarmsnorm(x, c, W1, b1, W2, b2, eps, return_gate=True)
+    x, xp = _f(x); Wqkv, wp = _f(Wqkv)
+    R, D = x.shape
+    Nout = Wqkv.shape[0]
+    assert Nout == (Hq + 2 * Hkv) * d and Wqkv.shape[1] == D
+    out = np.empty((R, Nout), np.float64)
+    rc = lib().reflex_oracle_adarmsnorm_linear(xp, _dptr(g), wp, R, D, Nout, float(eps), _dptr(out))
+    if rc != 0:
+        raise MemoryError("oracle adarmsnorm_linear")
+    nq, nk = Hq * d, Hkv * d
+    return out[:, :nq].reshape(R, Hq, d), out[:, nq:nq + nk].reshape(R, Hkv, d), out[:, nq + nk:].reshape(R, Hkv, d)
 
 
 def flow_step(x, v, K):
