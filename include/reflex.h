@@ -182,6 +182,26 @@ int reflex_adarmsnorm_noalloc(const void *x, void *y, const void *cond, const vo
                               const void *W2, const void *b2, int B, int R, int D, int Cd, int Hd, float eps,
                               int dtype, void *stream);
 
+/* Sec. 3.3 "System Optimizations" (the query, key and value projections as one packed matrix W_QKV = [W_Q; W_K; W_V])
+ * with the adaptive norm of Eq. 2 folded in (Sec. 4 "Operator Fusion Impact": the norm combined with the linear layer
+ * after it, the norm output never written to memory). For every row r of stream b:
+ *   y = x[r] / RMS(x[r]) * gamma_b,   [q | k_dyn | v_dyn][r] = W_QKV y
+ * One launch; the outputs have the layouts reflex_partitioned_attention reads.
+ *   cache    a cache whose status word records a device-side wait that ran out (reflex_cache_check_status), or NULL
+ *   x        device [B][R][D] dtype
+ *   gate     device fp32 [B][D]: gamma of every stream, as reflex_adarmsnorm_gate writes it
+ *   Wqkv     device [(Hq + 2 Hkv) d][D] dtype: one row per output feature; rows of W_Q (head-major) first, then W_K, then W_V
+ *   q        device [B][R][Hq][d] dtype;   k_dyn, v_dyn  device [B][R][Hkv][d] dtype   (written; all rows)
+ *   impl     0: tensor cores when dtype is bf16 and D % 64 == 0, else the plain kernel; 1: the plain kernel (fp32 FMAs)
+ * Arithmetic on the tensor-core path: products of bf16(x * gamma) and W_QKV accumulated in fp32, the row's 1/RMS applied
+ * to the accumulator, one rounding to bf16 at the end.
+ * Requirements: D % 8 == 0, D <= 8192; d % 8 == 0; Hq % Hkv == 0; (Hq + 2 Hkv) d <= 65536; 16-byte aligned pointers.
+ * Errors: REFLEX_ERR_INVALID_ARG (NULL pointer, unknown dtype or impl, eps < 0), REFLEX_ERR_SHAPE, REFLEX_ERR_ALIGN;
+ * nothing is launched and nothing written on error. */
+int reflex_adarmsnorm_qkv(reflex_cache_t *cache, const void *x, const float *gate, const void *Wqkv, void *q,
+                          void *k_dyn, void *v_dyn, int B, int R, int D, int Hq, int Hkv, int d, float eps,
+                          int dtype, int impl, void *stream);
+
 /* Eq. 1 / App. A Prop. 1: for every stream b, KV head j and its G*T query rows,
  *   out = softmax(scale * Q [K_pin; K_slide; K_dyn]^T) [V_pin; V_slide; V_dyn]
  * over static rows [0, static_len[b]), the live ring slots (physical order; softmax does not depend

@@ -26,7 +26,8 @@ EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
-    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_partitioned_attention", "reflex_flow_step",
+    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_partitioned_attention",
+    "reflex_flow_step",
 ]
 
 
@@ -70,6 +71,7 @@ def load():
     lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_adarmsnorm_gate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, vp]
     lib.reflex_adarmsnorm_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
+    lib.reflex_adarmsnorm_qkv.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
     for name in EXPORTS:
@@ -238,6 +240,16 @@ def reflex_adarmsnorm_noalloc(x, y, cond, W1, b1, W2, b2, eps=1e-6, stream=None)
     _check(load().reflex_adarmsnorm_noalloc(_ptr(x), _ptr(y), _ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2),
                                             B, R, D, int(Cd), int(Hd), float(eps), dtype_code(x), _stream(stream)))
     return y
+
+
+def reflex_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, eps=1e-6, impl=0, cache=None, stream=None):
+    """x [B][R][D], gate fp32 [B][D], Wqkv [(Hq + 2 Hkv) d][D] -> q [B][R][Hq][d], k_dyn / v_dyn [B][R][Hkv][d]."""
+    B, R, D = x.shape
+    Hq, d = int(q.shape[2]), int(q.shape[3])
+    Hkv = int(k_dyn.shape[2])
+    _check(load().reflex_adarmsnorm_qkv(cache.handle if cache is not None else None, _ptr(x), _ptr(gate), _ptr(Wqkv), _ptr(q), _ptr(k_dyn),
+                                        _ptr(v_dyn), B, R, D, Hq, Hkv, d, float(eps), dtype_code(x), int(impl), _stream(stream)))
+    return q, k_dyn, v_dyn
 
 
 def reflex_partitioned_attention(cache: Cache, layer, q, k_dyn, v_dyn, out, scale=0.0, dyn_mask=0, stream=None):

@@ -347,6 +347,25 @@ int reflex_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, con
     return REFLEX_OK;
 }
 
+int reflex_adarmsnorm_qkv(reflex_cache_t *c, const void *x, const float *gate, const void *Wqkv, void *q, void *k_dyn, void *v_dyn,
+                          int B, int R, int D, int Hq, int Hkv, int d, float eps, int dtype, int impl, void *stream)
+{
+    if (dtype != REFLEX_DTYPE_BF16 && dtype != REFLEX_DTYPE_F32) return fail(REFLEX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (impl != 0 && impl != 1) return fail(REFLEX_ERR_INVALID_ARG, "impl must be 0 (auto) or 1 (plain kernel)");
+    if (!x || !gate || !Wqkv || !q || !k_dyn || !v_dyn) return fail(REFLEX_ERR_INVALID_ARG, "NULL argument");
+    if (B < 1 || R < 1 || (long long)B * R > 0x7FFFFFFF / 2) return fail(REFLEX_ERR_SHAPE, "B=%d, R=%d", B, R);
+    if (D < 8 || D % 8 != 0 || D > 8192) return fail(REFLEX_ERR_SHAPE, "D=%d must be a multiple of 8 in [8, 8192]", D);
+    if (Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || d < 8 || d % 8 != 0 || (long long)(Hq + 2 * Hkv) * d > 65536)
+        return fail(REFLEX_ERR_SHAPE, "Hq=%d, Hkv=%d, d=%d: need Hq %% Hkv == 0, d a multiple of 8, (Hq + 2 Hkv) d <= 65536", Hq, Hkv, d);
+    if (!(eps >= 0.f)) return fail(REFLEX_ERR_INVALID_ARG, "eps must be >= 0");
+    if (!aligned16(x) || !aligned16(gate) || !aligned16(Wqkv) || !aligned16(q) || !aligned16(k_dyn) || !aligned16(v_dyn))
+        return fail(REFLEX_ERR_ALIGN, "x / gate / Wqkv / q / k_dyn / v_dyn not 16-byte aligned");
+    uint32_t *status = c ? (uint32_t *)(c->ws + c->lay.status_off) : nullptr;
+    cudaError_t e = launch_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, B, R, D, Hq * d, Hkv * d, eps, dtype, impl, status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "adarmsnorm qkv launch");
+    return REFLEX_OK;
+}
+
 int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, const void *k_dyn, const void *v_dyn,
                                  void *out, int T, float scale, int dyn_mask, void *stream)
 {

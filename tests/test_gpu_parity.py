@@ -395,3 +395,64 @@ def test_gate_for_all_layers_matches_per_layer_calls_and_oracle(U):
         rb.reflex_adarmsnorm(dx, y2, dcond, W1s[l], b1s[l], W2s[l], b2s[l], gate_buf=one)
         assert torch.equal(y1, y2)
         U.check_close(U.to_host(y1), orc.adarmsnorm_batched(x, cond, *Ws[l], 1e-6), w.dtype, f"rows with step gates, layer {l}", rel_clause=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# adaptive norm folded into the packed Q/K/V projection
+# ------------------------------------------------------------------------------------------------
+def _norm_qkv_case(U, w, impl, what, t=0.3, eps=1e-6):
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    x = synth.norm_input(w, 0, 0)
+    cond = synth.cond_vectors(w, t)
+    W1, b1, W2, b2 = synth.gate_weights(w, 0)          # gate near 1: unit-variance outputs, which the bf16 contract presumes
+    Wp = synth.qkv_weights(w, 0)
+    gb = torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=U.DEV)
+    rb.reflex_adarmsnorm_gate(U.to_dev(cond, w.dtype), U.to_dev(W1, w.dtype), U.to_dev(b1, w.dtype), U.to_dev(W2, w.dtype), U.to_dev(b2, w.dtype), gb)
+    dt = rb.torch_dtype(w.dtype)
+    q = torch.full((w.B, w.T, w.Hq, w.d), float("nan"), dtype=dt, device=U.DEV)
+    k = torch.full((w.B, w.T, w.Hkv, w.d), float("nan"), dtype=dt, device=U.DEV)
+    v = torch.full((w.B, w.T, w.Hkv, w.d), float("nan"), dtype=dt, device=U.DEV)
+    rb.reflex_adarmsnorm_qkv(U.to_dev(x, w.dtype), gb[: w.B * w.D].view(w.B, w.D), U.to_dev(Wp, w.dtype), q, k, v, eps=eps, impl=impl)
+    torch.cuda.synchronize()
+    for b in range(w.B):
+        wq, wk, wv = orc.adarmsnorm_qkv(x[b], cond[b], W1, b1, W2, b2, Wp, w.Hq, w.Hkv, w.d, eps)
+        for got, want, name in ((q, wq, "q"), (k, wk, "k"), (v, wv, "v")):
+            U.check_close(U.to_host(got[b]), want, w.dtype, f"{what} {name} stream {b}", rel_clause=True)
+
+
+def test_norm_qkv_fp32_plain_kernel(U):
+    _norm_qkv_case(U, synth.CONFIGS["cfg1"].with_(B=3), 0, "norm+qkv fp32")
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_norm_qkv_bf16_action_expert_shape(U, impl):
+    """cfg2 shapes (D = 1024, 8 + 1 + 1 heads of 256) for 7 streams of 50 rows: 350 rows = one full 256-row tile pair and a
+    second with 94 rows (its second CTA entirely past the end), 10 column tiles, rows of several streams in one tile."""
+    _norm_qkv_case(U, synth.CONFIGS["cfg2"].with_(B=7), impl, f"norm+qkv bf16 impl {impl}")
+
+
+def test_norm_qkv_bf16_ragged_columns_and_outliers(U):
+    """320 output columns (a second column tile with 64 of 256 live), head_dim 64, D = 192 (three contraction steps, fewer
+    than the stage ring), 300 rows per stream, and x with outliers x1000 as in the long-context configuration."""
+    w = synth.CONFIGS["cfg5"].with_(B=2, T=300, Hq=3, Hkv=1, d=64, D=192, L=1)
+    _norm_qkv_case(U, w, 0, "norm+qkv ragged", t=1e-3)
+
+
+def test_norm_qkv_error_paths(U):
+    rb = U.rb
+    z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device=U.DEV)
+    x, g, W = z(2, 4, 64), torch.ones((2, 64), dtype=torch.float32, device=U.DEV), z(4 * 16, 64)
+    q, k = z(2, 4, 2, 16), z(2, 4, 1, 16)
+    rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k.clone())
+    for bad in (lambda: rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k, impl=2),
+                lambda: rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k, eps=-1.0)):
+        with pytest.raises(rb.ReflexError) as e:
+            bad()
+        assert e.value.code == rb.ERR_INVALID_ARG
+    with pytest.raises(rb.ReflexError) as e:
+        rb.reflex_adarmsnorm_qkv(x, g, W, z(2, 4, 2, 12), z(2, 4, 1, 12), z(2, 4, 1, 12))     # head_dim not a multiple of 8
+    assert e.value.code == rb.ERR_SHAPE
+    with pytest.raises(rb.ReflexError) as e:
+        rb.reflex_adarmsnorm_qkv(x.view(-1)[4:4 + 2 * 3 * 64].view(2, 3, 64), g, W, q[:, :3].contiguous(), k[:, :3].contiguous(), k[:, :3].contiguous())
+    assert e.value.code == rb.ERR_ALIGN
