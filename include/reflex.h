@@ -192,7 +192,9 @@ int reflex_adarmsnorm_noalloc(const void *x, void *y, const void *cond, const vo
  *   gate     device fp32 [B][D]: gamma of every stream, as reflex_adarmsnorm_gate writes it
  *   Wqkv     device [(Hq + 2 Hkv) d][D] dtype: one row per output feature; rows of W_Q (head-major) first, then W_K, then W_V
  *   q        device [B][R][Hq][d] dtype;   k_dyn, v_dyn  device [B][R][Hkv][d] dtype   (written; all rows)
- *   impl     0: tensor cores when dtype is bf16 and D % 64 == 0, else the plain kernel; 1: the plain kernel (fp32 FMAs)
+ *   impl     0: tensor cores when dtype is bf16, D % 64 == 0 and the gates of the streams under 128 consecutive rows fit in
+ *               shared memory ((127 / R + 2) * D * 4 bytes <= 64 KiB), else the plain kernel; 1: the plain kernel (fp32 FMAs);
+ *               2: like 0 but never the 512-column tiles that 0 picks for large problems
  * Arithmetic on the tensor-core path: products of bf16(x * gamma) and W_QKV accumulated in fp32, the row's 1/RMS applied
  * to the accumulator, one rounding to bf16 at the end.
  * Requirements: D % 8 == 0, D <= 8192; d % 8 == 0; Hq % Hkv == 0; (Hq + 2 Hkv) d <= 65536; 16-byte aligned pointers.

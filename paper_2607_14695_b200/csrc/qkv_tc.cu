@@ -3,18 +3,20 @@
 // never reaches memory):
 //     [q | k_dyn | v_dyn][r][n] = (1 / RMS(x_r)) * sum_i (x[r][i] * gamma_b[i]) * W_QKV[n][i]          (Eq. 2 + projection)
 //
-// bf16 path: a pair of CTAs (cta_group::2) owns a 256 x 256 output tile and walks the contraction axis in 64-column
-// steps through a ring of stages. Per step and CTA, TMA brings 128 rows of x and 128 rows of W_QKV into shared memory.
-// Eight warps (two threads per row) read their half row of x, multiply by the stream's gate (staged in shared memory
-// once per CTA), round to bf16 and store the result into a ring of A stages in TENSOR memory (tcgen05.st; the MMA takes
-// its A operand from there), accumulating the row's sum of squares on the way. One elected thread of the leader CTA
-// issues the MMAs into a 256-column fp32 accumulator. The row scale 1/RMS does not depend on the contraction index, so
-// it multiplies the accumulator in the epilogue: the threads that summed a row's squares read that row out of tensor
-// memory, scale, round to bf16 and write it to the Q, K or V tensor its columns belong to.
-// Measured on the way (3200 x 2560 x 1024): x rewritten in place in shared memory as the A operand, gate from global
-// memory: 29.5 us (shared memory carried 96 KB per step and CTA against the 64 KB it moves in a 512-cycle MMA step, and
-// every step waited for an L2 round trip of gate values); x loaded from global memory by the row-owning threads: 40 us
-// (32 different cache lines per load instruction).
+// bf16 path: a pair of CTAs (cta_group::2) owns 256 rows and NACC x 256 output columns (NACC fp32 accumulators of 256
+// columns in tensor memory) and walks the contraction axis in 64-column steps through a ring of shared-memory stages.
+// Per step and CTA, TMA brings 128 rows of x and NACC x 128 rows of W_QKV. Eight warps (two threads per row) multiply
+// the x tile by the stream's gate in place (bf16(x * gamma), the A operand; the gates of the CTA's streams are staged
+// in shared memory once), accumulating the row's sum of squares on the way; one elected thread of the leader CTA
+// issues the tcgen05 MMAs. The row scale 1/RMS does not depend on the contraction index, so it multiplies the
+// accumulator in the epilogue: the threads that summed a row's squares read that row out of tensor memory, scale and
+// round to bf16; the tile is staged in shared memory and written as whole 512-byte rows to the Q, K or V tensor.
+// NACC = 2 where 256-column tiles would not fit the SM pairs in one wave: the gate multiply (ALU work that every column
+// tile of the same rows repeats) is then spread over twice the MMA work, and 3200 x 2560 becomes 65 tiles on 74 pairs.
+// Measured on the way (3200 x 2560 x 1024, NACC = 1, 130 tiles in two waves): in-place rewrite with the gate read from
+// global memory 29.5 us (an L2 round trip of gate values per step on the critical path); x loaded from global memory by
+// the row-owning threads 40 us (32 cache lines per load instruction); A operand stored to tensor memory instead of back
+// to shared memory 23.2 us (the gate multiply, about 700 cycles per step, stayed above the 512 cycles of the MMAs).
 //
 // Any other dtype or shape: a plain kernel (one block per row, fp32 FMAs) with the same semantics.
 #include <cuda.h>
@@ -33,24 +35,24 @@ namespace {
 
 constexpr int kQkThreads = 64 + 256;   // producer warp, MMA warp, eight transform / epilogue warps (two threads per row)
 constexpr int kQkBM = 128;             // rows of x per CTA (256 per pair)
-constexpr int kQkBN = 256;             // output columns per pair (each CTA loads 128 rows of W_QKV)
-constexpr int kQkBK = 64;              // contraction step: one 128-byte swizzled row of W_QKV
-constexpr int kQkStages = 5;
-constexpr int kQkColA = kQkBN;         // tensor memory: accumulator in columns [0, 256), A stages of 32 columns behind it
-constexpr int kQkTmemCols = 512;
-static_assert(kQkColA + kQkStages * (kQkBK / 2) <= kQkTmemCols, "tensor memory budget");
+constexpr int kQkBN = 256;             // output columns per accumulator (each CTA loads 128 rows of W_QKV for it)
+constexpr int kQkBK = 64;              // contraction step: one 128-byte swizzled row
+constexpr int kQkStages = 4;
 constexpr unsigned long long kQkWaitNs = 1000000000ull;
 
+template <int NACC>
 struct QkSmem {
     static constexpr uint32_t X_STAGE = kQkBM * 128;
-    static constexpr uint32_t B_STAGE = (kQkBN / 2) * 128;
+    static constexpr uint32_t B_HALF = (kQkBN / 2) * 128;     // 128 rows of W_QKV: this CTA's half of one accumulator's B operand
+    static constexpr uint32_t B_STAGE = NACC * B_HALF;
     static constexpr uint32_t OFF_X = 0;
     static constexpr uint32_t OFF_B = kQkStages * X_STAGE;
     static constexpr uint32_t OFF_BAR = OFF_B + kQkStages * B_STAGE;
     static constexpr uint32_t OFF_SS = OFF_BAR + 512;         // [2][128] partial sums of squares
     static constexpr uint32_t OFF_GATE = OFF_SS + 1024;       // gates of the streams this CTA's rows belong to, [n][D] fp32
-    static constexpr uint32_t GATE_MAX = 48 * 1024;
+    static constexpr uint32_t GATE_MAX = (NACC == 1 ? 64u : 28u) * 1024u;
     static constexpr uint32_t TOTAL = OFF_GATE + GATE_MAX + 1024;   // + slack for the 1024-byte alignment
+    static_assert(TOTAL <= 227u * 1024u, "shared memory budget");
 };
 enum { Q_XFULL = 0, Q_BFULL = kQkStages, Q_AREADY = 2 * kQkStages, Q_EMPTY = 3 * kQkStages, Q_ACC = 4 * kQkStages, Q_COUNT };
 
@@ -77,10 +79,11 @@ __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *ma
                  : "memory");
 }
 
+template <int NACC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kQkThreads, 1)
 norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, QkParams p)
 {
-    using S = QkSmem;
+    using S = QkSmem<NACC>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
@@ -92,7 +95,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1;
     const int m0 = (pair % p.m_tiles) * (2 * kQkBM) + (int)rank * kQkBM;   // this CTA's first row
-    const int n0 = (pair / p.m_tiles) * kQkBN;                              // the pair's first output column
+    const int n0 = (pair / p.m_tiles) * (NACC * kQkBN);                     // the pair's first output column
     const int nk_steps = p.D / kQkBK;
 
     if (threadIdx.x == 0) {
@@ -107,7 +110,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         fence_mbar_init();
         prefetch_tmap(&tm_x); prefetch_tmap(&tm_w);
     }
-    if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), kQkTmemCols);
+    if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), NACC * kQkBN);
     tc_fence_before();
     __syncthreads();
     cluster_arrive();
@@ -146,7 +149,10 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 mbar_expect_tx(bar(Q_XFULL + s), S::X_STAGE);
                 tma_load_2d(base + S::OFF_X + s * S::X_STAGE, &tm_x, bar(Q_XFULL + s), ks * kQkBK, m0);
                 if (rank == 0) mbar_expect_tx(bar(Q_BFULL + s), 2 * S::B_STAGE);
-                tma2_load_2d(base + S::OFF_B + s * S::B_STAGE, &tm_w, bar(Q_BFULL + s) & kPeerBitMask, ks * kQkBK, n0 + (int)rank * (kQkBN / 2));
+#pragma unroll
+                for (int j = 0; j < NACC; ++j)
+                    tma2_load_2d(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, &tm_w, bar(Q_BFULL + s) & kPeerBitMask, ks * kQkBK,
+                                 n0 + j * kQkBN + (int)rank * (kQkBN / 2));
             }
         }
     } else if (warp == 1) {
@@ -164,12 +170,16 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 if (lane == 0) QK_TRACE(1, ks, 2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_tmem = tmem + kQkColA + s * (kQkBK / 2);
-                uint64_t bd = umma_desc_sw128(base + S::OFF_B + s * S::B_STAGE, 16, 1024);
 #pragma unroll
-                for (int kk = 0; kk < kQkBK / 16; ++kk) {
-                    umma2_ts_elect(tmem, a_tmem + kk * 8, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);   // 16 bf16 of K = 8 columns of A
-                    umma_desc_advance(bd, 32);
+                for (int j = 0; j < NACC; ++j) {
+                    uint64_t ad = umma_desc_sw128(base + S::OFF_X + s * S::X_STAGE, 16, 1024);
+                    uint64_t bd = umma_desc_sw128(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, 16, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < kQkBK / 16; ++kk) {
+                        umma2_ss_elect(tmem + j * kQkBN, ad, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                        umma_desc_advance(ad, 32);
+                        umma_desc_advance(bd, 32);
+                    }
                 }
                 umma2_commit_mc_elect(bar(Q_EMPTY + s), (uint16_t)3);
                 if (lane == 0) QK_TRACE(1, ks, 3);
@@ -201,27 +211,24 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint64_t ss2 = 0ull;
         bool ok = true;
-        // operands of one step in registers: this thread's half row of x (four 16-byte chunks) and the 32 gate values for it
-        struct Ops { uint4 x[4]; ulonglong2 g[8]; };
-        auto load = [&](int ks, Ops &o) {
-            const int s = ks % kQkStages;
-            ok = ok && wait(Q_XFULL + s, (uint32_t)(ks / kQkStages) & 1u, 6);
-            const uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + row * 128;
-#pragma unroll
-            for (int c = 0; c < 4; ++c)   // 128-byte swizzle: chunk j of row r sits at j ^ (r % 8)
-                o.x[c] = *reinterpret_cast<const uint4 *>(rowp + (((4 * half + c) ^ (row & 7)) << 4));
-            const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + ks * kQkBK);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) o.g[i] = g2[i];
-        };
-        auto step = [&](int ks, const Ops &o) {
+        for (int ks = 0; ks < nk_steps; ++ks) {
             if (threadIdx.x == 64) QK_TRACE(2, ks, 0);
             const int s = ks % kQkStages;
-            uint32_t packed[16];
+            const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + ks * kQkBK);
+            ulonglong2 gq[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) gq[i] = g2[i];      // 32 gate values, read before the wait for the tile
+            ok = ok && wait(Q_XFULL + s, (uint32_t)(ks / kQkStages) & 1u, 4);
+            if (threadIdx.x == 64) QK_TRACE(2, ks, 1);
+            uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + row * 128;
+            uint4 xr[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)   // 128-byte swizzle: chunk j of row r sits at j ^ (r % 8)
+                xr[c] = *reinterpret_cast<const uint4 *>(rowp + (((4 * half + c) ^ (row & 7)) << 4));
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const uint64_t gg[4] = {o.g[2 * c].x, o.g[2 * c].y, o.g[2 * c + 1].x, o.g[2 * c + 1].y};
-                const uint32_t vv[4] = {o.x[c].x, o.x[c].y, o.x[c].z, o.x[c].w};
+                const uint64_t gg[4] = {gq[2 * c].x, gq[2 * c].y, gq[2 * c + 1].x, gq[2 * c + 1].y};
+                uint32_t vv[4] = {xr[c].x, xr[c].y, xr[c].z, xr[c].w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const uint64_t x2 = pack_f32x2(__uint_as_float(vv[k] << 16), __uint_as_float(vv[k] & 0xFFFF0000u));
@@ -229,35 +236,15 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     float y0, y1;
                     unpack_f32x2(mul_f32x2(x2, gg[k]), y0, y1);
                     __nv_bfloat162 y2 = __floats2bfloat162_rn(y0, y1);
-                    packed[4 * c + k] = *reinterpret_cast<uint32_t *>(&y2);
+                    vv[k] = *reinterpret_cast<uint32_t *>(&y2);
                 }
-            }
-            if (threadIdx.x == 64) QK_TRACE(2, ks, 1);
-            // the A stage is free once the MMAs that read it (kQkStages steps ago) are complete
-            if (ks >= kQkStages) {
-                ok = ok && wait(Q_EMPTY + s, (uint32_t)(ks / kQkStages - 1) & 1u, 4);
-                tc_fence_after();
+                *reinterpret_cast<uint4 *>(rowp + (((4 * half + c) ^ (row & 7)) << 4)) = make_uint4(vv[0], vv[1], vv[2], vv[3]);
             }
             if (threadIdx.x == 64) QK_TRACE(2, ks, 2);
-            tmem_st16(tmem + lane_addr + kQkColA + s * (kQkBK / 2) + half * 16, packed);
-            tmem_wait_st();
-            if (threadIdx.x == 64) QK_TRACE(2, ks, 3);
-            tc_fence_before();
+            fence_proxy_async_smem();   // the tensor pipe reads what these threads wrote
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(leader_aready0 + 8u * (uint32_t)s);
             if (threadIdx.x == 64) QK_TRACE(2, ks, 4);
-        };
-        {
-            // the next step's operands are read from shared memory before this step's result is handed over, so their
-            // latency runs under the store to tensor memory and the barrier traffic
-            Ops oa, ob;
-            load(0, oa);
-            for (int ks = 0; ks < nk_steps; ks += 2) {       // (the conditions are uniform over the CTA)
-                if (ks + 1 < nk_steps) load(ks + 1, ob);
-                step(ks, oa);
-                if (ks + 2 < nk_steps) load(ks + 2, oa);
-                if (ks + 1 < nk_steps) step(ks + 1, ob);
-            }
         }
         // the row's sum of squares: both halves meet through shared memory
         float *ssm = reinterpret_cast<float *>(smem + S::OFF_SS);
@@ -281,39 +268,43 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         uint4 *stg = reinterpret_cast<uint4 *>(smem + S::OFF_X);      // [128 rows][32 pieces of 8 columns]
         static_assert(kQkBM * kQkBN * 2 <= (int)(S::OFF_BAR - S::OFF_X), "staging area of the epilogue");
 #pragma unroll 1
-        for (int c = 0; c < kQkBN / 64; ++c) {
-            uint32_t acc[32];
-            tmem_ld32(tmem + lane_addr + half * (kQkBN / 2) + c * 32, acc);      // warp-wide: every lane takes part, whatever its row
-            tmem_wait_ld();
+        for (int j = 0; j < NACC; ++j) {
+#pragma unroll 1
+            for (int c = 0; c < kQkBN / 64; ++c) {
+                uint32_t acc[32];
+                tmem_ld32(tmem + lane_addr + j * kQkBN + half * (kQkBN / 2) + c * 32, acc);   // warp-wide: every lane takes part, whatever its row
+                tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint4 o;
-                uint32_t *oo = reinterpret_cast<uint32_t *>(&o);
+                for (int i = 0; i < 4; ++i) {
+                    uint4 o;
+                    uint32_t *oo = reinterpret_cast<uint32_t *>(&o);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[8 * i + 2 * k]) * rs, __uint_as_float(acc[8 * i + 2 * k + 1]) * rs);
-                    oo[k] = *reinterpret_cast<uint32_t *>(&h);
+                    for (int k = 0; k < 4; ++k) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[8 * i + 2 * k]) * rs, __uint_as_float(acc[8 * i + 2 * k + 1]) * rs);
+                        oo[k] = *reinterpret_cast<uint32_t *>(&h);
+                    }
+                    const int piece = half * 16 + c * 4 + i;
+                    stg[row * 32 + (piece ^ (row & 31))] = o;
                 }
-                const int piece = half * 16 + c * 4 + i;
-                stg[row * 32 + (piece ^ (row & 31))] = o;
             }
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        {
-            const int n = n0 + lane * 8;            // this lane's 8 columns: they never straddle Q, K and V (head_dim % 8 == 0)
-            __nv_bfloat16 *dst0 = nullptr;          // column n of row 0 of the tensor it belongs to
-            size_t pitch = 0;
-            if (n < p.nq) { dst0 = p.q + n; pitch = (size_t)p.nq; }
-            else if (n < p.nq + p.nk) { dst0 = p.k + (n - p.nq); pitch = (size_t)p.nk; }
-            else if (n < n_out) { dst0 = p.v + (n - p.nq - p.nk); pitch = (size_t)p.nk; }
-            const int w8 = warp - 2;                // 0..7: rows w8, w8 + 8, ...
-            if (ok && dst0) {
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            {
+                const int n = n0 + j * kQkBN + lane * 8;   // this lane's 8 columns: they never straddle Q, K and V (head_dim % 8 == 0)
+                __nv_bfloat16 *dst0 = nullptr;              // column n of row 0 of the tensor it belongs to
+                size_t pitch = 0;
+                if (n < p.nq) { dst0 = p.q + n; pitch = (size_t)p.nq; }
+                else if (n < p.nq + p.nk) { dst0 = p.k + (n - p.nq); pitch = (size_t)p.nk; }
+                else if (n < n_out) { dst0 = p.v + (n - p.nq - p.nk); pitch = (size_t)p.nk; }
+                const int w8 = warp - 2;                    // 0..7: rows w8, w8 + 8, ...
+                if (ok && dst0) {
 #pragma unroll 4
-                for (int r = w8; r < kQkBM; r += 8) {
-                    if (m0 + r >= p.M) break;
-                    *reinterpret_cast<uint4 *>(dst0 + (size_t)(m0 + r) * pitch) = stg[r * 32 + (lane ^ (r & 31))];
+                    for (int r = w8; r < kQkBM; r += 8) {
+                        if (m0 + r >= p.M) break;
+                        *reinterpret_cast<uint4 *>(dst0 + (size_t)(m0 + r) * pitch) = stg[r * 32 + (lane ^ (r & 31))];
+                    }
                 }
             }
+            if (j + 1 < NACC) asm volatile("bar.sync 1, 256;" ::: "memory");   // the staging area is rewritten by the next round
         }
     }
 
@@ -322,7 +313,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     __syncthreads();
     cluster_arrive();
     cluster_wait();   // neither CTA retires while its partner can still touch its shared memory or barriers
-    if (warp == 1) tmem_dealloc2(tmem, kQkTmemCols);
+    if (warp == 1) tmem_dealloc2(tmem, NACC * kQkBN);
 }
 
 // Any dtype, any shape: one block per row. y = x * gamma / RMS(x) in shared memory (fp32), then every thread takes output
@@ -393,18 +384,53 @@ cudaError_t launch_simt(const void *x, const float *gate, const void *W, void *q
 
 }  // namespace
 
+// 256-column tiles unless they would need more than one wave of SM pairs and the gates of a CTA's streams still fit
+// beside the larger stages
+static int qk_choose_nacc(int M, int R, int D, int n_out, int sm_count)
+{
+    const size_t gate_bytes = (size_t)((kQkBM - 1) / R + 2) * D * sizeof(float);
+    const long long m_tiles = (M + 2 * kQkBM - 1) / (2 * kQkBM);
+    const long long tiles1 = m_tiles * ((n_out + kQkBN - 1) / kQkBN);
+    if (tiles1 > sm_count / 2 && gate_bytes <= QkSmem<2>::GATE_MAX) return 2;
+    return gate_bytes <= QkSmem<1>::GATE_MAX ? 1 : 0;
+}
+
 bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk)
 {
     if (dtype != REFLEX_DTYPE_BF16 || B < 1 || R < 1) return false;
     if (D < kQkBK || D % kQkBK != 0) return false;
     if (nq % 8 != 0 || nk % 8 != 0) return false;
-    if ((size_t)((kQkBM - 1) / R + 2) * D * sizeof(float) > QkSmem::GATE_MAX) return false;   // gates of a CTA's streams in shared memory
-    const long long pairs = ((long long)B * R + 2 * kQkBM - 1) / (2 * kQkBM) * ((nq + 2 * nk + kQkBN - 1) / kQkBN);
-    return pairs <= 0x3FFFFFFF;
+    if ((long long)B * R > 0x3FFFFFFF) return false;
+    return qk_choose_nacc(B * R, R, D, nq + 2 * nk, 148) != 0;   // gates of a CTA's streams must fit in shared memory
+}
+
+template <int NACC>
+static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_out, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int n_tiles = (n_out + NACC * kQkBN - 1) / (NACC * kQkBN);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
+    cfg.blockDim = dim3(kQkThreads);
+    cfg.dynamicSmemBytes = QkSmem<NACC>::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel<NACC>, mx, mw, p);
+    count_launch();
+    return e;
 }
 
 cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *Wqkv, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
-                                  float eps, int dtype, int impl, uint32_t *status, cudaStream_t st)
+                                  float eps, int dtype, int impl, int sm_count, uint32_t *status, cudaStream_t st)
 {
     const int M = B * R;
     const bool tc = impl != 1 && norm_qkv_tc_supported(dtype, B, R, D, nq, nk);
@@ -415,31 +441,14 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
     }
     CUtensorMap mx, mw;
     if (!tensor_map_2d_bf16(&mx, x, D, M, kQkBM) || !tensor_map_2d_bf16(&mw, Wqkv, D, nq + 2 * nk, kQkBN / 2)) return cudaErrorInvalidValue;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(norm_qkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
     QkParams p;
     p.gate = gate; p.q = (__nv_bfloat16 *)q; p.k = (__nv_bfloat16 *)k; p.v = (__nv_bfloat16 *)v;
     p.M = M; p.R = R; p.B = B; p.D = D; p.nq = nq; p.nk = nk;
     p.m_tiles = (M + 2 * kQkBM - 1) / (2 * kQkBM);
     p.eps = eps; p.status = status;
-    const int n_tiles = (nq + 2 * nk + kQkBN - 1) / kQkBN;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
-    cfg.blockDim = dim3(kQkThreads);
-    cfg.dynamicSmemBytes = QkSmem::TOTAL;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel, mx, mw, p);
-    count_launch();
-    return e;
+    int nacc = qk_choose_nacc(M, R, D, nq + 2 * nk, sm_count > 0 ? sm_count : 148);
+    if (impl == 2 && nacc == 2) nacc = 1;     // (forced 256-column tiles, for tests and timing)
+    return nacc == 2 ? launch_tc<2>(mx, mw, p, nq + 2 * nk, st) : launch_tc<1>(mx, mw, p, nq + 2 * nk, st);
 }
 
 }  // namespace reflex

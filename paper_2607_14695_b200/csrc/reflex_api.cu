@@ -351,7 +351,7 @@ int reflex_adarmsnorm_qkv(reflex_cache_t *c, const void *x, const float *gate, c
                           int B, int R, int D, int Hq, int Hkv, int d, float eps, int dtype, int impl, void *stream)
 {
     if (dtype != REFLEX_DTYPE_BF16 && dtype != REFLEX_DTYPE_F32) return fail(REFLEX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
-    if (impl != 0 && impl != 1) return fail(REFLEX_ERR_INVALID_ARG, "impl must be 0 (auto) or 1 (plain kernel)");
+    if (impl < 0 || impl > 2) return fail(REFLEX_ERR_INVALID_ARG, "impl must be 0 (auto), 1 (plain kernel) or 2 (tensor cores, 256-column tiles)");
     if (!x || !gate || !Wqkv || !q || !k_dyn || !v_dyn) return fail(REFLEX_ERR_INVALID_ARG, "NULL argument");
     if (B < 1 || R < 1 || (long long)B * R > 0x7FFFFFFF / 2) return fail(REFLEX_ERR_SHAPE, "B=%d, R=%d", B, R);
     if (D < 8 || D % 8 != 0 || D > 8192) return fail(REFLEX_ERR_SHAPE, "D=%d must be a multiple of 8 in [8, 8192]", D);
@@ -361,7 +361,8 @@ int reflex_adarmsnorm_qkv(reflex_cache_t *c, const void *x, const float *gate, c
     if (!aligned16(x) || !aligned16(gate) || !aligned16(Wqkv) || !aligned16(q) || !aligned16(k_dyn) || !aligned16(v_dyn))
         return fail(REFLEX_ERR_ALIGN, "x / gate / Wqkv / q / k_dyn / v_dyn not 16-byte aligned");
     uint32_t *status = c ? (uint32_t *)(c->ws + c->lay.status_off) : nullptr;
-    cudaError_t e = launch_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, B, R, D, Hq * d, Hkv * d, eps, dtype, impl, status, (cudaStream_t)stream);
+    cudaError_t e = launch_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, B, R, D, Hq * d, Hkv * d, eps, dtype, impl, c ? c->sm_count : 0, status,
+                                          (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "adarmsnorm qkv launch");
     return REFLEX_OK;
 }

@@ -400,7 +400,7 @@ def test_gate_for_all_layers_matches_per_layer_calls_and_oracle(U):
 # ------------------------------------------------------------------------------------------------
 # adaptive norm folded into the packed Q/K/V projection
 # ------------------------------------------------------------------------------------------------
-def _norm_qkv_case(U, w, impl, what, t=0.3, eps=1e-6):
+def _norm_qkv_case(U, w, impl, what, t=0.3, eps=1e-6, streams=None):
     from oracle import reflex_oracle as orc
     rb = U.rb
     x = synth.norm_input(w, 0, 0)
@@ -415,7 +415,7 @@ def _norm_qkv_case(U, w, impl, what, t=0.3, eps=1e-6):
     v = torch.full((w.B, w.T, w.Hkv, w.d), float("nan"), dtype=dt, device=U.DEV)
     rb.reflex_adarmsnorm_qkv(U.to_dev(x, w.dtype), gb[: w.B * w.D].view(w.B, w.D), U.to_dev(Wp, w.dtype), q, k, v, eps=eps, impl=impl)
     torch.cuda.synchronize()
-    for b in range(w.B):
+    for b in (range(w.B) if streams is None else streams):
         wq, wk, wv = orc.adarmsnorm_qkv(x[b], cond[b], W1, b1, W2, b2, Wp, w.Hq, w.Hkv, w.d, eps)
         for got, want, name in ((q, wq, "q"), (k, wk, "k"), (v, wv, "v")):
             U.check_close(U.to_host(got[b]), want, w.dtype, f"{what} {name} stream {b}", rel_clause=True)
@@ -432,6 +432,13 @@ def test_norm_qkv_bf16_action_expert_shape(U, impl):
     _norm_qkv_case(U, synth.CONFIGS["cfg2"].with_(B=7), impl, f"norm+qkv bf16 impl {impl}")
 
 
+@pytest.mark.parametrize("impl", [0, 2])
+def test_norm_qkv_bf16_many_streams(U, impl):
+    """40 streams of 50 rows = 2000 rows: 8 row tiles x 10 column tiles exceed the SM pairs, so impl 0 takes the 512-column
+    tiles (two accumulators; 5 column tiles); impl 2 keeps 256-column tiles. A sample of streams is compared."""
+    _norm_qkv_case(U, synth.CONFIGS["cfg2"].with_(B=40), impl, f"norm+qkv bf16 40 streams impl {impl}", streams=[0, 5, 6, 20, 39])
+
+
 def test_norm_qkv_bf16_ragged_columns_and_outliers(U):
     """320 output columns (a second column tile with 64 of 256 live), head_dim 64, D = 192 (three contraction steps, fewer
     than the stage ring), 300 rows per stream, and x with outliers x1000 as in the long-context configuration."""
@@ -445,7 +452,7 @@ def test_norm_qkv_error_paths(U):
     x, g, W = z(2, 4, 64), torch.ones((2, 64), dtype=torch.float32, device=U.DEV), z(4 * 16, 64)
     q, k = z(2, 4, 2, 16), z(2, 4, 1, 16)
     rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k.clone())
-    for bad in (lambda: rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k, impl=2),
+    for bad in (lambda: rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k, impl=3),
                 lambda: rb.reflex_adarmsnorm_qkv(x, g, W, q, k, k, eps=-1.0)):
         with pytest.raises(rb.ReflexError) as e:
             bad()
