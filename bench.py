@@ -271,6 +271,15 @@ def main():
     # what the step itself launches for AdaRMSNorm: the gate MLPs of all L layers in one call (two kernels), then one rows kernel per layer
     gates_step_ms = avg_launch_ms(lambda v: runner.gates_of_step(v, sh()), 1)
     rows_avg_ms = avg_launch_ms(lambda v: [runner.rows(l, v, sh(), True) for l in range(w.L)], w.L)
+    # ---- the next part of the layer: AdaRMSNorm folded into the packed Q/K/V projection, and a step chained through it ----
+    chained = None
+    if runner.tdt == torch.bfloat16:
+        qkv_avg_ms = avg_launch_ms(lambda v: [runner.norm_qkv(l, v, sh()) for l in range(w.L)], w.L)
+        chained_ms = avg_launch_ms(lambda v: runner.step_chained(v), 1)
+        n_out = (w.Hq + 2 * w.Hkv) * w.d
+        chained = {"norm_qkv_avg_us": qkv_avg_ms * 1e3, "norm_qkv_tflops": 2.0 * w.B * w.T * w.D * n_out / (qkv_avg_ms * 1e-3) / 1e12,
+                   "norm_qkv_shape_mnk": [w.B * w.T, n_out, w.D], "ms_per_step": chained_ms,
+                   "what": "every layer: AdaRMSNorm + packed W_QKV projection in one launch, its Q/K/V read by that layer's attention; then the Euler update"}
     step_marks = []
     for k in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -353,6 +362,7 @@ def main():
                      "frac_of_nominal_8TBs": attn_gbs / 8000.0,
                      "tensor": {"achieved_tflops": attn_tflops, "peak_tflops_sustained": peaks["bf16_tflops_sustained"],
                                 "frac": attn_tflops / peaks["bf16_tflops_sustained"]}},
+        "chained_layer": chained,
         "kernels": {"attention_avg_us": attn_avg_ms * 1e3, "adarmsnorm_rows_avg_us": rows_avg_ms * 1e3,
                     "adarmsnorm_gates_of_step_us": gates_step_ms * 1e3,
                     "adarmsnorm_rows_gbs": alg["norm_bytes_per_launch"] / (rows_avg_ms * 1e-3) / 1e9,

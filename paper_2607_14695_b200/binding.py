@@ -299,6 +299,13 @@ def prepare_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf):
     return _prepared(load().reflex_adarmsnorm_gate, args)
 
 
+def prepare_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, eps=1e-6, impl=0, cache=None):
+    B, R, D = x.shape
+    args = (cache.handle if cache is not None else None, _ptr(x), _ptr(gate), _ptr(Wqkv), _ptr(q), _ptr(k_dyn), _ptr(v_dyn), B, R, D,
+            int(q.shape[2]), int(k_dyn.shape[2]), int(q.shape[3]), float(eps), dtype_code(x), int(impl))
+    return _prepared(load().reflex_adarmsnorm_qkv, args)
+
+
 def prepare_partitioned_attention(cache: Cache, layer, q, k_dyn, v_dyn, out, scale=0.0, dyn_mask=0):
     args = (cache.handle, int(layer), _ptr(q), _ptr(k_dyn), _ptr(v_dyn), _ptr(out), int(q.shape[1]), float(scale), int(dyn_mask))
     return _prepared(load().reflex_partitioned_attention, args)

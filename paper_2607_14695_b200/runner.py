@@ -150,6 +150,38 @@ class StepRunner:
         self._call(("r", layer, variant, from_step_gates), lambda: rb.prepare_adarmsnorm(
             self.x[layer][variant], self.y, None, None, None, None, None, gate_buf=gate.view(w.B, w.D)))(sh)
 
+    # ---- chained layer: the norm output feeds the packed Q/K/V projection, whose output feeds attention ----
+    def _chained_buffers(self):
+        if not hasattr(self, "Wqkv"):
+            w = self.w
+            self.Wqkv = [self.rnd((w.Hq + 2 * w.Hkv) * w.d, w.D, std=float(w.D) ** -0.5) for _ in range(w.L)]
+            self.qc = torch.empty((w.B, w.T, w.Hq, w.d), dtype=self.tdt, device=self.device)
+            self.kc = torch.empty((w.B, w.T, w.Hkv, w.d), dtype=self.tdt, device=self.device)
+            self.vc = torch.empty((w.B, w.T, w.Hkv, w.d), dtype=self.tdt, device=self.device)
+
+    def norm_qkv(self, layer: int, variant: int, sh, impl: int = 0):
+        """AdaRMSNorm folded into the packed projection: x_l -> Q, K_dyn, V_dyn (gates from gates_of_step)."""
+        self._chained_buffers()
+        w = self.w
+        n = w.B * w.D
+        gate = self.gate_all[layer * n:(layer + 1) * n].view(w.B, w.D)
+        self._call(("q", layer, variant, impl), lambda: rb.prepare_adarmsnorm_qkv(
+            self.x[layer][variant], gate, self.Wqkv[layer], self.qc, self.kc, self.vc, impl=impl, cache=self.cache))(sh)
+
+    def attention_chained(self, layer: int, sh):
+        self._chained_buffers()
+        self._call(("ac", layer), lambda: rb.prepare_partitioned_attention(self.cache, layer, self.qc, self.kc, self.vc, self.out))(sh)
+
+    def step_chained(self, k: int):
+        """A denoising step in which every layer's norm + Q/K/V projection produces the tensors its attention reads."""
+        variant = k % self.variants
+        sh = rb.stream_handle(torch.cuda.current_stream())
+        self.gates_of_step(k, sh)
+        for layer in range(self.w.L):
+            self.norm_qkv(layer, variant, sh)
+            self.attention_chained(layer, sh)
+        self.flow(k, variant, sh)
+
     def step(self, k: int):
         """One denoising step over all layers and streams, inputs already in HBM."""
         variant = k % self.variants

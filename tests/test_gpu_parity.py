@@ -463,3 +463,32 @@ def test_norm_qkv_error_paths(U):
     with pytest.raises(rb.ReflexError) as e:
         rb.reflex_adarmsnorm_qkv(x.view(-1)[4:4 + 2 * 3 * 64].view(2, 3, 64), g, W, q[:, :3].contiguous(), k[:, :3].contiguous(), k[:, :3].contiguous())
     assert e.value.code == rb.ERR_ALIGN
+
+
+def test_chained_layer_norm_qkv_attention(U):
+    """The chained layer: AdaRMSNorm + packed projection writes Q, K_dyn, V_dyn, the partitioned attention reads them.
+    Against the oracle chain in fp64 throughout (no rounding of Q/K/V in between): the bf16 storage of Q/K/V moves a logit by
+    about 2e-3 and the output far less than the contract's tolerance."""
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"].with_(B=3)
+    tw = U.Twin(w, head0=[0, 5, 31], poison=True)
+    tw.init_static([0, 1, 2], [w.S, 700, 64])
+    for i in range(20):
+        tw.append([0, 1, 2] if i < 12 else [0, 1], 1, i)
+    x = synth.norm_input(w, 0, 3)
+    cond = synth.cond_vectors(w, 0.7)
+    W1, b1, W2, b2 = synth.gate_weights(w, 0)
+    Wp = synth.qkv_weights(w, 0)
+    gb = torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=U.DEV)
+    rb.reflex_adarmsnorm_gate(U.to_dev(cond, w.dtype), U.to_dev(W1, w.dtype), U.to_dev(b1, w.dtype), U.to_dev(W2, w.dtype), U.to_dev(b2, w.dtype), gb)
+    nan = lambda *s: torch.full(s, float("nan"), dtype=torch.bfloat16, device=U.DEV)
+    q, k, v, out = nan(w.B, w.T, w.Hq, w.d), nan(w.B, w.T, w.Hkv, w.d), nan(w.B, w.T, w.Hkv, w.d), nan(w.B, w.T, w.Hq, w.d)
+    rb.reflex_adarmsnorm_qkv(U.to_dev(x, w.dtype), gb[: w.B * w.D].view(w.B, w.D), U.to_dev(Wp, w.dtype), q, k, v, cache=tw.g)
+    rb.reflex_partitioned_attention(tw.g, 0, q, k, v, out, dyn_mask=1)
+    rb.reflex_cache_check_status(tw.g)
+    got = U.to_host(out)
+    for b in range(w.B):
+        wq, wk, wv = orc.adarmsnorm_qkv(x[b], cond[b], W1, b1, W2, b2, Wp, w.Hq, w.Hkv, w.d)
+        want = tw.o.attention(b, 0, wq.astype(np.float32), wk.astype(np.float32), wv.astype(np.float32), 1, None)
+        U.check_close(got[b], want, w.dtype, f"chained layer stream {b}")
