@@ -23,7 +23,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture (profiles/)
-NCU_TRAFFIC_BYTES = {("cfg4", "auto"): 76.8e6, ("cfg4", "tc2"): 76.8e6}
+NCU_TRAFFIC_BYTES = {("cfg4", "auto"): 76.3e6, ("cfg4", "tc2"): 76.3e6}
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -43,7 +43,7 @@ def measured_peaks():
 class ClockSampler(threading.Thread):
     """Reads (never sets) SM clock, power and clock-event reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples = []          # (wall time, sm_mhz, reasons bitmask, power W)
@@ -238,6 +238,9 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
+    t_wait = time.time()
+    while not sampler.samples and sampler.is_alive() and time.time() - t_wait < 10.0:   # NVML is up before the timed region starts
+        time.sleep(0.01)
     for k in range(args.warmup):
         do_step(k)
     barrier()
