@@ -216,6 +216,40 @@ int reflex_oracle_adarmsnorm_linear(const float *x, const double *gamma, const f
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Adaptive norm followed by the combined gate and up projections of a SwiGLU block (Sec. 3.3
+ * "System Optimizations": the Gate and Up projections of SwiGLU blocks fused into one kernel;
+ * Sec. 4 "Operator Fusion Impact": the norm combined with the linear layer after it):
+ *   y = AdaRMSNorm(x; gamma)                      (Eq. 2, in double)
+ *   h[r][f] = SiLU(sum_i y[r][i] Wg[f][i]) * (sum_i y[r][i] Wu[f][i]),  SiLU(z) = z / (1 + e^-z)
+ *   x [R][D]  gamma [D]  Wg, Wu [F][D]  ->  h [R][F]
+ * ------------------------------------------------------------------------------------------ */
+int reflex_oracle_adarmsnorm_swiglu(const float *x, const double *gamma, const float *Wg, const float *Wu,
+                                    int R, int D, int F, double eps, double *h)
+{
+    double *y = (double *)malloc(sizeof(double) * (size_t)R * (size_t)D);
+    if (!y) return -1;
+    for (int r = 0; r < R; ++r) {
+        const float *xr = x + (size_t)r * D;
+        double ss = 0.0;
+        for (int i = 0; i < D; ++i) ss += (double)xr[i] * (double)xr[i];
+        const double rms = sqrt(ss / (double)D + eps);
+        for (int i = 0; i < D; ++i) y[(size_t)r * D + i] = (double)xr[i] / rms * gamma[i];
+    }
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < R; ++r)
+        for (int f = 0; f < F; ++f) {
+            double g = 0.0, u = 0.0;
+            for (int i = 0; i < D; ++i) {
+                g += y[(size_t)r * D + i] * (double)Wg[(size_t)f * D + i];
+                u += y[(size_t)r * D + i] * (double)Wu[(size_t)f * D + i];
+            }
+            h[(size_t)r * F + f] = g / (1.0 + exp(-g)) * u;
+        }
+    free(y);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Flow-matching update (Sec. 2.1 "ODE integration", Sec. 3.2 x ~ N(0,I) at t = 1, Appendix C
  * "Flow matching steps 10"): forward Euler with K uniform steps from t = 1 to t = 0,
  *   x <- x + dt * v,  dt = -1/K.

@@ -56,6 +56,8 @@ def lib():
         _lib.reflex_oracle_adarmsnorm.restype = i
         _lib.reflex_oracle_adarmsnorm_linear.argtypes = [fp, dp, fp, i, i, i, d, dp]
         _lib.reflex_oracle_adarmsnorm_linear.restype = i
+        _lib.reflex_oracle_adarmsnorm_swiglu.argtypes = [fp, dp, fp, fp, i, i, i, d, dp]
+        _lib.reflex_oracle_adarmsnorm_swiglu.restype = i
         _lib.reflex_oracle_flow_step.argtypes = [dp, fp, ctypes.c_long, i]
         _lib.reflex_oracle_flow_step.restype = None
         _lib.reflex_oracle_flow_time.argtypes = [i, i]
@@ -142,6 +144,21 @@ def adarmsnorm_qkv(x, c, W1, b1, W2, b2, Wqkv, Hq, Hkv, d, eps=1e-6):
         raise MemoryError("oracle adarmsnorm_linear")
     nq, nk = Hq * d, Hkv * d
     return out[:, :nq].reshape(R, Hq, d), out[:, nq:nq + nk].reshape(R, Hkv, d), out[:, nq + nk:].reshape(R, Hkv, d)
+
+
+def adarmsnorm_swiglu(x, c, W1, b1, W2, b2, Wg, Wu, eps=1e-6):
+    """Eq. 2 followed by the fused gate / up projections of a SwiGLU block for one stream:
+    x [R][D], Wg, Wu [F][D] -> h = SiLU(y Wg^T) * (y Wu^T), [R][F] f64."""
+    _, g = adarmsnorm(x, c, W1, b1, W2, b2, eps, return_gate=True)
+    x, xp = _f(x); Wg, gp = _f(Wg); Wu, up = _f(Wu)
+    R, D = x.shape
+    F = Wg.shape[0]
+    assert Wg.shape == (F, D) and Wu.shape == (F, D)
+    h = np.empty((R, F), np.float64)
+    rc = lib().reflex_oracle_adarmsnorm_swiglu(xp, _dptr(g), gp, up, R, D, F, float(eps), _dptr(h))
+    if rc != 0:
+        raise MemoryError("oracle adarmsnorm_swiglu")
+    return h
 
 
 def flow_step(x, v, K):

@@ -79,3 +79,55 @@ def test_brute_force_and_row_scale_invariance():
     assert np.max(np.abs(q2 - q)) <= 1e-13 and np.max(np.abs(v2 - v)) <= 1e-13
     q3, _, _ = orc.adarmsnorm_qkv(x, c, W1, b1, W2, b2, W * np.float32(2.0), Hq, Hkv, d, eps=0.0)
     assert np.max(np.abs(q3 - 2 * q)) <= 1e-13
+
+
+# ---- adaptive norm + fused gate / up projections of a SwiGLU block (Sec. 3.3: "combine the Gate and Up projections") ----
+
+def test_swiglu_hand_worked_example():
+    """x = (3, 4), gate off, eps = 0: y = x / sqrt(12.5). Wg = [(1, 0)], Wu = [(0, 1)]: h = SiLU(y0) * y1."""
+    x = np.array([[3.0, 4.0]], np.float32)
+    z1 = np.zeros((1, 1), np.float32); zb = np.zeros(1, np.float32)
+    h = orc.adarmsnorm_swiglu(x, np.zeros(1, np.float32), z1, zb, np.zeros((2, 1), np.float32), np.zeros(2, np.float32),
+                              np.array([[1, 0]], np.float32), np.array([[0, 1]], np.float32), eps=0.0)
+    r = np.sqrt(12.5)
+    y0, y1 = 3 / r, 4 / r
+    assert abs(h[0, 0] - y0 / (1 + np.exp(-y0)) * y1) <= 1e-15
+
+
+def test_swiglu_matches_torch_fp64_and_is_not_symmetric():
+    """h == silu(linear(y, Wg)) * linear(y, Wu) from torch in fp64; swapping Wg and Wu changes the result (the activation sits
+    on the gate branch only), and a zero up-projection row gives exactly 0."""
+    rng = np.random.default_rng(6)
+    R, D, Cd, Hd, F = 5, 24, 4, 6, 10
+    x = rng.standard_normal((R, D)).astype(np.float32)
+    c = rng.standard_normal(Cd).astype(np.float32)
+    W1, b1, W2, b2 = _mlp(rng, D, Cd, Hd)
+    Wg = rng.standard_normal((F, D)).astype(np.float32) * np.float32(0.3)
+    Wu = rng.standard_normal((F, D)).astype(np.float32) * np.float32(0.3)
+    Wu[3] = 0
+    h = orc.adarmsnorm_swiglu(x, c, W1, b1, W2, b2, Wg, Wu)
+    y = torch.from_numpy(orc.adarmsnorm(x, c, W1, b1, W2, b2))
+    Fn = torch.nn.functional
+    want = (Fn.silu(Fn.linear(y, torch.from_numpy(Wg).double())) * Fn.linear(y, torch.from_numpy(Wu).double())).numpy()
+    assert np.max(np.abs(h - want)) <= 1e-12
+    assert np.all(h[:, 3] == 0.0)
+    assert np.max(np.abs(orc.adarmsnorm_swiglu(x, c, W1, b1, W2, b2, Wu, Wg) - h)) > 1e-3
+
+
+def test_swiglu_brute_force():
+    rng = np.random.default_rng(7)
+    R, D, Cd, Hd, F = 2, 5, 2, 3, 3
+    x = rng.standard_normal((R, D)).astype(np.float32)
+    c = rng.standard_normal(Cd).astype(np.float32)
+    W1, b1, W2, b2 = _mlp(rng, D, Cd, Hd)
+    Wg = rng.standard_normal((F, D)).astype(np.float32); Wu = rng.standard_normal((F, D)).astype(np.float32)
+    h = orc.adarmsnorm_swiglu(x, c, W1, b1, W2, b2, Wg, Wu, eps=1e-5)
+    hid = [sum(float(W1[j, e]) * float(c[e]) for e in range(Cd)) + float(b1[j]) for j in range(Hd)]
+    hid = [z / (1.0 + np.exp(-z)) for z in hid]
+    gam = [1.0 + sum(float(W2[i, j]) * hid[j] for j in range(Hd)) + float(b2[i]) for i in range(D)]
+    for r in range(R):
+        rms = np.sqrt(sum(float(x[r, i]) ** 2 for i in range(D)) / D + 1e-5)
+        y = [float(x[r, i]) / rms * gam[i] for i in range(D)]
+        for f in range(F):
+            g = sum(y[i] * float(Wg[f, i]) for i in range(D)); u = sum(y[i] * float(Wu[f, i]) for i in range(D))
+            assert abs(h[r, f] - g / (1.0 + np.exp(-g)) * u) <= 1e-13
