@@ -280,9 +280,12 @@ def main():
         qkv_avg_ms = avg_launch_ms(lambda v: [runner.norm_qkv(l, v, sh()) for l in range(w.L)], w.L)
         chained_ms = avg_launch_ms(lambda v: runner.step_chained(v), 1)
         n_out = (w.Hq + 2 * w.Hkv) * w.d
+        swiglu_avg_ms = avg_launch_ms(lambda v: [runner.norm_swiglu(l, v, sh()) for l in range(w.L)], w.L)
         chained = {"norm_qkv_avg_us": qkv_avg_ms * 1e3, "norm_qkv_tflops": 2.0 * w.B * w.T * w.D * n_out / (qkv_avg_ms * 1e-3) / 1e12,
                    "norm_qkv_shape_mnk": [w.B * w.T, n_out, w.D], "ms_per_step": chained_ms,
-                   "what": "every layer: AdaRMSNorm + packed W_QKV projection in one launch, its Q/K/V read by that layer's attention; then the Euler update"}
+                   "norm_swiglu_avg_us": swiglu_avg_ms * 1e3, "norm_swiglu_tflops": 2.0 * w.B * w.T * w.D * 8 * w.D / (swiglu_avg_ms * 1e-3) / 1e12,
+                   "norm_swiglu_shape_m_f_k": [w.B * w.T, 4 * w.D, w.D],
+                   "what": "ms_per_step: every layer AdaRMSNorm + packed W_QKV projection in one launch, its Q/K/V read by that layer's attention, then the Euler update; norm_swiglu: AdaRMSNorm + fused gate/up projections + SiLU(gate)*up in one launch, timed alone"}
     step_marks = []
     for k in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

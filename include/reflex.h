@@ -204,6 +204,22 @@ int reflex_adarmsnorm_qkv(reflex_cache_t *cache, const void *x, const float *gat
                           void *k_dyn, void *v_dyn, int B, int R, int D, int Hq, int Hkv, int d, float eps,
                           int dtype, int impl, void *stream);
 
+/* Sec. 3.3 "System Optimizations" (the Gate and Up projections of a SwiGLU block combined into one kernel), again with the
+ * adaptive norm of Eq. 2 folded in. For every row r of stream b:
+ *   y = x[r] / RMS(x[r]) * gamma_b,   h[r] = SiLU(W_gate y) * (W_up y),   SiLU(z) = z / (1 + e^-z)
+ * One launch; neither y nor the two projections reach memory.
+ *   cache    as in reflex_adarmsnorm_qkv (status word), or NULL
+ *   x        device [B][R][D] dtype;   gate  device fp32 [B][D]
+ *   Wgu      device [2F][D] dtype: rows [0, F) = W_gate, rows [F, 2F) = W_up (row f of each = hidden feature f)
+ *   h        device [B][R][F] dtype (written)
+ *   impl     0: tensor cores when dtype is bf16, D % 64 == 0 and (127 / R + 2) * D * 4 bytes <= 28 KiB, else the plain
+ *               kernel; 1: the plain kernel
+ * Arithmetic on the tensor-core path: as reflex_adarmsnorm_qkv; both fp32 accumulators are scaled by 1/RMS, the activation
+ * and the product are computed in fp32 and rounded to bf16 once.
+ * Requirements: D % 8 == 0, D <= 8192; F % 8 == 0; 16-byte aligned pointers. Errors as reflex_adarmsnorm_qkv. */
+int reflex_adarmsnorm_swiglu(reflex_cache_t *cache, const void *x, const float *gate, const void *Wgu, void *h,
+                             int B, int R, int D, int F, float eps, int dtype, int impl, void *stream);
+
 /* Eq. 1 / App. A Prop. 1: for every stream b, KV head j and its G*T query rows,
  *   out = softmax(scale * Q [K_pin; K_slide; K_dyn]^T) [V_pin; V_slide; V_dyn]
  * over static rows [0, static_len[b]), the live ring slots (physical order; softmax does not depend

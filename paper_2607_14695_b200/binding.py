@@ -26,7 +26,7 @@ EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
-    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_partitioned_attention",
+    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_adarmsnorm_swiglu", "reflex_partitioned_attention",
     "reflex_flow_step",
 ]
 
@@ -72,6 +72,7 @@ def load():
     lib.reflex_adarmsnorm_gate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, vp]
     lib.reflex_adarmsnorm_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_adarmsnorm_qkv.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, vp]
+    lib.reflex_adarmsnorm_swiglu.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
     for name in EXPORTS:
@@ -297,6 +298,22 @@ def prepare_adarmsnorm_gate(cond, W1, b1, W2, b2, gate_buf):
     L, B, D, Cd, Hd = _gate_dims(cond, W1, W2)
     args = (_ptr(cond), _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(gate_buf), L, B, D, Cd, Hd, dtype_code(cond))
     return _prepared(load().reflex_adarmsnorm_gate, args)
+
+
+def reflex_adarmsnorm_swiglu(x, gate, Wgu, h, eps=1e-6, impl=0, cache=None, stream=None):
+    """x [B][R][D], gate fp32 [B][D], Wgu [2F][D] = [W_gate; W_up] -> h [B][R][F] = SiLU(y W_gate^T) * (y W_up^T)."""
+    B, R, D = x.shape
+    F = int(h.shape[2])
+    _check(load().reflex_adarmsnorm_swiglu(cache.handle if cache is not None else None, _ptr(x), _ptr(gate), _ptr(Wgu), _ptr(h), B, R, D, F,
+                                           float(eps), dtype_code(x), int(impl), _stream(stream)))
+    return h
+
+
+def prepare_adarmsnorm_swiglu(x, gate, Wgu, h, eps=1e-6, impl=0, cache=None):
+    B, R, D = x.shape
+    args = (cache.handle if cache is not None else None, _ptr(x), _ptr(gate), _ptr(Wgu), _ptr(h), B, R, D, int(h.shape[2]), float(eps),
+            dtype_code(x), int(impl))
+    return _prepared(load().reflex_adarmsnorm_swiglu, args)
 
 
 def prepare_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, eps=1e-6, impl=0, cache=None):

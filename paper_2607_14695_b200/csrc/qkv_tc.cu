@@ -18,6 +18,10 @@
 // the row-owning threads 40 us (32 cache lines per load instruction); A operand stored to tensor memory instead of back
 // to shared memory 23.2 us (the gate multiply, about 700 cycles per step, stayed above the 512 cycles of the MMAs).
 //
+// The same kernel serves the fused gate / up projections of a SwiGLU block (Sec. 3.3: "combine the Gate and Up projections"):
+// accumulator 0 takes 256 rows of W_gate, accumulator 1 the same rows of W_up, and the epilogue writes
+// SiLU(gate) * up for those 256 hidden columns (swiglu_F > 0 in the parameters).
+//
 // Any other dtype or shape: a plain kernel (one block per row, fp32 FMAs) with the same semantics.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -61,6 +65,7 @@ struct QkParams {
     __nv_bfloat16 *q, *k, *v;   // [M][nq], [M][nk], [M][nk]
     int M, R, B, D, nq, nk;     // M = B * R rows; nq = Hq * d, nk = Hkv * d
     int m_tiles;                // 256-row tiles
+    int swiglu_F;               // 0: columns go to Q, K, V. F > 0: W holds [W_gate; W_up] ([2F][D]), out (= q, pitch nq = F) gets SiLU(g) * u
     float eps;
     uint32_t *status;
 };
@@ -95,7 +100,8 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1;
     const int m0 = (pair % p.m_tiles) * (2 * kQkBM) + (int)rank * kQkBM;   // this CTA's first row
-    const int n0 = (pair / p.m_tiles) * (NACC * kQkBN);                     // the pair's first output column
+    const bool swiglu = NACC == 2 && p.swiglu_F > 0;
+    const int n0 = (pair / p.m_tiles) * (swiglu ? kQkBN : NACC * kQkBN);   // the pair's first output column
     const int nk_steps = p.D / kQkBK;
 
     if (threadIdx.x == 0) {
@@ -152,7 +158,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 #pragma unroll
                 for (int j = 0; j < NACC; ++j)
                     tma2_load_2d(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, &tm_w, bar(Q_BFULL + s) & kPeerBitMask, ks * kQkBK,
-                                 n0 + j * kQkBN + (int)rank * (kQkBN / 2));
+                                 (swiglu ? j * p.swiglu_F + n0 : n0 + j * kQkBN) + (int)rank * (kQkBN / 2));
             }
         }
     } else if (warp == 1) {
@@ -268,19 +274,32 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         uint4 *stg = reinterpret_cast<uint4 *>(smem + S::OFF_X);      // [128 rows][32 pieces of 8 columns]
         static_assert(kQkBM * kQkBN * 2 <= (int)(S::OFF_BAR - S::OFF_X), "staging area of the epilogue");
 #pragma unroll 1
-        for (int j = 0; j < NACC; ++j) {
+        for (int j = 0; j < (swiglu ? 1 : NACC); ++j) {
 #pragma unroll 1
             for (int c = 0; c < kQkBN / 64; ++c) {
                 uint32_t acc[32];
                 tmem_ld32(tmem + lane_addr + j * kQkBN + half * (kQkBN / 2) + c * 32, acc);   // warp-wide: every lane takes part, whatever its row
-                tmem_wait_ld();
+                if (swiglu) {     // (uniform) the up projection of the same columns; acc <- SiLU(g) * u, both scaled by 1/RMS first
+                    uint32_t up[32];
+                    tmem_ld32(tmem + lane_addr + kQkBN + half * (kQkBN / 2) + c * 32, up);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float g = __uint_as_float(acc[i]) * rs, u = __uint_as_float(up[i]) * rs;
+                        acc[i] = __float_as_uint(__fdividef(g, 1.f + __expf(-g)) * u);
+                    }
+                } else {
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * rs);
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     uint4 o;
                     uint32_t *oo = reinterpret_cast<uint32_t *>(&o);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[8 * i + 2 * k]) * rs, __uint_as_float(acc[8 * i + 2 * k + 1]) * rs);
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[8 * i + 2 * k]), __uint_as_float(acc[8 * i + 2 * k + 1]));
                         oo[k] = *reinterpret_cast<uint32_t *>(&h);
                     }
                     const int piece = half * 16 + c * 4 + i;
@@ -304,7 +323,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     }
                 }
             }
-            if (j + 1 < NACC) asm volatile("bar.sync 1, 256;" ::: "memory");   // the staging area is rewritten by the next round
+            if (j + 1 < (swiglu ? 1 : NACC)) asm volatile("bar.sync 1, 256;" ::: "memory");   // the staging area is rewritten by the next round
         }
     }
 
@@ -330,7 +349,7 @@ template <> __device__ __forceinline__ __nv_bfloat16 qk_from_f<__nv_bfloat16>(fl
 template <typename T>
 __global__ void __launch_bounds__(256)
 norm_qkv_simt_kernel(const T *__restrict__ x, const float *__restrict__ gate, const T *__restrict__ W, T *q, T *k, T *v,
-                     int R, int D, int nq, int nk, float eps)
+                     int R, int D, int nq, int nk, int swiglu_F, float eps)
 {
     extern __shared__ float ysm[];    // [D] + 8 partial sums
     float *part = ysm + D;
@@ -351,6 +370,16 @@ norm_qkv_simt_kernel(const T *__restrict__ x, const float *__restrict__ gate, co
     float tot = 0.f;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += part[w];
     const float rs = rsqrtf(tot / (float)D + eps);
+    if (swiglu_F > 0) {     // W = [W_gate; W_up], q = out [M][F]
+        for (int f = threadIdx.x; f < swiglu_F; f += blockDim.x) {
+            const T *wg = W + (size_t)f * D, *wu = W + (size_t)(swiglu_F + f) * D;
+            float g = 0.f, u = 0.f;
+            for (int i = 0; i < D; ++i) { g = fmaf(ysm[i], qk_to_f<T>(wg[i]), g); u = fmaf(ysm[i], qk_to_f<T>(wu[i]), u); }
+            g *= rs; u *= rs;
+            q[r * swiglu_F + f] = qk_from_f<T>(g / (1.f + expf(-g)) * u);
+        }
+        return;
+    }
     const int n_out = nq + 2 * nk;
     for (int n = threadIdx.x; n < n_out; n += blockDim.x) {
         const T *wr = W + (size_t)n * D;
@@ -364,8 +393,8 @@ norm_qkv_simt_kernel(const T *__restrict__ x, const float *__restrict__ gate, co
 }
 
 template <typename T>
-cudaError_t launch_simt(const void *x, const float *gate, const void *W, void *q, void *k, void *v, int M, int R, int D, int nq, int nk, float eps,
-                        cudaStream_t st)
+cudaError_t launch_simt(const void *x, const float *gate, const void *W, void *q, void *k, void *v, int M, int R, int D, int nq, int nk, int swiglu_F,
+                        float eps, cudaStream_t st)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)M);
@@ -377,7 +406,7 @@ cudaError_t launch_simt(const void *x, const float *gate, const void *W, void *q
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_simt_kernel<T>, (const T *)x, gate, (const T *)W, (T *)q, (T *)k, (T *)v, R, D, nq, nk, eps);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_simt_kernel<T>, (const T *)x, gate, (const T *)W, (T *)q, (T *)k, (T *)v, R, D, nq, nk, swiglu_F, eps);
     count_launch();
     return e;
 }
@@ -405,7 +434,7 @@ bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk)
 }
 
 template <int NACC>
-static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_out, cudaStream_t st)
+static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_tiles, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -413,7 +442,6 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    const int n_tiles = (n_out + NACC * kQkBN - 1) / (NACC * kQkBN);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
     cfg.blockDim = dim3(kQkThreads);
@@ -429,26 +457,34 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
     return e;
 }
 
-cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *Wqkv, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
-                                  float eps, int dtype, int impl, int sm_count, uint32_t *status, cudaStream_t st)
+// swiglu_F = 0: W = W_QKV, outputs q / k / v with nq and nk columns. swiglu_F = F > 0: W = [W_gate; W_up] ([2F][D]),
+// q = the [M][F] output SiLU(gate) * up; nq, nk, k, v unused.
+cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *W, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
+                                  int swiglu_F, float eps, int dtype, int impl, int sm_count, uint32_t *status, cudaStream_t st)
 {
     const int M = B * R;
-    const bool tc = impl != 1 && norm_qkv_tc_supported(dtype, B, R, D, nq, nk);
+    if (swiglu_F > 0) { nq = swiglu_F; nk = 0; }
+    const size_t gate_bytes = (size_t)((kQkBM - 1) / R + 2) * D * sizeof(float);
+    const bool tc = impl != 1 && norm_qkv_tc_supported(dtype, B, R, D, nq, nk) && (swiglu_F == 0 || gate_bytes <= QkSmem<2>::GATE_MAX);
     if (!tc) {
         if ((size_t)(D + 8) * sizeof(float) > 48 * 1024) return cudaErrorInvalidValue;
-        return dtype == REFLEX_DTYPE_BF16 ? launch_simt<__nv_bfloat16>(x, gate, Wqkv, q, k, v, M, R, D, nq, nk, eps, st)
-                                          : launch_simt<float>(x, gate, Wqkv, q, k, v, M, R, D, nq, nk, eps, st);
+        return dtype == REFLEX_DTYPE_BF16 ? launch_simt<__nv_bfloat16>(x, gate, W, q, k, v, M, R, D, nq, nk, swiglu_F, eps, st)
+                                          : launch_simt<float>(x, gate, W, q, k, v, M, R, D, nq, nk, swiglu_F, eps, st);
     }
+    const int w_rows = swiglu_F > 0 ? 2 * swiglu_F : nq + 2 * nk;
     CUtensorMap mx, mw;
-    if (!tensor_map_2d_bf16(&mx, x, D, M, kQkBM) || !tensor_map_2d_bf16(&mw, Wqkv, D, nq + 2 * nk, kQkBN / 2)) return cudaErrorInvalidValue;
+    if (!tensor_map_2d_bf16(&mx, x, D, M, kQkBM) || !tensor_map_2d_bf16(&mw, W, D, w_rows, kQkBN / 2)) return cudaErrorInvalidValue;
     QkParams p;
     p.gate = gate; p.q = (__nv_bfloat16 *)q; p.k = (__nv_bfloat16 *)k; p.v = (__nv_bfloat16 *)v;
     p.M = M; p.R = R; p.B = B; p.D = D; p.nq = nq; p.nk = nk;
     p.m_tiles = (M + 2 * kQkBM - 1) / (2 * kQkBM);
+    p.swiglu_F = swiglu_F;
     p.eps = eps; p.status = status;
+    if (swiglu_F > 0) return launch_tc<2>(mx, mw, p, (swiglu_F + kQkBN - 1) / kQkBN, st);
     int nacc = qk_choose_nacc(M, R, D, nq + 2 * nk, sm_count > 0 ? sm_count : 148);
     if (impl == 2 && nacc == 2) nacc = 1;     // (forced 256-column tiles, for tests and timing)
-    return nacc == 2 ? launch_tc<2>(mx, mw, p, nq + 2 * nk, st) : launch_tc<1>(mx, mw, p, nq + 2 * nk, st);
+    const int n_out = nq + 2 * nk;
+    return nacc == 2 ? launch_tc<2>(mx, mw, p, (n_out + 2 * kQkBN - 1) / (2 * kQkBN), st) : launch_tc<1>(mx, mw, p, (n_out + kQkBN - 1) / kQkBN, st);
 }
 
 }  // namespace reflex

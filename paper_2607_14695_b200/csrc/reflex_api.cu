@@ -361,9 +361,27 @@ int reflex_adarmsnorm_qkv(reflex_cache_t *c, const void *x, const float *gate, c
     if (!aligned16(x) || !aligned16(gate) || !aligned16(Wqkv) || !aligned16(q) || !aligned16(k_dyn) || !aligned16(v_dyn))
         return fail(REFLEX_ERR_ALIGN, "x / gate / Wqkv / q / k_dyn / v_dyn not 16-byte aligned");
     uint32_t *status = c ? (uint32_t *)(c->ws + c->lay.status_off) : nullptr;
-    cudaError_t e = launch_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, B, R, D, Hq * d, Hkv * d, eps, dtype, impl, c ? c->sm_count : 0, status,
+    cudaError_t e = launch_adarmsnorm_qkv(x, gate, Wqkv, q, k_dyn, v_dyn, B, R, D, Hq * d, Hkv * d, 0, eps, dtype, impl, c ? c->sm_count : 0, status,
                                           (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "adarmsnorm qkv launch");
+    return REFLEX_OK;
+}
+
+int reflex_adarmsnorm_swiglu(reflex_cache_t *c, const void *x, const float *gate, const void *Wgu, void *h, int B, int R, int D, int F,
+                             float eps, int dtype, int impl, void *stream)
+{
+    if (dtype != REFLEX_DTYPE_BF16 && dtype != REFLEX_DTYPE_F32) return fail(REFLEX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (impl != 0 && impl != 1) return fail(REFLEX_ERR_INVALID_ARG, "impl must be 0 (auto) or 1 (plain kernel)");
+    if (!x || !gate || !Wgu || !h) return fail(REFLEX_ERR_INVALID_ARG, "NULL argument");
+    if (B < 1 || R < 1 || (long long)B * R > 0x7FFFFFFF / 2) return fail(REFLEX_ERR_SHAPE, "B=%d, R=%d", B, R);
+    if (D < 8 || D % 8 != 0 || D > 8192) return fail(REFLEX_ERR_SHAPE, "D=%d must be a multiple of 8 in [8, 8192]", D);
+    if (F < 8 || F % 8 != 0 || F > (1 << 20)) return fail(REFLEX_ERR_SHAPE, "F=%d must be a multiple of 8 in [8, 2^20]", F);
+    if (!(eps >= 0.f)) return fail(REFLEX_ERR_INVALID_ARG, "eps must be >= 0");
+    if (!aligned16(x) || !aligned16(gate) || !aligned16(Wgu) || !aligned16(h)) return fail(REFLEX_ERR_ALIGN, "x / gate / Wgu / h not 16-byte aligned");
+    uint32_t *status = c ? (uint32_t *)(c->ws + c->lay.status_off) : nullptr;
+    cudaError_t e = launch_adarmsnorm_qkv(x, gate, Wgu, h, nullptr, nullptr, B, R, D, 0, 0, F, eps, dtype, impl, c ? c->sm_count : 0, status,
+                                          (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "adarmsnorm swiglu launch");
     return REFLEX_OK;
 }
 

@@ -95,8 +95,9 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
 // adaptive norm + packed Q/K/V projection (qkv_tc.cu). impl: 0 = tensor cores where supported, 1 = plain kernel,
 // 2 = tensor cores with 256-column tiles only
 bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk);
-cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *Wqkv, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
-                                  float eps, int dtype, int impl, int sm_count, uint32_t *status, cudaStream_t st);
+// swiglu_F > 0: W = [W_gate; W_up] and q receives SiLU(gate) * up, [B*R][F]
+cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *W, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
+                                  int swiglu_F, float eps, int dtype, int impl, int sm_count, uint32_t *status, cudaStream_t st);
 bool gate_tc_supported(int B, int D, int Cd, int Hd);
 cudaError_t launch_gate_tc(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf, int L, int B,
                            int D, int Cd, int Hd, cudaStream_t st);

@@ -168,6 +168,18 @@ class StepRunner:
         self._call(("q", layer, variant, impl), lambda: rb.prepare_adarmsnorm_qkv(
             self.x[layer][variant], gate, self.Wqkv[layer], self.qc, self.kc, self.vc, impl=impl, cache=self.cache))(sh)
 
+    def norm_swiglu(self, layer: int, variant: int, sh, F: Optional[int] = None):
+        """AdaRMSNorm folded into the fused gate / up projections of the layer's SwiGLU block: x_l -> h [B][T][F]."""
+        w = self.w
+        F = 4 * w.D if F is None else F
+        if not hasattr(self, "Wgu") or self.Wgu[0].shape[0] != 2 * F:
+            self.Wgu = [self.rnd(2 * F, w.D, std=float(w.D) ** -0.5) for _ in range(w.L)]
+            self.hmlp = torch.empty((w.B, w.T, F), dtype=self.tdt, device=self.device)
+        n = w.B * w.D
+        gate = self.gate_all[layer * n:(layer + 1) * n].view(w.B, w.D)
+        self._call(("s", layer, variant, F), lambda: rb.prepare_adarmsnorm_swiglu(
+            self.x[layer][variant], gate, self.Wgu[layer], self.hmlp, cache=self.cache))(sh)
+
     def attention_chained(self, layer: int, sh):
         self._chained_buffers()
         self._call(("ac", layer), lambda: rb.prepare_partitioned_attention(self.cache, layer, self.qc, self.kc, self.vc, self.out))(sh)

@@ -76,7 +76,7 @@ CONFIGS = {
 # tensor ids for the seed sequence
 TID = {"k_static": 1, "v_static": 2, "k_new": 3, "v_new": 4, "q": 5, "k_dyn": 6, "v_dyn": 7, "x": 8,
        "cond_state": 9, "W1": 10, "b1": 11, "W2": 12, "b2": 13, "v_flow": 14, "noise": 15, "head0": 16,
-       "outlier_mask": 17, "misc": 18, "Wqkv": 19, "Wo": 20}
+       "outlier_mask": 17, "misc": 18, "Wqkv": 19, "Wo": 20, "Wgu": 21}
 
 
 def rng_for(w_or_seed, tensor: str, layer: int = 0, variant: int = 0) -> np.random.Generator:
@@ -163,6 +163,11 @@ def gate_weights(w: Workload, layer: int, std: float = 0.02):
 def qkv_weights(w: Workload, layer: int) -> np.ndarray:
     """Packed projection W_QKV = [W_Q; W_K; W_V], [(Hq + 2 Hkv) d][D], N(0, 1/D): unit-variance outputs for unit-variance inputs."""
     return normal(w, "Wqkv", ((w.Hq + 2 * w.Hkv) * w.d, w.D), layer, 0, float(w.D) ** -0.5)
+
+
+def swiglu_weights(w: Workload, layer: int, F: int) -> np.ndarray:
+    """[W_gate; W_up] of a SwiGLU block, [2F][D], N(0, 1/D)."""
+    return normal(w, "Wgu", (2 * F, w.D), layer, 0, float(w.D) ** -0.5)
 
 
 def ring_head0(w: Workload, B: int | None = None) -> np.ndarray:

@@ -492,3 +492,54 @@ def test_chained_layer_norm_qkv_attention(U):
         wq, wk, wv = orc.adarmsnorm_qkv(x[b], cond[b], W1, b1, W2, b2, Wp, w.Hq, w.Hkv, w.d)
         want = tw.o.attention(b, 0, wq.astype(np.float32), wk.astype(np.float32), wv.astype(np.float32), 1, None)
         U.check_close(got[b], want, w.dtype, f"chained layer stream {b}")
+
+
+# ------------------------------------------------------------------------------------------------
+# adaptive norm folded into the fused gate / up projections of a SwiGLU block
+# ------------------------------------------------------------------------------------------------
+def _norm_swiglu_case(U, w, F, impl, what, t=0.3, eps=1e-6, streams=None):
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    x = synth.norm_input(w, 0, 1)
+    cond = synth.cond_vectors(w, t)
+    W1, b1, W2, b2 = synth.gate_weights(w, 0)
+    Wgu = synth.swiglu_weights(w, 0, F)
+    gb = torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=U.DEV)
+    rb.reflex_adarmsnorm_gate(U.to_dev(cond, w.dtype), U.to_dev(W1, w.dtype), U.to_dev(b1, w.dtype), U.to_dev(W2, w.dtype), U.to_dev(b2, w.dtype), gb)
+    h = torch.full((w.B, w.T, F), float("nan"), dtype=rb.torch_dtype(w.dtype), device=U.DEV)
+    rb.reflex_adarmsnorm_swiglu(U.to_dev(x, w.dtype), gb[: w.B * w.D].view(w.B, w.D), U.to_dev(Wgu, w.dtype), h, eps=eps, impl=impl)
+    torch.cuda.synchronize()
+    for b in (range(w.B) if streams is None else streams):
+        want = orc.adarmsnorm_swiglu(x[b], cond[b], W1, b1, W2, b2, Wgu[:F], Wgu[F:], eps)
+        got = U.to_host(h[b])
+        if w.dtype != synth.DTYPE_BF16:
+            U.check_close(got, want, w.dtype, f"{what} stream {b}", rel_clause=True)
+            continue
+        # bf16: each projection reaches the activation with the operand-rounding error of a bf16 GEMM over D terms, at most
+        # delta = 6.3e-3 per unit of output scale (4.5 sigma of 1.4e-3); h = SiLU(g) u then moves by |SiLU'(g) u| delta +
+        # |SiLU(g)| delta (|SiLU'| <= 1.1), on top of the contract's allowance for the stored value itself
+        y = orc.adarmsnorm(x[b], cond[b], W1, b1, W2, b2, eps)
+        g, u = y @ Wgu[:F].astype(np.float64).T, y @ Wgu[F:].astype(np.float64).T
+        silu = g / (1.0 + np.exp(-g))
+        lim = np.maximum(U.BF16_MAX_ABS, 2.0 ** -7 * np.abs(want)) + 6.3e-3 * (1.1 * np.abs(u) + np.abs(silu))
+        err = np.abs(got - want)
+        assert np.isfinite(got).all() and not (err > lim).any(), f"{what} stream {b}: worst {err.max():.3e}, {(err > lim).sum()} beyond the bound"
+        assert err.mean() <= U.BF16_MEAN_ABS, f"{what} stream {b}: mean-abs {err.mean():.3e}"
+
+
+def test_norm_swiglu_fp32_plain_kernel(U):
+    _norm_swiglu_case(U, synth.CONFIGS["cfg1"].with_(B=2), 96, 0, "norm+swiglu fp32")
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_norm_swiglu_bf16(U, impl):
+    """D = 1024, F = 1024 hidden features (4 column tiles of 256, each with a gate and an up accumulator), 7 streams of 50
+    rows (a full 256-row tile pair and a ragged one)."""
+    _norm_swiglu_case(U, synth.CONFIGS["cfg2"].with_(B=7), 1024, impl, f"norm+swiglu bf16 impl {impl}")
+
+
+def test_norm_swiglu_bf16_ragged_hidden_width(U):
+    """F = 328: the second column tile has 72 live columns and its gate accumulator reads rows of W_up past W_gate's end
+    (never stored); D = 192."""
+    w = synth.CONFIGS["cfg2"].with_(B=3, T=120, D=192)
+    _norm_swiglu_case(U, w, 328, 0, "norm+swiglu ragged")
