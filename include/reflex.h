@@ -244,6 +244,42 @@ int reflex_partitioned_attention(reflex_cache_t *cache, int layer, const void *q
 int reflex_flow_step(void *x, const void *v, void *x_lowp, int B, int T, int A, int k, int K,
                      int dtype, void *stream);
 
+/* ---- Sec. 3.4 "Stream Throughput: Asynchronous Pipeline", Algorithm 1 (future-conditional overlap scheduling), Eq. 3 ----
+ * Host logic only; no device work. A control loop calls reflex_overlap_tick once per control period:
+ *   - the event names the action to execute (chunk index, position in the chunk; Algorithm 1 line 5);
+ *   - launch_now = 1 on the tick of action C - K (1-based; line 6), K = ceil(mean inference latency / control period)
+ *     fixed at the start of the chunk (line 3) from the last 8 measured latencies (the initial estimate before the
+ *     first) and clamped to [0, C - 1]: the caller then starts the next chunk's inference conditioned on the action
+ *     just commanded (Eq. 3: s_hat = a_cmd) and reports its completion with reflex_overlap_inference_done;
+ *   - when a chunk is used up and the next has not been reported, the tick is a stall (stalled = 1, the last action
+ *     is held) and the loop resumes with the first action of the new chunk on the first tick after the report.
+ * reflex_overlap_simulate runs the same policy over a trace of inference latencies in continuous time (one loop
+ * iteration = one control period, the launch at the end of the period of action C - K) and returns stall and
+ * staleness figures; mode 0 = adaptive K (Algorithm 1), 1 = synchronous (inference only after the chunk has ended),
+ * 2 = fixed K. Errors: REFLEX_ERR_INVALID_ARG, REFLEX_ERR_STATE (completion reported with nothing in flight). */
+typedef struct reflex_overlap reflex_overlap_t;
+typedef struct reflex_overlap_event {
+    int32_t chunk, action;      /* chunk index (from 0) and 0-based position of the action executed on this tick */
+    int32_t launch_now;         /* start the next chunk's inference now */
+    int32_t stalled;            /* no action available: the previous one is held */
+    int32_t lookahead;          /* K of the current chunk */
+    int32_t reserved;
+    int64_t stalls_total;       /* stalled ticks so far */
+} reflex_overlap_event;
+typedef struct reflex_overlap_stats {
+    int64_t chunks, stall_ticks;            /* chunks executed; control periods lost waiting (each stall rounded up) */
+    double stall_time_s, total_time_s;      /* time lost waiting; time until the last chunk's successor is available */
+    double mean_staleness_s;                /* mean age of the conditioning state when a chunk's first action runs */
+    double mean_lookahead;
+    int32_t min_lookahead, max_lookahead;
+} reflex_overlap_stats;
+int reflex_overlap_create(int C, double tau_step_s, double tau_inf_init_s, reflex_overlap_t **out);
+int reflex_overlap_destroy(reflex_overlap_t *sched);
+int reflex_overlap_tick(reflex_overlap_t *sched, reflex_overlap_event *ev);
+int reflex_overlap_inference_done(reflex_overlap_t *sched, double latency_s);
+int reflex_overlap_simulate(int C, double tau_step_s, double tau_inf_init_s, const double *tau_inf_s, int n_chunks,
+                            int mode, int fixed_K, reflex_overlap_stats *out);
+
 #ifdef __cplusplus
 }
 #endif

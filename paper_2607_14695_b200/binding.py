@@ -27,8 +27,19 @@ EXPORTS = [
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
     "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_adarmsnorm_swiglu", "reflex_partitioned_attention",
-    "reflex_flow_step",
+    "reflex_flow_step", "reflex_overlap_create", "reflex_overlap_destroy", "reflex_overlap_tick", "reflex_overlap_inference_done",
+    "reflex_overlap_simulate",
 ]
+
+
+class OverlapEvent(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("chunk", "action", "launch_now", "stalled", "lookahead", "reserved")] + [("stalls_total", ctypes.c_int64)]
+
+
+class OverlapStats(ctypes.Structure):
+    _fields_ = [("chunks", ctypes.c_int64), ("stall_ticks", ctypes.c_int64), ("stall_time_s", ctypes.c_double), ("total_time_s", ctypes.c_double),
+                ("mean_staleness_s", ctypes.c_double), ("mean_lookahead", ctypes.c_double), ("min_lookahead", ctypes.c_int32),
+                ("max_lookahead", ctypes.c_int32)]
 
 
 class CacheDesc(ctypes.Structure):
@@ -75,6 +86,12 @@ def load():
     lib.reflex_adarmsnorm_swiglu.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
+    dbl = ctypes.c_double
+    lib.reflex_overlap_create.argtypes = [i, dbl, dbl, ctypes.POINTER(vp)]
+    lib.reflex_overlap_destroy.argtypes = [vp]
+    lib.reflex_overlap_tick.argtypes = [vp, ctypes.POINTER(OverlapEvent)]
+    lib.reflex_overlap_inference_done.argtypes = [vp, dbl]
+    lib.reflex_overlap_simulate.argtypes = [i, dbl, dbl, ctypes.POINTER(dbl), i, i, i, ctypes.POINTER(OverlapStats)]
     for name in EXPORTS:
         getattr(lib, name)  # every declared symbol must resolve
     _lib = lib
@@ -332,3 +349,36 @@ def prepare_flow_step(x, v, x_lowp, k, K):
     B, T, A = x.shape
     args = (_ptr(x), _ptr(v), _ptr(x_lowp), B, T, A, int(k), int(K), dtype_code(v))
     return _prepared(load().reflex_flow_step, args)
+
+
+# ---- Algorithm 1: overlap scheduling (host logic) ----
+class OverlapScheduler:
+    """Thin wrapper over reflex_overlap_*: tick() once per control period, inference_done(latency) when a chunk arrives."""
+
+    def __init__(self, C: int, tau_step_s: float, tau_inf_init_s: float):
+        h = ctypes.c_void_p()
+        _check(load().reflex_overlap_create(int(C), float(tau_step_s), float(tau_inf_init_s), ctypes.byref(h)))
+        self.handle = h
+
+    def tick(self) -> dict:
+        ev = OverlapEvent()
+        _check(load().reflex_overlap_tick(self.handle, ctypes.byref(ev)))
+        return {n: getattr(ev, n) for n in ("chunk", "action", "launch_now", "stalled", "lookahead", "stalls_total")}
+
+    def inference_done(self, latency_s: float):
+        _check(load().reflex_overlap_inference_done(self.handle, float(latency_s)))
+
+    def __del__(self):
+        try:
+            if self.handle:
+                load().reflex_overlap_destroy(self.handle)
+                self.handle = None
+        except Exception:
+            pass
+
+
+def reflex_overlap_simulate(C, tau_step_s, tau_inf_init_s, tau_inf_s, mode=0, fixed_K=0) -> dict:
+    arr = (ctypes.c_double * len(tau_inf_s))(*[float(t) for t in tau_inf_s])
+    st = OverlapStats()
+    _check(load().reflex_overlap_simulate(int(C), float(tau_step_s), float(tau_inf_init_s), arr, len(tau_inf_s), int(mode), int(fixed_K), ctypes.byref(st)))
+    return {n: getattr(st, n) for n, _ in OverlapStats._fields_}
