@@ -781,7 +781,7 @@ static bool tc2_cluster_merge_ok(const AttnParams &p, int nsplit, int sm_count)
     const int active = tc2_active_clusters(p.d, 2 * nsplit);
     if (base_units > (nsplit == 4 ? active - active / 4 : active)) return false;
     if (tc2_partials_us(p, nsplit) <= kTc2MergedUs) return false;
-    return (p.d / 4 / nsplit / kTc2Parts) % 2 == 0 && p.d / 4 / nsplit / kTc2Parts >= 2;
+    return (p.d / nsplit / kTc2Parts) % 16 == 0 && p.d / nsplit / kTc2Parts >= 16;   // a thread reduces whole 16-column pieces
 }
 
 int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)

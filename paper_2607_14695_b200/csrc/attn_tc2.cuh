@@ -719,21 +719,26 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int q = 0; q < 8; ++q)
                 if (q == (int)(crank >> 1)) w_own = wgt[q];
             {
-                // (the tensor-memory loads are warp-wide: every lane takes part, whatever its own row's weight; a row without
-                // weight in this slice, or a slice without tiles whose accumulator was never written, stages nothing)
+                // Only the columns that OTHER pairs reduce are staged; this pair's own columns stay in tensor memory until the
+                // reduction below. (The tensor-memory loads are warp-wide: every lane takes part, whatever its own row's
+                // weight; a row without weight in this slice, or a slice without tiles whose accumulator was never written,
+                // stages nothing.)
                 tc_fence_after();
                 const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
                 constexpr int EC = HD / NP;
                 const bool mine = w_own > 0.f && fin_ok;
+                const int own_lo = (int)(crank >> 1) * (HD / ns), own_hi = own_lo + HD / ns;     // columns this pair reduces
 #pragma unroll 1
                 for (int c = 0; c < EC / 32; ++c) {
+                    const int col0 = part * EC + c * 32;
+                    if (col0 >= own_lo && col0 < own_hi) continue;        // (uniform over the CTA; HD / ns is a multiple of 32)
                     uint32_t o[32];
-                    tmem_ld32(tmem_base + lane_addr + kColO + part * EC + c * 32, o);
+                    tmem_ld32(tmem_base + lane_addr + kColO + col0, o);
                     tmem_wait_ld();
                     if (mine) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
-                            stage[((part * EC + c * 32) / 4 + i) * 128 + row] =
+                            stage[(col0 / 4 + i) * 128 + row] =
                                 make_float4(__uint_as_float(o[4 * i]) * w_own, __uint_as_float(o[4 * i + 1]) * w_own,
                                             __uint_as_float(o[4 * i + 2]) * w_own, __uint_as_float(o[4 * i + 3]) * w_own);
                     }
@@ -742,37 +747,55 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         cluster_arrive();
         cluster_wait();
-        if (warp >= 2 && fin_ok) {
-            // this pair's columns [crank/2 * HD/ns, +HD/ns), split between the NP threads of the row
+        if (warp >= 2) {
+            // this pair's columns [crank/2 * HD/ns, +HD/ns), split between the NP threads of the row: its own share comes
+            // straight from tensor memory, the other slices' shares from their staging areas
             const int uu = u_start / p.nsplit, pair = uu % n_pairs, kvh = (uu / n_pairs) % p.Hkv, b = uu / (n_pairs * p.Hkv);
             const int t_row = (2 * pair + (int)rank) * p.tile_tokens + row / p.G;
-            const int c4_thread = HD / 4 / ns / NP;                                    // float4 columns per thread
-            const int c4_0 = (int)(crank >> 1) * (HD / 4 / ns) + part * c4_thread;
-            if (t_row < p.T && l_all > 0.f) {
-                const float inv = 1.f / l_all;
-                __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + t_row) * p.Hq + kvh * p.G + row % p.G) * HD + c4_0 * 4;
-#pragma unroll 1
-                for (int c4 = 0; c4 < c4_thread; c4 += 2) {                          // 8 columns = one 16-byte store at a time
-                    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            const int own = (int)(crank >> 1);
+            const int cols_thread = HD / ns / NP;                                       // columns per thread: 16, 32 or 64
+            const int col_0 = own * (HD / ns) + part * cols_thread;
+            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+            const bool live = fin_ok && t_row < p.T && l_all > 0.f;
+            float w_own = 0.f;
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (q < ns && wgt[q] > 0.f) {
-                            const uint32_t a = mapa(smem_u32(stage + (c4_0 + c4) * 128 + row), (uint32_t)(2 * q) + rank);
-                            float4 v0, v1;
-                            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v0.x), "=f"(v0.y), "=f"(v0.z), "=f"(v0.w) : "r"(a) : "memory");
-                            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v1.x), "=f"(v1.y), "=f"(v1.z), "=f"(v1.w) : "r"(a + 128 * 16) : "memory");
-                            acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
-                            acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+            for (int q = 0; q < 8; ++q)
+                if (q == own) w_own = wgt[q];
+            if (!(fin_l > 0.f)) w_own = 0.f;                                            // an accumulator that was never written
+            const float inv = live ? 1.f / l_all : 0.f;
+            __nv_bfloat16 *orow = (__nv_bfloat16 *)p.out + (((size_t)b * p.T + (live ? t_row : 0)) * p.Hq + kvh * p.G + row % p.G) * HD + col_0;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < cols_thread; c0 += 16) {
+                uint32_t o[16];
+                tmem_ld16(tmem_base + lane_addr + kColO + col_0 + c0, o);              // warp-wide, whatever the row's state
+                tmem_wait_ld();
+                if (!live) continue;
+                float acc[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = w_own > 0.f ? __uint_as_float(o[i]) * w_own : 0.f;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (q < ns && q != own && wgt[q] > 0.f) {
+                        const uint32_t a = mapa(smem_u32(stage + ((col_0 + c0) / 4) * 128 + row), (uint32_t)(2 * q) + rank);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float4 v;
+                            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a + j * 128 * 16) : "memory");
+                            acc[4 * j] += v.x; acc[4 * j + 1] += v.y; acc[4 * j + 2] += v.z; acc[4 * j + 3] += v.w;
                         }
                     }
+                }
+#pragma unroll
+                for (int h8 = 0; h8 < 2; ++h8) {
                     uint4 v;
                     uint32_t *vv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
+                        __nv_bfloat162 h = __floats2bfloat162_rn(acc[8 * h8 + 2 * k] * inv, acc[8 * h8 + 2 * k + 1] * inv);
                         vv[k] = *reinterpret_cast<uint32_t *>(&h);
                     }
-                    *reinterpret_cast<uint4 *>(orow + c4 * 4) = v;
+                    *reinterpret_cast<uint4 *>(orow + c0 + 8 * h8) = v;
                 }
             }
         }
