@@ -543,3 +543,13 @@ def test_norm_swiglu_bf16_ragged_hidden_width(U):
     (never stored); D = 192."""
     w = synth.CONFIGS["cfg2"].with_(B=3, T=120, D=192)
     _norm_swiglu_case(U, w, 328, 0, "norm+swiglu ragged")
+
+
+def test_norm_qkv_short_streams_and_fallback(U):
+    """Rows per stream far below the tile height: with R = 13 a 128-row tile covers 11 streams (all their gates in shared
+    memory); with R = 3 the gates of a tile's 44 streams no longer fit beside the stages and the call falls back to the plain
+    kernel. Both against the oracle."""
+    w13 = synth.CONFIGS["cfg2"].with_(B=23, T=13)
+    _norm_qkv_case(U, w13, 0, "norm+qkv R=13", streams=[0, 9, 10, 22])
+    w3 = synth.CONFIGS["cfg2"].with_(B=50, T=3)
+    _norm_qkv_case(U, w3, 0, "norm+qkv R=3 (plain kernel)", streams=[0, 42, 43, 49])
