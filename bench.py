@@ -331,6 +331,31 @@ def main():
         stream_stats = {"ticks": n_ticks, "steps_per_tick": w.K, "tick_ms_p50": tms[len(tms) // 2], "tick_ms_p95": tms[min(len(tms) - 1, int(0.95 * len(tms)))],
                         "tick_ms_max": tms[-1], "budget_ms": 20.0, "sustains_50hz": tms[-1] < 20.0, "kernels_per_tick": runner.kernels_per_tick,
                         "note": "one tick = ring append (all layers) + noise + K steps, replayed as one CUDA graph; a new static prefix every 10 ticks; cache stays L2-resident across a tick by nature"}
+        # the same trace with the asynchronous hand-over: every 10 ticks a producer stream stages the next prefix in the
+        # idle static bank while ticks keep running, and the consumer flips banks at the following tick boundary
+        r2 = StepRunner(w, device=f"cuda:{local_rank}", static_banks=2)
+        r2.capture_tick()
+        producer = torch.cuda.Stream()
+        tick_ev2, staged = [], False
+        for tck in range(n_ticks + 5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            if staged:
+                stream.wait_stream(producer)
+                r2.commit_static()
+                staged = False
+            if tck % 10 == 0:
+                r2.stage_static(w.S if (tck // 10) % 2 == 0 else w.S - 16, producer)
+                staged = True
+            r2.tick_graph.replay()
+            b.record(stream)
+            tick_ev2.append((a, b))
+        barrier()
+        rb.reflex_cache_check_status(r2.cache)
+        tms2 = sorted(a.elapsed_time(b) for a, b in tick_ev2[5:])
+        stream_stats["async_prefix"] = {"tick_ms_p50": tms2[len(tms2) // 2], "tick_ms_max": tms2[-1],
+                                        "note": "new prefix staged on a second stream into the idle static bank during the ticks, committed (index flip) at the next tick boundary"}
+        del r2
     sampler.stop()
 
     from paper_2607_14695_b200 import multi

@@ -63,6 +63,8 @@ typedef struct {
     int32_t N;       /* capacity of the sliding ring, tokens                    */
     int32_t T_max;   /* largest number of dynamic (action) tokens per call      */
     int32_t dtype;   /* REFLEX_DTYPE_*                                           */
+    int32_t static_banks; /* 0 or 1: one static region; 2: two banks, so that a new prefix can be staged while the
+                             current one is being read (reflex_cache_stage_static / reflex_cache_commit_static) */
 } reflex_cache_desc;
 
 const char *reflex_last_error_string(void);
@@ -72,9 +74,10 @@ unsigned long long reflex_kernel_launch_count(void);
 
 /* ---- helpers around the five hot-path calls -------------------------------------------------- */
 
-/* Bytes of ONE slab (K or V; the caller allocates two): [L][B][S_max + N][Hkv][d] elements of
- * dtype. Rows [0, S_max) of a (layer, stream) block are the static region, rows [S_max, S_max+N)
- * the ring in physical slot order. The dynamic suffix is never copied into the slab: attention
+/* Bytes of ONE slab (K or V; the caller allocates two): [L][B][banks * S_max + N][Hkv][d] elements of
+ * dtype (banks = 2 with static_banks == 2, else 1). Rows [0, banks * S_max) of a (layer, stream) block are
+ * the static region (bank k at rows [k S_max, (k + 1) S_max)), the N rows after them the ring in physical
+ * slot order. The dynamic suffix is never copied into the slab: attention
  * reads it from the caller's tensors in place. Returns 0 for an invalid descriptor. */
 size_t reflex_cache_slab_bytes(const reflex_cache_desc *desc);
 
@@ -122,6 +125,23 @@ int reflex_cache_check_status(reflex_cache_t *cache, void *stream);
 int reflex_cache_init_static(reflex_cache_t *cache, const int32_t *stream_ids, int n_streams,
                              const void *k_static, const void *v_static, int S_src, const int32_t *S,
                              void *stream);
+
+/* Sec. 3.4 "Stream Throughput: Asynchronous Pipeline": the vision thread (producer) pushes the K,V of a new observation
+ * while the policy thread (consumer) keeps denoising against the current one. With static_banks == 2:
+ *   reflex_cache_stage_static   writes a new prefix into the bank that attention is NOT reading (arguments as
+ *                               reflex_cache_init_static) and records its length as staged; attention launched
+ *                               before or after it on any stream still reads the current prefix, so this call may
+ *                               run on the producer's stream concurrently with the consumer's denoising steps;
+ *   reflex_cache_commit_static  makes the staged prefix of the listed streams the current one: an index flip and
+ *                               a length update by a tiny kernel on `stream`, no copy. Order it after the staging
+ *                               (an event wait on the consumer's stream) and between two chunks.
+ * The host mirror follows the calls (static_len as returned by reflex_cache_get_state is the committed length).
+ * Errors: REFLEX_ERR_STATE when the cache has one bank or nothing is staged for a listed stream; else as
+ * reflex_cache_init_static. */
+int reflex_cache_stage_static(reflex_cache_t *cache, const int32_t *stream_ids, int n_streams,
+                              const void *k_static, const void *v_static, int S_src, const int32_t *S,
+                              void *stream);
+int reflex_cache_commit_static(reflex_cache_t *cache, const int32_t *stream_ids, int n_streams, void *stream);
 
 /* Sec. 3.1 "Sliding History ... FIFO queue of the last N"; Sec. 3.4 circular pointer arithmetic into
  * the pre-allocated buffer; App. B.1 "returns eviction count". Appends m tokens per stream in place,

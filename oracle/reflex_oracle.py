@@ -207,6 +207,24 @@ class OracleCache:
         self.v_static[:, b, :S] = v_s
         self.static_len[b] = S
 
+    # Sec. 3.4 "Asynchronous Pipeline": the producer hands over a new prefix while the consumer still reads the current one.
+    # By definition: staging changes nothing that attention sees; committing replaces the prefix as a whole.
+    def stage_static(self, b, k_s, v_s):
+        if not (0 <= k_s.shape[1] <= self.S_max):
+            raise ValueError("S out of range")
+        if not hasattr(self, "_staged"):
+            self._staged = {}
+        self._staged[b] = (np.array(k_s, np.float32), np.array(v_s, np.float32))
+
+    def commit_static(self, b):
+        k_s, v_s = self._staged.pop(b)
+        S = k_s.shape[1]
+        self.k_static[:, b] = np.nan            # the previous prefix is gone entirely (a read of stale rows shows up)
+        self.v_static[:, b] = np.nan
+        self.k_static[:, b, :S] = k_s
+        self.v_static[:, b, :S] = v_s
+        self.static_len[b] = S
+
     # Sec. 3.4 / App. B.1-B.2: circular write pointer, FIFO eviction of the oldest tokens, in all layers.
     def append_sliding(self, b, k_n, v_n):
         """k_n, v_n [L][m][Hkv][d]. Returns the number of tokens evicted."""

@@ -25,7 +25,8 @@ ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT
 EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
-    "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_append_sliding",
+    "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_stage_static",
+    "reflex_cache_commit_static", "reflex_cache_append_sliding",
     "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_adarmsnorm_swiglu", "reflex_partitioned_attention",
     "reflex_flow_step", "reflex_overlap_create", "reflex_overlap_destroy", "reflex_overlap_tick", "reflex_overlap_inference_done",
     "reflex_overlap_simulate",
@@ -43,7 +44,7 @@ class OverlapStats(ctypes.Structure):
 
 
 class CacheDesc(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("L", "B", "Hq", "Hkv", "d", "S_max", "N", "T_max", "dtype")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("L", "B", "Hq", "Hkv", "d", "S_max", "N", "T_max", "dtype", "static_banks")]
 
 
 class ReflexError(RuntimeError):
@@ -78,6 +79,8 @@ def load():
     lib.reflex_cache_set_attention_impl.argtypes = [vp, i]
     lib.reflex_cache_check_status.argtypes = [vp, vp]
     lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
+    lib.reflex_cache_stage_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
+    lib.reflex_cache_commit_static.argtypes = [vp, i32p, i, vp]
     lib.reflex_cache_append_sliding.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_adarmsnorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_adarmsnorm_gate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, vp]
@@ -155,16 +158,17 @@ class Cache:
     """Owns the device memory the library borrows (two slabs + workspace, allocated once through
     torch) and the opaque handle."""
 
-    def __init__(self, L, B, Hq, Hkv, d, S_max, N, T_max, dtype, device="cuda:0", ring_head0=None, stream=None):
+    def __init__(self, L, B, Hq, Hkv, d, S_max, N, T_max, dtype, device="cuda:0", ring_head0=None, stream=None, static_banks=1):
         lib = load()
-        self.desc = CacheDesc(L, B, Hq, Hkv, d, S_max, N, T_max, dtype)
+        self.desc = CacheDesc(L, B, Hq, Hkv, d, S_max, N, T_max, dtype, static_banks)
+        self.ring_off = (2 if static_banks == 2 else 1) * S_max     # first ring row of a (layer, stream) block
         slab = reflex_cache_slab_bytes(self.desc)
         wsb = reflex_workspace_bytes(self.desc)
         if slab == 0 or wsb == 0:
             raise ReflexError(ERR_SHAPE, "invalid cache descriptor")
         self.device = torch.device(device)
         tdt = torch_dtype(dtype)
-        self.k_slab = torch.zeros((L, B, S_max + N, Hkv, d), dtype=tdt, device=self.device)
+        self.k_slab = torch.zeros((L, B, self.ring_off + N, Hkv, d), dtype=tdt, device=self.device)
         self.v_slab = torch.zeros_like(self.k_slab)
         assert self.k_slab.numel() * self.k_slab.element_size() == slab
         self.workspace = torch.zeros((wsb,), dtype=torch.uint8, device=self.device)
@@ -213,6 +217,19 @@ def reflex_cache_init_static(cache: Cache, stream_ids, k_static, v_static, S=Non
     S_src = int(k_static.shape[2]) if k_static is not None else 0
     _check(load().reflex_cache_init_static(cache.handle, _i32(stream_ids), n, _ptr(k_static), _ptr(v_static), S_src,
                                            _i32(S), _stream(stream)))
+
+
+def reflex_cache_stage_static(cache: Cache, stream_ids, k_static, v_static, S=None, stream=None):
+    """Write a new prefix into the static bank that attention is not reading (cache created with static_banks=2)."""
+    n = len(stream_ids)
+    S_src = int(k_static.shape[2]) if k_static is not None else 0
+    _check(load().reflex_cache_stage_static(cache.handle, _i32(stream_ids), n, _ptr(k_static), _ptr(v_static), S_src,
+                                            _i32(S), _stream(stream)))
+
+
+def reflex_cache_commit_static(cache: Cache, stream_ids, stream=None):
+    """Make the staged prefix of these streams the one attention reads (index flip on `stream`)."""
+    _check(load().reflex_cache_commit_static(cache.handle, _i32(stream_ids), len(stream_ids), _stream(stream)))
 
 
 def reflex_cache_append_sliding(cache: Cache, stream_ids, k_new, v_new, stream=None):

@@ -94,7 +94,8 @@ attn_simt_kernel(AttnParams p)
     if (oldest < 0) oldest += N;
 
     const size_t row_elems = (size_t)p.Hkv * d;
-    const size_t blk = ((size_t)p.layer * p.B + b) * (size_t)(p.S_max + N);
+    const size_t blk = ((size_t)p.layer * p.B + b) * (size_t)(p.ring_off + N);
+    const size_t s_row0 = (size_t)st.bank * p.S_max;     // first row of the static bank in use
     const T *k_blk = (const T *)p.k_slab + blk * row_elems + (size_t)kv * d;
     const T *v_blk = (const T *)p.v_slab + blk * row_elems + (size_t)kv * d;
     const T *k_dyn = (const T *)p.k_dyn + (size_t)b * p.T * row_elems + (size_t)kv * d;
@@ -118,13 +119,13 @@ attn_simt_kernel(AttnParams p)
         const int idx = tile * 32 + lane;
         const T *kp = nullptr, *vp = nullptr;
         if (idx < S) {
-            kp = k_blk + (size_t)idx * row_elems; vp = v_blk + (size_t)idx * row_elems;
+            kp = k_blk + (s_row0 + idx) * row_elems; vp = v_blk + (s_row0 + idx) * row_elems;
         } else if (idx < S + N) {
             const int slot = idx - S;
             int age = slot - oldest;
             if (age < 0) age += N;
             if (age < st.count) {
-                kp = k_blk + (size_t)(p.S_max + slot) * row_elems; vp = v_blk + (size_t)(p.S_max + slot) * row_elems;
+                kp = k_blk + (size_t)(p.ring_off + slot) * row_elems; vp = v_blk + (size_t)(p.ring_off + slot) * row_elems;
             }
         } else if (idx < n_keys) {
             const int j = idx - S - N;

@@ -41,6 +41,7 @@ struct TcParams {
     float *partials;
     uint32_t *status;
     int B, L, Hq, Hkv, G, S_max, N, T, layer;
+    int ring_off;      // first ring row of a (layer, stream) block: S_max times the number of static banks
     int dyn_mask;
     float scale, scale_log2;
     int nsplit;
@@ -73,12 +74,12 @@ struct TileRef {
 };
 
 struct TileGeom {
-    int S, N, T, count, oldest, ns, nr, nd, row_base, S_max, b;
+    int S, N, T, count, oldest, ns, nr, nd, row_base, s_off, ring_off, b;   // s_off: first row of the static bank in use
     __device__ __forceinline__ TileRef decode(int it) const
     {
         TileRef t;
-        if (it < ns) { t.dyn = 0; t.kind = 0; t.idx = it; t.row0 = row_base + it * kBN; }
-        else if (it < ns + nr) { t.dyn = 0; t.kind = 1; t.idx = it - ns; t.row0 = row_base + S_max + t.idx * kBN; }
+        if (it < ns) { t.dyn = 0; t.kind = 0; t.idx = it; t.row0 = row_base + s_off + it * kBN; }
+        else if (it < ns + nr) { t.dyn = 0; t.kind = 1; t.idx = it - ns; t.row0 = row_base + ring_off + t.idx * kBN; }
         else { t.dyn = 1; t.kind = 2; t.idx = it - ns - nr; t.row0 = b * T + t.idx * kBN; }
         return t;
     }
@@ -160,8 +161,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         g.ns = (g.S + kBN - 1) / kBN;
         g.nr = g.count > 0 ? (p.N + kBN - 1) / kBN : 0;
         g.nd = (p.T + kBN - 1) / kBN;
-        g.row_base = (p.layer * p.B + b) * (p.S_max + p.N);
-        g.S_max = p.S_max; g.b = b;
+        g.row_base = (p.layer * p.B + b) * (p.ring_off + p.N);
+        g.s_off = st.bank * p.S_max; g.ring_off = p.ring_off; g.b = b;
     }
     const int n_tiles = g.ns + g.nr + g.nd;
     const int per = (n_tiles + p.nsplit - 1) / p.nsplit;
@@ -723,7 +724,7 @@ bool tc_supported(const AttnParams &p)
     const int G = p.Hq / p.Hkv;
     if (G > kBM || (kBM % G) != 0) return false;
     if (p.B > 65535 || p.T > 65535) return false;
-    if ((uint64_t)p.L * p.B * (uint64_t)(p.S_max + p.N) > 0x7FFFFFFFull || (uint64_t)p.B * p.T > 0x7FFFFFFFull) return false;
+    if ((uint64_t)p.L * p.B * (uint64_t)(p.ring_off + p.N) > 0x7FFFFFFFull || (uint64_t)p.B * p.T > 0x7FFFFFFFull) return false;
     return encode_fn() != nullptr;
 }
 
@@ -812,7 +813,7 @@ int tc2_choose_splits(const AttnParams &p, size_t partial_bytes, int sm_count)
 cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_cta, int sm_count, cudaStream_t st)
 {
     const int G = p.Hq / p.Hkv;
-    const int rows_slab = p.L * p.B * (p.S_max + p.N);
+    const int rows_slab = p.L * p.B * (p.ring_off + p.N);
     CUtensorMap mk, mv, mkd, mvd, mq;
     if (!cache().get(&mk, p.k_slab, 0, rows_slab, p.Hkv, p.d, 0, mk_slab) || !cache().get(&mv, p.v_slab, 0, rows_slab, p.Hkv, p.d, 0, mk_slab) ||
         !cache().get(&mkd, p.k_dyn, 0, p.B * p.T, p.Hkv, p.d, 0, mk_slab) || !cache().get(&mvd, p.v_dyn, 0, p.B * p.T, p.Hkv, p.d, 0, mk_slab) ||
@@ -821,6 +822,7 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     TcParams tp;
     tp.state = p.state; tp.out = p.out; tp.partials = p.partials; tp.status = status;
     tp.B = p.B; tp.L = p.L; tp.Hq = p.Hq; tp.Hkv = p.Hkv; tp.G = G; tp.S_max = p.S_max; tp.N = p.N; tp.T = p.T; tp.layer = p.layer;
+    tp.ring_off = p.ring_off;
     tp.dyn_mask = p.dyn_mask; tp.scale = p.scale; tp.scale_log2 = p.scale * 1.4426950408889634f;
     tp.nsplit = p.nsplit;
     tp.tile_tokens = kBM / G;

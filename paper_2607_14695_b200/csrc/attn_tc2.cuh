@@ -177,8 +177,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         g.ns = (g.S + kBN - 1) / kBN;
         g.nr = g.count > 0 ? (p.N + kBN - 1) / kBN : 0;
         g.nd = (p.T + kBN - 1) / kBN;
-        g.row_base = (p.layer * p.B + w.b) * (p.S_max + p.N);
-        g.S_max = p.S_max; g.b = w.b;
+        g.row_base = (p.layer * p.B + w.b) * (p.ring_off + p.N);
+        g.s_off = st.bank * p.S_max; g.ring_off = p.ring_off; g.b = w.b;
         w.H = g.ns + g.nr + g.nd;          // 64-key halves
         const int all_tiles = (w.H + 1) / 2;   // >= 1: there is always a dynamic half
         const int per = (all_tiles + p.nsplit - 1) / p.nsplit;

@@ -16,6 +16,8 @@ __global__ void state_init_kernel(StreamState *state, int64_t *total, uint32_t *
     s.head = ((h % N) + N) % N;
     s.count = 0;
     s.ticket = 0;
+    s.bank = 0;
+    s.staged_len = -1;
     state[b] = s;
     total[b] = 0;
 }
@@ -33,23 +35,28 @@ cudaError_t launch_state_init(StreamState *state, int64_t *total, uint32_t *stat
 __global__ void __launch_bounds__(256)
 init_static_kernel(uint4 *__restrict__ k_slab, uint4 *__restrict__ v_slab, const uint4 *__restrict__ k_src,
                    const uint4 *__restrict__ v_src, StreamState *state, StreamBatch batch, int src_stream0, int L, int B,
-                   int rows_per_block /* S_max + N */, int S_src, int row_units)
+                   int rows_per_block /* ring_off + N */, int S_max, int S_src, int row_units, int to_other_bank)
 {
     const int i = blockIdx.z, l = blockIdx.y;
     const int b = batch.id[i];
     const int S = batch.len[i];
     const size_t units = (size_t)S * row_units;
     const size_t src_off = ((size_t)(src_stream0 + i) * L + l) * S_src * row_units;
-    const size_t dst_off = ((size_t)l * B + b) * rows_per_block * row_units;
+    // the bank attention reads, or (staging a new prefix while the current one is in use) the other one
+    const int bank = ((const volatile StreamState *)state)[b].bank ^ (to_other_bank ? 1 : 0);
+    const size_t dst_off = (((size_t)l * B + b) * rows_per_block + (size_t)bank * S_max) * row_units;
     for (size_t u = (size_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (size_t)gridDim.x * blockDim.x) {
         k_slab[dst_off + u] = k_src[src_off + u];
         v_slab[dst_off + u] = v_src[src_off + u];
     }
-    if (blockIdx.x == 0 && l == 0 && threadIdx.x == 0) state[b].static_len = S;
+    if (blockIdx.x == 0 && l == 0 && threadIdx.x == 0) {
+        if (to_other_bank) state[b].staged_len = S;
+        else state[b].static_len = S;
+    }
 }
 
 cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
-                               const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max, int N, int S_src,
+                               const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max, int ring_off, int N, int S_src, int to_other_bank,
                                size_t row_bytes, cudaStream_t st)
 {
     const int row_units = (int)(row_bytes / 16);
@@ -59,7 +66,7 @@ cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, co
     if (chunks > 64) chunks = 64;
     dim3 grid(chunks, L, n);
     init_static_kernel<<<grid, 256, 0, st>>>((uint4 *)k_slab, (uint4 *)v_slab, (const uint4 *)k_src, (const uint4 *)v_src,
-                                             state, batch, src_stream0, L, B, S_max + N, S_src, row_units);
+                                             state, batch, src_stream0, L, B, ring_off + N, S_max, S_src, row_units, to_other_bank);
     count_launch();
     return cudaGetLastError();
 }
@@ -70,7 +77,7 @@ cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, co
 __global__ void __launch_bounds__(256)
 append_sliding_kernel(uint4 *__restrict__ k_slab, uint4 *__restrict__ v_slab, const uint4 *__restrict__ k_src,
                       const uint4 *__restrict__ v_src, StreamState *state, int64_t *total, StreamBatch batch,
-                      int src_stream0, int L, int B, int S_max, int N, int m, int row_units)
+                      int src_stream0, int L, int B, int ring_off, int N, int m, int row_units)
 {
     const int i = blockIdx.y;
     const int b = batch.id[i];
@@ -80,7 +87,7 @@ append_sliding_kernel(uint4 *__restrict__ k_slab, uint4 *__restrict__ v_slab, co
     const int head = s_head;
     const size_t units = (size_t)L * m * row_units;
     const size_t src_base = (size_t)(src_stream0 + i) * L * m * row_units;
-    const int rows_per_block = S_max + N;
+    const int rows_per_block = ring_off + N;
     for (size_t u = (size_t)blockIdx.x * blockDim.x + threadIdx.x; u < units; u += (size_t)gridDim.x * blockDim.x) {
         const int off = (int)(u % row_units);
         const size_t r = u / row_units;
@@ -88,7 +95,7 @@ append_sliding_kernel(uint4 *__restrict__ k_slab, uint4 *__restrict__ v_slab, co
         const int l = (int)(r / m);
         int slot = head + tok;
         if (slot >= N) slot -= N;
-        const size_t dst = (((size_t)l * B + b) * rows_per_block + S_max + slot) * row_units + off;
+        const size_t dst = (((size_t)l * B + b) * rows_per_block + ring_off + slot) * row_units + off;
         k_slab[dst] = k_src[src_base + u];
         v_slab[dst] = v_src[src_base + u];
     }
@@ -109,7 +116,7 @@ append_sliding_kernel(uint4 *__restrict__ k_slab, uint4 *__restrict__ v_slab, co
 }
 
 cudaError_t launch_append_sliding(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
-                                  int64_t *total, const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max,
+                                  int64_t *total, const StreamBatch &batch, int n, int src_stream0, int L, int B, int ring_off,
                                   int N, int m, size_t row_bytes, cudaStream_t st)
 {
     const int row_units = (int)(row_bytes / 16);
@@ -119,8 +126,30 @@ cudaError_t launch_append_sliding(void *k_slab, void *v_slab, const void *k_src,
     if (chunks > 32) chunks = 32;
     dim3 grid(chunks, n);
     append_sliding_kernel<<<grid, 256, 0, st>>>((uint4 *)k_slab, (uint4 *)v_slab, (const uint4 *)k_src,
-                                                (const uint4 *)v_src, state, total, batch, src_stream0, L, B, S_max, N, m,
+                                                (const uint4 *)v_src, state, total, batch, src_stream0, L, B, ring_off, N, m,
                                                 row_units);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// The staged prefix becomes the one attention reads: flip the bank, take over the staged length.
+__global__ void commit_static_kernel(StreamState *state, StreamBatch batch, int n)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int b = batch.id[i];
+    StreamState s = state[b];
+    if (s.staged_len >= 0) {
+        s.bank ^= 1;
+        s.static_len = s.staged_len;
+        s.staged_len = -1;
+        state[b] = s;
+    }
+}
+
+cudaError_t launch_commit_static(StreamState *state, const StreamBatch &batch, int n, cudaStream_t st)
+{
+    commit_static_kernel<<<(n + 127) / 128, 128, 0, st>>>(state, batch, n);
     count_launch();
     return cudaGetLastError();
 }

@@ -18,6 +18,7 @@ struct reflex_cache {
     WorkspaceLayout lay;
     std::vector<int32_t> static_len, head, count;
     std::vector<int64_t> total;
+    std::vector<int32_t> staged_len;   // host mirror of the length staged in the other static bank, -1 = none
     int attn_impl;
     int sm_count;
 };
@@ -49,10 +50,13 @@ bool desc_ok(const reflex_cache_desc *d)
     if (d->Hq % d->Hkv != 0) return false;
     if (!(d->d == 32 || d->d == 64 || d->d == 128 || d->d == 256)) return false;
     if (d->dtype != REFLEX_DTYPE_BF16 && d->dtype != REFLEX_DTYPE_F32) return false;
+    if (d->static_banks < 0 || d->static_banks > 2) return false;
     return true;
 }
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline int ring_off(const reflex_cache_desc &d) { return (d.static_banks == 2 ? 2 : 1) * d.S_max; }
 
 int check_stream_ids(const reflex_cache *c, const int32_t *ids, int n)
 {
@@ -121,7 +125,7 @@ unsigned long long reflex_kernel_launch_count(void) { return g_launches.load(std
 size_t reflex_cache_slab_bytes(const reflex_cache_desc *d)
 {
     if (!desc_ok(d)) return 0;
-    return (size_t)d->L * d->B * (size_t)(d->S_max + d->N) * d->Hkv * d->d * elem_size(d->dtype);
+    return (size_t)d->L * d->B * (size_t)(ring_off(*d) + d->N) * d->Hkv * d->d * elem_size(d->dtype);
 }
 
 size_t reflex_workspace_bytes(const reflex_cache_desc *d)
@@ -149,6 +153,7 @@ int reflex_cache_create(const reflex_cache_desc *desc, void *k_slab, void *v_sla
     c->k_slab = k_slab; c->v_slab = v_slab; c->ws = (char *)workspace;
     c->lay = workspace_layout(*desc);
     c->static_len.assign(desc->B, -1);
+    c->staged_len.assign(desc->B, -1);
     c->head.assign(desc->B, 0);
     c->count.assign(desc->B, 0);
     c->total.assign(desc->B, 0);
@@ -194,6 +199,7 @@ int reflex_cache_get_state(reflex_cache_t *c, int32_t *static_len, int32_t *head
     if (e != cudaSuccess) return cuda_fail(e, "state read-back");
     for (int b = 0; b < B; ++b) {
         c->static_len[b] = s[b].static_len; c->head[b] = s[b].head; c->count[b] = s[b].count; c->total[b] = tot[b];
+        c->staged_len[b] = s[b].staged_len;
         if (static_len) static_len[b] = s[b].static_len;
         if (head) head[b] = s[b].head;
         if (count) count[b] = s[b].count;
@@ -242,13 +248,14 @@ int reflex_cache_set_attention_impl(reflex_cache_t *c, int impl)
     return REFLEX_OK;
 }
 
-int reflex_cache_init_static(reflex_cache_t *c, const int32_t *stream_ids, int n_streams, const void *k_static,
-                             const void *v_static, int S_src, const int32_t *S, void *stream)
+static int write_static(reflex_cache_t *c, const int32_t *stream_ids, int n_streams, const void *k_static, const void *v_static, int S_src,
+                        const int32_t *S, int to_other_bank, void *stream)
 {
     if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");
     int rc = check_stream_ids(c, stream_ids, n_streams);
     if (rc) return rc;
     const reflex_cache_desc &d = c->desc;
+    if (to_other_bank && d.static_banks != 2) return fail(REFLEX_ERR_STATE, "the cache was created with one static bank (static_banks = 2 needed)");
     if (S_src < 0) return fail(REFLEX_ERR_SHAPE, "S_src=%d is negative", S_src);
     bool any = false;
     for (int i = 0; i < n_streams; ++i) {
@@ -267,9 +274,42 @@ int reflex_cache_init_static(reflex_cache_t *c, const int32_t *stream_ids, int n
         memset(&batch, 0, sizeof(batch));
         for (int i = 0; i < n; ++i) { batch.id[i] = stream_ids[i0 + i]; batch.len[i] = S ? S[i0 + i] : S_src; }
         cudaError_t e = launch_init_static(c->k_slab, c->v_slab, k_static, v_static, (StreamState *)(c->ws + c->lay.state_off),
-                                           batch, n, i0, d.L, d.B, d.S_max, d.N, S_src, row_bytes, st);
+                                           batch, n, i0, d.L, d.B, d.S_max, ring_off(d), d.N, S_src, to_other_bank, row_bytes, st);
         if (e != cudaSuccess) return cuda_fail(e, "init_static launch");
-        for (int i = 0; i < n; ++i) c->static_len[batch.id[i]] = batch.len[i];
+        for (int i = 0; i < n; ++i) (to_other_bank ? c->staged_len : c->static_len)[batch.id[i]] = batch.len[i];
+    }
+    return REFLEX_OK;
+}
+
+int reflex_cache_init_static(reflex_cache_t *c, const int32_t *stream_ids, int n_streams, const void *k_static,
+                             const void *v_static, int S_src, const int32_t *S, void *stream)
+{
+    return write_static(c, stream_ids, n_streams, k_static, v_static, S_src, S, 0, stream);
+}
+
+int reflex_cache_stage_static(reflex_cache_t *c, const int32_t *stream_ids, int n_streams, const void *k_static,
+                              const void *v_static, int S_src, const int32_t *S, void *stream)
+{
+    return write_static(c, stream_ids, n_streams, k_static, v_static, S_src, S, 1, stream);
+}
+
+int reflex_cache_commit_static(reflex_cache_t *c, const int32_t *stream_ids, int n_streams, void *stream)
+{
+    if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");
+    int rc = check_stream_ids(c, stream_ids, n_streams);
+    if (rc) return rc;
+    if (c->desc.static_banks != 2) return fail(REFLEX_ERR_STATE, "the cache was created with one static bank (static_banks = 2 needed)");
+    for (int i = 0; i < n_streams; ++i)
+        if (c->staged_len[stream_ids[i]] < 0) return fail(REFLEX_ERR_STATE, "stream %d: nothing staged", stream_ids[i]);
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int i0 = 0; i0 < n_streams; i0 += kStreamsPerLaunch) {
+        const int n = (n_streams - i0 < kStreamsPerLaunch) ? n_streams - i0 : kStreamsPerLaunch;
+        StreamBatch batch;
+        memset(&batch, 0, sizeof(batch));
+        for (int i = 0; i < n; ++i) batch.id[i] = stream_ids[i0 + i];
+        cudaError_t e = launch_commit_static((StreamState *)(c->ws + c->lay.state_off), batch, n, st);
+        if (e != cudaSuccess) return cuda_fail(e, "commit_static launch");
+        for (int i = 0; i < n; ++i) { c->static_len[batch.id[i]] = c->staged_len[batch.id[i]]; c->staged_len[batch.id[i]] = -1; }
     }
     return REFLEX_OK;
 }
@@ -292,7 +332,7 @@ int reflex_cache_append_sliding(reflex_cache_t *c, const int32_t *stream_ids, in
         memset(&batch, 0, sizeof(batch));
         for (int i = 0; i < n; ++i) batch.id[i] = stream_ids[i0 + i];
         cudaError_t e = launch_append_sliding(c->k_slab, c->v_slab, k_new, v_new, (StreamState *)(c->ws + c->lay.state_off),
-                                              (int64_t *)(c->ws + c->lay.total_off), batch, n, i0, d.L, d.B, d.S_max, d.N, m,
+                                              (int64_t *)(c->ws + c->lay.total_off), batch, n, i0, d.L, d.B, ring_off(d), d.N, m,
                                               row_bytes, st);
         if (e != cudaSuccess) return cuda_fail(e, "append_sliding launch");
         for (int i = 0; i < n; ++i) {
@@ -405,6 +445,7 @@ int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, co
     p.state = (const StreamState *)(c->ws + c->lay.state_off);
     p.partials = (float *)(c->ws + c->lay.partial_off);
     p.L = d.L; p.B = d.B; p.Hq = d.Hq; p.Hkv = d.Hkv; p.d = d.d; p.S_max = d.S_max; p.N = d.N; p.T = T; p.layer = layer;
+    p.ring_off = ring_off(d);
     p.dyn_mask = dyn_mask;
     p.scale = scale > 0.f ? scale : 1.0f / sqrtf((float)d.d);
     p.dtype = d.dtype;

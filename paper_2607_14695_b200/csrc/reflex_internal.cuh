@@ -17,6 +17,8 @@ struct StreamState {
     int32_t head;        // next ring slot to write
     int32_t count;       // live ring tokens
     int32_t ticket;      // arrival counter of the append kernel (always 0 between launches)
+    int32_t bank;        // which static bank attention reads (0 unless the cache has two banks)
+    int32_t staged_len;  // rows written to the other bank by the last stage call, -1 = nothing staged
 };
 
 // Layout of the caller-lent workspace.
@@ -49,6 +51,7 @@ struct AttnParams {
     const StreamState *state;
     float *partials;               // split-K scratch
     int L, B, Hq, Hkv, d, S_max, N, T, layer;
+    int ring_off;                  // first ring row of a (layer, stream) block: S_max times the number of static banks
     int dyn_mask;
     float scale;
     int nsplit;
@@ -71,10 +74,11 @@ void count_launch(int n = 1);
 cudaError_t launch_state_init(StreamState *state, int64_t *total, uint32_t *status, const int32_t *head0_dev_or_null,
                               int B, int N, cudaStream_t st);
 cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
-                               const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max, int N, int S_src,
+                               const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max, int ring_off, int N, int S_src, int to_other_bank,
                                size_t row_bytes, cudaStream_t st);
+cudaError_t launch_commit_static(StreamState *state, const StreamBatch &batch, int n, cudaStream_t st);
 cudaError_t launch_append_sliding(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
-                                  int64_t *total, const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max,
+                                  int64_t *total, const StreamBatch &batch, int n, int src_stream0, int L, int B, int ring_off,
                                   int N, int m, size_t row_bytes, cudaStream_t st);
 cudaError_t launch_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, const void *b1, const void *W2,
                               const void *b2, float *gate_buf, int B, int R, int D, int Cd, int Hd, float eps, int dtype,

@@ -17,7 +17,8 @@ from . import synth
 
 class StepRunner:
     def __init__(self, w: synth.Workload, device: str = "cuda:0", variants: int = 2, attn_impl: int = rb.ATTN_AUTO,
-                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, gate_mode: str = "step"):
+                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, gate_mode: str = "step",
+                 static_banks: int = 1):
         self.w = w
         self.device = torch.device(device)
         self.variants = variants
@@ -35,7 +36,7 @@ class StepRunner:
 
         self.rnd = rnd
         head0 = [int(h) for h in synth.ring_head0(w)]
-        self.cache = rb.Cache(w.L, w.B, w.Hq, w.Hkv, w.d, w.S_max, w.N, w.T, w.dtype, device=device, ring_head0=head0)
+        self.cache = rb.Cache(w.L, w.B, w.Hq, w.Hkv, w.d, w.S_max, w.N, w.T, w.dtype, device=device, ring_head0=head0, static_banks=static_banks)
         rb.reflex_cache_set_attention_impl(self.cache, attn_impl)
         ids = list(range(w.B))
         # static prefix, a few streams at a time to bound the staging tensors
@@ -268,6 +269,19 @@ class StepRunner:
             self._static_src = (self.rnd(w.B, w.L, w.S_max, w.Hkv, w.d), self.rnd(w.B, w.L, w.S_max, w.Hkv, w.d))
         ks, vs = self._static_src
         rb.reflex_cache_init_static(self.cache, list(range(w.B)), ks, vs, S=[S] * w.B)
+
+    def stage_static(self, S: int, stream):
+        """Producer side of the asynchronous pipeline: the next observation's prefix goes to the idle static bank on
+        `stream` while the denoising steps keep reading the current one (cache created with static_banks=2)."""
+        w = self.w
+        if not hasattr(self, "_static_src"):
+            self._static_src = (self.rnd(w.B, w.L, w.S_max, w.Hkv, w.d), self.rnd(w.B, w.L, w.S_max, w.Hkv, w.d))
+        ks, vs = self._static_src
+        rb.reflex_cache_stage_static(self.cache, list(range(w.B)), ks, vs, S=[S] * w.B, stream=stream)
+
+    def commit_static(self):
+        """Consumer side, between two ticks: the staged prefix becomes the current one (index flip)."""
+        rb.reflex_cache_commit_static(self.cache, list(range(self.w.B)))
 
     def step_graph(self, k: int):
         self.step_graphs[k % len(self.step_graphs)].replay()

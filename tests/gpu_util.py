@@ -50,11 +50,12 @@ def check_close(got: np.ndarray, want: np.ndarray, dtype: int, what: str, rel_cl
 class Twin:
     """The same partitioned cache on both sides: OracleCache (CPU) and rb.Cache (CUDA)."""
 
-    def __init__(self, w: synth.Workload, head0=None, T_max=None, poison=False):
+    def __init__(self, w: synth.Workload, head0=None, T_max=None, poison=False, static_banks=1):
         self.w = w
         self.o = orc.OracleCache(w.L, w.B, w.Hkv, w.d, w.S_max, w.N, head0=head0)
         self.g = rb.Cache(w.L, w.B, w.Hq, w.Hkv, w.d, w.S_max, w.N, T_max or w.T, w.dtype, device=DEV,
-                          ring_head0=None if head0 is None else [int(h) for h in head0])
+                          ring_head0=None if head0 is None else [int(h) for h in head0], static_banks=static_banks)
+        self.bank = [0] * w.B       # which static bank of the slab holds each stream's current prefix
         if poison:  # stale / empty rows hold NaN on both sides: any read of them shows up
             self.g.k_slab.fill_(float("nan")); self.g.v_slab.fill_(float("nan"))
             for a in (self.o.k_static, self.o.v_static, self.o.k_ring, self.o.v_ring):
@@ -68,6 +69,24 @@ class Twin:
         for i, b in enumerate(ids):
             self.o.init_static(b, ks[i][:, : S_list[i]], vs[i][:, : S_list[i]])
         rb.reflex_cache_init_static(self.g, ids, to_dev(ks, w.dtype), to_dev(vs, w.dtype), S=S_list)
+
+    def stage_static(self, ids, S_list, variant, stream=None):
+        """A new prefix for these streams goes to the bank that is not being read, on both sides."""
+        w = self.w
+        S_src = max(S_list)
+        ks = synth.normal(w, "k_static", (len(ids), w.L, S_src, w.Hkv, w.d), 0, variant)
+        vs = synth.normal(w, "v_static", (len(ids), w.L, S_src, w.Hkv, w.d), 0, variant)
+        for i, b in enumerate(ids):
+            self.o.stage_static(b, ks[i][:, : S_list[i]], vs[i][:, : S_list[i]])
+        dk, dv = to_dev(ks, w.dtype), to_dev(vs, w.dtype)
+        rb.reflex_cache_stage_static(self.g, ids, dk, dv, S=S_list, stream=stream)
+        return dk, dv        # (kept alive by the caller while a side stream may still read them)
+
+    def commit_static(self, ids, stream=None):
+        for b in ids:
+            self.o.commit_static(b)
+            self.bank[b] ^= 1
+        rb.reflex_cache_commit_static(self.g, ids, stream=stream)
 
     def append(self, ids, m, variant):
         w = self.w
@@ -87,10 +106,12 @@ class Twin:
         for b in range(w.B):
             assert rb.reflex_cache_slot_map(self.g, b) == self.o.slot_map(b)
             S = max(self.o.static_len[b], 0)
-            assert np.array_equal(ks[:, b, :S], self.o.k_static[:, b, :S]) and np.array_equal(vs[:, b, :S], self.o.v_static[:, b, :S])
+            s0 = self.bank[b] * w.S_max
+            assert np.array_equal(ks[:, b, s0:s0 + S], self.o.k_static[:, b, :S]) and np.array_equal(vs[:, b, s0:s0 + S], self.o.v_static[:, b, :S])
             live = self.o.slot_map(b)[: self.o.count[b]]
-            assert np.array_equal(ks[:, b, w.S_max:][:, live], self.o.k_ring[:, b, live])
-            assert np.array_equal(vs[:, b, w.S_max:][:, live], self.o.v_ring[:, b, live])
+            r0 = self.g.ring_off
+            assert np.array_equal(ks[:, b, r0:][:, live], self.o.k_ring[:, b, live])
+            assert np.array_equal(vs[:, b, r0:][:, live], self.o.v_ring[:, b, live])
 
     def attention(self, layer, variant, dyn_mask=0, T=None, streams=None, scale=0.0, what="attention", partitioned=False, q_scale=1.0, rel_clause=False):
         w = self.w

@@ -553,3 +553,49 @@ def test_norm_qkv_short_streams_and_fallback(U):
     _norm_qkv_case(U, w13, 0, "norm+qkv R=13", streams=[0, 9, 10, 22])
     w3 = synth.CONFIGS["cfg2"].with_(B=50, T=3)
     _norm_qkv_case(U, w3, 0, "norm+qkv R=3 (plain kernel)", streams=[0, 42, 43, 49])
+
+
+# ------------------------------------------------------------------------------------------------
+# producer / consumer: a new prefix staged in the second static bank while the current one is read
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", ["simt", "tc", "tc2"])
+def test_double_banked_static_prefix(U, impl):
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"].with_(B=3, S=300, S_max=320)
+    tw = U.Twin(w, head0=[0, 9, 31], poison=True, static_banks=2)
+    rb.reflex_cache_set_attention_impl(tw.g, {"simt": rb.ATTN_SIMT, "tc": rb.ATTN_TC, "tc2": rb.ATTN_TC2}[impl])
+    tw.init_static([0, 1, 2], [300, 257, 64])
+    for i in range(3):
+        tw.append([0, 1, 2], 7, i)
+    tw.check_state()
+    tw.attention(0, 0, what="banked: first prefix")
+    # the producer stages new prefixes for streams 0 and 2 on its own stream; the consumer's attention, launched right
+    # behind it on the main stream without any ordering between the two, still sees the first prefix
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        keep = tw.stage_static([0, 2], [320, 100], 5, stream=side)
+    tw.attention(0, 1, dyn_mask=1, what="banked: staged but not committed")
+    tw.append([0, 1, 2], 30, 7)                                   # the ring moves on independently of the banks
+    tw.attention(0, 2, what="banked: staged, ring advanced")
+    # hand-over between two chunks: the consumer waits for the producer's writes, then flips
+    torch.cuda.current_stream().wait_stream(side)
+    tw.commit_static([0, 2])
+    tw.check_state()
+    tw.attention(0, 3, dyn_mask=1, what="banked: committed")
+    # and back into the first bank, with a shorter prefix for stream 0 only
+    keep2 = tw.stage_static([0], [48], 6)
+    tw.attention(0, 4, what="banked: second staging")
+    tw.commit_static([0])
+    tw.check_state()
+    tw.attention(0, 5, what="banked: second commit")
+    sl, _, _, _ = rb.reflex_cache_get_state(tw.g)
+    assert sl == [48, 257, 100]
+    with pytest.raises(rb.ReflexError) as e:
+        tw_err = rb.reflex_cache_commit_static(tw.g, [1])          # nothing staged for stream 1
+    assert e.value.code == rb.ERR_STATE
+    single = U.Twin(w.with_(B=1))
+    with pytest.raises(rb.ReflexError) as e:
+        rb.reflex_cache_commit_static(single.g, [0])
+    assert e.value.code == rb.ERR_STATE
+    del keep, keep2
