@@ -599,3 +599,19 @@ def test_double_banked_static_prefix(U, impl):
         rb.reflex_cache_commit_static(single.g, [0])
     assert e.value.code == rb.ERR_STATE
     del keep, keep2
+
+
+@pytest.mark.parametrize("frames,T", [(1, 75), (5, 50), (50, 25)])
+def test_context_window_and_chunk_sweep(U, frames, T):
+    """Points of the paper's context-window (1 to 50 frames of 256 tokens in the sliding history) and action-chunk (25 to 100
+    tokens) ablations: the ring is filled frame by frame past its capacity, with a partly filled second stream."""
+    N = frames * 256
+    w = synth.Workload("sweep", 43, synth.DTYPE_BF16, B=2, L=1, Hq=8, Hkv=1, d=256, S=300, S_max=320, N=N, T=T, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w, head0=[0, N - 100], poison=True)
+    tw.init_static([0, 1], [300, 129])
+    n_app = min(frames + 2, 7)            # past the capacity for the small windows, partly filled for the largest
+    for i in range(n_app):
+        tw.append([0, 1] if i % 3 != 2 else [0], 256, i)
+    tw.check_state()
+    tw.attention(0, 0, dyn_mask=0, what=f"sweep {frames} frames, T={T}")
+    tw.attention(0, 1, dyn_mask=1, what=f"sweep {frames} frames, T={T}, causal")
