@@ -625,26 +625,29 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // that all clusters hit at the same moment: 4.4 k cycles per unit.)
             const float inv = 1.f / l;
             const bool store_unit = w.t0 < p.T;   // an idle partner tile (odd tile count) has nothing to write
-            constexpr int SC = 128 / NP;           // columns per thread and round: a round stages 128 columns of O
+            // Rounds of 64 columns, alternating between the two 16 KB halves of the staging area: the TMA store of one round
+            // reads its half while the threads convert the next round into the other (one store of 32 KB per 128 columns made
+            // every second round wait about 900 cycles for the first to be read).
+            constexpr int SC = 64 / NP;            // columns per thread and round
+            static_assert(SC == 32 || SC == 16, "columns per thread and epilogue round");
 #pragma unroll 1
-            for (int rnd = 0; rnd < HD / 128; ++rnd) {
+            for (int rnd = 0; rnd < HD / 64; ++rnd) {
                 uint32_t o[SC];
-                const uint32_t o_addr = tmem_base + lane_addr + kColO + rnd * 128 + part * SC;
-#pragma unroll
-                for (int q = 0; q < SC / 32; ++q) tmem_ld32(o_addr + 32 * q, *reinterpret_cast<uint32_t(*)[32]>(o + 32 * q));
-                // the staging area may still be read by the stores of the previous round or unit
-                if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                const uint32_t o_addr = tmem_base + lane_addr + kColO + rnd * 64 + part * SC;
+                if constexpr (SC == 32) tmem_ld32(o_addr, *reinterpret_cast<uint32_t(*)[32]>(o));
+                else tmem_ld16(o_addr, *reinterpret_cast<uint32_t(*)[16]>(o));
+                // this half may still be read by the store issued two rounds ago (this unit's or the previous one's)
+                if (threadIdx.x == 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 tmem_wait_ld();
-                if (rnd == HD / 128 - 1) {
+                if (rnd == HD / 64 - 1) {
                     // all of O is in registers: the next unit's first P V may overwrite the accumulator
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(leader_ofree);
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
-                const int col0 = part * SC;
-                uint8_t *srow = smem + L::OFF_STAGE + (col0 >> 6) * (128 * 128) + row * 128;
-                const int c16 = (col0 & 63) >> 3;
+                uint8_t *srow = smem + L::OFF_STAGE + (rnd & 1) * (128 * 128) + row * 128;
+                const int c16 = part * (SC / 8);
 #pragma unroll
                 for (int c = 0; c < SC / 8; ++c) {
                     uint4 v;
@@ -659,11 +662,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 fence_proxy_async_smem();
                 asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
                 if (threadIdx.x == 64) {
-                    if (store_unit) {
-#pragma unroll
-                        for (int hh = 0; hh < 2; ++hh)
-                            tma_store_4d(&tm_o, base + L::OFF_STAGE + hh * (128 * 128), rnd * 128 + hh * 64, w.kvh * p.G, w.t0, w.b);
-                    }
+                    if (store_unit) tma_store_4d(&tm_o, base + L::OFF_STAGE + (rnd & 1) * (128 * 128), rnd * 64, w.kvh * p.G, w.t0, w.b);
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
