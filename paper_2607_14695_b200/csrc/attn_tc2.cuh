@@ -394,8 +394,13 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         bool ok = true;
         int gt = 0;
         [[maybe_unused]] int ui_s = 0;
+        // (the next unit's geometry -- a global load of the stream state and a handful of integer divisions, about 800 cycles --
+        // is worked out while this unit's last P V completes, not at the top of the next unit)
+        Unit w_next;
+        bool have_next = false;
         for (int u = u_start; u < n_units; u += u_stride, ++ui_s) {
-            const Unit w = load_unit(u);
+            const Unit w = have_next ? w_next : load_unit(u);
+            have_next = false;
             const int t_row = w.t0 + row / p.G;
             if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 0);
             const int rows_total = p.T * p.Hq;
@@ -571,6 +576,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 SM_EV(9);
             }
             gt += w.n_tiles;
+            if (u + u_stride < n_units) { w_next = load_unit(u + u_stride); have_next = true; }
             // ---- epilogue of the unit ----
             // (before this cluster's last epilogue: let the next kernel on the stream be scheduled; it waits for this grid's end)
             if (threadIdx.x == 64 && u + u_stride >= n_units) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
