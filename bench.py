@@ -279,13 +279,18 @@ def main():
     if runner.tdt == torch.bfloat16:
         qkv_avg_ms = avg_launch_ms(lambda v: [runner.norm_qkv(l, v, sh()) for l in range(w.L)], w.L)
         chained_ms = avg_launch_ms(lambda v: runner.step_chained(v), 1)
+        # a whole action-expert step: the fused calls above plus library GEMMs for the four plain projections
+        from paper_2607_14695_b200 import expert as ex
+        model = ex.ActionExpert(w, runner.cache, ex.random_weights_device(w, 4 * w.D, device=f"cuda:{local_rank}"), 4 * w.D, device=f"cuda:{local_rank}")
+        expert_ms = avg_launch_ms(lambda v: model.step(runner.xa, runner.cond[v % w.K], v % w.K), 1)
+        del model
         n_out = (w.Hq + 2 * w.Hkv) * w.d
         swiglu_avg_ms = avg_launch_ms(lambda v: [runner.norm_swiglu(l, v, sh()) for l in range(w.L)], w.L)
         chained = {"norm_qkv_avg_us": qkv_avg_ms * 1e3, "norm_qkv_tflops": 2.0 * w.B * w.T * w.D * n_out / (qkv_avg_ms * 1e-3) / 1e12,
                    "norm_qkv_shape_mnk": [w.B * w.T, n_out, w.D], "ms_per_step": chained_ms,
                    "norm_swiglu_avg_us": swiglu_avg_ms * 1e3, "norm_swiglu_tflops": 2.0 * w.B * w.T * w.D * 8 * w.D / (swiglu_avg_ms * 1e-3) / 1e12,
-                   "norm_swiglu_shape_m_f_k": [w.B * w.T, 4 * w.D, w.D],
-                   "what": "ms_per_step: every layer AdaRMSNorm + packed W_QKV projection in one launch, its Q/K/V read by that layer's attention, then the Euler update; norm_swiglu: AdaRMSNorm + fused gate/up projections + SiLU(gate)*up in one launch, timed alone"}
+                   "norm_swiglu_shape_m_f_k": [w.B * w.T, 4 * w.D, w.D], "expert_step_ms": expert_ms,
+                   "what": "ms_per_step: every layer AdaRMSNorm + packed W_QKV projection in one launch, its Q/K/V read by that layer's attention, then the Euler update; norm_swiglu: AdaRMSNorm + fused gate/up projections + SiLU(gate)*up in one launch, timed alone; expert_step_ms: a whole action-expert denoising step (input projection, L x (norm+QKV, attention, output projection, norm+SwiGLU, down projection), velocity head, Euler update; F = 4 D; the plain projections are library GEMMs)"}
     step_marks = []
     for k in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -615,3 +615,46 @@ def test_context_window_and_chunk_sweep(U, frames, T):
     tw.check_state()
     tw.attention(0, 0, dyn_mask=0, what=f"sweep {frames} frames, T={T}")
     tw.attention(0, 1, dyn_mask=1, what=f"sweep {frames} frames, T={T}, causal")
+
+
+# ------------------------------------------------------------------------------------------------
+# a whole action-expert denoising step chained from the library's calls
+# ------------------------------------------------------------------------------------------------
+def _expert_case(U, w, F, tol_v, what):
+    from oracle import expert_oracle as eo
+    from paper_2607_14695_b200 import expert as ex
+    rb = U.rb
+    tw = U.Twin(w, head0=[3] * w.B, poison=True)
+    tw.init_static(list(range(w.B)), [w.S] * w.B)
+    for i in range(3):
+        tw.append(list(range(w.B)), 2, i)
+    W = ex.expert_weights(w, F, std_scale=0.5)
+    dW = {n: U.to_dev(v, w.dtype) for n, v in W.items()}
+    model = ex.ActionExpert(w, tw.g, dW, F, device=U.DEV)
+    a0 = synth.normal(w, "noise", (w.B, w.T, w.A)).astype(np.float64)
+    if w.dtype == synth.DTYPE_BF16:          # the step reads the chunk through a storage-dtype mirror: start from representable values
+        a0 = synth.round_storage(a0.astype(np.float32), w.dtype).astype(np.float64)
+    cond = synth.cond_vectors(w, 0.6)
+    a_gpu = torch.from_numpy(a0.astype(np.float32)).to(U.DEV)
+    model.step(a_gpu, U.to_dev(cond, w.dtype), 1)
+    rb.reflex_cache_check_status(tw.g)
+    want_a, want_v = eo.expert_step(tw.o, W, a0, cond, w.K, w.Hq, w.Hkv, w.d, F)
+    got_v = U.to_host(model.vel)
+    rel = np.linalg.norm(got_v - want_v) / np.linalg.norm(want_v)
+    assert np.isfinite(got_v).all() and rel <= tol_v, f"{what}: velocity off by {rel:.3e} (relative Frobenius)"
+    err_a = np.abs(a_gpu.double().cpu().numpy() - want_a).max()
+    assert err_a <= tol_v * max(1.0, float(np.abs(want_v).max())) / w.K + 1e-6, f"{what}: action chunk off by {err_a:.3e}"
+    return rel
+
+
+def test_expert_step_fp32(U):
+    """Two layers in fp32 (plain kernels + fp32 library GEMMs): the chain agrees with the double-precision chain to fp32 rounding."""
+    w = synth.CONFIGS["cfg1"].with_(B=2, L=2)
+    _expert_case(U, w, 256, 2e-5, "expert fp32")
+
+
+def test_expert_step_bf16(U):
+    """Two layers at the action-expert widths in bf16 (tensor-core kernels, bf16 residual stream): a few roundings per layer
+    accumulate; the velocity stays within 2 % of the double-precision chain."""
+    w = synth.CONFIGS["cfg2"].with_(B=2, L=2, S=200, S_max=208)
+    _expert_case(U, w, 1024, 2e-2, "expert bf16")
