@@ -335,6 +335,239 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     if (warp == 1) tmem_dealloc2(tmem, NACC * kQkBN);
 }
 
+// ---- few rows (one or two streams): weights as the A operand ----------------------------------------------------------------
+// With at most 128 rows in all, tiles of 256 rows would be mostly padding and the launch a chain of sixteen dependent steps
+// on a handful of CTAs. Here the roles are swapped: out^T [features][rows] = W [features][D] . y'^T [D][rows]. A CTA owns 128
+// output features (the M of a cta_group::1 MMA; for SwiGLU 128 hidden features with a gate and an up accumulator), the rows
+// are the N (64 or 128), so the grid is features / 128 CTAs that each stream their own slice of the weights once (the
+// whole cost of the call) while eight warps rewrite the small x tile of every step as the gated B operand.
+constexpr int kSmThreads = 64 + 256;   // producer warp, MMA warp, eight warps that rewrite x and run the epilogue
+
+template <int NT, int NACC>      // NT: rows (tokens) padded to 64 or 128; NACC: 1, or 2 for SwiGLU (gate and up rows)
+struct SmSmem {
+    static constexpr int STAGES = NACC == 2 ? 4 : (NT == 64 ? 8 : 6);
+    static constexpr uint32_t W_TILE = 128 * 128;                 // 128 feature rows x 64 k
+    static constexpr uint32_t W_STAGE = NACC * W_TILE;
+    static constexpr uint32_t X_STAGE = NT * 128;                 // NT rows x 64 k
+    static constexpr uint32_t OFF_W = 0;
+    static constexpr uint32_t OFF_X = STAGES * W_STAGE;
+    static constexpr uint32_t OFF_BAR = OFF_X + STAGES * X_STAGE;
+    static constexpr uint32_t OFF_SS = OFF_BAR + 512;             // [4][128] partial sums of squares per row, then [128] 1/RMS
+    static constexpr uint32_t OFF_GATE = OFF_SS + 2560;
+    static constexpr uint32_t GATE_MAX = 16 * 1024;               // gates of the (at most 4) streams the rows belong to
+    static constexpr uint32_t TOTAL = OFF_GATE + GATE_MAX + 1024;
+    static_assert(TOTAL <= 227u * 1024u, "shared memory budget");
+    // mbarrier indices
+    static constexpr int S_XFULL = 0, S_BREADY = STAGES, S_EMPTY = 2 * STAGES, S_ACC = 3 * STAGES, S_COUNT = S_ACC + 1;
+};
+
+template <int NT, int NACC>
+__global__ void __launch_bounds__(kSmThreads, 1)
+norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, QkParams p)
+{
+    using S = SmSmem<NT, NACC>;
+    constexpr int kSmStages = S::STAGES;
+    constexpr int S_XFULL = S::S_XFULL, S_BREADY = S::S_BREADY, S_EMPTY = S::S_EMPTY, S_ACC = S::S_ACC, S_COUNT = S::S_COUNT;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    auto bar = [&](int i) -> uint32_t { return base + S::OFF_BAR + 8u * (uint32_t)i; };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + S::OFF_BAR + 8 * S_COUNT);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool swiglu = NACC == 2;
+    const int f0 = blockIdx.x * 128;                  // first output feature (hidden feature for SwiGLU) of this CTA
+    const int nk_steps = p.D / kQkBK;
+    constexpr int TP = 256 / NT;                      // transform threads per row: 4 (64 rows) or 2 (128 rows)
+    constexpr uint32_t kCols = NACC * NT < 32 ? 32 : NACC * NT;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kSmStages; ++s) {
+            mbar_init(bar(S_XFULL + s), 1);
+            mbar_init(bar(S_BREADY + s), 8);          // one arrival per transform warp
+            mbar_init(bar(S_EMPTY + s), 1);
+        }
+        mbar_init(bar(S_ACC), 1);
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tmap(&tm_x); prefetch_tmap(&tm_w);
+    }
+    if (warp == 1) tmem_alloc(smem_u32((const void *)tmem_slot), kCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    if (threadIdx.x == 64) QK_TRACE(2, 30, 0);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (threadIdx.x == 64) QK_TRACE(2, 30, 1);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool {
+        if (mbar_try_wait(bar(i), parity)) return true;
+        const unsigned long long t_start = globaltimer_ns();
+        for (uint32_t n = 1;; ++n) {
+            if (mbar_try_wait(bar(i), parity)) return true;
+            if ((n & 255u) == 0u) {
+                if (*abort_flag) return false;
+                if (globaltimer_ns() - t_start > kQkWaitNs) break;
+            }
+        }
+        *abort_flag = 1u;
+        if (p.status) atomicCAS(p.status, 0u, 0x80000000u | ((code + 112u) << 16) | (blockIdx.x & 0xFFFFu));
+        return false;
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int ks = 0; ks < nk_steps && ok; ++ks) {
+                const int s = ks % kSmStages;
+                if (ks >= kSmStages) ok = wait(S_EMPTY + s, (uint32_t)(ks / kSmStages - 1) & 1u, 1);
+                if (!ok) break;
+                // one barrier for both operands of the step: the threads that rewrite x wait for it, so their hand-over to the
+                // MMA warp also says that the weights are in place (one wait less per step in the issuing loop)
+                mbar_expect_tx(bar(S_XFULL + s), S::X_STAGE + S::W_STAGE);
+                tma_load_2d(base + S::OFF_X + s * S::X_STAGE, &tm_x, bar(S_XFULL + s), ks * kQkBK, 0);
+#pragma unroll
+                for (int j = 0; j < NACC; ++j)
+                    tma_load_2d(base + S::OFF_W + s * S::W_STAGE + j * S::W_TILE, &tm_w, bar(S_XFULL + s), ks * kQkBK, j * p.swiglu_F + f0);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (the warp stays converged, one elected lane issues) ----------------
+        constexpr uint32_t idesc = umma_idesc_bf16(128, NT, false);
+        bool ok = true;
+        for (int ks = 0; ks < nk_steps && ok; ++ks) {
+            const int s = ks % kSmStages;
+            const uint32_t ph = (uint32_t)(ks / kSmStages) & 1u;
+            if (lane == 0) QK_TRACE(1, ks, 0);
+            ok = wait(S_BREADY + s, ph, 3);
+            if (lane == 0) QK_TRACE(1, ks, 2);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int j = 0; j < NACC; ++j) {
+                uint64_t ad = umma_desc_sw128(base + S::OFF_W + s * S::W_STAGE + j * S::W_TILE, 16, 1024);
+                uint64_t bd = umma_desc_sw128(base + S::OFF_X + s * S::X_STAGE, 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < kQkBK / 16; ++kk) {
+                    umma_ss_elect(tmem + j * NT, ad, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    umma_desc_advance(ad, 32);
+                    umma_desc_advance(bd, 32);
+                }
+            }
+            umma_commit_elect(bar(S_EMPTY + s));
+        }
+        umma_commit_elect(bar(S_ACC));    // also after a wait that ran out: the epilogue warps must not wait for nothing
+    } else {
+        // ---------------- gate multiply (B operand) and epilogue ----------------
+        const int tid = threadIdx.x - 64;              // 0..255
+        const int row = tid % NT;                      // row (token) this thread rewrites
+        const int kpart = tid / NT;                    // which 64 / TP columns of every step
+        constexpr int KW = kQkBK / TP;                 // columns per thread and step: 16 or 32
+        const int b = min(row / p.R, p.B - 1);
+        float *gsm = reinterpret_cast<float *>(smem + S::OFF_GATE);
+        {
+            const int n4 = p.B * p.D / 4;              // (at most 4 streams: checked by the launcher)
+            const float4 *src = reinterpret_cast<const float4 *>(p.gate);
+            for (int i = tid; i < n4; i += 256) reinterpret_cast<float4 *>(gsm)[i] = __ldg(src + i);
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
+        if (threadIdx.x == 64) QK_TRACE(2, 30, 2);
+        const float *grow = gsm + (size_t)b * p.D + kpart * KW;
+        uint64_t ss2 = 0ull;
+        bool ok = true;
+        for (int ks = 0; ks < nk_steps; ++ks) {
+            const int s = ks % kSmStages;
+            const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + ks * kQkBK);
+            if (threadIdx.x == 64) QK_TRACE(2, ks, 0);
+            ok = ok && wait(S_XFULL + s, (uint32_t)(ks / kSmStages) & 1u, 4);
+            if (threadIdx.x == 64) QK_TRACE(2, ks, 1);
+            uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + row * 128;
+#pragma unroll
+            for (int c = 0; c < KW / 8; ++c) {
+                uint4 *cp = reinterpret_cast<uint4 *>(rowp + (((kpart * (KW / 8) + c) ^ (row & 7)) << 4));   // 128-byte swizzle
+                const uint4 xv = *cp;
+                const ulonglong2 ga = g2[2 * c], gb = g2[2 * c + 1];
+                const uint64_t gg[4] = {ga.x, ga.y, gb.x, gb.y};
+                uint32_t vv[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint64_t x2 = pack_f32x2(__uint_as_float(vv[k] << 16), __uint_as_float(vv[k] & 0xFFFF0000u));
+                    ss2 = fma_f32x2(x2, x2, ss2);
+                    float y0, y1;
+                    unpack_f32x2(mul_f32x2(x2, gg[k]), y0, y1);
+                    __nv_bfloat162 y2 = __floats2bfloat162_rn(y0, y1);
+                    vv[k] = *reinterpret_cast<uint32_t *>(&y2);
+                }
+                *cp = make_uint4(vv[0], vv[1], vv[2], vv[3]);
+            }
+            fence_proxy_async_smem();   // the tensor pipe reads what these threads wrote
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(S_BREADY + s));
+            if (threadIdx.x == 64) QK_TRACE(2, ks, 4);
+        }
+        // 1 / RMS of every row (a column of the accumulator), shared by all threads
+        float *ssm = reinterpret_cast<float *>(smem + S::OFF_SS);
+        {
+            float s0, s1;
+            unpack_f32x2(ss2, s0, s1);
+            ssm[kpart * 128 + row] = s0 + s1;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // ... as a table, one entry per row, behind the partial sums
+        float *rsm = ssm + 512;
+        if (tid < NT) {
+            float ssr = 0.f;
+#pragma unroll
+            for (int t = 0; t < TP; ++t) ssr += ssm[t * 128 + tid];
+            rsm[tid] = rsqrtf(ssr * (1.f / (float)p.D) + p.eps);
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (threadIdx.x == 64) QK_TRACE(2, 31, 0);
+        ok = wait(S_ACC, 0u, 5) && ok;
+        if (threadIdx.x == 64) QK_TRACE(2, 31, 1);
+        tc_fence_after();
+        // epilogue: thread = output feature (TMEM lane), columns = rows of x; the two warps of a lane quarter take alternate
+        // blocks of 32 rows
+        const int quarter = warp & 3;
+        const int egroup = (warp - 2) >> 2;
+        const int f = f0 + quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int n_feat = swiglu ? p.swiglu_F : p.nq + 2 * p.nk;
+        __nv_bfloat16 *dst0 = nullptr;            // row 0 of this feature's column in the tensor it belongs to
+        size_t pitch = 0;
+        if (swiglu || f < p.nq) { dst0 = p.q + f; pitch = (size_t)p.nq; }
+        else if (f < p.nq + p.nk) { dst0 = p.k + (f - p.nq); pitch = (size_t)p.nk; }
+        else { dst0 = p.v + (f - p.nq - p.nk); pitch = (size_t)p.nk; }
+#pragma unroll 1
+        for (int c = egroup; c < NT / 32; c += 2) {
+            uint32_t acc[32], up[32];
+            tmem_ld32(tmem + lane_addr + c * 32, acc);          // warp-wide: every lane takes part
+            if (swiglu) tmem_ld32(tmem + lane_addr + NT + c * 32, up);
+            tmem_wait_ld();
+            if (!ok || f >= n_feat) continue;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int r = c * 32 + i;
+                if (r < p.M) {                      // (no early exit: the accumulator stays in registers)
+                    const float rs = rsm[r];
+                    float val = __uint_as_float(acc[i]) * rs;
+                    if (swiglu) { const float u = __uint_as_float(up[i]) * rs; val = __fdividef(val, 1.f + __expf(-val)) * u; }
+                    dst0[(size_t)r * pitch] = __float2bfloat16_rn(val);     // a warp writes 64 contiguous bytes per row
+                }
+            }
+        }
+    }
+
+    if (threadIdx.x == 64) QK_TRACE(2, 31, 2);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kCols);
+}
+
 // Any dtype, any shape: one block per row. y = x * gamma / RMS(x) in shared memory (fp32), then every thread takes output
 // features n = tid, tid + 256, ... as plain dot products.
 template <typename T>
@@ -457,6 +690,30 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
     return e;
 }
 
+template <int NT, int NACC>
+static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, unsigned grid, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(norm_linear_small_kernel<NT, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmSmem<NT, NACC>::TOTAL);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kSmThreads);
+    cfg.dynamicSmemBytes = SmSmem<NT, NACC>::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_linear_small_kernel<NT, NACC>, mx, mw, p);
+    count_launch();
+    return e;
+}
+
 // swiglu_F = 0: W = W_QKV, outputs q / k / v with nq and nk columns. swiglu_F = F > 0: W = [W_gate; W_up] ([2F][D]),
 // q = the [M][F] output SiLU(gate) * up; nq, nk, k, v unused.
 cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *W, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
@@ -472,6 +729,20 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
                                           : launch_simt<float>(x, gate, W, q, k, v, M, R, D, nq, nk, swiglu_F, eps, st);
     }
     const int w_rows = swiglu_F > 0 ? 2 * swiglu_F : nq + 2 * nk;
+    if (impl == 0 && M <= 128 && (size_t)B * D * sizeof(float) <= SmSmem<64, 1>::GATE_MAX) {
+        // few rows: weights as the A operand, one CTA per 128 output features
+        const int NT = M <= 64 ? 64 : 128;
+        CUtensorMap sx, sw;
+        if (!tensor_map_2d_bf16(&sx, x, D, M, NT) || !tensor_map_2d_bf16(&sw, W, D, w_rows, 128)) return cudaErrorInvalidValue;
+        QkParams sp;
+        sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
+        sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.swiglu_F = swiglu_F;
+        sp.eps = eps; sp.status = status;
+        const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
+        const unsigned grid = (unsigned)((n_feat + 127) / 128);
+        if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, st) : launch_small<128, 2>(sx, sw, sp, grid, st);
+        return NT == 64 ? launch_small<64, 1>(sx, sw, sp, grid, st) : launch_small<128, 1>(sx, sw, sp, grid, st);
+    }
     CUtensorMap mx, mw;
     if (!tensor_map_2d_bf16(&mx, x, D, M, kQkBM) || !tensor_map_2d_bf16(&mw, W, D, w_rows, kQkBN / 2)) return cudaErrorInvalidValue;
     QkParams p;

@@ -658,3 +658,15 @@ def test_expert_step_bf16(U):
     accumulate; the velocity stays within 2 % of the double-precision chain."""
     w = synth.CONFIGS["cfg2"].with_(B=2, L=2, S=200, S_max=208)
     _expert_case(U, w, 1024, 2e-2, "expert bf16")
+
+
+@pytest.mark.parametrize("B", [1, 2])
+def test_norm_qkv_and_swiglu_few_rows(U, B):
+    """One or two streams of 50 rows (at most 128 rows in all): the kernel with the weights as the A operand, 64 or 128
+    row columns; Q/K/V routing with 20 feature tiles, SwiGLU with ragged hidden width."""
+    w = synth.CONFIGS["cfg2"].with_(B=B)
+    _norm_qkv_case(U, w, 0, f"norm+qkv {B * w.T} rows")
+    _norm_swiglu_case(U, w, 1024, 0, f"norm+swiglu {B * w.T} rows")
+    w2 = synth.CONFIGS["cfg2"].with_(B=B, Hq=3, Hkv=1, d=64, D=192)
+    _norm_qkv_case(U, w2, 0, f"norm+qkv {B * w.T} rows, 320 features")
+    _norm_swiglu_case(U, w2, 328, 0, f"norm+swiglu {B * w.T} rows, 328 hidden features")
