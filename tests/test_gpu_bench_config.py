@@ -70,3 +70,15 @@ def test_full_size_step_graph_sampled_outputs(cfg, streams):
     oc = _oracle_for_stream(runner, mid, b)
     want = oc.attention(0, 0, f(runner.q[mid][0][b]), f(runner.kd[mid][0][b]), f(runner.vd[mid][0][b]))
     U.check_close(runner.out[b].float().cpu().numpy().astype(np.float64), want, w.dtype, f"{cfg} attention layer {mid} direct")
+
+
+def test_fused_projections_at_bench_size():
+    """The two fused projections at the size and launch configuration `bench.py` times them (64 streams x 50 rows, D = 1024,
+    2560 Q/K/V features in 512-column tiles; F = 4096 hidden features), compared on a sample of streams."""
+    from paper_2607_14695_b200 import build as rbuild
+    rbuild.build()
+    import gpu_util as U
+    import test_gpu_parity as tp
+    w = synth.CONFIGS["cfg4"]
+    tp._norm_qkv_case(U, w, 0, "bench-size norm+qkv", streams=[0, 17, 63])
+    tp._norm_swiglu_case(U, w, 4 * w.D, 0, "bench-size norm+swiglu", streams=[5, 40])
