@@ -113,6 +113,12 @@ int reflex_cache_set_attention_impl(reflex_cache_t *cache, int impl);
  * created again. */
 int reflex_cache_check_status(reflex_cache_t *cache, void *stream);
 
+/* Self-test of that convention, safe by construction: launches one thread that waits on a barrier nothing will ever
+ * complete, gives up after limit_us microseconds (1..100000) and raises the cache's status word (wait site 127) exactly as
+ * a real kernel would. reflex_cache_check_status then returns REFLEX_ERR_TIMEOUT; the CUDA context stays usable, and a
+ * cache created anew over the same memory starts with a clear status word. */
+int reflex_cache_selftest_wait_limit(reflex_cache_t *cache, int limit_us, void *stream);
+
 /* ---- the five hot-path calls ------------------------------------------------------------------ */
 
 /* Sec. 3.1 "Static Prefix ... computed once and permanently pinned"; timestep invariance of the

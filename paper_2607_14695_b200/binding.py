@@ -25,7 +25,7 @@ ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_NOT
 EXPORTS = [
     "reflex_last_error_string", "reflex_version", "reflex_kernel_launch_count", "reflex_cache_slab_bytes", "reflex_workspace_bytes",
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
-    "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_init_static", "reflex_cache_stage_static",
+    "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_selftest_wait_limit", "reflex_cache_init_static", "reflex_cache_stage_static",
     "reflex_cache_commit_static", "reflex_cache_append_sliding",
     "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_adarmsnorm_swiglu", "reflex_partitioned_attention",
     "reflex_flow_step", "reflex_overlap_create", "reflex_overlap_destroy", "reflex_overlap_tick", "reflex_overlap_inference_done",
@@ -78,6 +78,7 @@ def load():
     lib.reflex_cache_slot_map.argtypes = [vp, i, i32p]
     lib.reflex_cache_set_attention_impl.argtypes = [vp, i]
     lib.reflex_cache_check_status.argtypes = [vp, vp]
+    lib.reflex_cache_selftest_wait_limit.argtypes = [vp, i, vp]
     lib.reflex_cache_init_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_cache_stage_static.argtypes = [vp, i32p, i, vp, vp, i, i32p, vp]
     lib.reflex_cache_commit_static.argtypes = [vp, i32p, i, vp]
@@ -209,6 +210,11 @@ def reflex_cache_set_attention_impl(cache: Cache, impl: int):
 
 def reflex_cache_check_status(cache: Cache, stream=None):
     _check(load().reflex_cache_check_status(cache.handle, _stream(stream)))
+
+
+def reflex_cache_selftest_wait_limit(cache: Cache, limit_us: int = 2000, stream=None):
+    """Launch the bounded-wait probe: its wait runs out after limit_us and raises the cache's status word."""
+    _check(load().reflex_cache_selftest_wait_limit(cache.handle, int(limit_us), _stream(stream)))
 
 
 def reflex_cache_init_static(cache: Cache, stream_ids, k_static, v_static, S=None, stream=None):

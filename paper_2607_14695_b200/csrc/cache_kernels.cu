@@ -2,6 +2,7 @@
 // sliding-ring append with circular pointer arithmetic (Sec. 3.4, App. B.2). Byte movers: rows are
 // opaque 16-byte units, so one kernel serves bf16 and fp32 storage.
 #include "reflex_internal.cuh"
+#include "sm100_ptx.cuh"
 
 namespace reflex {
 
@@ -150,6 +151,34 @@ __global__ void commit_static_kernel(StreamState *state, StreamBatch batch, int 
 cudaError_t launch_commit_static(StreamState *state, const StreamBatch &batch, int n, cudaStream_t st)
 {
     commit_static_kernel<<<(n + 127) / 128, 128, 0, st>>>(state, batch, n);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// Self-test of the bounded-wait convention every kernel of the library follows: one thread waits on an mbarrier that
+// nothing will ever complete, with a time limit, and on expiry records the wait site in the status word and returns.
+// Nothing here can hang: the limit is clamped by the launcher, and the loop leaves on its own.
+__global__ void wait_limit_probe_kernel(uint32_t *status, unsigned long long limit_ns, uint32_t code)
+{
+    __shared__ __align__(8) unsigned long long probe_bar;
+    using namespace ptx;
+    const uint32_t bar = smem_u32(&probe_bar);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        fence_mbar_init();
+        const unsigned long long t_start = globaltimer_ns();
+        bool done = false;
+        for (uint32_t n = 1; !done; ++n) {
+            if (mbar_try_wait(bar, 0)) done = true;                                   // (never: nothing arrives)
+            else if ((n & 63u) == 0u && globaltimer_ns() - t_start > limit_ns) break;
+        }
+        if (!done) atomicCAS(status, 0u, 0x80000000u | (code << 16) | (blockIdx.x & 0xFFFFu));
+    }
+}
+
+cudaError_t launch_wait_limit_probe(uint32_t *status, unsigned long long limit_ns, cudaStream_t st)
+{
+    wait_limit_probe_kernel<<<1, 32, 0, st>>>(status, limit_ns, 127u);
     count_launch();
     return cudaGetLastError();
 }

@@ -239,6 +239,15 @@ int reflex_cache_check_status(reflex_cache_t *c, void *stream)
     return REFLEX_OK;
 }
 
+int reflex_cache_selftest_wait_limit(reflex_cache_t *c, int limit_us, void *stream)
+{
+    if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");
+    if (limit_us < 1 || limit_us > 100000) return fail(REFLEX_ERR_INVALID_ARG, "limit_us=%d outside [1, 100000]", limit_us);
+    cudaError_t e = launch_wait_limit_probe((uint32_t *)(c->ws + c->lay.status_off), (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "wait-limit probe launch");
+    return REFLEX_OK;
+}
+
 int reflex_cache_set_attention_impl(reflex_cache_t *c, int impl)
 {
     if (!c) return fail(REFLEX_ERR_INVALID_ARG, "cache is NULL");

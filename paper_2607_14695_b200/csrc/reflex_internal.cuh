@@ -76,6 +76,7 @@ cudaError_t launch_state_init(StreamState *state, int64_t *total, uint32_t *stat
 cudaError_t launch_init_static(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
                                const StreamBatch &batch, int n, int src_stream0, int L, int B, int S_max, int ring_off, int N, int S_src, int to_other_bank,
                                size_t row_bytes, cudaStream_t st);
+cudaError_t launch_wait_limit_probe(uint32_t *status, unsigned long long limit_ns, cudaStream_t st);
 cudaError_t launch_commit_static(StreamState *state, const StreamBatch &batch, int n, cudaStream_t st);
 cudaError_t launch_append_sliding(void *k_slab, void *v_slab, const void *k_src, const void *v_src, StreamState *state,
                                   int64_t *total, const StreamBatch &batch, int n, int src_stream0, int L, int B, int ring_off,

@@ -670,3 +670,29 @@ def test_norm_qkv_and_swiglu_few_rows(U, B):
     w2 = synth.CONFIGS["cfg2"].with_(B=B, Hq=3, Hkv=1, d=64, D=192)
     _norm_qkv_case(U, w2, 0, f"norm+qkv {B * w.T} rows, 320 features")
     _norm_swiglu_case(U, w2, 328, 0, f"norm+swiglu {B * w.T} rows, 328 hidden features")
+
+
+def test_bounded_wait_reports_and_context_survives(U):
+    """A device-side wait that nothing completes gives up after its limit, raises the status word and returns: the next
+    status check reports REFLEX_ERR_TIMEOUT with the wait site, the CUDA context keeps working, and a cache created anew
+    starts clean. (The probe is the library's own self-test kernel; nothing is hung or faulted.)"""
+    import time
+    rb = U.rb
+    w = synth.CONFIGS["cfg2"]
+    tw = U.Twin(w)
+    tw.init_static([0], [w.S])
+    tw.append([0], 3, 0)
+    rb.reflex_cache_check_status(tw.g)                      # clean
+    t0 = time.time()
+    rb.reflex_cache_selftest_wait_limit(tw.g, 2000)         # 2 ms
+    with pytest.raises(rb.ReflexError) as e:
+        rb.reflex_cache_check_status(tw.g)
+    assert e.value.code == rb.ERR_TIMEOUT and "wait site 127" in str(e.value)
+    assert time.time() - t0 < 5.0
+    with pytest.raises(rb.ReflexError):
+        rb.reflex_cache_selftest_wait_limit(tw.g, 0)
+    # the context is alive: a fresh cache over new memory computes correctly and reports a clear status
+    tw2 = U.Twin(w)
+    tw2.init_static([0], [w.S])
+    tw2.append([0], 3, 0)
+    tw2.attention(0, 0, what="after a reported timeout")
