@@ -345,10 +345,13 @@ constexpr int kSmThreads = 64 + 256;   // producer warp, MMA warp, eight warps t
 
 template <int NT, int NACC>      // NT: rows (tokens) padded to 64 or 128; NACC: 1, or 2 for SwiGLU (gate and up rows)
 struct SmSmem {
-    static constexpr int STAGES = NACC == 2 ? 4 : (NT == 64 ? 8 : 6);
+    static constexpr int CPS = NACC == 2 ? 1 : 2;                 // 64-column chunks of the contraction axis per step: fewer, longer
+                                                                  // steps where the stages allow (every step costs ~560 cycles of hand-overs)
+    static constexpr int STAGES = NACC == 2 ? 4 : (NT == 64 ? 4 : 3);
     static constexpr uint32_t W_TILE = 128 * 128;                 // 128 feature rows x 64 k
-    static constexpr uint32_t W_STAGE = NACC * W_TILE;
-    static constexpr uint32_t X_STAGE = NT * 128;                 // NT rows x 64 k
+    static constexpr uint32_t W_STAGE = NACC * CPS * W_TILE;
+    static constexpr uint32_t X_TILE = NT * 128;                  // NT rows x 64 k
+    static constexpr uint32_t X_STAGE = CPS * X_TILE;
     static constexpr uint32_t OFF_W = 0;
     static constexpr uint32_t OFF_X = STAGES * W_STAGE;
     static constexpr uint32_t OFF_BAR = OFF_X + STAGES * X_STAGE;
@@ -378,7 +381,9 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool swiglu = NACC == 2;
     const int f0 = blockIdx.x * 128;                  // first output feature (hidden feature for SwiGLU) of this CTA
-    const int nk_steps = p.D / kQkBK;
+    constexpr int CPS = S::CPS;
+    const int n_chunks = p.D / kQkBK;
+    const int nk_steps = (n_chunks + CPS - 1) / CPS;       // (a last step may hold one chunk only: TMA zero-fills the other)
     constexpr int TP = 256 / NT;                      // transform threads per row: 4 (64 rows) or 2 (128 rows)
     constexpr uint32_t kCols = NACC * NT < 32 ? 32 : NACC * NT;
 
@@ -429,10 +434,14 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
                 // one barrier for both operands of the step: the threads that rewrite x wait for it, so their hand-over to the
                 // MMA warp also says that the weights are in place (one wait less per step in the issuing loop)
                 mbar_expect_tx(bar(S_XFULL + s), S::X_STAGE + S::W_STAGE);
-                tma_load_2d(base + S::OFF_X + s * S::X_STAGE, &tm_x, bar(S_XFULL + s), ks * kQkBK, 0);
 #pragma unroll
-                for (int j = 0; j < NACC; ++j)
-                    tma_load_2d(base + S::OFF_W + s * S::W_STAGE + j * S::W_TILE, &tm_w, bar(S_XFULL + s), ks * kQkBK, j * p.swiglu_F + f0);
+                for (int cc = 0; cc < CPS; ++cc) {
+                    const int col = (ks * CPS + cc) * kQkBK;
+                    tma_load_2d(base + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE, &tm_x, bar(S_XFULL + s), col, 0);
+#pragma unroll
+                    for (int j = 0; j < NACC; ++j)
+                        tma_load_2d(base + S::OFF_W + s * S::W_STAGE + (j * CPS + cc) * S::W_TILE, &tm_w, bar(S_XFULL + s), col, j * p.swiglu_F + f0);
+                }
             }
         }
     } else if (warp == 1) {
@@ -449,13 +458,16 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             tc_fence_after();
 #pragma unroll
             for (int j = 0; j < NACC; ++j) {
-                uint64_t ad = umma_desc_sw128(base + S::OFF_W + s * S::W_STAGE + j * S::W_TILE, 16, 1024);
-                uint64_t bd = umma_desc_sw128(base + S::OFF_X + s * S::X_STAGE, 16, 1024);
 #pragma unroll
-                for (int kk = 0; kk < kQkBK / 16; ++kk) {
-                    umma_ss_elect(tmem + j * NT, ad, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
-                    umma_desc_advance(ad, 32);
-                    umma_desc_advance(bd, 32);
+                for (int cc = 0; cc < CPS; ++cc) {
+                    uint64_t ad = umma_desc_sw128(base + S::OFF_W + s * S::W_STAGE + (j * CPS + cc) * S::W_TILE, 16, 1024);
+                    uint64_t bd = umma_desc_sw128(base + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE, 16, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < kQkBK / 16; ++kk) {
+                        umma_ss_elect(tmem + j * NT, ad, bd, idesc, (ks > 0 || cc > 0 || kk > 0) ? 1u : 0u);
+                        umma_desc_advance(ad, 32);
+                        umma_desc_advance(bd, 32);
+                    }
                 }
             }
             umma_commit_elect(bar(S_EMPTY + s));
@@ -481,28 +493,47 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
         bool ok = true;
         for (int ks = 0; ks < nk_steps; ++ks) {
             const int s = ks % kSmStages;
-            const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + ks * kQkBK);
             if (threadIdx.x == 64) QK_TRACE(2, ks, 0);
             ok = ok && wait(S_XFULL + s, (uint32_t)(ks / kSmStages) & 1u, 4);
             if (threadIdx.x == 64) QK_TRACE(2, ks, 1);
-            uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + row * 128;
+            // all loads of the step first (x pieces and gate values of every chunk), then the arithmetic and the stores: the
+            // stores could alias the later loads for all the compiler knows, and with a few independent loads per thread the
+            // shared-memory latency was most of a step
+            constexpr int NPC = KW / 8;                 // 16-byte pieces per thread and chunk
+            uint4 xv[CPS * NPC];
+            ulonglong2 gv[CPS * NPC * 2];
 #pragma unroll
-            for (int c = 0; c < KW / 8; ++c) {
-                uint4 *cp = reinterpret_cast<uint4 *>(rowp + (((kpart * (KW / 8) + c) ^ (row & 7)) << 4));   // 128-byte swizzle
-                const uint4 xv = *cp;
-                const ulonglong2 ga = g2[2 * c], gb = g2[2 * c + 1];
-                const uint64_t gg[4] = {ga.x, ga.y, gb.x, gb.y};
-                uint32_t vv[4] = {xv.x, xv.y, xv.z, xv.w};
+            for (int cc = 0; cc < CPS; ++cc) {
+                const int chunk = min(ks * CPS + cc, n_chunks - 1);      // (a chunk past the end: loaded but never used)
+                const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + chunk * kQkBK);
+                const uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE + row * 128;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const uint64_t x2 = pack_f32x2(__uint_as_float(vv[k] << 16), __uint_as_float(vv[k] & 0xFFFF0000u));
-                    ss2 = fma_f32x2(x2, x2, ss2);
-                    float y0, y1;
-                    unpack_f32x2(mul_f32x2(x2, gg[k]), y0, y1);
-                    __nv_bfloat162 y2 = __floats2bfloat162_rn(y0, y1);
-                    vv[k] = *reinterpret_cast<uint32_t *>(&y2);
+                for (int c = 0; c < NPC; ++c) {
+                    xv[cc * NPC + c] = *reinterpret_cast<const uint4 *>(rowp + (((kpart * NPC + c) ^ (row & 7)) << 4));   // 128-byte swizzle
+                    gv[(cc * NPC + c) * 2] = g2[2 * c];
+                    gv[(cc * NPC + c) * 2 + 1] = g2[2 * c + 1];
                 }
-                *cp = make_uint4(vv[0], vv[1], vv[2], vv[3]);
+            }
+#pragma unroll
+            for (int cc = 0; cc < CPS; ++cc) {
+                if (ks * CPS + cc < n_chunks) {         // (uniform; a chunk past the end holds TMA's zeros and stays as it is)
+                    uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE + row * 128;
+#pragma unroll
+                    for (int c = 0; c < NPC; ++c) {
+                        const uint64_t gg[4] = {gv[(cc * NPC + c) * 2].x, gv[(cc * NPC + c) * 2].y, gv[(cc * NPC + c) * 2 + 1].x, gv[(cc * NPC + c) * 2 + 1].y};
+                        uint32_t vv[4] = {xv[cc * NPC + c].x, xv[cc * NPC + c].y, xv[cc * NPC + c].z, xv[cc * NPC + c].w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const uint64_t x2 = pack_f32x2(__uint_as_float(vv[k] << 16), __uint_as_float(vv[k] & 0xFFFF0000u));
+                            ss2 = fma_f32x2(x2, x2, ss2);
+                            float y0, y1;
+                            unpack_f32x2(mul_f32x2(x2, gg[k]), y0, y1);
+                            __nv_bfloat162 y2 = __floats2bfloat162_rn(y0, y1);
+                            vv[k] = *reinterpret_cast<uint32_t *>(&y2);
+                        }
+                        *reinterpret_cast<uint4 *>(rowp + (((kpart * NPC + c) ^ (row & 7)) << 4)) = make_uint4(vv[0], vv[1], vv[2], vv[3]);
+                    }
+                }
             }
             fence_proxy_async_smem();   // the tensor pipe reads what these threads wrote
             __syncwarp();
