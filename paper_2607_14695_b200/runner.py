@@ -17,7 +17,7 @@ from . import synth
 
 class StepRunner:
     def __init__(self, w: synth.Workload, device: str = "cuda:0", variants: int = 2, attn_impl: int = rb.ATTN_AUTO,
-                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, gate_mode: str = "step",
+                 host_inputs: bool = False, ring_fill: Optional[int] = None, gate_scratch: bool = True, gate_mode: str = "tick",
                  static_banks: int = 1):
         self.w = w
         self.device = torch.device(device)
@@ -70,8 +70,13 @@ class StepRunner:
         #             layer's row kernel then takes its slice as a ready gate;
         #   "overlap" the gate of layer l+1 is computed on a second stream while layer l's attention runs;
         #   "inline"  each layer's reflex_adarmsnorm call computes its own gate (three launches per layer).
+        #   "tick"    one call per control tick computes the gates of all K steps and all L layers: c_k = [emb(t_k), s_t] is
+        #             known for the whole schedule when the tick starts (the streams' K conditioning vectors are stacked as
+        #             K * B "streams" of the gate kernels).
         self.gate_mode = gate_mode if gate_scratch else "inline"
         if gate_scratch:
+            self.cond_all = torch.cat(self.cond, dim=0).contiguous()                     # [K * B][Cd]
+            self.gate_tick = torch.empty((w.L * w.K * w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device)
             self.gate_all = torch.empty((w.L * w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device)
             self.gate_bufs = [torch.empty((w.B * (w.D + w.Hd),), dtype=torch.float32, device=self.device) for _ in range(2)]
             self.side = torch.cuda.Stream(device=self.device)
@@ -144,10 +149,20 @@ class StepRunner:
         kk = k % self.w.K
         self._call(("G", kk), lambda: rb.prepare_adarmsnorm_gate(self.cond[kk], self.W1s, self.b1s, self.W2s, self.b2s, self.gate_all))(sh)
 
-    def rows(self, layer: int, variant: int, sh, from_step_gates: bool = False):
+    def gates_of_tick(self, sh):
+        """gamma_l(c_k) for all layers and all K steps of the tick in one call."""
+        self._call(("T",), lambda: rb.prepare_adarmsnorm_gate(self.cond_all, self.W1s, self.b1s, self.W2s, self.b2s, self.gate_tick))(sh)
+
+    def rows(self, layer: int, variant: int, sh, from_step_gates=False, k: int = 0):
+        """from_step_gates: False (this layer's own gate buffer), True (gates_of_step), "tick" (gates_of_tick, step k)."""
         w = self.w
         n = w.B * w.D
-        gate = self.gate_all[layer * n:(layer + 1) * n] if from_step_gates else self.gate_bufs[layer & 1][:n]
+        if from_step_gates == "tick":
+            o = (layer * w.K + k % w.K) * n
+            gate = self.gate_tick[o:o + n]
+            from_step_gates = ("tick", k % w.K)
+        else:
+            gate = self.gate_all[layer * n:(layer + 1) * n] if from_step_gates else self.gate_bufs[layer & 1][:n]
         self._call(("r", layer, variant, from_step_gates), lambda: rb.prepare_adarmsnorm(
             self.x[layer][variant], self.y, None, None, None, None, None, gate_buf=gate.view(w.B, w.D)))(sh)
 
@@ -200,7 +215,13 @@ class StepRunner:
         variant = k % self.variants
         main = torch.cuda.current_stream()
         sh = rb.stream_handle(main)
-        if self.gate_mode == "step":
+        if self.gate_mode == "tick":
+            if k % self.w.K == 0:
+                self.gates_of_tick(sh)
+            for layer in range(self.w.L):
+                self.rows(layer, variant, sh, "tick", k)
+                self.attention(layer, variant, sh)
+        elif self.gate_mode == "step":
             self.gates_of_step(k, sh)
             for layer in range(self.w.L):
                 self.rows(layer, variant, sh, True)
@@ -237,10 +258,11 @@ class StepRunner:
         """One graph per distinct step (conditioning index x input variant)."""
         import math
         period = self.w.K * self.variants // math.gcd(self.w.K, self.variants)
-        self.step_graphs, self.kernels_per_step = [], 0
+        self.step_graphs, self.kernels_per_step, self.kernels_each = [], 0, []
         for k in range(period):
             g, n = self.capture(lambda k=k: self.step(k))
             self.step_graphs.append(g)
+            self.kernels_each.append(n)
             self.kernels_per_step = n
         return self.step_graphs
 
