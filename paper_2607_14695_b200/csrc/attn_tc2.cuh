@@ -453,12 +453,14 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     // as this CTA's V half has landed. (Doing it at the end of the tile, where every thread waits for V anyway,
                     // puts the clearing stores and their proxy fence in front of the P-ready arrival: measured slower.)
                     ok = ok && wait(C_VLAND + st, vph, 12);
-                    if (koff == 0 && row < 64 && !((tmask >> row) & 1ull)) {
+                    // (all 128 threads of the slice share the stores: thread `row` takes half of V row `row % 64`. Two warps
+                    // clearing a whole dead half alone, 32 stores each, held their next shared-memory load for 700 cycles.)
+                    if (koff == 0 && !((tmask >> (row & 63)) & 1ull)) {
 #pragma unroll
                         for (int c = 0; c < VCH; ++c) {
-                            uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (half * 64 + row) * 128);
+                            uint4 *vr = reinterpret_cast<uint4 *>(smem + L::OFF_V + st * L::V_STAGE + c * (128 * 128) + (half * 64 + (row & 63)) * 128) + (row >> 6) * 4;
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) vr[i] = make_uint4(0, 0, 0, 0);
+                            for (int i = 0; i < 4; ++i) vr[i] = make_uint4(0, 0, 0, 0);
                         }
                     }
                 }
