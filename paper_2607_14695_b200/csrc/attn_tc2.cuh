@@ -361,8 +361,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const uint32_t p_tmem = tmem_base + kColS + buf * kTc2Keys;
                     uint64_t vd = vdesc0;
                     umma_desc_advance(vd, (uint32_t)st * L::V_STAGE);
-#pragma unroll
-                    for (int kk = 0; kk < kTc2Keys / 16; ++kk) {
+                    // a tile whose second 64-key half lies past the unit's last key (odd number of halves) contributes
+                    // nothing from it: its P is zero and its V rows were never loaded, so those four MMAs are left out
+                    const int ksteps = (2 * (w.tile0 + jj) + 1 < w.H) ? kTc2Keys / 16 : kTc2Keys / 32;
+#pragma unroll 4
+                    for (int kk = 0; kk < ksteps; ++kk) {
                         umma2_ts_elect(tmem_base + kColO, p_tmem + kk * 8, vd, idesc_pv, (jj > 0 || kk > 0) ? 1u : 0u);
                         umma_desc_advance(vd, 16 * 128);   // the next 16 keys
                     }
@@ -448,7 +451,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int c = 0; c < KT; ++c) s[c] = __uint_as_float(r[c]);
                 }
                 SM_EV(2);
-                if (tmask != ~0ull) {
+                if (tmask != ~0ull && h < w.H) {   // (a half past the unit's last key is never read by P V: nothing to clear)
                     // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows as soon
                     // as this CTA's V half has landed. (Doing it at the end of the tile, where every thread waits for V anyway,
                     // puts the clearing stores and their proxy fence in front of the P-ready arrival: measured slower.)
@@ -567,7 +570,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // reading O out. Their parity test stays unambiguous because S(g) exists only after P V(g-2) completed, so the
                 // barrier of tile g-1 has finished the phase of tile g-3 and cannot have passed that of tile g+1.)
                 // the arrive below also tells the leader that this CTA's V half is in place
-                if (tmask == ~0ull) ok = ok && wait(C_VLAND + st, vph, 12);
+                if (tmask == ~0ull || h >= w.H) ok = ok && wait(C_VLAND + st, vph, 12);
                 SM_EV(8);
                 fence_proxy_async_smem();   // V rows cleared above are read by the tensor pipe
                 tc_fence_before();
