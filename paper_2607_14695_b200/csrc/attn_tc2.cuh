@@ -23,6 +23,7 @@
 // softmax arrivals through shared::cluster arrives); completions fan out with multicast commits.
 // Included by attn_tc.cu (shares its tile geometry and tensor maps).
 #pragma once
+#include <type_traits>
 
 namespace reflex {
 
@@ -417,14 +418,17 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             float m_ref = -INFINITY, l = 0.f;
             const int full_halves = w.g.S / kBN;      // 64-key halves that lie entirely inside the static prefix
-            for (int jj = 0; jj < w.n_tiles; ++jj) {
+            // one tile of the softmax, compiled twice: for a half that lies entirely inside the static prefix (every key live:
+            // no masks, nothing to clear) and for the rest
+            auto tile = [&](auto full_c, const int jj) {
+                constexpr bool FULL = decltype(full_c)::value;
                 const int gi = gt + jj, buf = gi & 1, st = gi % NVS;
                 const uint32_t vph = (uint32_t)(gi / NVS) & 1u;
                 const int h = 2 * (w.tile0 + jj) + half;
-                uint64_t tmask = 0ull, rmask = 0ull;   // liveness of the 64 keys of this half: for every row / for this row
-                if (h < full_halves) {
-                    tmask = rmask = ~0ull;             // inside the static prefix, before its last (partial) half: the common case
-                } else if (h < w.H) {
+                uint64_t tmask = ~0ull, rmask = ~0ull;   // liveness of the 64 keys of this half: for every row / for this row
+                if constexpr (!FULL) {
+                  tmask = rmask = 0ull;
+                  if (h < w.H) {
                     const TileRef tr = w.g.decode(h);
                     tmask = w.g.tile_mask(tr);
                     rmask = tmask;
@@ -432,8 +436,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         const int lim = t_row - tr.idx * kBN;
                         rmask &= (lim < 0) ? 0ull : (lim >= 63 ? ~0ull : ((2ull << lim) - 1ull));
                     }
+                  }
                 }
-                const uint64_t smask = (rmask >> koff) & kSliceFull;   // this thread's KT keys
+                const uint64_t smask = FULL ? kSliceFull : ((rmask >> koff) & kSliceFull);   // this thread's KT keys
 #define SM_EV(ev) do { if (threadIdx.x == 64 && ui_s == 0) TC2_TRACE(3, jj, ev); } while (0)
                 SM_EV(0);
                 ok = ok && wait(C_SFULL + buf, (uint32_t)(gi >> 1) & 1u, 9);
@@ -451,7 +456,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int c = 0; c < KT; ++c) s[c] = __uint_as_float(r[c]);
                 }
                 SM_EV(2);
-                if (tmask != ~0ull && h < w.H) {   // (a half past the unit's last key is never read by P V: nothing to clear)
+                if (!FULL && tmask != ~0ull && h < w.H) {   // (a half past the unit's last key is never read by P V: nothing to clear)
                     // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows as soon
                     // as this CTA's V half has landed. (Doing it at the end of the tile, where every thread waits for V anyway,
                     // puts the clearing stores and their proxy fence in front of the P-ready arrival: measured slower.)
@@ -467,7 +472,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
-                if (smask != kSliceFull) apply_slice_mask<KT>(s, smask);
+                if (!FULL && smask != kSliceFull) apply_slice_mask<KT>(s, smask);
                 // three-input maxima: half the instructions of a two-input chain (the single MMA-issuing thread shares its
                 // scheduler with two of these warps, and every issue slot they do not take is one it can have)
                 float mx4[4] = {s[0], s[1], s[2], s[3]};
@@ -544,7 +549,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), a, b);
                     l += a + b;
                 }
-                if (kTc2PolyEighths > 0 && smask != kSliceFull) {
+                if (!FULL && kTc2PolyEighths > 0 && smask != kSliceFull) {
                     // the polynomial gives a masked key 2^-125 instead of 0 (nothing for the sum, but P must be exactly 0
                     // there): clear those halves of the packed words
 #pragma unroll
@@ -570,7 +575,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // reading O out. Their parity test stays unambiguous because S(g) exists only after P V(g-2) completed, so the
                 // barrier of tile g-1 has finished the phase of tile g-3 and cannot have passed that of tile g+1.)
                 // the arrive below also tells the leader that this CTA's V half is in place
-                if (tmask == ~0ull || h >= w.H) ok = ok && wait(C_VLAND + st, vph, 12);
+                if (FULL || tmask == ~0ull || h >= w.H) ok = ok && wait(C_VLAND + st, vph, 12);
                 SM_EV(8);
                 fence_proxy_async_smem();   // V rows cleared above are read by the tensor pipe
                 tc_fence_before();
@@ -579,6 +584,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // barrier a CTA one tile ahead would complete this tile's phase with its arrivals for the next)
                 if (lane == 0) mbar_arrive_cluster(leader_pfull[buf]);
                 SM_EV(9);
+            };
+            for (int jj = 0; jj < w.n_tiles; ++jj) {
+                if (2 * (w.tile0 + jj) + half < full_halves) tile(std::true_type{}, jj);
+                else tile(std::false_type{}, jj);
             }
             gt += w.n_tiles;
             if (u + u_stride < n_units) { w_next = load_unit(u + u_stride); have_next = true; }
