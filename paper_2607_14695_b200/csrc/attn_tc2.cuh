@@ -420,8 +420,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int full_halves = w.g.S / kBN;      // 64-key halves that lie entirely inside the static prefix
             // one tile of the softmax, compiled twice: for a half that lies entirely inside the static prefix (every key live:
             // no masks, nothing to clear) and for the rest
-            auto tile = [&](auto full_c, const int jj) {
-                constexpr bool FULL = decltype(full_c)::value;
+            auto tile = [&](auto mode_c, const int jj) {
+                constexpr bool FULL = decltype(mode_c)::value == 0;
+                // a half past the unit's last key (odd number of halves: second half of the last tile) has no logits to read and
+                // no P to write: its threads only take part in the row exchange, rescale their columns of O and arrive
+                constexpr bool DEAD = decltype(mode_c)::value == 2;
                 const int gi = gt + jj, buf = gi & 1, st = gi % NVS;
                 const uint32_t vph = (uint32_t)(gi / NVS) & 1u;
                 const int h = 2 * (w.tile0 + jj) + half;
@@ -441,12 +444,12 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint64_t smask = FULL ? kSliceFull : ((rmask >> koff) & kSliceFull);   // this thread's KT keys
 #define SM_EV(ev) do { if (threadIdx.x == 64 && ui_s == 0) TC2_TRACE(3, jj, ev); } while (0)
                 SM_EV(0);
-                ok = ok && wait(C_SFULL + buf, (uint32_t)(gi >> 1) & 1u, 9);
-                SM_EV(1);
-                if (threadIdx.x == 64 && jj == 0) TC2_TRACE(2, ui_s, 1);
-                tc_fence_after();
                 float s[KT];
-                {
+                if constexpr (!DEAD) {
+                    ok = ok && wait(C_SFULL + buf, (uint32_t)(gi >> 1) & 1u, 9);
+                    SM_EV(1);
+                    if (threadIdx.x == 64 && jj == 0) TC2_TRACE(2, ui_s, 1);
+                    tc_fence_after();
                     const uint32_t s_addr = tmem_base + lane_addr + kColS + buf * kTc2Keys + part * KT;
                     uint32_t r[KT];
 #pragma unroll
@@ -456,7 +459,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int c = 0; c < KT; ++c) s[c] = __uint_as_float(r[c]);
                 }
                 SM_EV(2);
-                if (!FULL && tmask != ~0ull && h < w.H) {   // (a half past the unit's last key is never read by P V: nothing to clear)
+                if (!FULL && !DEAD && tmask != ~0ull) {   // (a half past the unit's last key is never read by P V: nothing to clear)
                     // dead keys get weight 0, but 0 x (stale NaN/Inf bytes) would still poison O: clear their V rows as soon
                     // as this CTA's V half has landed. (Doing it at the end of the tile, where every thread waits for V anyway,
                     // puts the clearing stores and their proxy fence in front of the P-ready arrival: measured slower.)
@@ -472,6 +475,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                 }
+                float mx = -INFINITY;
+                if constexpr (!DEAD) {
                 if (!FULL && smask != kSliceFull) apply_slice_mask<KT>(s, smask);
                 // three-input maxima: half the instructions of a two-input chain (the single MMA-issuing thread shares its
                 // scheduler with two of these warps, and every issue slot they do not take is one it can have)
@@ -485,7 +490,8 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if constexpr ((KT - 4) % 8 == 4) {
                     mx4[0] = max3_f32(mx4[0], s[KT - 4], s[KT - 3]); mx4[1] = max3_f32(mx4[1], s[KT - 2], s[KT - 1]);
                 }
-                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                }
                 // meet the threads that hold the other keys of this row: every one of them publishes its maximum rounded up
                 // to bf16 and takes the largest of the NP published values, so all agree. Past this barrier every thread of the
                 // row has its logits in registers, so P may overwrite them in tensor memory.
@@ -529,6 +535,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // the running sums, the polynomial). A quarter of the key pairs take a cubic on the FMA pipe, the rest the MUFU
                 // unit (4 results per clock and scheduler): measured 2/8 35.4 us, 0/8 35.6, 3/8 35.9, 4/8 36.4 per launch.
                 SM_EV(6);
+                if constexpr (!DEAD) {
                 const uint64_t sc2 = pack_f32x2(p.scale_log2, p.scale_log2), nm2 = pack_f32x2(-mr, -mr);
                 const Ex2PolyConsts pk = ex2_poly_consts();
                 uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
@@ -570,12 +577,13 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     else tmem_st16(p_addr, *reinterpret_cast<const uint32_t(*)[16]>(packed));
                     tmem_wait_st();
                 }
+                }
                 SM_EV(7);
                 // (The waits on a P V barrier, one barrier per S/P buffer, come at irregular times: before rescaling O and before
                 // reading O out. Their parity test stays unambiguous because S(g) exists only after P V(g-2) completed, so the
                 // barrier of tile g-1 has finished the phase of tile g-3 and cannot have passed that of tile g+1.)
                 // the arrive below also tells the leader that this CTA's V half is in place
-                if (FULL || tmask == ~0ull || h >= w.H) ok = ok && wait(C_VLAND + st, vph, 12);
+                if (FULL || DEAD || tmask == ~0ull) ok = ok && wait(C_VLAND + st, vph, 12);
                 SM_EV(8);
                 fence_proxy_async_smem();   // V rows cleared above are read by the tensor pipe
                 tc_fence_before();
@@ -586,8 +594,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 SM_EV(9);
             };
             for (int jj = 0; jj < w.n_tiles; ++jj) {
-                if (2 * (w.tile0 + jj) + half < full_halves) tile(std::true_type{}, jj);
-                else tile(std::false_type{}, jj);
+                const int hh = 2 * (w.tile0 + jj) + half;
+                if (hh < full_halves) tile(std::integral_constant<int, 0>{}, jj);
+                else if (hh < w.H) tile(std::integral_constant<int, 1>{}, jj);
+                else tile(std::integral_constant<int, 2>{}, jj);
             }
             gt += w.n_tiles;
             if (u + u_stride < n_units) { w_next = load_unit(u + u_stride); have_next = true; }
