@@ -269,14 +269,15 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         tma2_load_3d(base + L::OFF_K + st * L::K_STAGE + ch * (64 * 128), tr.dyn ? &tm_kd : &tm_k,
                                      bar(C_KFULL + st) & kPeerBitMask, ch * 64, w.kvh, tr.row0);
                 }
-                if (c.jj == 0) {
-                    // this unit's Q tile, once the last Q K^T of the previous unit has drained the buffer
-                    if (c.ui >= 1) ok = wait(C_QEMPTY, (uint32_t)(c.ui - 1) & 1u, 14);
-                    if (!ok) return;
-                    if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
-                    for (int ch = 0; ch < CH; ++ch)
-                        tma2_load_4d(base + L::OFF_Q + ch * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, ch * 64, w.kvh * p.G, w.t0, w.b);
-                }
+            };
+            auto issue_q = [&](const Cursor &c) {
+                // a unit's Q tile, once the last Q K^T of the previous unit has drained the buffer
+                const Unit &w = c.w;
+                if (c.ui >= 1) ok = wait(C_QEMPTY, (uint32_t)(c.ui - 1) & 1u, 14);
+                if (!ok) return;
+                if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
+                for (int ch = 0; ch < CH; ++ch)
+                    tma2_load_4d(base + L::OFF_Q + ch * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, ch * 64, w.kvh * p.G, w.t0, w.b);
             };
             auto issue_v = [&](const Cursor &c) {
                 const Unit &w = c.w;
@@ -300,14 +301,19 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ck.u = u_start; ck.ui = 0; ck.jj = 0; ck.g = 0;
             settle(ck);
             cv = ck;
-            if (kLead == 1 && ck.valid) { issue_k(ck); advance(ck); }
+            if (kLead == 1 && ck.valid) { issue_k(ck); issue_q(ck); advance(ck); }
+            // At a unit boundary the pipe's completions come as QK(last - 1) PV(last - 2) QK(last): the next unit's first K
+            // tile, the V tile of this unit's last P V and then the next unit's Q tile go out in that order, and the next
+            // unit's geometry (a global load and some divisions) is worked out only after the V tile is on its way.
             while (cv.valid && ok) {
-                if (ck.valid) {
-                    issue_k(ck);
-                    if (!ok) break;
+                const bool k_now = ck.valid;
+                if (k_now) { issue_k(ck); if (!ok) break; }
+                issue_v(cv);
+                if (!ok) break;
+                if (k_now) {
+                    if (ck.jj == 0) { issue_q(ck); if (!ok) break; }
                     advance(ck);
                 }
-                issue_v(cv);
                 advance(cv);
             }
         }
