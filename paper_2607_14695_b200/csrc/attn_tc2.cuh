@@ -299,9 +299,19 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             };
             Cursor ck, cv;
             ck.u = u_start; ck.ui = 0; ck.jj = 0; ck.g = 0;
+            // Where a Q tile lies follows from the unit's number alone: with unsplit keys (no unit is ever empty) the first
+            // one is requested before the stream state, which everything else about the unit hangs on, has come in.
+            const bool q_early = p.nsplit == 1 && u_start < n_units;
+            if (q_early) {
+                const int pair = u_start % n_pairs, kvh = (u_start / n_pairs) % p.Hkv, b = u_start / (n_pairs * p.Hkv);
+                if (rank == 0) mbar_expect_tx(bar(C_QFULL), 2 * L::Q_BYTES);
+                for (int ch = 0; ch < CH; ++ch)
+                    tma2_load_4d(base + L::OFF_Q + ch * (128 * 128), &tm_q, bar(C_QFULL) & kPeerBitMask, ch * 64, kvh * p.G,
+                                 (2 * pair + (int)rank) * p.tile_tokens, b);
+            }
             settle(ck);
             cv = ck;
-            if (kLead == 1 && ck.valid) { issue_k(ck); issue_q(ck); advance(ck); }
+            if (kLead == 1 && ck.valid) { issue_k(ck); if (!q_early) issue_q(ck); advance(ck); }
             // At a unit boundary the pipe's completions come as QK(last - 1) PV(last - 2) QK(last): the next unit's first K
             // tile, the V tile of this unit's last P V and then the next unit's Q tile go out in that order, and the next
             // unit's geometry (a global load and some divisions) is worked out only after the V tile is on its way.
@@ -311,7 +321,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 issue_v(cv);
                 if (!ok) break;
                 if (k_now) {
-                    if (ck.jj == 0) { issue_q(ck); if (!ok) break; }
+                    if (ck.jj == 0 && !(q_early && ck.ui == 0)) { issue_q(ck); if (!ok) break; }
                     advance(ck);
                 }
                 advance(cv);
