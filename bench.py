@@ -23,7 +23,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture (profiles/)
-NCU_TRAFFIC_BYTES = {("cfg4", "auto"): 76.6e6, ("cfg4", "tc2"): 76.6e6}
+NCU_TRAFFIC_BYTES = {("cfg4", "auto"): 76.0e6, ("cfg4", "tc2"): 76.0e6}
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
