@@ -24,6 +24,13 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture (profiles/)
 NCU_TRAFFIC_BYTES = {("cfg4", "auto"): 76.0e6, ("cfg4", "tc2"): 76.0e6}
+
+
+def workload_name(w):
+    """The one description of a workload that both arms print in `config.workload`."""
+    return (f"{w.name}: B={w.B} streams x L={w.L} layers, Hq={w.Hq}/Hkv={w.Hkv}, d={w.d}, static S={w.S}, ring N={w.N}, "
+            f"dynamic T={w.T}, D={w.D}, K={w.K}; one step = L x (AdaRMSNorm + partitioned attention) + Euler update")
+
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 
@@ -148,7 +155,7 @@ def run_reference(args, w):
     line = {"impl": "reference", "metric": "denoising_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "B": w.B, "L": w.L, "S": w.S, "N": w.N, "T": w.T},
+            "config": {"workload": workload_name(w), "B": w.B, "L": w.L, "S": w.S, "N": w.N, "T": w.T},
             "cpu_baseline": {"value": value, "unit": "steps/s", "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -401,8 +408,7 @@ def main():
         "metric": "denoising_steps_per_s", "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "us_per_step": ms_per_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == synth.DTYPE_BF16 else "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: B={w.B} streams x L={w.L} layers, Hq={w.Hq}/Hkv={w.Hkv}, d={w.d}, static S={w.S}, ring N={w.N}, "
-                               f"dynamic T={w.T}, D={w.D}, K={w.K}; one step = L x (AdaRMSNorm + partitioned attention) + Euler update",
+        "config": {"workload": workload_name(w),
                    "parallelism": "replicas only (independent streams per GPU, no collective)" if world > 1 else "single GPU",
                    "attention_impl": args.attn, "launch": "CUDA graph replay, one graph per step" if use_graph else "direct launches",
                    "gates": "gate MLPs of all K steps and L layers once per tick of K steps (the first step of every K carries the two gate launches)",
