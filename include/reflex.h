@@ -185,7 +185,11 @@ int reflex_adarmsnorm(const void *x, void *y, const void *cond, const void *W1, 
  * layer then calls reflex_adarmsnorm with cond == NULL and its slice gate_buf + l*B*D. L = 1 is the single-layer case.
  *   cond [B][Cd]; W1 [L][Hd][Cd], b1 [L][Hd], W2 [L][D][Hd], b2 [L][D]   device, dtype
  *   gate_buf  device fp32, L*B*(D+Hd) floats: gates [L][B][D] first, then scratch for the hidden activations
- * Requirements: D % 8 == 0, Cd and Hd multiples of 8 in [8, 1024], 1 <= L <= 65535. */
+ * Requirements: D % 8 == 0, Cd and Hd multiples of 8 in [8, 1024], 1 <= L <= 65535. Widths above 632 do not fit the
+ * staged kernels' shared memory and take a per-stream kernel, one launch per layer.
+ * bf16 with Cd, Hd multiples of 16 up to 320 runs on the tensor cores; should one of that kernel's bounded waits run
+ * out, its part of the gates is written as NaN (there is no cache handle to carry a status word), so the failure
+ * shows in everything computed from them. */
 int reflex_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2,
                            float *gate_buf, int L, int B, int D, int Cd, int Hd, int dtype, void *stream);
 
@@ -256,7 +260,11 @@ int reflex_adarmsnorm_swiglu(reflex_cache_t *cache, const void *x, const float *
  *   T              1..T_max
  *   scale          <= 0 selects 1/sqrt(d)
  *   dyn_mask       0: every query sees all T dynamic keys (Eq. 1 as printed);
- *                  1: dynamic key j hidden from dynamic query i when j > i (causal suffix, Prop. 1) */
+ *                  1: dynamic key j hidden from dynamic query i when j > i (causal suffix, Prop. 1)
+ * Calls on one cache must be ordered on a single stream (or by events): when the keys are split, all layers share the
+ * cache's one area of partial results in the workspace, and two calls that overlap on the GPU would race in it.
+ * Kernel attributes are set up the first time a kernel is used on each device, so one process may drive several
+ * devices (each with its own caches). */
 int reflex_partitioned_attention(reflex_cache_t *cache, int layer, const void *q, const void *k_dyn,
                                  const void *v_dyn, void *out, int T, float scale, int dyn_mask,
                                  void *stream);

@@ -618,12 +618,11 @@ template <int HD>
 cudaError_t launch_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
                      const CUtensorMap *mvd, const TcParams &tp, dim3 grid, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcSmem<HD>::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
+        return cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TcSmem<HD>::TOTAL);
+    });
+    if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(kTcThreads);
@@ -645,12 +644,11 @@ template <int HD>
 cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtensorMap *mv, const CUtensorMap *mkd,
                       const CUtensorMap *mvd, const CUtensorMap *mo, const TcParams &tp, dim3 grid, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Tc2Smem<HD>::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
+        return cudaFuncSetAttribute(attn_tc2_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Tc2Smem<HD>::TOTAL);
+    });
+    if (e0 != cudaSuccess) return e0;
     // programmatic stream serialisation: the grid may be scheduled while the preceding kernel drains; it waits
     // (griddepcontrol.wait) before it touches global memory
     cudaLaunchConfig_t cfg = {};
@@ -675,8 +673,11 @@ cudaError_t launch2_t(const CUtensorMap *mq, const CUtensorMap *mk, const CUtens
 template <int HD>
 int tc2_active_clusters_t(int cluster_ctas)
 {
-    static int cached[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    static int cached_dev[64][9] = {};          // per device ordinal (modulo 64): the answer depends on the device
     if (cluster_ctas < 2 || cluster_ctas > 8) return 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    int *cached = cached_dev[dev & 63];
     if (cached[cluster_ctas] != 0) return cached[cluster_ctas] > 0 ? cached[cluster_ctas] : 0;
     int n = 0;
     cudaLaunchConfig_t cfg = {};

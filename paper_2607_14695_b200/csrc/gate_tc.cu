@@ -122,6 +122,16 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     tmem_ld32(tmem + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(acc));
     tmem_ld32(tmem + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(acc + 32));
     tmem_wait_ld();
+    if (!ok && u < units) {
+        // a bounded wait ran out: this CTA's slice of the output is marked invalid (quiet NaN) instead of keeping the previous
+        // call's values, so whatever consumes the gates shows it
+        const int nb = min(kGtStreams, B - b0);
+        for (int n = 0; n < nb; ++n) {
+            const size_t o = ((size_t)layer * B + b0 + n) * units + u;
+            if (SILU) { out_hi[o] = __float2bfloat16_rn(__int_as_float(0x7fc00000)); out_lo[o] = __float2bfloat16_rn(0.f); }
+            else out_f32[o] = __int_as_float(0x7fc00000);
+        }
+    }
     if (ok && u < units) {
         const float bi = __bfloat162float(bias[(size_t)layer * units + u]);
         const int nb = min(kGtStreams, B - b0);
@@ -149,12 +159,11 @@ template <bool SILU, int PASSES>
 cudaError_t launch_one(const CUtensorMap &mw, const CUtensorMap &mv0, const CUtensorMap &mv1, const __nv_bfloat16 *bias, float *out_f32,
                        __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, int L, int B, int len, int units, int vec_rows_per_layer, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(gate_tc_kernel<SILU, PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GateTcSmem::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
+        return cudaFuncSetAttribute(gate_tc_kernel<SILU, PASSES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GateTcSmem::TOTAL);
+    });
+    if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((units + kGtUnits - 1) / kGtUnits, (B + kGtStreams - 1) / kGtStreams, L);
     cfg.blockDim = dim3(128);

@@ -383,13 +383,13 @@ static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const 
     const size_t smem_h = (size_t)(upb * Cd + kGateStreams * (Cd + 4)) * 4;
     const size_t smem_g = (size_t)(upb * Hd + kGateStreams * (Hd + 4)) * 4;
     float *hid = gate_buf + (size_t)L * B * D;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
         cudaError_t e = cudaFuncSetAttribute(gate_layer_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gate_layer_kernel<T, float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+        return e;
+    });
+    if (e0 != cudaSuccess) return e0;
     if constexpr (sizeof(T) == 2) {
         // bf16: both layers on the tensor cores, whatever L is (one call for L layers and L calls give the same bits); the
         // FMA kernels below remain for fp32 and for widths the tensor-core kernel does not take
@@ -402,13 +402,13 @@ static cudaError_t launch_gate_t(const T *cond, const T *W1, const T *b1, const 
     const size_t tiled_h = (size_t)(kTileUnits + kGateStreams) * (Cd + 4) * 4, tiled_g = (size_t)(kTileUnits + kGateStreams) * (Hd + 4) * 4;
     if (L > 1 && tiled_h <= 200 * 1024 && tiled_g <= 200 * 1024) {
         // many layers in one call: throughput of the whole batch matters more than the latency of one small grid
-        static bool tiled_attr_set = false;
-        if (!tiled_attr_set) {
+        static std::atomic<unsigned long long> tiled_attr_set{0};
+        e0 = once_per_device(tiled_attr_set, [] {
             cudaError_t e = cudaFuncSetAttribute(gate_layer_tiled_kernel<T, T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(gate_layer_tiled_kernel<T, float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e != cudaSuccess) return e;
-            tiled_attr_set = true;
-        }
+            return e;
+        });
+        if (e0 != cudaSuccess) return e0;
         gate_layer_tiled_kernel<T, T, true><<<dim3((Hd + kTileUnits - 1) / kTileUnits, groups, L), 256, tiled_h, st>>>(
             cond, W1, b1, hid, B, Cd, Hd, 0, (size_t)0, (size_t)B * Hd);
         count_launch();
@@ -521,10 +521,32 @@ __global__ void flow_step_kernel(float *__restrict__ x, const T *__restrict__ v,
     }
 }
 
+template <typename T>
+static cudaError_t launch_gate_wide_t(const T *cond, const T *W1, const T *b1, const T *W2, const T *b2, float *gate_buf, int L, int B,
+                                      int D, int Cd, int Hd, cudaStream_t st)
+{
+    const int cols = 64;
+    for (int l = 0; l < L; ++l) {
+        gate_kernel<T><<<dim3((D + cols - 1) / cols, B), 256, (size_t)(Cd + Hd) * 4, st>>>(
+            cond, W1 + (size_t)l * Hd * Cd, b1 + (size_t)l * Hd, W2 + (size_t)l * D * Hd, b2 + (size_t)l * D, gate_buf + (size_t)l * B * D, D, Cd, Hd, cols);
+        count_launch();
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
 cudaError_t launch_adarmsnorm_gate(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf,
                                    int L, int B, int D, int Cd, int Hd, int dtype, cudaStream_t st)
 {
-    if (!gate_scratch_fits(Cd, Hd)) return cudaErrorNotSupported;
+    if (!gate_scratch_fits(Cd, Hd)) {
+        // conditioning or hidden layers too wide to stage 32 streams' vectors in shared memory: the per-stream kernel, layer by layer
+        if (dtype == REFLEX_DTYPE_BF16)
+            return launch_gate_wide_t<__nv_bfloat16>((const __nv_bfloat16 *)cond, (const __nv_bfloat16 *)W1, (const __nv_bfloat16 *)b1,
+                                                     (const __nv_bfloat16 *)W2, (const __nv_bfloat16 *)b2, gate_buf, L, B, D, Cd, Hd, st);
+        return launch_gate_wide_t<float>((const float *)cond, (const float *)W1, (const float *)b1, (const float *)W2, (const float *)b2,
+                                         gate_buf, L, B, D, Cd, Hd, st);
+    }
     if (dtype == REFLEX_DTYPE_BF16)
         return launch_gate_t<__nv_bfloat16>((const __nv_bfloat16 *)cond, (const __nv_bfloat16 *)W1, (const __nv_bfloat16 *)b1,
                                             (const __nv_bfloat16 *)W2, (const __nv_bfloat16 *)b2, gate_buf, L, B, D, Cd, Hd, st);

@@ -700,12 +700,11 @@ bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk)
 template <int NACC>
 static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_tiles, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
+        return cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
+    });
+    if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
     cfg.blockDim = dim3(kQkThreads);
@@ -724,12 +723,11 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
 template <int NT, int NACC>
 static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, unsigned grid, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(norm_linear_small_kernel<NT, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmSmem<NT, NACC>::TOTAL);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
+        return cudaFuncSetAttribute(norm_linear_small_kernel<NT, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmSmem<NT, NACC>::TOTAL);
+    });
+    if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kSmThreads);

@@ -7,6 +7,8 @@
 
 #include <cuda.h>
 
+#include <atomic>
+
 #include "reflex.h"
 
 namespace reflex {
@@ -66,6 +68,23 @@ __host__ __device__ inline float *partial_ml(float *base, size_t n_slots, size_t
 
 // Records a failure for reflex_last_error_string() and returns `code` (printf-style message).
 int api_fail(int code, const char *fmt, ...);
+
+// Kernel attributes (the dynamic shared-memory limit) belong to a device's context, not to the process: a launcher runs its
+// set-up the first time it is used on each device. `done` is the launcher's function-local bit mask of devices (ordinals
+// modulo 64); several host threads may race to run the same idempotent set-up.
+template <typename F>
+inline cudaError_t once_per_device(std::atomic<unsigned long long> &done, F &&setup)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+    e = setup();
+    if (e != cudaSuccess) return e;
+    done.fetch_or(bit, std::memory_order_release);
+    return cudaSuccess;
+}
 
 // Number of kernels this library has launched in this process (every launcher bumps it).
 void count_launch(int n = 1);

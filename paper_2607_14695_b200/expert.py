@@ -75,8 +75,8 @@ def expert_weights(w: synth.Workload, F: int, std_scale: float = 1.0) -> dict:
         "W_in": g("misc", (D, A), A ** -0.5, 0), "W_out": g("misc", (A, D), D ** -0.5, 1),
         "Wqkv": g("Wqkv", (L, (w.Hq + 2 * w.Hkv) * w.d, D), D ** -0.5), "Wo": g("Wo", (L, D, nq), std_scale * nq ** -0.5),
         "Wgu": g("Wgu", (L, 2 * F, D), D ** -0.5), "Wd": g("misc", (L, D, F), std_scale * F ** -0.5, 2),
-        "W1": g("W1", (n_norm, w.Hd, w.Cd), 0.02), "b1": synth.round_storage(0.0 * g("b1", (n_norm, w.Hd), 1.0), w.dtype),
-        "W2": g("W2", (n_norm, D, w.Hd), 0.02), "b2": synth.round_storage(0.0 * g("b2", (n_norm, D), 1.0), w.dtype),
+        "W1": g("W1", (n_norm, w.Hd, w.Cd), 0.02), "b1": g("b1", (n_norm, w.Hd), 0.1),
+        "W2": g("W2", (n_norm, D, w.Hd), 0.02), "b2": g("b2", (n_norm, D), 0.1),
     }
     return out
 
@@ -89,7 +89,6 @@ def random_weights_device(w: synth.Workload, F: int, device="cuda:0", seed: int 
     L, D, A = w.L, w.D, w.A
     nq, n_norm = w.Hq * w.d, 2 * w.L + 1
     r = lambda shape, std: (torch.randn(*shape, generator=g, device=device, dtype=torch.float32) * std).to(tdt).contiguous()
-    z = lambda *shape: torch.zeros(*shape, dtype=tdt, device=device)
     return {"W_in": r((D, A), A ** -0.5), "W_out": r((A, D), D ** -0.5), "Wqkv": r((L, (w.Hq + 2 * w.Hkv) * w.d, D), D ** -0.5),
             "Wo": r((L, D, nq), 0.5 * nq ** -0.5), "Wgu": r((L, 2 * F, D), D ** -0.5), "Wd": r((L, D, F), 0.5 * F ** -0.5),
-            "W1": r((n_norm, w.Hd, w.Cd), 0.02), "b1": z(n_norm, w.Hd), "W2": r((n_norm, D, w.Hd), 0.02), "b2": z(n_norm, D)}
+            "W1": r((n_norm, w.Hd, w.Cd), 0.02), "b1": r((n_norm, w.Hd), 0.1), "W2": r((n_norm, D, w.Hd), 0.02), "b2": r((n_norm, D), 0.1)}

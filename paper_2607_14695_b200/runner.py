@@ -57,8 +57,8 @@ class StepRunner:
         self.vd = [[rnd(w.B, w.T, w.Hkv, w.d) for _ in range(variants)] for _ in range(w.L)]
         self.vflow = [rnd(w.B, w.T, w.A) for _ in range(variants)]
         # gate-MLP parameters of all layers, stacked along a leading layer axis (self.W[l] are views of layer l)
-        self.W1s, self.b1s = rnd(w.L, w.Hd, w.Cd, std=0.02), torch.zeros(w.L, w.Hd, dtype=tdt, device=self.device)
-        self.W2s, self.b2s = rnd(w.L, w.D, w.Hd, std=0.02), torch.zeros(w.L, w.D, dtype=tdt, device=self.device)
+        self.W1s, self.b1s = rnd(w.L, w.Hd, w.Cd, std=0.02), rnd(w.L, w.Hd, std=0.1)
+        self.W2s, self.b2s = rnd(w.L, w.D, w.Hd, std=0.02), rnd(w.L, w.D, std=0.1)
         self.W = [[self.W1s[l], self.b1s[l], self.W2s[l], self.b2s[l]] for l in range(w.L)]
         self.cond = [torch.from_numpy(synth.cond_vectors(w, 1.0 - k / w.K)).to(self.device).to(tdt).contiguous() for k in range(w.K)]
         self.y = torch.empty((w.B, w.T, w.D), dtype=tdt, device=self.device)

@@ -150,13 +150,18 @@ def cond_vectors(w: Workload, t: float, B: int | None = None, variant: int = 0) 
     return round_storage(c, w.dtype)
 
 
-def gate_weights(w: Workload, layer: int, std: float = 0.02):
-    """Gate-MLP parameters W1[Hd][Cd], b1[Hd], W2[D][Hd], b2[D]: N(0, std^2) weights, zero biases,
-    so the gate 1+MLP(c) stays near 1."""
+def gate_weights(w: Workload, layer: int, std: float = 0.02, bias_std: float = 0.1):
+    """Gate-MLP parameters W1[Hd][Cd], b1[Hd], W2[D][Hd], b2[D] of Eq. 2: N(0, std^2) weights and N(0, bias_std^2)
+    biases, all rounded to the storage dtype. With the defaults the gate 1 + MLP(c) stays within about 1 +- 0.3 and
+    both biases move it visibly; a larger std makes the hidden layer and the second product carry the gate."""
     W1 = normal(w, "W1", (w.Hd, w.Cd), layer, 0, std)
     W2 = normal(w, "W2", (w.D, w.Hd), layer, 0, std)
-    b1 = np.zeros((w.Hd,), np.float32)
-    b2 = np.zeros((w.D,), np.float32)
+    if bias_std > 0.0:
+        b1 = normal(w, "b1", (w.Hd,), layer, 0, bias_std)
+        b2 = normal(w, "b2", (w.D,), layer, 0, bias_std)
+    else:
+        b1 = np.zeros((w.Hd,), np.float32)
+        b2 = np.zeros((w.D,), np.float32)
     return W1, b1, W2, b2
 
 
