@@ -254,6 +254,27 @@ int reflex_oracle_adarmsnorm_swiglu(const float *x, const double *gamma, const f
  * "Flow matching steps 10"): forward Euler with K uniform steps from t = 1 to t = 0,
  *   x <- x + dt * v,  dt = -1/K.
  * ------------------------------------------------------------------------------------------ */
+/* ------------------------------------------------------------------------------------------
+ * A plain projection of the action expert with its residual connection (Sec. 3.3 lists the expert's
+ * linear layers; the attention output projection and the down projection of the SwiGLU block each
+ * add their result to the residual stream):
+ *     out[r][n] = res[r][n] + sum_i a[r][i] * W[n][i]
+ *   a [M][K], W [N][K] (one row per output feature), res [M][N] or NULL (no residual), out [M][N].
+ * Plain triple loop, double accumulator, nothing rounded.
+ * ------------------------------------------------------------------------------------------ */
+int reflex_oracle_linear_residual(const float *a, const float *W, const float *res, int M, int K, int N, double *out)
+{
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < M; ++r) {
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int i = 0; i < K; ++i) acc += (double)a[(size_t)r * K + i] * (double)W[(size_t)n * K + i];
+            out[(size_t)r * N + n] = acc + (res ? (double)res[(size_t)r * N + n] : 0.0);
+        }
+    }
+    return 0;
+}
+
 void reflex_oracle_flow_step(double *x, const float *v, long n, int K)
 {
     const double dt = -1.0 / (double)K;

@@ -58,6 +58,8 @@ def lib():
         _lib.reflex_oracle_adarmsnorm_linear.restype = i
         _lib.reflex_oracle_adarmsnorm_swiglu.argtypes = [fp, dp, fp, fp, i, i, i, d, dp]
         _lib.reflex_oracle_adarmsnorm_swiglu.restype = i
+        _lib.reflex_oracle_linear_residual.argtypes = [fp, fp, fp, i, i, i, dp]
+        _lib.reflex_oracle_linear_residual.restype = i
         _lib.reflex_oracle_flow_step.argtypes = [dp, fp, ctypes.c_long, i]
         _lib.reflex_oracle_flow_step.restype = None
         _lib.reflex_oracle_flow_time.argtypes = [i, i]
@@ -159,6 +161,23 @@ def adarmsnorm_swiglu(x, c, W1, b1, W2, b2, Wg, Wu, eps=1e-6):
     if rc != 0:
         raise MemoryError("oracle adarmsnorm_swiglu")
     return h
+
+
+def linear_residual(a, W, res=None):
+    """A plain projection with its residual: a [M][K], W [N][K], res [M][N] or None -> res + a W^T, [M][N] f64."""
+    a, ap = _f(a); W, wp = _f(W)
+    M, K = a.shape
+    N = W.shape[0]
+    assert W.shape == (N, K)
+    rp = None
+    if res is not None:
+        res, rp = _f(res)
+        assert res.shape == (M, N)
+    out = np.empty((M, N), np.float64)
+    rc = lib().reflex_oracle_linear_residual(ap, wp, rp, M, K, N, _dptr(out))
+    if rc != 0:
+        raise MemoryError("oracle linear_residual")
+    return out
 
 
 def flow_step(x, v, K):
