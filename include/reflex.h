@@ -250,6 +250,26 @@ int reflex_adarmsnorm_qkv(reflex_cache_t *cache, const void *x, const float *gat
 int reflex_adarmsnorm_swiglu(reflex_cache_t *cache, const void *x, const float *gate, const void *Wgu, void *h,
                              int B, int R, int D, int F, float eps, int dtype, int impl, void *stream);
 
+/* Sec. 3.3 "System Optimizations" lists the linear layers of the action expert; the two that close a residual branch --
+ * the attention output projection and the down projection of the SwiGLU block -- are this call:
+ *   out[r][n] = res[r][n] + sum_i a[r][i] * W[n][i]
+ * One launch; products of bf16 operands accumulated in fp32, the residual added in fp32, one rounding to dtype.
+ *   cache    a cache whose status word records a device-side wait that ran out (reflex_cache_check_status), or NULL
+ *            (without a cache such a failure shows as NaN in the tile it hit)
+ *   a        device [M][K] dtype (M = streams x tokens)
+ *   W        device [N][K] dtype: one row per output feature
+ *   res      device [M][N] dtype, or NULL for a projection without residual
+ *   out      device [M][N] dtype (written); may be the same buffer as res (in-place update of the residual stream),
+ *            must not overlap a
+ *   impl     0: tensor cores when dtype is bf16 (256 x 256 output tiles per pair of SMs; a kernel with the weights as the
+ *               stationary operand when M <= 128 and K % 64 == 0), else the plain kernel; 1: the plain kernel (fp32
+ *               FMAs, K <= 12288); 2: like 0 but always the 256-row tiles
+ * Requirements: K % 8 == 0, 8 <= K <= 12288; N % 8 == 0; 16-byte aligned pointers.
+ * Errors: REFLEX_ERR_INVALID_ARG (NULL pointer, unknown dtype or impl, out == a), REFLEX_ERR_SHAPE, REFLEX_ERR_ALIGN;
+ * nothing is launched and nothing written on error. */
+int reflex_linear_residual(reflex_cache_t *cache, const void *a, const void *W, const void *res, void *out, int M,
+                           int K, int N, int dtype, int impl, void *stream);
+
 /* Eq. 1 / App. A Prop. 1: for every stream b, KV head j and its G*T query rows,
  *   out = softmax(scale * Q [K_pin; K_slide; K_dyn]^T) [V_pin; V_slide; V_dyn]
  * over static rows [0, static_len[b]), the live ring slots (physical order; softmax does not depend

@@ -27,7 +27,7 @@ EXPORTS = [
     "reflex_cache_create", "reflex_cache_destroy", "reflex_cache_get_state", "reflex_cache_slot_map",
     "reflex_cache_set_attention_impl", "reflex_cache_check_status", "reflex_cache_selftest_wait_limit", "reflex_cache_init_static", "reflex_cache_stage_static",
     "reflex_cache_commit_static", "reflex_cache_append_sliding",
-    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_adarmsnorm_swiglu", "reflex_partitioned_attention",
+    "reflex_adarmsnorm", "reflex_adarmsnorm_gate", "reflex_adarmsnorm_noalloc", "reflex_adarmsnorm_qkv", "reflex_adarmsnorm_swiglu", "reflex_linear_residual", "reflex_partitioned_attention",
     "reflex_flow_step", "reflex_overlap_create", "reflex_overlap_destroy", "reflex_overlap_tick", "reflex_overlap_inference_done",
     "reflex_overlap_simulate",
 ]
@@ -88,6 +88,7 @@ def load():
     lib.reflex_adarmsnorm_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, f, i, vp]
     lib.reflex_adarmsnorm_qkv.argtypes = [vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, vp]
     lib.reflex_adarmsnorm_swiglu.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, i, vp]
+    lib.reflex_linear_residual.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     lib.reflex_partitioned_attention.argtypes = [vp, i, vp, vp, vp, vp, i, f, i, vp]
     lib.reflex_flow_step.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
     dbl = ctypes.c_double
@@ -347,6 +348,21 @@ def reflex_adarmsnorm_swiglu(x, gate, Wgu, h, eps=1e-6, impl=0, cache=None, stre
     _check(load().reflex_adarmsnorm_swiglu(cache.handle if cache is not None else None, _ptr(x), _ptr(gate), _ptr(Wgu), _ptr(h), B, R, D, F,
                                            float(eps), dtype_code(x), int(impl), _stream(stream)))
     return h
+
+
+def reflex_linear_residual(a, W, res, out, impl=0, cache=None, stream=None):
+    """a [..., K] (all leading axes are rows), W [N][K], res [..., N] or None -> out [..., N] = res + a W^T; out may be res."""
+    K, N = int(a.shape[-1]), int(W.shape[0])
+    M = a.numel() // K
+    _check(load().reflex_linear_residual(cache.handle if cache is not None else None, _ptr(a), _ptr(W), _ptr(res), _ptr(out), M, K, N,
+                                         dtype_code(a), int(impl), _stream(stream)))
+    return out
+
+
+def prepare_linear_residual(a, W, res, out, impl=0, cache=None):
+    K, N = int(a.shape[-1]), int(W.shape[0])
+    args = (cache.handle if cache is not None else None, _ptr(a), _ptr(W), _ptr(res), _ptr(out), a.numel() // K, K, N, dtype_code(a), int(impl))
+    return _prepared(load().reflex_linear_residual, args)
 
 
 def prepare_adarmsnorm_swiglu(x, gate, Wgu, h, eps=1e-6, impl=0, cache=None):

@@ -1,0 +1,319 @@
+// A plain projection of the action expert with its residual connection (Sec. 3.3 names the expert's linear layers; the
+// attention output projection and the down projection of the SwiGLU block each add their result to the residual stream):
+//     out[r][n] = res[r][n] + sum_i a[r][i] * W[n][i]
+//
+// bf16 path: one pair of CTAs (tcgen05.mma.cta_group::2, M = 256) per 256 x 256 output tile. Each CTA stages its own 128
+// rows of a and its 128 rows of W (its half of the B operand) per 64-column contraction step through a ring of five
+// 32 KB stages filled by TMA; one elected thread of the leader CTA issues the MMAs into a 256-column fp32 accumulator in
+// tensor memory. The residual tile (128 rows x 256 columns, 64 KB) is fetched by TMA into a buffer of its own while the
+// main loop runs; the epilogue adds the accumulator to it in place (fp32 add, one rounding to bf16) and the same buffer
+// leaves through TMA stores, which clip rows and columns past the end. out may alias res: a tile is read and written
+// by one CTA only.
+// The contraction is long (2048 or 4096) and the output small (3200 x 1024 at 64 streams): 52 tiles on 74 SM pairs in
+// one wave, so the kernel is not persistent.
+//
+// Few rows (at most 128 in all): the weights-as-A-operand kernel of the fused projections with the gate stage switched off
+// (qkv_tc.cu). Any other dtype or shape: a plain kernel, one block per row, fp32 FMAs.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "reflex_internal.cuh"
+#include "sm100_ptx.cuh"
+
+namespace reflex {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int kLinThreads = 64 + 256;   // producer warp, MMA warp, eight epilogue warps (two threads per row)
+constexpr int kLinBM = 128;             // rows per CTA (256 per pair)
+constexpr int kLinBK = 64;              // contraction step: one 128-byte swizzled row
+constexpr unsigned long long kLinWaitNs = 1000000000ull;
+
+template <int BN>
+struct LinSmem {
+    static constexpr int NST = 5;
+    static constexpr uint32_t A_STAGE = kLinBM * 128;
+    static constexpr uint32_t B_STAGE = (BN / 2) * 128;            // this CTA's half of the B operand: BN / 2 rows of W
+    static constexpr uint32_t CHUNK = kLinBM * 128;                // 128 rows x 64 columns of the residual / output tile
+    static constexpr uint32_t OFF_A = 0;
+    static constexpr uint32_t OFF_B = NST * A_STAGE;
+    static constexpr uint32_t OFF_RES = OFF_B + NST * B_STAGE;
+    static constexpr uint32_t RES_BYTES = (BN / 64) * CHUNK;
+    static constexpr uint32_t OFF_BAR = OFF_RES + RES_BYTES;
+    static constexpr uint32_t TOTAL = OFF_BAR + 256 + 1024;        // + slack for the 1024-byte alignment
+    static constexpr int C_FULL = 0, C_EMPTY = NST, C_ACC = 2 * NST, C_RES = 2 * NST + 1, C_COUNT = 2 * NST + 2;
+    static_assert(TOTAL <= 227u * 1024u && 8 * C_COUNT + 8 <= 256, "shared memory budget");
+};
+
+struct LinParams {
+    int M, K, N;
+    int m_tiles;          // 256-row tiles
+    int has_res;
+    uint32_t *status;     // status word of a cache, or NULL
+};
+
+__device__ __forceinline__ void lin_tma2_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(leader_bar), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void lin_tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+
+template <int BN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kLinThreads, 1)
+linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                     const __grid_constant__ CUtensorMap tm_res, const __grid_constant__ CUtensorMap tm_out, LinParams p)
+{
+    using S = LinSmem<BN>;
+    constexpr int NST = S::NST;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw_addr);
+    auto bar = [&](int i) -> uint32_t { return base + S::OFF_BAR + 8u * (uint32_t)i; };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + S::OFF_BAR + 8 * S::C_COUNT);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1;
+    const int m0 = (pair % p.m_tiles) * (2 * kLinBM) + (int)rank * kLinBM;   // this CTA's first row
+    const int n0 = (pair / p.m_tiles) * BN;                                  // the pair's first output column
+    const int nk_steps = (p.K + kLinBK - 1) / kLinBK;                        // (columns past K come in as TMA's zeros)
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < S::C_COUNT; ++i) mbar_init(bar(i), 1);
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tmap(&tm_a); prefetch_tmap(&tm_w); prefetch_tmap(&tm_out);
+        if (p.has_res) prefetch_tmap(&tm_res);
+    }
+    if (warp == 1) tmem_alloc2(smem_u32((const void *)tmem_slot), BN);
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();   // both CTAs' barriers exist before anything crosses the pair
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    // programmatic dependent launch: whatever produced a and res is complete from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool {
+        if (mbar_try_wait(bar(i), parity)) return true;
+        const unsigned long long t_start = globaltimer_ns();
+        for (uint32_t n = 1;; ++n) {
+            if (mbar_try_wait(bar(i), parity)) return true;
+            if ((n & 255u) == 0u) {
+                if (*abort_flag) return false;
+                if (globaltimer_ns() - t_start > kLinWaitNs) break;
+            }
+        }
+        *abort_flag = 1u;
+        if (p.status) atomicCAS(p.status, 0u, 0x80000000u | ((code + 80u) << 16) | (blockIdx.x & 0xFFFFu));
+        return false;
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs) ----------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int ks = 0; ks < nk_steps && ok; ++ks) {
+                const int s = ks % NST;
+                if (ks >= NST) ok = wait(S::C_EMPTY + s, (uint32_t)(ks / NST - 1) & 1u, 1);
+                if (!ok) break;
+                // both CTAs' loads complete on the leader's barrier: the issuing thread there waits for all four at once
+                if (rank == 0) mbar_expect_tx(bar(S::C_FULL + s), 2 * (S::A_STAGE + S::B_STAGE));
+                lin_tma2_load_2d(base + S::OFF_A + s * S::A_STAGE, &tm_a, bar(S::C_FULL + s) & kPeerBitMask, ks * kLinBK, m0);
+                lin_tma2_load_2d(base + S::OFF_B + s * S::B_STAGE, &tm_w, bar(S::C_FULL + s) & kPeerBitMask, ks * kLinBK, n0 + (int)rank * (BN / 2));
+            }
+            if (p.has_res && ok) {
+                // the residual tile goes last: it is not needed before the epilogue, and ahead of the main loop's operands it
+                // would hold them up for the time 64 KB take to come in (measured: 0.7 us per launch)
+                mbar_expect_tx(bar(S::C_RES), S::RES_BYTES);
+#pragma unroll
+                for (int ch = 0; ch < BN / 64; ++ch) tma_load_2d(base + S::OFF_RES + ch * S::CHUNK, &tm_res, bar(S::C_RES), n0 + ch * 64, m0);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader CTA; the warp stays converged, one elected lane issues) ----------------
+        if (rank == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(2 * kLinBM, BN, false);
+            bool ok = true;
+            for (int ks = 0; ks < nk_steps && ok; ++ks) {
+                const int s = ks % NST;
+                ok = wait(S::C_FULL + s, (uint32_t)(ks / NST) & 1u, 2);
+                if (!ok) break;
+                tc_fence_after();
+                uint64_t ad = umma_desc_sw128(base + S::OFF_A + s * S::A_STAGE, 16, 1024);
+                uint64_t bd = umma_desc_sw128(base + S::OFF_B + s * S::B_STAGE, 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < kLinBK / 16; ++kk) {
+                    umma2_ss_elect(tmem, ad, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                    umma_desc_advance(ad, 32);
+                    umma_desc_advance(bd, 32);
+                }
+                umma2_commit_mc_elect(bar(S::C_EMPTY + s), (uint16_t)3);
+            }
+            umma2_commit_mc_elect(bar(S::C_ACC), (uint16_t)3);   // also after a wait that ran out: the epilogue warps must not wait for nothing
+        }
+    } else {
+        // ---------------- epilogue: two threads per row, each owns BN / 2 columns ----------------
+        const int quarter = warp & 3;                 // the TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        bool ok = true;
+        if (p.has_res) ok = wait(S::C_RES, 0u, 3);
+        ok = wait(S::C_ACC, 0u, 4) && ok;
+        tc_fence_after();
+        constexpr int CPT = BN / 2 / 64;              // 64-column chunks per thread
+#pragma unroll 1
+        for (int cc = 0; cc < CPT; ++cc) {
+            const int ch = half * CPT + cc;
+            uint8_t *rowp = smem + S::OFF_RES + ch * S::CHUNK + row * 128;
+#pragma unroll 1
+            for (int g = 0; g < 2; ++g) {             // 32 columns at a time
+                uint32_t acc[32];
+                tmem_ld32(tmem + lane_addr + ch * 64 + g * 32, acc);   // warp-wide: every lane takes part, whatever its row
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // 128-byte swizzle of the TMA boxes: 16-byte piece j of row r sits at j ^ (r % 8)
+                    uint4 *pc = reinterpret_cast<uint4 *>(rowp + (((g * 4 + i) ^ (row & 7)) << 4));
+                    uint32_t rv[4] = {0u, 0u, 0u, 0u};
+                    if (p.has_res) { const uint4 t = *pc; rv[0] = t.x; rv[1] = t.y; rv[2] = t.z; rv[3] = t.w; }
+                    uint32_t ov[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        float v0 = __uint_as_float(acc[8 * i + 2 * k]) + __uint_as_float(rv[k] << 16);
+                        float v1 = __uint_as_float(acc[8 * i + 2 * k + 1]) + __uint_as_float(rv[k] & 0xFFFF0000u);
+                        if (!ok) v0 = v1 = __int_as_float(0x7fc00000);   // a wait ran out: the tile is marked invalid, not left stale
+                        __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                        ov[k] = *reinterpret_cast<uint32_t *>(&h);
+                    }
+                    *pc = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+                }
+            }
+            // this half's chunk is complete once its 128 threads are through: one of them hands it to the TMA engine
+            fence_proxy_async_smem();
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + half) : "memory");
+            if (quarter == 0 && lane == 0 && m0 < p.M && n0 + ch * 64 < p.N) {
+                lin_tma_store_2d(&tm_out, base + S::OFF_RES + ch * S::CHUNK, n0 + ch * 64, m0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+        }
+        if (quarter == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the stores of this thread are complete
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();   // neither CTA retires while its partner can still touch its shared memory or barriers
+    if (warp == 1) tmem_dealloc2(tmem, BN);
+}
+
+// Any dtype, any shape: one block per row; the row of a in shared memory (fp32), every thread takes output features
+// n = tid, tid + 256, ... as plain dot products.
+template <typename T> __device__ __forceinline__ float lin_to_f(T v);
+template <> __device__ __forceinline__ float lin_to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float lin_to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T lin_from_f(float v);
+template <> __device__ __forceinline__ float lin_from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 lin_from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+linear_res_simt_kernel(const T *__restrict__ a, const T *__restrict__ W, const T *res, T *out, int K, int N)
+{
+    extern __shared__ float asm_row[];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const size_t r = blockIdx.x;
+    for (int i = threadIdx.x; i < K; i += blockDim.x) asm_row[i] = lin_to_f<T>(a[r * K + i]);
+    __syncthreads();
+    for (int n = threadIdx.x; n < N; n += blockDim.x) {
+        const T *wr = W + (size_t)n * K;
+        float acc = 0.f;
+        for (int i = 0; i < K; ++i) acc = fmaf(asm_row[i], lin_to_f<T>(wr[i]), acc);
+        if (res) acc += lin_to_f<T>(res[r * N + n]);
+        out[r * N + n] = lin_from_f<T>(acc);
+    }
+}
+
+template <typename T>
+cudaError_t launch_lin_simt(const void *a, const void *W, const void *res, void *out, int M, int K, int N, cudaStream_t st)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)M);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = (size_t)K * sizeof(float);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_res_simt_kernel<T>, (const T *)a, (const T *)W, (const T *)res, (T *)out, K, N);
+    count_launch();
+    return e;
+}
+
+template <int BN>
+cudaError_t launch_lin_tc(const CUtensorMap &ma, const CUtensorMap &mw, const CUtensorMap &mr, const CUtensorMap &mo, const LinParams &p, int n_tiles,
+                          cudaStream_t st)
+{
+    static std::atomic<unsigned long long> attr_set{0};
+    cudaError_t e0 = once_per_device(attr_set, [] {
+        return cudaFuncSetAttribute(linear_res_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LinSmem<BN>::TOTAL);
+    });
+    if (e0 != cudaSuccess) return e0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
+    cfg.blockDim = dim3(kLinThreads);
+    cfg.dynamicSmemBytes = LinSmem<BN>::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_res_tc_kernel<BN>, ma, mw, mr, mo, p);
+    count_launch();
+    return e;
+}
+
+}  // namespace
+
+bool linear_tc_supported(int dtype, int M, int K, int N)
+{
+    return dtype == REFLEX_DTYPE_BF16 && M >= 1 && K >= 8 && K % 8 == 0 && N >= 8 && N % 8 == 0 && (long long)M * N <= 0x3FFFFFFF;
+}
+
+// impl: 0 = tensor cores where supported, 1 = plain kernel, 2 = tensor cores, the 256-row tiles whatever M is
+cudaError_t launch_linear_residual(const void *a, const void *W, const void *res, void *out, int M, int K, int N, int dtype, int impl,
+                                   uint32_t *status, cudaStream_t st)
+{
+    const bool tc = impl != 1 && linear_tc_supported(dtype, M, K, N);
+    if (!tc) {
+        if ((size_t)K * sizeof(float) > 48 * 1024) return cudaErrorInvalidValue;
+        return dtype == REFLEX_DTYPE_BF16 ? launch_lin_simt<__nv_bfloat16>(a, W, res, out, M, K, N, st) : launch_lin_simt<float>(a, W, res, out, M, K, N, st);
+    }
+    if (impl == 0 && M <= 128 && K % 64 == 0) return launch_linear_small(a, W, res, out, M, K, N, status, st);
+    CUtensorMap ma, mw, mr, mo;
+    if (!tensor_map_2d_bf16(&ma, a, K, M, kLinBM) || !tensor_map_2d_bf16(&mw, W, K, N, 128) || !tensor_map_2d_bf16(&mo, out, N, M, kLinBM)) return cudaErrorInvalidValue;
+    if (res) { if (!tensor_map_2d_bf16(&mr, res, N, M, kLinBM)) return cudaErrorInvalidValue; }
+    else mr = mo;
+    LinParams p;
+    p.M = M; p.K = K; p.N = N; p.m_tiles = (M + 2 * kLinBM - 1) / (2 * kLinBM); p.has_res = res ? 1 : 0; p.status = status;
+    return launch_lin_tc<256>(ma, mw, mr, mo, p, (N + 255) / 256, st);
+}
+
+}  // namespace reflex

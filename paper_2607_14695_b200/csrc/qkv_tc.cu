@@ -68,6 +68,8 @@ struct QkParams {
     int swiglu_F;               // 0: columns go to Q, K, V. F > 0: W holds [W_gate; W_up] ([2F][D]), out (= q, pitch nq = F) gets SiLU(g) * u
     float eps;
     uint32_t *status;
+    const __nv_bfloat16 *res;   // plain projection only (few-rows kernel with PLAIN): residual [M][nq] added to the output, or NULL
+    int ksplit;                 // plain projection only: CTAs of a cluster that share one feature tile, each taking a slice of the contraction
 };
 
 #ifdef REFLEX_QK_TRACE
@@ -364,7 +366,9 @@ struct SmSmem {
     static constexpr int S_XFULL = 0, S_BREADY = STAGES, S_EMPTY = 2 * STAGES, S_ACC = 3 * STAGES, S_COUNT = S_ACC + 1;
 };
 
-template <int NT, int NACC>
+// PLAIN: no norm at all (out = res + x W^T, the expert's output / down projections for one or two streams): the eight warps
+// only pass each landed step on to the MMA warp, and the epilogue adds the residual instead of scaling by 1/RMS.
+template <int NT, int NACC, bool PLAIN = false>
 __global__ void __launch_bounds__(kSmThreads, 1)
 norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, QkParams p)
 {
@@ -380,9 +384,16 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
     volatile uint32_t *abort_flag = tmem_slot + 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool swiglu = NACC == 2;
-    const int f0 = blockIdx.x * 128;                  // first output feature (hidden feature for SwiGLU) of this CTA
+    // PLAIN with ksplit > 1: the ksplit CTAs of a cluster own the same 128 features and a slice of the contraction axis each
+    // (whole steps only: the launcher picks ksplit so that the chunks divide), and add up their accumulators through
+    // distributed shared memory at the end
+    const int ksplit = PLAIN ? p.ksplit : 1;
+    const int krank = (PLAIN && ksplit > 1) ? (int)cluster_ctarank() : 0;
+    const int f0 = (blockIdx.x / ksplit) * 128;       // first output feature (hidden feature for SwiGLU) of this CTA
     constexpr int CPS = S::CPS;
-    const int n_chunks = p.D / kQkBK;
+    const int all_chunks = p.D / kQkBK;
+    const int chunk0 = krank * (all_chunks / ksplit);      // this CTA's first 64-column chunk of the contraction axis
+    const int n_chunks = ksplit > 1 ? all_chunks / ksplit : all_chunks;
     const int nk_steps = (n_chunks + CPS - 1) / CPS;       // (a last step may hold one chunk only: TMA zero-fills the other)
     constexpr int TP = 256 / NT;                      // transform threads per row: 4 (64 rows) or 2 (128 rows)
     constexpr uint32_t kCols = NACC * NT < 32 ? 32 : NACC * NT;
@@ -436,7 +447,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
                 mbar_expect_tx(bar(S_XFULL + s), S::X_STAGE + S::W_STAGE);
 #pragma unroll
                 for (int cc = 0; cc < CPS; ++cc) {
-                    const int col = (ks * CPS + cc) * kQkBK;
+                    const int col = (chunk0 + ks * CPS + cc) * kQkBK;
                     tma_load_2d(base + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE, &tm_x, bar(S_XFULL + s), col, 0);
 #pragma unroll
                     for (int j = 0; j < NACC; ++j)
@@ -481,7 +492,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
         constexpr int KW = kQkBK / TP;                 // columns per thread and step: 16 or 32
         const int b = min(row / p.R, p.B - 1);
         float *gsm = reinterpret_cast<float *>(smem + S::OFF_GATE);
-        {
+        if constexpr (!PLAIN) {
             const int n4 = p.B * p.D / 4;              // (at most 4 streams: checked by the launcher)
             const float4 *src = reinterpret_cast<const float4 *>(p.gate);
             for (int i = tid; i < n4; i += 256) reinterpret_cast<float4 *>(gsm)[i] = __ldg(src + i);
@@ -496,6 +507,11 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             if (threadIdx.x == 64) QK_TRACE(2, ks, 0);
             ok = ok && wait(S_XFULL + s, (uint32_t)(ks / kSmStages) & 1u, 4);
             if (threadIdx.x == 64) QK_TRACE(2, ks, 1);
+            if constexpr (PLAIN) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(S_BREADY + s));
+                continue;
+            }
             // all loads of the step first (x pieces and gate values of every chunk), then the arithmetic and the stores: the
             // stores could alias the later loads for all the compiler knows, and with a few independent loads per thread the
             // shared-memory latency was most of a step
@@ -554,7 +570,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             float ssr = 0.f;
 #pragma unroll
             for (int t = 0; t < TP; ++t) ssr += ssm[t * 128 + tid];
-            rsm[tid] = rsqrtf(ssr * (1.f / (float)p.D) + p.eps);
+            rsm[tid] = PLAIN ? 1.f : rsqrtf(ssr * (1.f / (float)p.D) + p.eps);
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (threadIdx.x == 64) QK_TRACE(2, 31, 0);
@@ -579,6 +595,18 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             tmem_ld32(tmem + lane_addr + c * 32, acc);          // warp-wide: every lane takes part
             if (swiglu) tmem_ld32(tmem + lane_addr + NT + c * 32, up);
             tmem_wait_ld();
+            if constexpr (PLAIN) {
+                if (ksplit > 1) {
+                    // this CTA's share of the sums goes to shared memory (the stage ring is idle: every load has been consumed
+                    // and every MMA has completed), [row][feature] so that a warp writes 128 contiguous bytes
+                    float *part = reinterpret_cast<float *>(smem + S::OFF_W);
+                    static_assert(S::STAGES * S::W_STAGE >= (uint32_t)NT * 128 * 4, "partial sums fit in the stage ring");
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        part[(c * 32 + i) * 128 + quarter * 32 + lane] = ok ? __uint_as_float(acc[i]) : __int_as_float(0x7fc00000);
+                    continue;
+                }
+            }
             if (!ok || f >= n_feat) continue;
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -587,12 +615,43 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
                     const float rs = rsm[r];
                     float val = __uint_as_float(acc[i]) * rs;
                     if (swiglu) { const float u = __uint_as_float(up[i]) * rs; val = __fdividef(val, 1.f + __expf(-val)) * u; }
+                    if constexpr (PLAIN) { if (p.res) val += __bfloat162float(p.res[(size_t)r * pitch + f]); }
                     dst0[(size_t)r * pitch] = __float2bfloat16_rn(val);     // a warp writes 64 contiguous bytes per row
                 }
             }
         }
     }
 
+    if constexpr (PLAIN) {
+        if (ksplit > 1) {
+            // (cluster barriers are warp-aligned: the lanes of the producer warp that idled while lane 0 ran the loads must
+            // not reach them before lane 0 does, so the CTA meets first)
+            __syncthreads();
+            cluster_arrive();
+            cluster_wait();
+            if (warp >= 2) {
+                // CTA krank adds up rows [krank, krank + 1) * NT / ksplit of all slices, adds the residual and writes bf16
+                const float *part = reinterpret_cast<const float *>(smem + S::OFF_W);
+                const int rows_mine = NT / ksplit, r0 = krank * rows_mine;
+                for (int e = threadIdx.x - 64; e < rows_mine * 128; e += 256) {
+                    const int r = r0 + e / 128, fl = e % 128;
+                    if (r >= p.M || f0 + fl >= p.nq) continue;
+                    float sum = 0.f;
+                    const uint32_t a0 = smem_u32(part + r * 128 + fl);
+                    for (int q = 0; q < ksplit; ++q) {
+                        float v;
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(mapa(a0, (uint32_t)q)) : "memory");
+                        sum += v;
+                    }
+                    const size_t o = (size_t)r * p.nq + f0 + fl;
+                    if (p.res) sum += __bfloat162float(p.res[o]);
+                    p.q[o] = __float2bfloat16_rn(sum);
+                }
+            }
+            cluster_arrive();
+            cluster_wait();   // no CTA retires while a peer may still read its partial sums
+        }
+    }
     if (threadIdx.x == 64) QK_TRACE(2, 31, 2);
     tc_fence_before();
     __syncthreads();
@@ -720,12 +779,12 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
     return e;
 }
 
-template <int NT, int NACC>
+template <int NT, int NACC, bool PLAIN = false>
 static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, unsigned grid, cudaStream_t st)
 {
     static std::atomic<unsigned long long> attr_set{0};
     cudaError_t e0 = once_per_device(attr_set, [] {
-        return cudaFuncSetAttribute(norm_linear_small_kernel<NT, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmSmem<NT, NACC>::TOTAL);
+        return cudaFuncSetAttribute(norm_linear_small_kernel<NT, NACC, PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SmSmem<NT, NACC>::TOTAL);
     });
     if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
@@ -733,12 +792,14 @@ static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, Qk
     cfg.blockDim = dim3(kSmThreads);
     cfg.dynamicSmemBytes = SmSmem<NT, NACC>::TOTAL;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // plain projection: the CTAs that split one feature tile's contraction
+    attr[1].val.clusterDim.x = (unsigned)(PLAIN ? p.ksplit : 1); attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_linear_small_kernel<NT, NACC>, mx, mw, p);
+    cfg.numAttrs = (PLAIN && p.ksplit > 1) ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_linear_small_kernel<NT, NACC, PLAIN>, mx, mw, p);
     count_launch();
     return e;
 }
@@ -766,7 +827,7 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
         QkParams sp;
         sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
         sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.swiglu_F = swiglu_F;
-        sp.eps = eps; sp.status = status;
+        sp.eps = eps; sp.status = status; sp.res = nullptr; sp.ksplit = 1;
         const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
         const unsigned grid = (unsigned)((n_feat + 127) / 128);
         if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, st) : launch_small<128, 2>(sx, sw, sp, grid, st);
@@ -779,12 +840,32 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
     p.M = M; p.R = R; p.B = B; p.D = D; p.nq = nq; p.nk = nk;
     p.m_tiles = (M + 2 * kQkBM - 1) / (2 * kQkBM);
     p.swiglu_F = swiglu_F;
-    p.eps = eps; p.status = status;
+    p.eps = eps; p.status = status; p.res = nullptr; p.ksplit = 1;
     if (swiglu_F > 0) return launch_tc<2>(mx, mw, p, (swiglu_F + kQkBN - 1) / kQkBN, st);
     int nacc = qk_choose_nacc(M, R, D, nq + 2 * nk, sm_count > 0 ? sm_count : 148);
     if (impl == 2 && nacc == 2) nacc = 1;     // (forced 256-column tiles, for tests and timing)
     const int n_out = nq + 2 * nk;
     return nacc == 2 ? launch_tc<2>(mx, mw, p, (n_out + 2 * kQkBN - 1) / (2 * kQkBN), st) : launch_tc<1>(mx, mw, p, (n_out + kQkBN - 1) / kQkBN, st);
+}
+
+// out [M][N] = res + a [M][K] W [N][K]^T for at most 128 rows (K a multiple of 64): the few-rows kernel without its norm stage
+cudaError_t launch_linear_small(const void *a, const void *W, const void *res, void *out, int M, int K, int N, uint32_t *status, cudaStream_t st)
+{
+    const int NT = M <= 64 ? 64 : 128;
+    CUtensorMap sx, sw;
+    if (!tensor_map_2d_bf16(&sx, a, K, M, NT) || !tensor_map_2d_bf16(&sw, W, K, N, 128)) return cudaErrorInvalidValue;
+    QkParams sp;
+    sp.gate = nullptr; sp.q = (__nv_bfloat16 *)out; sp.k = nullptr; sp.v = nullptr;
+    sp.M = M; sp.R = M; sp.B = 1; sp.D = K; sp.nq = N; sp.nk = 0; sp.m_tiles = 1; sp.swiglu_F = 0;
+    sp.eps = 0.f; sp.status = status; sp.res = (const __nv_bfloat16 *)res;
+    // split the contraction over up to 8 CTAs per feature tile while every slice keeps whole steps of two 64-column chunks and
+    // the grid stays within the SMs
+    const int chunks = K / kQkBK, ftiles = (N + 127) / 128;
+    int ks = 1;
+    while (ks < 8 && chunks % (4 * ks) == 0 && chunks / (2 * ks) >= 2 && ftiles * 2 * ks <= 148) ks *= 2;
+    sp.ksplit = ks;
+    const unsigned grid = (unsigned)(ftiles * ks);
+    return NT == 64 ? launch_small<64, 1, true>(sx, sw, sp, grid, st) : launch_small<128, 1, true>(sx, sw, sp, grid, st);
 }
 
 }  // namespace reflex

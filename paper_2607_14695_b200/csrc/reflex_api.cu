@@ -434,6 +434,23 @@ int reflex_adarmsnorm_swiglu(reflex_cache_t *c, const void *x, const float *gate
     return REFLEX_OK;
 }
 
+int reflex_linear_residual(reflex_cache_t *c, const void *a, const void *W, const void *res, void *out, int M, int K, int N, int dtype,
+                           int impl, void *stream)
+{
+    if (dtype != REFLEX_DTYPE_BF16 && dtype != REFLEX_DTYPE_F32) return fail(REFLEX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (impl < 0 || impl > 2) return fail(REFLEX_ERR_INVALID_ARG, "impl must be 0 (auto), 1 (plain kernel) or 2 (tensor cores, 256-row tiles)");
+    if (!a || !W || !out) return fail(REFLEX_ERR_INVALID_ARG, "NULL argument");
+    if (M < 1 || (long long)M * N > 0x3FFFFFFF) return fail(REFLEX_ERR_SHAPE, "M=%d, N=%d", M, N);
+    if (K < 8 || K % 8 != 0 || K > 12288) return fail(REFLEX_ERR_SHAPE, "K=%d must be a multiple of 8 in [8, 12288]", K);
+    if (N < 8 || N % 8 != 0) return fail(REFLEX_ERR_SHAPE, "N=%d must be a multiple of 8", N);
+    if (!aligned16(a) || !aligned16(W) || !aligned16(out) || (res && !aligned16(res))) return fail(REFLEX_ERR_ALIGN, "a / W / res / out not 16-byte aligned");
+    if (a == out) return fail(REFLEX_ERR_INVALID_ARG, "out may alias res, not a");
+    uint32_t *status = c ? (uint32_t *)(c->ws + c->lay.status_off) : nullptr;
+    cudaError_t e = launch_linear_residual(a, W, res, out, M, K, N, dtype, impl, status, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "linear residual launch");
+    return REFLEX_OK;
+}
+
 int reflex_partitioned_attention(reflex_cache_t *c, int layer, const void *q, const void *k_dyn, const void *v_dyn,
                                  void *out, int T, float scale, int dyn_mask, void *stream)
 {

@@ -122,6 +122,11 @@ bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk);
 // swiglu_F > 0: W = [W_gate; W_up] and q receives SiLU(gate) * up, [B*R][F]
 cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *W, void *q, void *k, void *v, int B, int R, int D, int nq, int nk,
                                   int swiglu_F, float eps, int dtype, int impl, int sm_count, uint32_t *status, cudaStream_t st);
+// plain projection with residual (linear_tc.cu): out [M][N] = res + a [M][K] W [N][K]^T. impl: 0 = tensor cores where supported,
+// 1 = plain kernel, 2 = tensor cores with 256-row tiles whatever M is
+cudaError_t launch_linear_residual(const void *a, const void *W, const void *res, void *out, int M, int K, int N, int dtype, int impl,
+                                   uint32_t *status, cudaStream_t st);
+cudaError_t launch_linear_small(const void *a, const void *W, const void *res, void *out, int M, int K, int N, uint32_t *status, cudaStream_t st);
 bool gate_tc_supported(int B, int D, int Cd, int Hd);
 cudaError_t launch_gate_tc(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf, int L, int B,
                            int D, int Cd, int Hd, cudaStream_t st);

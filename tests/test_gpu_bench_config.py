@@ -82,3 +82,7 @@ def test_fused_projections_at_bench_size():
     w = synth.CONFIGS["cfg4"]
     tp._norm_qkv_case(U, w, 0, "bench-size norm+qkv", streams=[0, 17, 63])
     tp._norm_swiglu_case(U, w, 4 * w.D, 0, "bench-size norm+swiglu", streams=[5, 40])
+    # the output and down projections at the same size (3200 rows onto D = 1024 from 2048 and 4096), a sample of rows
+    rows = [0, 255, 256, 1700, 3071, 3072, 3199]
+    tp._linear_case(U, w.dtype, w.B * w.T, w.Hq * w.d, w.D, 0, "bench-size output projection", in_place=True, rows=rows)
+    tp._linear_case(U, w.dtype, w.B * w.T, 4 * w.D, w.D, 0, "bench-size down projection", in_place=True, rows=rows)

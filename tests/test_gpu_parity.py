@@ -621,6 +621,79 @@ def test_norm_qkv_short_streams_and_fallback(U):
 
 
 # ------------------------------------------------------------------------------------------------
+# plain projections with residual (attention output projection, SwiGLU down projection)
+# ------------------------------------------------------------------------------------------------
+def _linear_case(U, dtype, M, K, N, impl, what, residual=True, in_place=False, rows=None, seed=61):
+    """out = res + a W^T against the oracle's triple loop. a ~ N(0,1), W ~ N(0, 1/K), res ~ N(0,1): outputs of variance 2
+    (1 without residual). The operands are exact in the storage dtype and accumulate in fp32, so what is left is the
+    rounding of the output: the bf16 contract with its output-spacing clause, mean-abs scaled to the output's rms."""
+    from oracle import reflex_oracle as orc
+    rb = U.rb
+    w = synth.Workload("lin", seed, dtype, B=1, L=1, Hq=1, Hkv=1, d=8, S=1, S_max=1, N=1, T=1, D=8, Cd=8, Hd=8, A=4, K=1)
+    a = synth.normal(w, "x", (M, K), 0, 0)
+    W = synth.normal(w, "Wo", (N, K), 0, 0, float(K) ** -0.5)
+    res = synth.normal(w, "misc", (M, N), 0, 0) if residual else None
+    da, dW = U.to_dev(a, dtype), U.to_dev(W, dtype)
+    dres = U.to_dev(res, dtype) if residual else None
+    out = dres if in_place else torch.full((M, N), float("nan"), dtype=rb.torch_dtype(dtype), device=U.DEV)
+    rb.reflex_linear_residual(da, dW, dres, out, impl=impl)
+    torch.cuda.synchronize()
+    rows = list(range(M)) if rows is None else rows
+    want = orc.linear_residual(a[rows], W, res[rows] if residual else None)
+    U.check_close(U.to_host(out)[rows], want, dtype, what, rel_clause=True, out_scale=float(np.sqrt(np.mean(want ** 2))))
+    if not in_place and residual:
+        assert torch.equal(dres, U.to_dev(res, dtype))      # the residual itself is only read
+
+
+def test_linear_residual_fp32_plain_kernel(U):
+    _linear_case(U, synth.DTYPE_F32, 37, 136, 72, 0, "linear fp32")
+    _linear_case(U, synth.DTYPE_F32, 5, 64, 8, 0, "linear fp32, no residual", residual=False)
+
+
+@pytest.mark.parametrize("K", [2048, 4096])
+def test_linear_residual_bf16_output_and_down_projection(U, K):
+    """The expert's output projection (K = Hq d = 2048) and down projection (K = F = 4096) onto D = 1024 for 7 streams of 50
+    rows: a full 256-row tile pair and one with 94 rows (its second CTA entirely past the end), four column tiles; in place
+    and out of place, against the plain kernel's path as well."""
+    _linear_case(U, synth.DTYPE_BF16, 350, K, 1024, 0, f"linear bf16 K={K}")
+    _linear_case(U, synth.DTYPE_BF16, 350, K, 1024, 0, f"linear bf16 K={K} in place", in_place=True)
+    _linear_case(U, synth.DTYPE_BF16, 350, K, 1024, 1, f"linear bf16 K={K} plain kernel", rows=[0, 127, 128, 255, 256, 349])
+
+
+def test_linear_residual_bf16_ragged_shapes(U):
+    """Column count 328 (a second column tile with 72 live columns, its last 64-column piece clipped at 8), contraction 200
+    (not a multiple of the 64-column step: the tail arrives as zeros), 300 rows; and without residual."""
+    _linear_case(U, synth.DTYPE_BF16, 300, 200, 328, 0, "linear ragged")
+    _linear_case(U, synth.DTYPE_BF16, 300, 200, 328, 0, "linear ragged, no residual", residual=False)
+    _linear_case(U, synth.DTYPE_BF16, 129, 64, 8, 0, "linear one step, 8 columns")
+
+
+@pytest.mark.parametrize("M", [50, 100])
+def test_linear_residual_bf16_few_rows(U, M):
+    """One or two streams of 50 rows: the kernel with the weights as the stationary operand (64 or 128 row columns), and the
+    same shapes forced through the 256-row tiles."""
+    _linear_case(U, synth.DTYPE_BF16, M, 2048, 1024, 0, f"linear {M} rows")
+    _linear_case(U, synth.DTYPE_BF16, M, 4096, 1024, 0, f"linear {M} rows K=4096 in place", in_place=True)
+    _linear_case(U, synth.DTYPE_BF16, M, 192, 328, 0, f"linear {M} rows ragged", residual=False)
+    _linear_case(U, synth.DTYPE_BF16, M, 2048, 1024, 2, f"linear {M} rows, 256-row tiles")
+
+
+def test_linear_residual_error_paths(U):
+    rb = U.rb
+    z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device=U.DEV)
+    a, W, r = z(4, 64), z(16, 64), z(4, 16)
+    rb.reflex_linear_residual(a, W, r, r)
+    for bad, code in ((lambda: rb.reflex_linear_residual(a, W, r, r, impl=3), rb.ERR_INVALID_ARG),
+                      (lambda: rb.reflex_linear_residual(a, W, r, a), rb.ERR_INVALID_ARG),                      # out aliases a
+                      (lambda: rb.reflex_linear_residual(z(4, 60), z(16, 60), r, r), rb.ERR_SHAPE),             # K % 8
+                      (lambda: rb.reflex_linear_residual(a, z(12, 64), z(4, 12), z(4, 12)), rb.ERR_SHAPE),      # N % 8
+                      (lambda: rb.reflex_linear_residual(a.view(-1)[4:4 + 3 * 64].view(3, 64), W, r[:3].contiguous(), r[:3].contiguous()), rb.ERR_ALIGN)):
+        with pytest.raises(rb.ReflexError) as e:
+            bad()
+        assert e.value.code == code
+
+
+# ------------------------------------------------------------------------------------------------
 # producer / consumer: a new prefix staged in the second static bank while the current one is read
 # ------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("impl", ["simt", "tc", "tc2"])
