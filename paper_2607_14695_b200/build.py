@@ -1,6 +1,9 @@
 """Builds libreflex_b200.so (the C-ABI library, sm_100a only) in-tree with nvcc.
 
     python -m paper_2607_14695_b200.build [--force] [--verbose]
+
+Extra compiler flags (debug builds with in-kernel timelines: -DREFLEX_TRACE, -DREFLEX_QK_TRACE, -DREFLEX_LIN_TRACE) can be
+given in the environment variable REFLEX_NVCC_FLAGS.
 """
 from __future__ import annotations
 
@@ -40,7 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "--threads", "0", "-o", tmp] + sources()
+           "--threads", "0", "-o", tmp] + os.environ.get("REFLEX_NVCC_FLAGS", "").split() + sources()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -5,10 +5,13 @@
 // bf16 path: one pair of CTAs (tcgen05.mma.cta_group::2, M = 256) per 256 x 256 output tile. Each CTA stages its own 128
 // rows of a and its 128 rows of W (its half of the B operand) per 64-column contraction step through a ring of five
 // 32 KB stages filled by TMA; one elected thread of the leader CTA issues the MMAs into a 256-column fp32 accumulator in
-// tensor memory. The residual tile (128 rows x 256 columns, 64 KB) is fetched by TMA into a buffer of its own while the
-// main loop runs; the epilogue adds the accumulator to it in place (fp32 add, one rounding to bf16) and the same buffer
-// leaves through TMA stores, which clip rows and columns past the end. out may alias res: a tile is read and written
-// by one CTA only.
+// tensor memory. The residual tile (128 rows x 256 columns, 64 KB) comes in by TMA behind the last operand tiles into a
+// buffer of its own; the epilogue threads (two per row) take it into registers while the last stages are multiplied, add
+// the accumulator (fp32 add, one rounding to bf16) and write the result back into the same buffer, which leaves through
+// TMA stores (they clip rows and columns past the end). out may alias res: a tile is read and written by one CTA only.
+// What bounds the kernel: without multicast every CTA fetches its own operand tiles, 52 tiles x 64 KB per contraction step
+// = 105 MB through the L2 for the 3200 x 1024 x 2048 problem, and the L2 delivers about 10 TB/s: 10.5 us for the main loop
+// against 8.3 us of tensor-pipe time.
 // The contraction is long (2048 or 4096) and the output small (3200 x 1024 at 64 streams): 52 tiles on 74 SM pairs in
 // one wave, so the kernel is not persistent.
 //
@@ -56,6 +59,14 @@ struct LinParams {
     uint32_t *status;     // status word of a cache, or NULL
 };
 
+// Optional timeline (debug builds only: -DREFLEX_LIN_TRACE): %globaltimer stamps of every CTA's milestones.
+#ifdef REFLEX_LIN_TRACE
+__device__ unsigned long long g_lin_trace[512 * 8];
+#define LIN_TRACE(ev) do { if (blockIdx.x < 512) g_lin_trace[blockIdx.x * 8 + (ev)] = globaltimer_ns(); } while (0)
+#else
+#define LIN_TRACE(ev) do { } while (0)
+#endif
+
 __device__ __forceinline__ void lin_tma2_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1)
 {
     asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -87,6 +98,7 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     const int m0 = (pair % p.m_tiles) * (2 * kLinBM) + (int)rank * kLinBM;   // this CTA's first row
     const int n0 = (pair / p.m_tiles) * BN;                                  // the pair's first output column
     const int nk_steps = (p.K + kLinBK - 1) / kLinBK;                        // (columns past K come in as TMA's zeros)
+    if (threadIdx.x == 64) LIN_TRACE(0);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < S::C_COUNT; ++i) mbar_init(bar(i), 1);
@@ -102,9 +114,11 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     cluster_wait();   // both CTAs' barriers exist before anything crosses the pair
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (threadIdx.x == 64) LIN_TRACE(1);
     // programmatic dependent launch: whatever produced a and res is complete from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 64) LIN_TRACE(2);
 
     auto wait = [&](int i, uint32_t parity, uint32_t code) -> bool {
         if (mbar_try_wait(bar(i), parity)) return true;
@@ -134,12 +148,16 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 lin_tma2_load_2d(base + S::OFF_A + s * S::A_STAGE, &tm_a, bar(S::C_FULL + s) & kPeerBitMask, ks * kLinBK, m0);
                 lin_tma2_load_2d(base + S::OFF_B + s * S::B_STAGE, &tm_w, bar(S::C_FULL + s) & kPeerBitMask, ks * kLinBK, n0 + (int)rank * (BN / 2));
             }
-            if (p.has_res && ok) {
+            if (ok) {
                 // the residual tile goes last: it is not needed before the epilogue, and ahead of the main loop's operands it
                 // would hold them up for the time 64 KB take to come in (measured: 0.7 us per launch)
-                mbar_expect_tx(bar(S::C_RES), S::RES_BYTES);
+                if (p.has_res) {
+                    mbar_expect_tx(bar(S::C_RES), S::RES_BYTES);
 #pragma unroll
-                for (int ch = 0; ch < BN / 64; ++ch) tma_load_2d(base + S::OFF_RES + ch * S::CHUNK, &tm_res, bar(S::C_RES), n0 + ch * 64, m0);
+                    for (int ch = 0; ch < BN / 64; ++ch) tma_load_2d(base + S::OFF_RES + ch * S::CHUNK, &tm_res, bar(S::C_RES), n0 + ch * 64, m0);
+                } else {
+                    mbar_arrive(bar(S::C_RES));
+                }
             }
         }
     } else if (warp == 1) {
@@ -151,6 +169,7 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 const int s = ks % NST;
                 ok = wait(S::C_FULL + s, (uint32_t)(ks / NST) & 1u, 2);
                 if (!ok) break;
+                if (ks == 0 && lane == 0) LIN_TRACE(3);
                 tc_fence_after();
                 uint64_t ad = umma_desc_sw128(base + S::OFF_A + s * S::A_STAGE, 16, 1024);
                 uint64_t bd = umma_desc_sw128(base + S::OFF_B + s * S::B_STAGE, 16, 1024);
@@ -170,26 +189,36 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const int half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        bool ok = true;
-        if (p.has_res) ok = wait(S::C_RES, 0u, 3);
-        ok = wait(S::C_ACC, 0u, 4) && ok;
-        tc_fence_after();
+        // The residual tile comes in by TMA behind the last operand tiles; every thread takes its BN / 2 columns of its row
+        // out of shared memory into registers while the last stages are multiplied, so that after the accumulator is final
+        // only tensor-memory loads, adds and the stores into the same staging buffer remain. (As global loads by these
+        // threads, 16 bytes per row and instruction, the residual cost the main loop 2.5 us: the L2's bandwidth is what
+        // limits this kernel, and half-used sectors waste it.)
+        bool ok = wait(S::C_RES, 0u, 3);
         constexpr int CPT = BN / 2 / 64;              // 64-column chunks per thread
-#pragma unroll 1
+        uint4 rr[CPT * 8];
+#pragma unroll
+        for (int j = 0; j < CPT * 8; ++j) {
+            // 128-byte swizzle of the TMA box: 16-byte piece j of row r sits at j ^ (r % 8)
+            rr[j] = make_uint4(0u, 0u, 0u, 0u);
+            if (p.has_res) rr[j] = *reinterpret_cast<const uint4 *>(smem + S::OFF_RES + (half * CPT + j / 8) * S::CHUNK + row * 128 + (((j & 7) ^ (row & 7)) << 4));
+        }
+        ok = wait(S::C_ACC, 0u, 4) && ok;
+        if (threadIdx.x == 64) LIN_TRACE(4);
+        tc_fence_after();
+#pragma unroll
         for (int cc = 0; cc < CPT; ++cc) {
             const int ch = half * CPT + cc;
             uint8_t *rowp = smem + S::OFF_RES + ch * S::CHUNK + row * 128;
-#pragma unroll 1
+#pragma unroll
             for (int g = 0; g < 2; ++g) {             // 32 columns at a time
                 uint32_t acc[32];
                 tmem_ld32(tmem + lane_addr + ch * 64 + g * 32, acc);   // warp-wide: every lane takes part, whatever its row
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    // 128-byte swizzle of the TMA boxes: 16-byte piece j of row r sits at j ^ (r % 8)
-                    uint4 *pc = reinterpret_cast<uint4 *>(rowp + (((g * 4 + i) ^ (row & 7)) << 4));
-                    uint32_t rv[4] = {0u, 0u, 0u, 0u};
-                    if (p.has_res) { const uint4 t = *pc; rv[0] = t.x; rv[1] = t.y; rv[2] = t.z; rv[3] = t.w; }
+                    const uint4 t = rr[cc * 8 + g * 4 + i];
+                    const uint32_t rv[4] = {t.x, t.y, t.z, t.w};
                     uint32_t ov[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
@@ -199,7 +228,8 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                         __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
                         ov[k] = *reinterpret_cast<uint32_t *>(&h);
                     }
-                    *pc = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+                    // 128-byte swizzle of the TMA box: 16-byte piece j of row r sits at j ^ (r % 8)
+                    *reinterpret_cast<uint4 *>(rowp + (((g * 4 + i) ^ (row & 7)) << 4)) = make_uint4(ov[0], ov[1], ov[2], ov[3]);
                 }
             }
             // this half's chunk is complete once its 128 threads are through: one of them hands it to the TMA engine
@@ -210,7 +240,10 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
         }
-        if (quarter == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the stores of this thread are complete
+        if (threadIdx.x == 64) LIN_TRACE(5);
+        // (the staging buffer has been read; the writes themselves are complete when the grid is)
+        if (quarter == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        if (warp == 4 && lane == 0) LIN_TRACE(6);
     }
 
     tc_fence_before();
@@ -218,6 +251,7 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     cluster_arrive();
     cluster_wait();   // neither CTA retires while its partner can still touch its shared memory or barriers
     if (warp == 1) tmem_dealloc2(tmem, BN);
+    if (threadIdx.x == 64) LIN_TRACE(7);
 }
 
 // Any dtype, any shape: one block per row; the row of a in shared memory (fp32), every thread takes output features
@@ -317,3 +351,10 @@ cudaError_t launch_linear_residual(const void *a, const void *W, const void *res
 }
 
 }  // namespace reflex
+
+#ifdef REFLEX_LIN_TRACE
+extern "C" int reflex_debug_lin_trace(unsigned long long *out)
+{
+    return (int)cudaMemcpyFromSymbol(out, reflex::g_lin_trace, sizeof(unsigned long long) * 512 * 8);
+}
+#endif
