@@ -48,15 +48,6 @@ constexpr int kTc2Parts = REFLEX_TC2_NP;            // softmax threads per query
 constexpr int kTc2Threads = 64 + 128 * kTc2Parts;   // producer warp, MMA warp, 4 * kTc2Parts softmax warps
 static_assert(kTc2Parts == 2 || kTc2Parts == 4, "softmax threads per row");
 
-// Round a float up to the next bf16 value, as raw upper 16 bits (the softmax threads of a row exchange their
-// maxima in this form: any common reference >= the true maximum serves, and 16 bits keep the exchange area small).
-__device__ __forceinline__ uint32_t bf16_bits_round_up(float x)
-{
-    uint32_t u = __float_as_uint(x);
-    if (!(u >> 31) && (u & 0xFFFFu)) u += 0x10000u;   // positive: towards +inf; negative: truncation already rounds up
-    return u >> 16;
-}
-
 // s[c] = -inf for every key c < K of a slice that `mask` marks dead
 template <int K>
 __device__ __forceinline__ void apply_slice_mask(float (&s)[K], uint64_t mask)
@@ -92,15 +83,16 @@ template <int HD> struct Tc2Smem {
     static constexpr uint32_t STAGE_BYTES = 2 * 128 * 128;
     static constexpr uint32_t OFF_BAR = OFF_STAGE + STAGE_BYTES;
     static constexpr uint32_t BAR_BYTES = 256;
-    static constexpr uint32_t OFF_XMAX = OFF_BAR + BAR_BYTES;                   // row maxima: 2 buffers x 128 rows x NP 16-bit values
-    static constexpr uint32_t XMAX_BYTES = 2 * 128 * kTc2Parts * 2;
-    static constexpr uint32_t XSUM_BYTES = kTc2Parts * 128 * 4;                 // row sums: NP x 128 rows fp32
+    // Row maxima of the NP threads of a row: 2 buffers (one per S/P buffer) x 128 rows x NP fp32, exact (rounded to 16 bits
+    // the common reference overshot the true maximum by up to |max| / 128, which empties a row by underflow once logits
+    // reach tens of thousands). The row sums exchanged at the end of a unit (NP x 128 fp32: one buffer's size) use the
+    // buffer the unit's last tile did NOT use: every thread is past its last read of it, and the next tile writes to it
+    // only after the barriers of the epilogue, which every thread reaches after it has read the sums.
+    static constexpr uint32_t OFF_XMAX = OFF_BAR + BAR_BYTES;
+    static constexpr uint32_t XBUF_BYTES = 128 * kTc2Parts * 4;
+    static constexpr uint32_t XMAX_BYTES = 2 * XBUF_BYTES;
     static constexpr uint32_t TOTAL = 232448;                                   // the whole opt-in shared memory of an SM (227 KB)
-    // the sums get an area of their own when it fits, else they reuse the maxima's (with two more barriers per unit)
-    static constexpr bool XSUM_OWN = OFF_XMAX + XMAX_BYTES + XSUM_BYTES <= TOTAL;
-    static constexpr uint32_t OFF_XSUM = XSUM_OWN ? OFF_XMAX + XMAX_BYTES : OFF_XMAX;
-    static constexpr uint32_t NEED = XSUM_OWN ? OFF_XSUM + XSUM_BYTES
-                                              : OFF_XMAX + (XMAX_BYTES > XSUM_BYTES ? XMAX_BYTES : XSUM_BYTES);   // from the 1024-byte aligned base
+    static constexpr uint32_t NEED = OFF_XMAX + XMAX_BYTES;                     // from the 1024-byte aligned base
     static_assert(NEED <= TOTAL, "shared memory budget");
     // mbarrier indices
     static constexpr int C_QFULL = 0, C_QEMPTY = 1, C_KFULL = 2, C_KEMPTY = C_KFULL + NKS, C_VLAND = C_KEMPTY + NKS,
@@ -409,8 +401,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const uint32_t leader_pfull[2] = {mapa(bar(C_PFULL), lead), mapa(bar(C_PFULL + 1), lead)};
         const uint32_t leader_ofree = mapa(bar(C_OFREE), lead);
-        uint16_t *xmax = reinterpret_cast<uint16_t *>(smem + L::OFF_XMAX);   // [2 buffers][128 rows][NP], bf16 bit patterns
-        float *xsum = reinterpret_cast<float *>(smem + L::OFF_XSUM);         // [NP][128 rows]
+        float *xmax = reinterpret_cast<float *>(smem + L::OFF_XMAX);         // [2 buffers][128 rows][NP]
         bool ok = true;
         int gt = 0;
         [[maybe_unused]] int ui_s = 0;
@@ -508,18 +499,18 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 }
-                // meet the threads that hold the other keys of this row: every one of them publishes its maximum rounded up
-                // to bf16 and takes the largest of the NP published values, so all agree. Past this barrier every thread of the
-                // row has its logits in registers, so P may overwrite them in tensor memory.
+                // meet the threads that hold the other keys of this row: every one of them publishes its maximum and takes the
+                // largest of the NP published values, so all agree. Past this barrier every thread of the row has its logits
+                // in registers, so P may overwrite them in tensor memory.
                 SM_EV(3);
-                xmax[(buf * 128 + row) * NP + part] = (uint16_t)bf16_bits_round_up(mx);
+                xmax[(buf * 128 + row) * NP + part] = mx;
                 asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
                 SM_EV(4);
                 {
-                    const uint16_t *xr = xmax + (buf * 128 + row) * NP;
-                    mx = -INFINITY;
+                    const float *xr = xmax + (buf * 128 + row) * NP;
+                    mx = xr[0];
 #pragma unroll
-                    for (int q = 0; q < NP; ++q) mx = fmaxf(mx, __uint_as_float((uint32_t)xr[q] << 16));
+                    for (int q = 1; q < NP; ++q) mx = fmaxf(mx, xr[q]);
                 }
                 if (jj == 0) {
                     m_ref = mx;
@@ -626,12 +617,11 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int g_last = gt - 1;
             ok = ok && wait(C_PVDONE + (g_last & 1), (uint32_t)(g_last >> 1) & 1u, 13);
             if (threadIdx.x == 64) { TC2_TRACE(2, 15, 3); TC2_TRACE(2, ui_s, 3); }
-            if constexpr (!L::XSUM_OWN) asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // the maxima of the last tile have been read
+            float *xsum = xmax + ((g_last & 1) ^ 1) * (128 * NP);      // [NP][128 rows], in the maxima buffer the last tile did not use
             xsum[part * 128 + row] = l;
             asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");
 #pragma unroll
             for (int q = 1; q < NP; ++q) l += xsum[((part + q) % NP) * 128 + row];
-            if constexpr (!L::XSUM_OWN) asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // ... and the sums, before new maxima land there
             tc_fence_after();
             if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 5);
             const bool row_live = t_row < p.T;
@@ -663,6 +653,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         for (int i = 0; i < 4; ++i) st_global_v8(po + c * 32 + 8 * i, *reinterpret_cast<const uint32_t(*)[8]>(o + 8 * i));
                     }
                 }
+                asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // every thread has read the row sums before the next unit's maxima land there
                 continue;
             }
             // O / l goes out through a 32 KB staging area laid out like a Q tile (two 64-column chunks of 128 swizzled rows)

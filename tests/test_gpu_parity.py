@@ -143,6 +143,66 @@ def test_cfg3_stream_ticks(U):
                 tw.attention(layer, tick, what=f"cfg3 tick {tick}")
 
 
+def test_cfg3_500_tick_stream_graph_replay(U):
+    """The batch-1 streaming trace in full: 500 control ticks, one token appended to the ring in all 18 layers per tick, a
+    new static prefix every 10 ticks with lengths alternating 816 / 800 (a shorter prefix leaves stale rows behind). From
+    tick 1 on a tick is ONE CUDA-graph replay (ring append + 18 attention launches) fed through fixed device buffers; the
+    oracle is advanced on the host with the same bytes. Ring state, slot map and cache bytes are compared exactly and the
+    attention outputs element-wise on ticks 0, 1, 9, 10, 11, 31, 32, 33 and 499 (the ring has wrapped 15 times by then)."""
+    rb = U.rb
+    w = synth.CONFIGS["cfg3"]
+    tw = U.Twin(w, head0=[30], poison=True)
+    dt = rb.torch_dtype(w.dtype)
+    e = lambda *s: torch.empty(s, dtype=dt, device=U.DEV)
+    kn_buf, vn_buf = e(1, w.L, 1, w.Hkv, w.d), e(1, w.L, 1, w.Hkv, w.d)
+    q_buf, kd_buf, vd_buf = e(w.L, 1, w.T, w.Hq, w.d), e(w.L, 1, w.T, w.Hkv, w.d), e(w.L, 1, w.T, w.Hkv, w.d)
+    out_buf = e(w.L, 1, w.T, w.Hq, w.d)
+
+    def tick_calls():
+        rb.reflex_cache_append_sliding(tw.g, [0], kn_buf, vn_buf)
+        for layer in range(w.L):
+            rb.reflex_partitioned_attention(tw.g, layer, q_buf[layer], kd_buf[layer], vd_buf[layer], out_buf[layer])
+
+    def fill_inputs(tick):
+        host = {}
+        for layer in range(w.L):
+            host[layer] = tuple(synth.normal(w, n, (1, w.T, h, w.d), layer, tick) for n, h in (("q", w.Hq), ("k_dyn", w.Hkv), ("v_dyn", w.Hkv)))
+            for buf, a in zip((q_buf, kd_buf, vd_buf), host[layer]):
+                buf[layer].copy_(U.to_dev(a, w.dtype))
+        return host
+
+    compare = {0, 1, 9, 10, 11, 31, 32, 33, 499}
+    graph = None
+    fill_inputs(0)
+    for tick in range(500):
+        if tick % 10 == 0:
+            tw.init_static([0], [816 if (tick // 10) % 2 == 0 else 800], variant=tick)
+        kn = synth.normal(w, "k_new", (1, w.L, 1, w.Hkv, w.d), 0, tick)
+        vn = synth.normal(w, "v_new", (1, w.L, 1, w.Hkv, w.d), 0, tick)
+        tw.o.append_sliding(0, kn[0], vn[0])
+        kn_buf.copy_(U.to_dev(kn, w.dtype)); vn_buf.copy_(U.to_dev(vn, w.dtype))
+        host = fill_inputs(tick) if tick in compare else None
+        if tick == 0:
+            tick_calls()                       # direct launches; the graph is captured afterwards (capture launches nothing)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                tick_calls()
+        else:
+            graph.replay()
+        if tick in compare:
+            torch.cuda.synchronize()
+            rb.reflex_cache_check_status(tw.g)
+            tw.check_state()                   # (reads the ring state back from the device: replays do not touch the host mirror)
+            assert tw.o.total[0] == tick + 1 and tw.o.count[0] == min(tick + 1, w.N) and tw.o.head[0] == (30 + tick + 1) % w.N
+            got = U.to_host(out_buf)
+            assert np.isfinite(got).all()
+            for layer in (range(w.L) if tick in (10, 32, 499) else (0, 17)):
+                q, kd, vd = host[layer]
+                want = tw.o.attention(0, layer, q[0], kd[0], vd[0])
+                U.check_close(got[layer, 0], want, w.dtype, f"cfg3 tick {tick} layer {layer}")
+
+
 # ------------------------------------------------------------------------------------------------
 # config 4 shapes: 64 streams with random ring offsets and mixed fill levels
 # ------------------------------------------------------------------------------------------------
@@ -182,6 +242,54 @@ def test_cfg5_long_context(U, impl):
         x = synth.norm_input(w, 0, int(t * 1000))
         assert (np.abs(x) > 100).any()
         _norm_case(U, w, x, synth.cond_vectors(w, t), what=f"cfg5 norm t={t}")
+
+
+def test_cfg5b_outliers_in_queries_and_keys(U):
+    """The labelled stress run beside the long-context configuration: 0.1 % of the elements of Q, of the dynamic K and of the
+    cached K (prefix and ring) are multiplied by 1000, V stays N(0, 1). Logits reach tens of thousands and the softmax is
+    one-hot for the rows an outlier touches: every output must be finite, and the outputs are compared with the oracle
+    under the output-spacing clause (a one-hot row returns a single V row, |v| up to 4.5). This is a finiteness and
+    relative-error stress outside the absolute-error contract; the worst relative error is printed."""
+    rb = U.rb
+    w = synth.CONFIGS["cfg5"].with_(L=1, B=3)
+    tw = U.Twin(w, head0=synth.ring_head0(w), poison=True)
+
+    def spiked(name, shape, layer, variant):
+        a = synth.normal(w, name, shape, layer, variant)
+        mask = synth.rng_for(w, "outlier_mask", layer, variant + 100 * synth.TID[name]).random(size=a.shape) < w.outlier_frac
+        return synth.round_storage(np.where(mask, a * np.float32(w.outlier_mult), a).astype(np.float32), w.dtype)
+
+    ids = list(range(w.B))
+    ks, vs = spiked("k_static", (w.B, w.L, w.S, w.Hkv, w.d), 0, 0), synth.normal(w, "v_static", (w.B, w.L, w.S, w.Hkv, w.d), 0, 0)
+    for b in ids:
+        tw.o.init_static(b, ks[b], vs[b])
+    rb.reflex_cache_init_static(tw.g, ids, U.to_dev(ks, w.dtype), U.to_dev(vs, w.dtype))
+    for i in range(3):
+        kn, vn = spiked("k_new", (w.B, w.L, 100, w.Hkv, w.d), 0, i), synth.normal(w, "v_new", (w.B, w.L, 100, w.Hkv, w.d), 0, i)
+        for b in ids:
+            tw.o.append_sliding(b, kn[b], vn[b])
+        rb.reflex_cache_append_sliding(tw.g, ids, U.to_dev(kn, w.dtype), U.to_dev(vn, w.dtype))
+    tw.check_state()
+    q, kd = spiked("q", (w.B, w.T, w.Hq, w.d), 0, 0), spiked("k_dyn", (w.B, w.T, w.Hkv, w.d), 0, 0)
+    vd = synth.normal(w, "v_dyn", (w.B, w.T, w.Hkv, w.d), 0, 0)
+    assert (np.abs(q) > 100).any() and (np.abs(ks) > 100).any() and (np.abs(kd) > 100).any()
+    worst_rel = 0.0
+    for impl in (rb.ATTN_AUTO, rb.ATTN_SIMT):
+        rb.reflex_cache_set_attention_impl(tw.g, impl)
+        for dyn_mask in (0, 1):
+            out = torch.full((w.B, w.T, w.Hq, w.d), float("nan"), dtype=torch.bfloat16, device=U.DEV)
+            rb.reflex_partitioned_attention(tw.g, 0, U.to_dev(q, w.dtype), U.to_dev(kd, w.dtype), U.to_dev(vd, w.dtype), out, dyn_mask=dyn_mask)
+            rb.reflex_cache_check_status(tw.g)
+            got = U.to_host(out)
+            assert np.isfinite(got).all(), "cfg5b: non-finite output"
+            for b in ids:
+                want = tw.o.attention(b, 0, q[b], kd[b], vd[b], dyn_mask, None)
+                U.check_close(got[b], want, w.dtype, f"cfg5b stream {b} mask {dyn_mask} impl {impl}", rel_clause=True)
+                big = np.abs(want) > 0.5
+                if big.any():
+                    worst_rel = max(worst_rel, float((np.abs(got[b] - want)[big] / np.abs(want)[big]).max()))
+    print(f"cfg5b: worst relative error on |o| > 0.5: {worst_rel:.3e}")
+    assert worst_rel <= U.BF16_MAX_ABS / 0.5          # (what the element-wise bound above allows at |o| = 0.5)
 
 
 # ------------------------------------------------------------------------------------------------
