@@ -69,3 +69,27 @@ def test_reference_arm_prints_one_json_line():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "cfg2", "--steps", "1"],
                          capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_roofline_picks_the_binding_roof_and_both_arms_print_the_same_config():
+    """cfg4's attention launch: 85.07 MB and 23.54 GFLOP; at the measured peaks the tensor floor (17.4 us sustained) is above
+    the HBM floor (13.2 us), so the bound is the tensor pipe and frac = tensor floor / measured; a copy-like launch is HBM-bound."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench_mod", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    from paper_2607_14695_b200 import synth
+    w = synth.CONFIGS["cfg4"]
+    alg = bench.algorithmic_work(w)
+    assert alg["attn_bytes_per_launch"] == 85065728 and abs(alg["attn_flops_per_launch"] - 23.5405e9) < 1e7
+    peaks = {"hbm_gbs": 6459.3, "bf16_tflops": 1635.6, "bf16_tflops_sustained": 1354.9, "source": "measured"}
+    r = bench.roofline_of(alg["attn_flops_per_launch"], alg["attn_bytes_per_launch"], 30e-6, peaks, "sustained")
+    assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and abs(r["frac"] - 17.374e-6 / 30e-6) < 1e-3
+    assert abs(r["frac_hbm"] - 85065728 / 30e-6 / 1e9 / 6459.3) < 1e-9 and abs(r["achieved"] - 784.7) < 0.1
+    r2 = bench.roofline_of(1e6, 13.8e6, 4.5e-6, peaks, "burst")
+    assert r2["bound"] == "hbm" and r2["unit"] == "GB/s" and abs(r2["frac"] - r2["frac_hbm"]) < 1e-12
+    cfg = bench.config_of(w)
+    assert cfg["workload"].startswith("cfg4:") and "larger than L2" in cfg["l2_policy"] and cfg["flops_per_step"] == 18 * alg["attn_flops_per_launch"]
+    assert "flushed" in bench.config_of(synth.CONFIGS["cfg2"])["l2_policy"]
+    traffic, src = bench.ncu_traffic(w, "auto")
+    assert traffic and traffic < alg["attn_bytes_per_launch"] and "profiles/" in src
