@@ -663,7 +663,8 @@ def main():
                     "adarmsnorm_rows_gbs": alg["norm_bytes_per_launch"] / (rows_avg_ms * 1e-3) / 1e9,
                     "adarmsnorm_rows_frac_hbm": alg["norm_bytes_per_launch"] / (rows_avg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                     "adarmsnorm_standalone_call_avg_us": norm_avg_ms * 1e3,
-                    "attention_share_of_step": attn_avg_ms * w.L / (statistics.mean(step_ms))},
+                    "attention_share_of_step": (attn["burst"]["us"] * w.L / regimes["step_burst"]["us"]) if "step_burst" in regimes
+                                               else attn["burst"]["us"] * 1e-3 * w.L / statistics.mean(step_ms)},
         "clocks": clocks,
     }
     if stream_stats is not None:
