@@ -69,7 +69,7 @@ struct QkParams {
     float eps;
     uint32_t *status;
     const __nv_bfloat16 *res;   // plain projection only (few-rows kernel with PLAIN): residual [M][nq] added to the output, or NULL
-    int ksplit;                 // plain projection only: CTAs of a cluster that share one feature tile, each taking a slice of the contraction
+    int ksplit;                 // few-rows kernel: CTAs of a cluster that share one feature tile, each taking a slice of the contraction
 };
 
 #ifdef REFLEX_QK_TRACE
@@ -384,11 +384,12 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
     volatile uint32_t *abort_flag = tmem_slot + 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool swiglu = NACC == 2;
-    // PLAIN with ksplit > 1: the ksplit CTAs of a cluster own the same 128 features and a slice of the contraction axis each
-    // (whole steps only: the launcher picks ksplit so that the chunks divide), and add up their accumulators through
-    // distributed shared memory at the end
-    const int ksplit = PLAIN ? p.ksplit : 1;
-    const int krank = (PLAIN && ksplit > 1) ? (int)cluster_ctarank() : 0;
+    // ksplit > 1: the ksplit CTAs of a cluster own the same 128 features and a slice of the contraction axis each (whole
+    // steps only: the launcher picks ksplit so that the chunks divide), and add up their accumulators -- and, with the
+    // norm, their shares of every row's sum of squares -- through distributed shared memory at the end. With a handful of
+    // CTAs streaming the weights the launch is a chain of dependent steps; split, 80 to 128 CTAs share it.
+    const int ksplit = p.ksplit;
+    const int krank = ksplit > 1 ? (int)cluster_ctarank() : 0;
     const int f0 = (blockIdx.x / ksplit) * 128;       // first output feature (hidden feature for SwiGLU) of this CTA
     constexpr int CPS = S::CPS;
     const int all_chunks = p.D / kQkBK;
@@ -520,7 +521,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             ulonglong2 gv[CPS * NPC * 2];
 #pragma unroll
             for (int cc = 0; cc < CPS; ++cc) {
-                const int chunk = min(ks * CPS + cc, n_chunks - 1);      // (a chunk past the end: loaded but never used)
+                const int chunk = chunk0 + min(ks * CPS + cc, n_chunks - 1);      // (a chunk past the end: loaded but never used)
                 const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + chunk * kQkBK);
                 const uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE + row * 128;
 #pragma unroll
@@ -570,7 +571,8 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             float ssr = 0.f;
 #pragma unroll
             for (int t = 0; t < TP; ++t) ssr += ssm[t * 128 + tid];
-            rsm[tid] = PLAIN ? 1.f : rsqrtf(ssr * (1.f / (float)p.D) + p.eps);
+            // (contraction split over a cluster: this CTA has seen its slice of the row only; the shares meet in the reduction)
+            rsm[tid] = PLAIN ? 1.f : (ksplit > 1 ? ssr : rsqrtf(ssr * (1.f / (float)p.D) + p.eps));
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (threadIdx.x == 64) QK_TRACE(2, 31, 0);
@@ -595,17 +597,18 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             tmem_ld32(tmem + lane_addr + c * 32, acc);          // warp-wide: every lane takes part
             if (swiglu) tmem_ld32(tmem + lane_addr + NT + c * 32, up);
             tmem_wait_ld();
-            if constexpr (PLAIN) {
-                if (ksplit > 1) {
-                    // this CTA's share of the sums goes to shared memory (the stage ring is idle: every load has been consumed
-                    // and every MMA has completed), [row][feature] so that a warp writes 128 contiguous bytes
-                    float *part = reinterpret_cast<float *>(smem + S::OFF_W);
-                    static_assert(S::STAGES * S::W_STAGE >= (uint32_t)NT * 128 * 4, "partial sums fit in the stage ring");
+            if (ksplit > 1) {
+                // this CTA's share of the sums goes to shared memory (the stage ring is idle: every load has been consumed
+                // and every MMA has completed), [row][feature] so that a warp writes 128 contiguous bytes; the up projection's
+                // share behind it
+                float *part = reinterpret_cast<float *>(smem + S::OFF_W);
+                static_assert(S::STAGES * S::W_STAGE >= (uint32_t)NACC * NT * 128 * 4, "partial sums fit in the stage ring");
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        part[(c * 32 + i) * 128 + quarter * 32 + lane] = ok ? __uint_as_float(acc[i]) : __int_as_float(0x7fc00000);
-                    continue;
+                for (int i = 0; i < 32; ++i) {
+                    part[(c * 32 + i) * 128 + quarter * 32 + lane] = ok ? __uint_as_float(acc[i]) : __int_as_float(0x7fc00000);
+                    if (swiglu) part[(NT + c * 32 + i) * 128 + quarter * 32 + lane] = __uint_as_float(up[i]);
                 }
+                continue;
             }
             if (!ok || f >= n_feat) continue;
 #pragma unroll
@@ -622,35 +625,65 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
         }
     }
 
-    if constexpr (PLAIN) {
-        if (ksplit > 1) {
-            // (cluster barriers are warp-aligned: the lanes of the producer warp that idled while lane 0 ran the loads must
-            // not reach them before lane 0 does, so the CTA meets first)
-            __syncthreads();
-            cluster_arrive();
-            cluster_wait();
-            if (warp >= 2) {
-                // CTA krank adds up rows [krank, krank + 1) * NT / ksplit of all slices, adds the residual and writes bf16
-                const float *part = reinterpret_cast<const float *>(smem + S::OFF_W);
-                const int rows_mine = NT / ksplit, r0 = krank * rows_mine;
-                for (int e = threadIdx.x - 64; e < rows_mine * 128; e += 256) {
-                    const int r = r0 + e / 128, fl = e % 128;
-                    if (r >= p.M || f0 + fl >= p.nq) continue;
-                    float sum = 0.f;
-                    const uint32_t a0 = smem_u32(part + r * 128 + fl);
+    if (ksplit > 1) {
+        // (cluster barriers are warp-aligned: the lanes of the producer warp that idled while lane 0 ran the loads must
+        // not reach them before lane 0 does, so the CTA meets first)
+        __syncthreads();
+        cluster_arrive();
+        cluster_wait();
+        // CTA krank adds up rows [krank, krank + 1) * NT / ksplit of all slices and finishes them
+        const int rows_mine = NT / ksplit, r0 = krank * rows_mine;
+        float *ssm = reinterpret_cast<float *>(smem + S::OFF_SS);
+        float *rsm = ssm + 512;                  // [NT] this CTA's share of every row's sum of squares (1 for the plain projection)
+        float *rs_mine = ssm;                    // [rows_mine] 1 / RMS of this CTA's rows (the partial sums there have been consumed)
+        if (warp >= 2) {
+            if constexpr (!PLAIN) {
+                const int t = threadIdx.x - 64;
+                if (t < rows_mine) {
+                    float ss = 0.f;
+                    const uint32_t a0 = smem_u32(rsm + r0 + t);
                     for (int q = 0; q < ksplit; ++q) {
                         float v;
                         asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(mapa(a0, (uint32_t)q)) : "memory");
-                        sum += v;
+                        ss += v;
                     }
-                    const size_t o = (size_t)r * p.nq + f0 + fl;
-                    if (p.res) sum += __bfloat162float(p.res[o]);
-                    p.q[o] = __float2bfloat16_rn(sum);
+                    rs_mine[t] = rsqrtf(ss * (1.f / (float)p.D) + p.eps);
                 }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
             }
-            cluster_arrive();
-            cluster_wait();   // no CTA retires while a peer may still read its partial sums
+            const float *part = reinterpret_cast<const float *>(smem + S::OFF_W);
+            const int n_feat = swiglu ? p.swiglu_F : p.nq + 2 * p.nk;
+            for (int e = threadIdx.x - 64; e < rows_mine * 128; e += 256) {
+                const int r = r0 + e / 128, fl = e % 128, f = f0 + fl;
+                if (r >= p.M || f >= n_feat) continue;
+                float sum = 0.f, sum_up = 0.f;
+                const uint32_t a0 = smem_u32(part + r * 128 + fl);
+                for (int q = 0; q < ksplit; ++q) {
+                    float v;
+                    const uint32_t aq = mapa(a0, (uint32_t)q);
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(aq) : "memory");
+                    sum += v;
+                    if (swiglu) {
+                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(aq + (uint32_t)NT * 128 * 4) : "memory");
+                        sum_up += v;
+                    }
+                }
+                __nv_bfloat16 *dst;
+                if (swiglu || f < p.nq) dst = p.q + (size_t)r * p.nq + f;
+                else if (f < p.nq + p.nk) dst = p.k + (size_t)r * p.nk + (f - p.nq);
+                else dst = p.v + (size_t)r * p.nk + (f - p.nq - p.nk);
+                if constexpr (PLAIN) {
+                    if (p.res) sum += __bfloat162float(p.res[(size_t)r * p.nq + f]);
+                } else {
+                    const float rs = rs_mine[r - r0];
+                    sum *= rs;
+                    if (swiglu) sum = __fdividef(sum, 1.f + __expf(-sum)) * (sum_up * rs);
+                }
+                *dst = __float2bfloat16_rn(sum);
+            }
         }
+        cluster_arrive();
+        cluster_wait();   // no CTA retires while a peer may still read its partial sums
     }
     if (threadIdx.x == 64) QK_TRACE(2, 31, 2);
     tc_fence_before();
@@ -796,9 +829,9 @@ static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, Qk
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;      // plain projection: the CTAs that split one feature tile's contraction
-    attr[1].val.clusterDim.x = (unsigned)(PLAIN ? p.ksplit : 1); attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    attr[1].val.clusterDim.x = (unsigned)p.ksplit; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (PLAIN && p.ksplit > 1) ? 2 : 1;
+    cfg.numAttrs = p.ksplit > 1 ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, norm_linear_small_kernel<NT, NACC, PLAIN>, mx, mw, p);
     count_launch();
     return e;
@@ -827,9 +860,17 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
         QkParams sp;
         sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
         sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.swiglu_F = swiglu_F;
-        sp.eps = eps; sp.status = status; sp.res = nullptr; sp.ksplit = 1;
+        sp.eps = eps; sp.status = status; sp.res = nullptr;
         const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
-        const unsigned grid = (unsigned)((n_feat + 127) / 128);
+        // The contraction split over 4 CTAs per feature tile where the chain of steps is long enough to pay for a cluster
+        // launch and its two barriers (16 steps or more: SwiGLU at D = 1024, 11.1 -> 10.0 us for one stream; the packed
+        // projection's 8 steps got slower, 6.8 -> 8.3 us, and a split in two is slower than none for both), while every
+        // slice keeps whole steps and the grid stays within the SMs.
+        const int chunks = D / kQkBK, ftiles = (n_feat + 127) / 128, cps = swiglu_F > 0 ? 1 : 2;
+        int ks = 1;
+        if (chunks / cps >= 16 && chunks % (4 * cps) == 0 && ftiles * 4 <= (sm_count > 0 ? sm_count : 148)) ks = 4;
+        sp.ksplit = ks;
+        const unsigned grid = (unsigned)(ftiles * ks);
         if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, st) : launch_small<128, 2>(sx, sw, sp, grid, st);
         return NT == 64 ? launch_small<64, 1>(sx, sw, sp, grid, st) : launch_small<128, 1>(sx, sw, sp, grid, st);
     }
