@@ -61,6 +61,20 @@ def test_validation_before_launch(lib):
     assert lib.reflex_adarmsnorm(fake, fake, None, None, None, None, None, None, 1, 1, 128, 8, 8, 1e-6, 0, None) == rb.ERR_INVALID_ARG
     assert lib.reflex_adarmsnorm(odd, fake, fake, fake, fake, fake, fake, None, 1, 1, 128, 8, 8, 1e-6, 0, None) == rb.ERR_ALIGN
     assert lib.reflex_adarmsnorm(*a, 1, 1, 128, 8, 8, -1.0, 0, None) == rb.ERR_INVALID_ARG
+    # plain projection with residual
+    fake2 = ctypes.c_void_p(0x2000)
+    assert lib.reflex_linear_residual(None, fake, fake, fake2, fake2, 4, 64, 16, rb.DTYPE_BF16, 3, None) == rb.ERR_INVALID_ARG and "impl" in err()
+    assert lib.reflex_linear_residual(None, fake, fake, None, None, 4, 64, 16, rb.DTYPE_BF16, 0, None) == rb.ERR_INVALID_ARG      # out NULL
+    assert lib.reflex_linear_residual(None, fake, fake, None, fake, 4, 64, 16, rb.DTYPE_BF16, 0, None) == rb.ERR_INVALID_ARG      # out aliases a
+    assert lib.reflex_linear_residual(None, fake, fake, fake2, fake2, 4, 60, 16, rb.DTYPE_BF16, 0, None) == rb.ERR_SHAPE          # K % 8
+    assert lib.reflex_linear_residual(None, fake, fake, fake2, fake2, 4, 64, 12, rb.DTYPE_BF16, 0, None) == rb.ERR_SHAPE          # N % 8
+    assert lib.reflex_linear_residual(None, fake, fake, fake2, fake2, 0, 64, 16, rb.DTYPE_BF16, 0, None) == rb.ERR_SHAPE          # M < 1
+    assert lib.reflex_linear_residual(None, fake, odd, fake2, fake2, 4, 64, 16, rb.DTYPE_BF16, 0, None) == rb.ERR_ALIGN
+    assert lib.reflex_linear_residual(None, fake, fake, fake2, fake2, 4, 64, 16, 5, 0, None) == rb.ERR_INVALID_ARG               # dtype
+    # gate MLP for all layers
+    assert lib.reflex_adarmsnorm_gate(fake, fake, fake, fake, fake, fake, 0, 1, 128, 8, 8, 0, None) == rb.ERR_SHAPE              # L < 1
+    assert lib.reflex_adarmsnorm_gate(fake, fake, fake, fake, fake, fake, 1, 1, 128, 8, 1032, 0, None) == rb.ERR_SHAPE           # Hd > 1024
+    assert lib.reflex_adarmsnorm_gate(fake, fake, fake, fake, fake, None, 1, 1, 128, 8, 8, 0, None) == rb.ERR_INVALID_ARG
     # cache calls with a NULL handle
     assert lib.reflex_partitioned_attention(None, 0, fake, fake, fake, fake, 1, 0.0, 0, None) == rb.ERR_INVALID_ARG
     assert lib.reflex_cache_init_static(None, None, 0, fake, fake, 0, None, None) == rb.ERR_INVALID_ARG
