@@ -619,6 +619,8 @@ def main():
                                    "roofline": roofline_of(alg5["attn_flops_per_launch"], alg5["attn_bytes_per_launch"], m5["us"] * 1e-6, peaks,
                                                            "sustained" if "sustained" in a5 else "burst"),
                                    "roofline_burst": roofline_of(alg5["attn_flops_per_launch"], alg5["attn_bytes_per_launch"], a5["burst"]["us"] * 1e-6, peaks, "burst")}
+        t5, src5 = ncu_traffic(w5, args.attn)
+        extra["cfg5_attention"]["roofline"].update({"traffic": t5, "traffic_source": src5, "bytes_per_launch": alg5["attn_bytes_per_launch"]})
         rb.reflex_cache_check_status(r5.cache)
         del r5
     sampler.stop()
