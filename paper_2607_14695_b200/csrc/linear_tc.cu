@@ -341,12 +341,17 @@ cudaError_t launch_linear_residual(const void *a, const void *W, const void *res
         return dtype == REFLEX_DTYPE_BF16 ? launch_lin_simt<__nv_bfloat16>(a, W, res, out, M, K, N, st) : launch_lin_simt<float>(a, W, res, out, M, K, N, st);
     }
     if (impl == 0 && M <= 128 && K % 64 == 0) return launch_linear_small(a, W, res, out, M, K, N, status, st);
-    CUtensorMap ma, mw, mr, mo;
-    if (!tensor_map_2d_bf16(&ma, a, K, M, kLinBM) || !tensor_map_2d_bf16(&mw, W, K, N, 128) || !tensor_map_2d_bf16(&mo, out, N, M, kLinBM)) return cudaErrorInvalidValue;
-    if (res) { if (!tensor_map_2d_bf16(&mr, res, N, M, kLinBM)) return cudaErrorInvalidValue; }
-    else mr = mo;
     LinParams p;
     p.M = M; p.K = K; p.N = N; p.m_tiles = (M + 2 * kLinBM - 1) / (2 * kLinBM); p.has_res = res ? 1 : 0; p.status = status;
+    // 256-column tiles unless they would leave more than half of the SM pairs without one: then 128-column tiles, twice as
+    // many pairs at work on a contraction that is as long (every CTA then fetches 24 KB per step for half the MMA work)
+    const bool narrow = p.m_tiles * ((N + 255) / 256) * 2 <= 74;
+    CUtensorMap ma, mw, mr, mo;
+    if (!tensor_map_2d_bf16(&ma, a, K, M, kLinBM) || !tensor_map_2d_bf16(&mw, W, K, N, narrow ? 64 : 128) || !tensor_map_2d_bf16(&mo, out, N, M, kLinBM))
+        return cudaErrorInvalidValue;
+    if (res) { if (!tensor_map_2d_bf16(&mr, res, N, M, kLinBM)) return cudaErrorInvalidValue; }
+    else mr = mo;
+    if (narrow) return launch_lin_tc<128>(ma, mw, mr, mo, p, (N + 127) / 128, st);
     return launch_lin_tc<256>(ma, mw, mr, mo, p, (N + 255) / 256, st);
 }
 
