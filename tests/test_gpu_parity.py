@@ -774,6 +774,8 @@ def test_linear_residual_bf16_ragged_shapes(U):
     _linear_case(U, synth.DTYPE_BF16, 300, 200, 328, 0, "linear ragged")
     _linear_case(U, synth.DTYPE_BF16, 300, 200, 328, 0, "linear ragged, no residual", residual=False)
     _linear_case(U, synth.DTYPE_BF16, 129, 64, 8, 0, "linear one step, 8 columns")
+    _linear_case(U, synth.DTYPE_BF16, 130, 8, 72, 0, "linear contraction of 8 (narrower than a 64-column step)")
+    _linear_case(U, synth.DTYPE_BF16, 40, 72, 136, 0, "linear few rows, contraction not a multiple of 64 (256-row tile path)")
     # enough row tiles for the 256-column tiles (the smaller problems above take 128-column tiles): 2600 rows, a ragged last
     # row tile, three contraction steps
     _linear_case(U, synth.DTYPE_BF16, 2600, 192, 1024, 0, "linear 256-column tiles", in_place=True, rows=[0, 255, 256, 1300, 2559, 2560, 2599])
