@@ -9,9 +9,9 @@
 // buffer of its own; the epilogue threads (two per row) take it into registers while the last stages are multiplied, add
 // the accumulator (fp32 add, one rounding to bf16) and write the result back into the same buffer, which leaves through
 // TMA stores (they clip rows and columns past the end). out may alias res: a tile is read and written by one CTA only.
-// What bounds the kernel: without multicast every CTA fetches its own operand tiles, 52 tiles x 64 KB per contraction step
-// = 105 MB through the L2 for the 3200 x 1024 x 2048 problem, and the L2 delivers about 10 TB/s: 10.5 us for the main loop
-// against 8.3 us of tensor-pipe time.
+// What bounds the kernel: without multicast every CTA fetches its own operand tiles, 32 KB per contraction step against
+// 512 cycles of MMAs = 64 B/clk, and an SM takes in 50 to 58 B/clk from the L2: 10.75 us for the main loop of the
+// 3200 x 1024 x 2048 problem against 8.3 us of tensor-pipe time.
 // The contraction is long (2048 or 4096) and the output small (3200 x 1024 at 64 streams): 52 tiles on 74 SM pairs in
 // one wave, so the kernel is not persistent.
 //
@@ -192,8 +192,8 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // The residual tile comes in by TMA behind the last operand tiles; every thread takes its BN / 2 columns of its row
         // out of shared memory into registers while the last stages are multiplied, so that after the accumulator is final
         // only tensor-memory loads, adds and the stores into the same staging buffer remain. (As global loads by these
-        // threads, 16 bytes per row and instruction, the residual cost the main loop 2.5 us: the L2's bandwidth is what
-        // limits this kernel, and half-used sectors waste it.)
+        // threads, 16 bytes per row and instruction, the residual cost the main loop 2.5 us: what an SM takes in from
+        // the L2 is what limits this kernel, and half-used sectors waste it.)
         bool ok = wait(S::C_RES, 0u, 3);
         constexpr int CPT = BN / 2 / 64;              // 64-column chunks per thread
         uint4 rr[CPT * 8];
