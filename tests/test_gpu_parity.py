@@ -274,7 +274,7 @@ def test_cfg5b_outliers_in_queries_and_keys(U):
     vd = synth.normal(w, "v_dyn", (w.B, w.T, w.Hkv, w.d), 0, 0)
     assert (np.abs(q) > 100).any() and (np.abs(ks) > 100).any() and (np.abs(kd) > 100).any()
     worst_rel = 0.0
-    for impl in (rb.ATTN_AUTO, rb.ATTN_SIMT):
+    for impl in (rb.ATTN_AUTO, rb.ATTN_TC, rb.ATTN_SIMT):
         rb.reflex_cache_set_attention_impl(tw.g, impl)
         for dyn_mask in (0, 1):
             out = torch.full((w.B, w.T, w.Hq, w.d), float("nan"), dtype=torch.bfloat16, device=U.DEV)
