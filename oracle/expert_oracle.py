@@ -10,15 +10,16 @@ from . import reflex_oracle as orc
 
 
 def expert_step(ocache: "orc.OracleCache", W: dict, a: np.ndarray, cond: np.ndarray, K: int, Hq: int, Hkv: int, d: int, F: int,
-                eps: float = 1e-6, dyn_mask: int = 0):
-    """a [B][T][A] float64 (returned updated), cond [B][Cd]. Returns (a_new, v)."""
+                eps: float = 1e-6, dyn_mask: int = 0, streams=None):
+    """a [B][T][A] float64 (returned updated), cond [B][Cd]. Returns (a_new, v). streams: compute these streams only (the
+    streams are independent; the others keep their chunk and a zero velocity)."""
     B, T, A = a.shape
     L = W["Wqkv"].shape[0]
     f64 = lambda x: np.asarray(x, np.float64)
     f32 = lambda x: np.asarray(x, np.float32)
     a_new = a.copy()
-    v_all = np.empty_like(a)
-    for b in range(B):
+    v_all = np.zeros_like(a)
+    for b in (range(B) if streams is None else streams):
         h = a[b] @ f64(W["W_in"]).T                                             # [T][D]
         for l in range(L):
             g1 = (W["W1"][2 * l], W["b1"][2 * l], W["W2"][2 * l], W["b2"][2 * l])

@@ -871,7 +871,7 @@ def test_context_window_and_chunk_sweep(U, frames, T):
 # ------------------------------------------------------------------------------------------------
 # a whole action-expert denoising step chained from the library's calls
 # ------------------------------------------------------------------------------------------------
-def _expert_case(U, w, F, tol_v, what):
+def _expert_case(U, w, F, tol_v, what, streams=None):
     from oracle import expert_oracle as eo
     from paper_2607_14695_b200 import expert as ex
     rb = U.rb
@@ -889,8 +889,11 @@ def _expert_case(U, w, F, tol_v, what):
     a_gpu = torch.from_numpy(a0.astype(np.float32)).to(U.DEV)
     model.step(a_gpu, U.to_dev(cond, w.dtype), 1)
     rb.reflex_cache_check_status(tw.g)
-    want_a, want_v = eo.expert_step(tw.o, W, a0, cond, w.K, w.Hq, w.Hkv, w.d, F)
+    want_a, want_v = eo.expert_step(tw.o, W, a0, cond, w.K, w.Hq, w.Hkv, w.d, F, streams=streams)
     got_v = U.to_host(model.vel)
+    if streams is not None:          # a sample of the (independent) streams
+        got_v, want_v, want_a = got_v[streams], want_v[streams], want_a[streams]
+        a_gpu = a_gpu[streams]
     rel = np.linalg.norm(got_v - want_v) / np.linalg.norm(want_v)
     assert np.isfinite(got_v).all() and rel <= tol_v, f"{what}: velocity off by {rel:.3e} (relative Frobenius)"
     # element by element: the roundings that accumulate along the chain are independent, so an element's error is spread
@@ -914,6 +917,13 @@ def test_expert_step_bf16(U):
     accumulate; the velocity stays within 2 % of the double-precision chain."""
     w = synth.CONFIGS["cfg2"].with_(B=2, L=2, S=200, S_max=208)
     _expert_case(U, w, 1024, 2e-2, "expert bf16")
+
+
+def test_expert_step_bf16_batched(U):
+    """The same two-layer step for 64 streams (3200 rows: the 256-row tiles of every projection kernel, the two-CTA attention
+    in its batched form), three streams compared."""
+    w = synth.CONFIGS["cfg4"].with_(L=2, S=200, S_max=208)
+    _expert_case(U, w, 1024, 2e-2, "expert bf16, 64 streams", streams=[0, 31, 63])
 
 
 @pytest.mark.parametrize("B", [1, 2])
