@@ -14,7 +14,7 @@
 //           warp 1      MMA issuer (leader CTA only): S = Q K^T (M256 N128), O += P V (M256 N=d)
 //           warps 2..   softmax over this CTA's 128 rows x 128 keys: NP threads per row (128 / NP keys each),
 //                       P (bf16) written back into tensor memory over the logits it came from, lazy rescale
-//                       of O in tensor memory, and the epilogue: O / l straight from registers to global memory
+//                       of O in tensor memory, and the epilogue: O / l through a 32 KB staging area and TMA stores
 // P never touches shared memory: P V takes its A operand from tensor memory. With head_dim 256 the Q K^T
 // MMAs alone read shared memory at its full bandwidth (a 4 KB slice of Q plus 4 KB of K per 64-cycle
 // instruction), so every byte of shared-memory traffic that is not an operand read or a TMA fill stretches
