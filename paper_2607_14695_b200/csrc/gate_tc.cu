@@ -55,8 +55,16 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     const uint32_t bar_load = base + S::OFF_BAR, bar_mma = bar_load + 8;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + S::OFF_BAR + 16);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int layer = blockIdx.z, u0 = blockIdx.x * kGtUnits, b0 = blockIdx.y * kGtStreams;
+    const int layer = blockIdx.z, u0 = blockIdx.x * kGtUnits;
     const int chunks = (len + 63) / 64, ksteps = len / 16;
+    // A CTA keeps its 128 weight rows in shared memory and walks the groups of 64 streams that fall to it (blockIdx.y takes
+    // a contiguous share of the groups): with many streams -- the conditioning vectors of all steps of a control tick
+    // stacked -- the weights are fetched once per CTA instead of once per group, and the next group's vectors come in
+    // while this group's results are stored.
+    const int n_groups = (B + kGtStreams - 1) / kGtStreams;
+    const int gpc = (n_groups + (int)gridDim.y - 1) / (int)gridDim.y;
+    const int g_first = (int)blockIdx.y * gpc;
+    const int ng = max(0, min(n_groups, g_first + gpc) - g_first);
 
     if (threadIdx.x == 0) {
         mbar_init(bar_load, 1);
@@ -74,79 +82,93 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    auto wait = [&](uint32_t bar, uint32_t code) -> bool {
-        if (mbar_try_wait(bar, 0)) return true;
+    auto wait = [&](uint32_t bar, uint32_t parity, uint32_t code) -> bool {
+        if (mbar_try_wait(bar, parity)) return true;
         const unsigned long long t_start = globaltimer_ns();
         for (uint32_t n = 1;; ++n) {
-            if (mbar_try_wait(bar, 0)) return true;
+            if (mbar_try_wait(bar, parity)) return true;
             if ((n & 255u) == 0u && globaltimer_ns() - t_start > kGtWaitNs) break;
         }
         if (status) atomicCAS(status, 0u, 0x80000000u | ((code + 64u) << 16) | (blockIdx.x & 0xFFFFu));
         return false;
     };
+    auto load_vectors = [&](int g) {   // the (up to) 64 vectors of group g, one or two bf16 arrays
+        for (int c = 0; c < chunks; ++c) {
+            tma_load_2d(base + S::OFF_B + c * S::B_CHUNK, &tm_v0, bar_load, c * 64, layer * vec_rows_per_layer + g * kGtStreams);
+            if (PASSES == 2)
+                tma_load_2d(base + S::OFF_B + (kGtMaxChunks + c) * S::B_CHUNK, &tm_v1, bar_load, c * 64, layer * vec_rows_per_layer + g * kGtStreams);
+        }
+    };
 
     bool ok = true;
-    if (warp == 0) {
-        // the whole warp stays converged; one elected lane loads and issues
-        if (lane == 0) {
-            mbar_expect_tx(bar_load, (uint32_t)chunks * (S::A_CHUNK + PASSES * S::B_CHUNK));
-            for (int c = 0; c < chunks; ++c) {
-                tma_load_2d(base + S::OFF_A + c * S::A_CHUNK, &tm_w, bar_load, c * 64, layer * units + u0);
-                tma_load_2d(base + S::OFF_B + c * S::B_CHUNK, &tm_v0, bar_load, c * 64, layer * vec_rows_per_layer + b0);
-                if (PASSES == 2)
-                    tma_load_2d(base + S::OFF_B + (kGtMaxChunks + c) * S::B_CHUNK, &tm_v1, bar_load, c * 64, layer * vec_rows_per_layer + b0);
-            }
-        }
-        ok = wait(bar_load, 1);
-        tc_fence_after();
-        if (ok) {
-            constexpr uint32_t idesc = umma_idesc_bf16(kGtUnits, kGtStreams, false);
-#pragma unroll 1
-            for (int pass = 0; pass < PASSES; ++pass) {
-#pragma unroll 1
-                for (int kk = 0; kk < ksteps; ++kk) {
-                    const uint32_t a = base + S::OFF_A + (kk >> 2) * S::A_CHUNK + (kk & 3) * 32;
-                    const uint32_t b = base + S::OFF_B + (pass * kGtMaxChunks + (kk >> 2)) * S::B_CHUNK + (kk & 3) * 32;
-                    umma_ss_elect(tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(b, 16, 1024), idesc, (pass > 0 || kk > 0) ? 1u : 0u);
-                }
-            }
-        }
-        umma_commit_elect(bar_mma);   // also when the load never came: the other warps must not wait for nothing
+    if (warp == 0 && lane == 0 && ng > 0) {
+        mbar_expect_tx(bar_load, (uint32_t)chunks * (S::A_CHUNK + PASSES * S::B_CHUNK));
+        for (int c = 0; c < chunks; ++c) tma_load_2d(base + S::OFF_A + c * S::A_CHUNK, &tm_w, bar_load, c * 64, layer * units + u0);
+        load_vectors(g_first);
     }
-    ok = wait(bar_mma, 2) && ok;
-    tc_fence_after();
-    // epilogue: thread = weight row (TMEM lane), 64 columns = streams
     const int u = u0 + warp * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-    uint32_t acc[64];
-    tmem_ld32(tmem + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(acc));
-    tmem_ld32(tmem + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(acc + 32));
-    tmem_wait_ld();
-    if (!ok && u < units) {
-        // a bounded wait ran out: this CTA's slice of the output is marked invalid (quiet NaN) instead of keeping the previous
-        // call's values, so whatever consumes the gates shows it
-        const int nb = min(kGtStreams, B - b0);
-        for (int n = 0; n < nb; ++n) {
-            const size_t o = ((size_t)layer * B + b0 + n) * units + u;
-            if (SILU) { out_hi[o] = __float2bfloat16_rn(__int_as_float(0x7fc00000)); out_lo[o] = __float2bfloat16_rn(0.f); }
-            else out_f32[o] = __int_as_float(0x7fc00000);
+    const float bi = u < units ? __bfloat162float(bias[(size_t)layer * units + u]) : 0.f;
+#pragma unroll 1
+    for (int i = 0; i < ng; ++i) {
+        const int b0 = (g_first + i) * kGtStreams;
+        const uint32_t ph = (uint32_t)i & 1u;
+        if (warp == 0) {
+            // the whole warp stays converged; one elected lane issues
+            ok = ok && wait(bar_load, ph, 1);
+            tc_fence_after();
+            if (ok) {
+                constexpr uint32_t idesc = umma_idesc_bf16(kGtUnits, kGtStreams, false);
+#pragma unroll 1
+                for (int pass = 0; pass < PASSES; ++pass) {
+#pragma unroll 1
+                    for (int kk = 0; kk < ksteps; ++kk) {
+                        const uint32_t a = base + S::OFF_A + (kk >> 2) * S::A_CHUNK + (kk & 3) * 32;
+                        const uint32_t b = base + S::OFF_B + (pass * kGtMaxChunks + (kk >> 2)) * S::B_CHUNK + (kk & 3) * 32;
+                        umma_ss_elect(tmem, umma_desc_sw128(a, 16, 1024), umma_desc_sw128(b, 16, 1024), idesc, (pass > 0 || kk > 0) ? 1u : 0u);
+                    }
+                }
+            }
+            umma_commit_elect(bar_mma);   // also when the load never came: the other warps must not wait for nothing
         }
-    }
-    if (ok && u < units) {
-        const float bi = __bfloat162float(bias[(size_t)layer * units + u]);
+        ok = wait(bar_mma, ph, 2) && ok;
+        tc_fence_after();
+        // the MMAs that read this group's vectors are complete: the next group's may land on them
+        if (warp == 0 && lane == 0 && i + 1 < ng) {
+            mbar_expect_tx(bar_load, (uint32_t)chunks * (PASSES * S::B_CHUNK));
+            load_vectors(g_first + i + 1);
+        }
+        // epilogue: thread = weight row (TMEM lane), 64 columns = streams
+        uint32_t acc[64];
+        tmem_ld32(tmem + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(acc));
+        tmem_ld32(tmem + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(acc + 32));
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncthreads();      // every warp holds its accumulators in registers: the next group's MMAs may overwrite them
         const int nb = min(kGtStreams, B - b0);
+        if (!ok && u < units) {
+            // a bounded wait ran out: this CTA's slice of the output is marked invalid (quiet NaN) instead of keeping the
+            // previous call's values, so whatever consumes the gates shows it
+            for (int n = 0; n < nb; ++n) {
+                const size_t o = ((size_t)layer * B + b0 + n) * units + u;
+                if (SILU) { out_hi[o] = __float2bfloat16_rn(__int_as_float(0x7fc00000)); out_lo[o] = __float2bfloat16_rn(0.f); }
+                else out_f32[o] = __int_as_float(0x7fc00000);
+            }
+        }
+        if (ok && u < units) {
 #pragma unroll
-        for (int n = 0; n < kGtStreams; ++n) {
-            if (n >= nb) continue;   // (fully unrolled: the accumulator stays in registers)
-            const float z = __uint_as_float(acc[n]) + bi;
-            const size_t o = ((size_t)layer * B + b0 + n) * units + u;
-            if (SILU) {
-                const float h = z / (1.f + expf(-z));
-                const __nv_bfloat16 hi = __float2bfloat16_rn(h);
-                out_hi[o] = hi;
-                out_lo[o] = __float2bfloat16_rn(h - __bfloat162float(hi));
-            } else {
-                out_f32[o] = 1.f + z;
+            for (int n = 0; n < kGtStreams; ++n) {
+                if (n >= nb) continue;   // (fully unrolled: the accumulator stays in registers)
+                const float z = __uint_as_float(acc[n]) + bi;
+                const size_t o = ((size_t)layer * B + b0 + n) * units + u;
+                if (SILU) {
+                    const float h = z / (1.f + expf(-z));
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(h);
+                    out_hi[o] = hi;
+                    out_lo[o] = __float2bfloat16_rn(h - __bfloat162float(hi));
+                } else {
+                    out_f32[o] = 1.f + z;
+                }
             }
         }
     }
@@ -165,7 +187,12 @@ cudaError_t launch_one(const CUtensorMap &mw, const CUtensorMap &mv0, const CUte
     });
     if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((units + kGtUnits - 1) / kGtUnits, (B + kGtStreams - 1) / kGtStreams, L);
+    // groups of 64 streams are spread over blockIdx.y only as far as that adds CTAs the SMs can hold at once; beyond, a CTA
+    // walks several groups with its weights resident
+    const int ux = (units + kGtUnits - 1) / kGtUnits, n_groups = (B + kGtStreams - 1) / kGtStreams;
+    int gy = 148 / (ux * L);
+    gy = gy < 1 ? 1 : (gy > n_groups ? n_groups : gy);
+    cfg.gridDim = dim3(ux, gy, L);
     cfg.blockDim = dim3(128);
     cfg.dynamicSmemBytes = GateTcSmem::TOTAL;
     cfg.stream = st;
