@@ -79,6 +79,17 @@ __device__ long long g_qk_trace[3 * 32 * 8];
 #define QK_TRACE(role, step, ev) do { } while (0)
 #endif
 
+// SiLU(g) * u with one special-function operation per element: g / (1 + e^-g) = g (1 + tanh(g / 2)) / 2. The epilogue of the
+// gate/up kernel is bound by the special-function unit (16 results per clock and SM; 32 K elements per tile): with an
+// exponential and a reciprocal per element it took 7.7 k cycles of a 26 k-cycle tile. tanh.approx is accurate to about 2^-11,
+// a quarter of the spacing of the bf16 the result is rounded to.
+__device__ __forceinline__ float silu_mul(float g, float u)
+{
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
+    return fmaf(t, 0.5f * g, 0.5f * g) * u;
+}
+
 __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1)
 {
     asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -288,7 +299,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         const float g = __uint_as_float(acc[i]) * rs, u = __uint_as_float(up[i]) * rs;
-                        acc[i] = __float_as_uint(__fdividef(g, 1.f + __expf(-g)) * u);
+                        acc[i] = __float_as_uint(silu_mul(g, u));
                     }
                 } else {
                     tmem_wait_ld();
@@ -617,7 +628,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
                 if (r < p.M) {                      // (no early exit: the accumulator stays in registers)
                     const float rs = rsm[r];
                     float val = __uint_as_float(acc[i]) * rs;
-                    if (swiglu) { const float u = __uint_as_float(up[i]) * rs; val = __fdividef(val, 1.f + __expf(-val)) * u; }
+                    if (swiglu) { const float u = __uint_as_float(up[i]) * rs; val = silu_mul(val, u); }
                     if constexpr (PLAIN) { if (p.res) val += __bfloat162float(p.res[(size_t)r * pitch + f]); }
                     dst0[(size_t)r * pitch] = __float2bfloat16_rn(val);     // a warp writes 64 contiguous bytes per row
                 }
@@ -677,7 +688,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
                 } else {
                     const float rs = rs_mine[r - r0];
                     sum *= rs;
-                    if (swiglu) sum = __fdividef(sum, 1.f + __expf(-sum)) * (sum_up * rs);
+                    if (swiglu) sum = silu_mul(sum, sum_up * rs);
                 }
                 *dst = __float2bfloat16_rn(sum);
             }
