@@ -70,6 +70,7 @@ struct QkParams {
     uint32_t *status;
     const __nv_bfloat16 *res;   // plain projection only (few-rows kernel with PLAIN): residual [M][nq] added to the output, or NULL
     int ksplit;                 // few-rows kernel: CTAs of a cluster that share one feature tile, each taking a slice of the contraction
+    int tma_out;                // 256-row kernel: the output tile leaves through TMA stores (tensor maps over q / k / v given)
 };
 
 #ifdef REFLEX_QK_TRACE
@@ -90,6 +91,11 @@ __device__ __forceinline__ float silu_mul(float g, float u)
     return fmaf(t, 0.5f * g, 0.5f * g) * u;
 }
 
+__device__ __forceinline__ void qk_tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+
 __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1)
 {
     asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -99,7 +105,8 @@ __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *ma
 
 template <int NACC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kQkThreads, 1)
-norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, QkParams p)
+norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
+                   const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QkParams p)
 {
     using S = QkSmem<NACC>;
     extern __shared__ uint8_t smem_raw[];
@@ -280,6 +287,66 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         tc_fence_after();
         const float rs = rsqrtf(ss / (float)p.D + p.eps);
         const int n_out = p.nq + 2 * p.nk;
+        if (p.tma_out) {
+            // The tile goes out through shared memory and TMA stores. The stage ring is idle now (every load has been consumed and
+            // every MMA has completed): accumulator j is staged in the x stages (j = 0) or the weight stages (j = 1) as four
+            // chunks of 128 rows x 64 columns in the layout of a 128-byte-swizzled TMA box, each thread dropping its half row,
+            // scaled and rounded, as 16-byte pieces; a chunk is handed to the TMA engine as soon as the 128 threads that fill it
+            // are through, and the stores drain while the next chunk is converted. (With every warp copying whole rows from
+            // the staging area to global memory the epilogue took 6.4 k cycles of a 25 k-cycle tile.)
+            static_assert(S::OFF_B - S::OFF_X >= 4u * 128u * 128u && S::OFF_BAR - S::OFF_B >= 4u * 128u * 128u, "staging areas of the epilogue");
+#pragma unroll 1
+            for (int j = 0; j < (swiglu ? 1 : NACC); ++j) {
+                const uint32_t stage_off = j == 0 ? S::OFF_X : S::OFF_B;
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int ch = half * 2 + cc;                 // 64-column chunk of the accumulator
+                    uint8_t *rowp = smem + stage_off + ch * (128 * 128) + row * 128;
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t acc[32];
+                        tmem_ld32(tmem + lane_addr + j * kQkBN + ch * 64 + g * 32, acc);   // warp-wide: every lane takes part, whatever its row
+                        if (swiglu) {     // (uniform) the up projection of the same columns; acc <- SiLU(g) * u, both scaled by 1/RMS first
+                            uint32_t up[32];
+                            tmem_ld32(tmem + lane_addr + kQkBN + ch * 64 + g * 32, up);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(silu_mul(__uint_as_float(acc[i]) * rs, __uint_as_float(up[i]) * rs));
+                        } else {
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * rs);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 o;
+                            uint32_t *oo = reinterpret_cast<uint32_t *>(&o);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(acc[8 * i + 2 * k]), __uint_as_float(acc[8 * i + 2 * k + 1]));
+                                oo[k] = *reinterpret_cast<uint32_t *>(&h);
+                            }
+                            // 128-byte swizzle of the TMA box: 16-byte piece p of row r sits at p ^ (r % 8)
+                            *reinterpret_cast<uint4 *>(rowp + (((g * 4 + i) ^ (row & 7)) << 4)) = o;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    asm volatile("bar.sync %0, 128;" ::"r"(2 + half) : "memory");   // the chunk's 128 threads
+                    if (quarter == 0 && lane == 0 && ok && m0 < p.M) {
+                        const int n = n0 + j * kQkBN + ch * 64;     // first output column of the chunk (chunks never straddle Q, K and V:
+                                                                    // the launcher takes this path only when their widths are multiples of 64)
+                        const uint32_t src = base + stage_off + ch * (128 * 128);
+                        if (swiglu) { if (n < p.swiglu_F) qk_tma_store_2d(&tm_q, src, n, m0); }
+                        else if (n < p.nq) qk_tma_store_2d(&tm_q, src, n, m0);
+                        else if (n < p.nq + p.nk) qk_tma_store_2d(&tm_k, src, n - p.nq, m0);
+                        else if (n < n_out) qk_tma_store_2d(&tm_v, src, n - p.nq - p.nk, m0);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                }
+            }
+            // (the staging areas have been read; the writes themselves are complete when the grid is)
+            if (quarter == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        } else {
         // The tile goes out through shared memory (the stage ring is idle now: every load has been consumed and every MMA
         // has completed): each thread drops its half row, scaled and rounded, as 16-byte pieces at [row][piece ^ (row % 32)]
         // (conflict-free for 32 rows at a time), then every warp writes whole 512-byte rows, 16 bytes per lane. (Straight
@@ -337,6 +404,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 }
             }
             if (j + 1 < (swiglu ? 1 : NACC)) asm volatile("bar.sync 1, 256;" ::: "memory");   // the staging area is rewritten by the next round
+        }
         }
     }
 
@@ -803,6 +871,15 @@ bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk)
 template <int NACC>
 static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_tiles, cudaStream_t st)
 {
+    // tensor maps over the outputs when every tensor's width is a multiple of the 64-column chunks the epilogue stores
+    CUtensorMap mq = mx, mk = mx, mv = mx;
+    p.tma_out = 0;
+    if (p.swiglu_F > 0) {
+        p.tma_out = tensor_map_2d_bf16(&mq, p.q, p.swiglu_F, p.M, kQkBM) ? 1 : 0;
+    } else if (p.nq % 64 == 0 && p.nk % 64 == 0) {
+        p.tma_out = (tensor_map_2d_bf16(&mq, p.q, p.nq, p.M, kQkBM) && tensor_map_2d_bf16(&mk, p.k, p.nk, p.M, kQkBM) &&
+                     tensor_map_2d_bf16(&mv, p.v, p.nk, p.M, kQkBM)) ? 1 : 0;
+    }
     static std::atomic<unsigned long long> attr_set{0};
     cudaError_t e0 = once_per_device(attr_set, [] {
         return cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
@@ -818,7 +895,7 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel<NACC>, mx, mw, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel<NACC>, mx, mw, mq, mk, mv, p);
     count_launch();
     return e;
 }
@@ -871,7 +948,7 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
         QkParams sp;
         sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
         sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.swiglu_F = swiglu_F;
-        sp.eps = eps; sp.status = status; sp.res = nullptr;
+        sp.eps = eps; sp.status = status; sp.res = nullptr; sp.tma_out = 0;
         const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
         // The contraction split over 4 CTAs per feature tile where the chain of steps is long enough to pay for a cluster
         // launch and its two barriers (16 steps or more: SwiGLU at D = 1024, 11.1 -> 10.0 us for one stream; the packed
@@ -892,7 +969,7 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
     p.M = M; p.R = R; p.B = B; p.D = D; p.nq = nq; p.nk = nk;
     p.m_tiles = (M + 2 * kQkBM - 1) / (2 * kQkBM);
     p.swiglu_F = swiglu_F;
-    p.eps = eps; p.status = status; p.res = nullptr; p.ksplit = 1;
+    p.eps = eps; p.status = status; p.res = nullptr; p.ksplit = 1; p.tma_out = 0;
     if (swiglu_F > 0) return launch_tc<2>(mx, mw, p, (swiglu_F + kQkBN - 1) / kQkBN, st);
     int nacc = qk_choose_nacc(M, R, D, nq + 2 * nk, sm_count > 0 ? sm_count : 148);
     if (impl == 2 && nacc == 2) nacc = 1;     // (forced 256-column tiles, for tests and timing)
@@ -909,7 +986,7 @@ cudaError_t launch_linear_small(const void *a, const void *W, const void *res, v
     QkParams sp;
     sp.gate = nullptr; sp.q = (__nv_bfloat16 *)out; sp.k = nullptr; sp.v = nullptr;
     sp.M = M; sp.R = M; sp.B = 1; sp.D = K; sp.nq = N; sp.nk = 0; sp.m_tiles = 1; sp.swiglu_F = 0;
-    sp.eps = 0.f; sp.status = status; sp.res = (const __nv_bfloat16 *)res;
+    sp.eps = 0.f; sp.status = status; sp.res = (const __nv_bfloat16 *)res; sp.tma_out = 0;
     // split the contraction over up to 8 CTAs per feature tile while every slice keeps whole steps of two 64-column chunks and
     // the grid stays within the SMs
     const int chunks = K / kQkBK, ftiles = (N + 127) / 128;
