@@ -20,7 +20,9 @@
 //
 // The same kernel serves the fused gate / up projections of a SwiGLU block (Sec. 3.3: "combine the Gate and Up projections"):
 // accumulator 0 takes 256 rows of W_gate, accumulator 1 the same rows of W_up, and the epilogue writes
-// SiLU(gate) * up for those 256 hidden columns (swiglu_F > 0 in the parameters).
+// SiLU(gate) * up for those 256 hidden columns (swiglu_F > 0 in the parameters). With more tiles than SM pairs (3200 rows x
+// 4096 hidden columns: 208) the grid is one CTA pair per SM pair and every pair walks its tiles (WALK): 48.8 -> 44.7 us,
+// the loads of a tile's first steps and the set-up of a wave no longer waiting behind the last tile's epilogue.
 //
 // Any other dtype or shape: a plain kernel (one block per row, fp32 FMAs) with the same semantics.
 #include <cuda.h>
@@ -58,13 +60,14 @@ struct QkSmem {
     static constexpr uint32_t TOTAL = OFF_GATE + GATE_MAX + 1024;   // + slack for the 1024-byte alignment
     static_assert(TOTAL <= 227u * 1024u, "shared memory budget");
 };
-enum { Q_XFULL = 0, Q_BFULL = kQkStages, Q_AREADY = 2 * kQkStages, Q_EMPTY = 3 * kQkStages, Q_ACC = 4 * kQkStages, Q_COUNT };
+enum { Q_XFULL = 0, Q_BFULL = kQkStages, Q_AREADY = 2 * kQkStages, Q_EMPTY = 3 * kQkStages, Q_ACC = 4 * kQkStages, Q_ACCFREE, Q_STAGEFREE, Q_COUNT };
 
 struct QkParams {
     const float *gate;          // [B][D]
     __nv_bfloat16 *q, *k, *v;   // [M][nq], [M][nk], [M][nk]
     int M, R, B, D, nq, nk;     // M = B * R rows; nq = Hq * d, nk = Hkv * d
     int m_tiles;                // 256-row tiles
+    int n_tiles;                // column tiles (256-row kernel: a CTA pair walks tiles pair, pair + pairs, ... of m_tiles x n_tiles)
     int swiglu_F;               // 0: columns go to Q, K, V. F > 0: W holds [W_gate; W_up] ([2F][D]), out (= q, pitch nq = F) gets SiLU(g) * u
     float eps;
     uint32_t *status;
@@ -103,7 +106,7 @@ __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *ma
                  : "memory");
 }
 
-template <int NACC>
+template <int NACC, bool WALK>      // WALK: more tiles than CTA pairs (otherwise one tile per pair, and the tile loops fold away)
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kQkThreads, 1)
 norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
                    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, QkParams p)
@@ -119,10 +122,18 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1;
-    const int m0 = (pair % p.m_tiles) * (2 * kQkBM) + (int)rank * kQkBM;   // this CTA's first row
     const bool swiglu = NACC == 2 && p.swiglu_F > 0;
-    const int n0 = (pair / p.m_tiles) * (swiglu ? kQkBN : NACC * kQkBN);   // the pair's first output column
     const int nk_steps = p.D / kQkBK;
+    // A pair takes tiles pair, pair + pairs, ... (row tiles fastest, so that the pairs working at the same time share weight
+    // rows in L2). With more tiles than pairs the grid is one pair per SM pair and the roles below run ahead of each other
+    // across tile boundaries: the producer refills the weight stages and the tensor pipe starts the next tile's first
+    // steps while the eight warps still convert and store the last tile. The stage ring, its barrier phases and the
+    // accumulator hand-over all count steps and tiles from the start of the kernel.
+    const int n_pairs = (int)(gridDim.x >> 1);
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int my_tiles = !WALK ? 1 : pair < total_tiles ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+    auto tile_m0 = [&](int it) -> int { return ((pair + it * n_pairs) % p.m_tiles) * (2 * kQkBM) + (int)rank * kQkBM; };    // this CTA's first row
+    auto tile_n0 = [&](int it) -> int { return ((pair + it * n_pairs) / p.m_tiles) * (swiglu ? kQkBN : NACC * kQkBN); };   // the pair's first output column
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kQkStages; ++s) {
@@ -132,6 +143,8 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             mbar_init(bar(Q_EMPTY + s), 1);
         }
         mbar_init(bar(Q_ACC), 1);
+        mbar_init(bar(Q_ACCFREE), 16);      // one arrival per epilogue warp of either CTA: the accumulators have been read
+        mbar_init(bar(Q_STAGEFREE), 2);     // the two threads that hand this CTA's staged chunks to the TMA engine: all of them read
         *abort_flag = 0u;
         fence_mbar_init();
         prefetch_tmap(&tm_x); prefetch_tmap(&tm_w);
@@ -167,18 +180,51 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
             bool ok = true;
-            for (int ks = 0; ks < nk_steps && ok; ++ks) {
-                const int s = ks % kQkStages;
-                if (ks >= kQkStages) ok = wait(Q_EMPTY + s, (uint32_t)(ks / kQkStages - 1) & 1u, 1);
-                if (!ok) break;
-                QK_TRACE(0, ks, 0);
-                mbar_expect_tx(bar(Q_XFULL + s), S::X_STAGE);
-                tma_load_2d(base + S::OFF_X + s * S::X_STAGE, &tm_x, bar(Q_XFULL + s), ks * kQkBK, m0);
-                if (rank == 0) mbar_expect_tx(bar(Q_BFULL + s), 2 * S::B_STAGE);
+            // the epilogue stages accumulator 0 in the x stages and (packed projection, two accumulators) accumulator 1 in the
+            // weight stages: loads into either wait until the last tile's stores have read them
+            const bool w_staged = !swiglu && NACC == 2;
+            for (int it = 0; it < my_tiles && ok; ++it) {
+                const int m0 = tile_m0(it), n0 = tile_n0(it);
+                const int g0 = it * nk_steps;
+                auto stage_free = [&](int ks) -> bool {     // the MMAs that read the stage of step ks four steps ago are complete
+                    const int g = g0 + ks;
+                    return g < kQkStages || wait(Q_EMPTY + g % kQkStages, (uint32_t)(g / kQkStages - 1) & 1u, 1);
+                };
+                auto load_x = [&](int ks) {
+                    const int s = (g0 + ks) % kQkStages;
+                    mbar_expect_tx(bar(Q_XFULL + s), S::X_STAGE);
+                    tma_load_2d(base + S::OFF_X + s * S::X_STAGE, &tm_x, bar(Q_XFULL + s), ks * kQkBK, m0);
+                };
+                auto load_w = [&](int ks) {
+                    const int s = (g0 + ks) % kQkStages;
+                    if (rank == 0) mbar_expect_tx(bar(Q_BFULL + s), 2 * S::B_STAGE);
 #pragma unroll
-                for (int j = 0; j < NACC; ++j)
-                    tma2_load_2d(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, &tm_w, bar(Q_BFULL + s) & kPeerBitMask, ks * kQkBK,
-                                 (swiglu ? j * p.swiglu_F + n0 : n0 + j * kQkBN) + (int)rank * (kQkBN / 2));
+                    for (int j = 0; j < NACC; ++j)
+                        tma2_load_2d(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, &tm_w, bar(Q_BFULL + s) & kPeerBitMask, ks * kQkBK,
+                                     (swiglu ? j * p.swiglu_F + n0 : n0 + j * kQkBN) + (int)rank * (kQkBN / 2));
+                };
+                int ks = 0;
+                if (it > 0) {
+                    // head of a later tile: the weights of its first steps go out while the last tile's epilogue still owns the
+                    // x stages, the x tiles follow once its stores have read them
+                    const int nh = nk_steps < kQkStages ? nk_steps : kQkStages;
+                    const uint32_t ph = (uint32_t)(it - 1) & 1u;
+                    if (w_staged) ok = wait(Q_STAGEFREE, ph, 7);
+                    for (int h = 0; h < nh && ok; ++h) {
+                        ok = stage_free(h);
+                        if (ok) load_w(h);
+                    }
+                    if (ok && !w_staged) ok = wait(Q_STAGEFREE, ph, 7);
+                    for (int h = 0; h < nh && ok; ++h) load_x(h);
+                    ks = nh;
+                }
+                for (; ks < nk_steps && ok; ++ks) {
+                    ok = stage_free(ks);
+                    if (!ok) break;
+                    QK_TRACE(0, ks, 0);
+                    load_x(ks);
+                    load_w(ks);
+                }
             }
         }
     } else if (warp == 1) {
@@ -186,31 +232,36 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         if (rank == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(2 * kQkBM, kQkBN, false);
             bool ok = true;
-            for (int ks = 0; ks < nk_steps && ok; ++ks) {
-                const int s = ks % kQkStages;
-                const uint32_t ph = (uint32_t)(ks / kQkStages) & 1u;
-                if (lane == 0) QK_TRACE(1, ks, 0);
-                ok = wait(Q_BFULL + s, ph, 2);
-                if (lane == 0) QK_TRACE(1, ks, 1);
-                ok = ok && wait(Q_AREADY + s, ph, 3);
-                if (lane == 0) QK_TRACE(1, ks, 2);
-                if (!ok) break;
-                tc_fence_after();
+            for (int it = 0; it < my_tiles && ok; ++it) {
+                // the epilogue warps of both CTAs have read the last tile's accumulators
+                if (it > 0) ok = wait(Q_ACCFREE, (uint32_t)(it - 1) & 1u, 6);
+                for (int ks = 0; ks < nk_steps && ok; ++ks) {
+                    const int g = it * nk_steps + ks;
+                    const int s = g % kQkStages;
+                    const uint32_t ph = (uint32_t)(g / kQkStages) & 1u;
+                    if (lane == 0) QK_TRACE(1, ks, 0);
+                    ok = wait(Q_BFULL + s, ph, 2);
+                    if (lane == 0) QK_TRACE(1, ks, 1);
+                    ok = ok && wait(Q_AREADY + s, ph, 3);
+                    if (lane == 0) QK_TRACE(1, ks, 2);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
-                for (int j = 0; j < NACC; ++j) {
-                    uint64_t ad = umma_desc_sw128(base + S::OFF_X + s * S::X_STAGE, 16, 1024);
-                    uint64_t bd = umma_desc_sw128(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, 16, 1024);
+                    for (int j = 0; j < NACC; ++j) {
+                        uint64_t ad = umma_desc_sw128(base + S::OFF_X + s * S::X_STAGE, 16, 1024);
+                        uint64_t bd = umma_desc_sw128(base + S::OFF_B + s * S::B_STAGE + j * S::B_HALF, 16, 1024);
 #pragma unroll
-                    for (int kk = 0; kk < kQkBK / 16; ++kk) {
-                        umma2_ss_elect(tmem + j * kQkBN, ad, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
-                        umma_desc_advance(ad, 32);
-                        umma_desc_advance(bd, 32);
+                        for (int kk = 0; kk < kQkBK / 16; ++kk) {
+                            umma2_ss_elect(tmem + j * kQkBN, ad, bd, idesc, (ks > 0 || kk > 0) ? 1u : 0u);
+                            umma_desc_advance(ad, 32);
+                            umma_desc_advance(bd, 32);
+                        }
                     }
+                    umma2_commit_mc_elect(bar(Q_EMPTY + s), (uint16_t)3);
+                    if (lane == 0) QK_TRACE(1, ks, 3);
                 }
-                umma2_commit_mc_elect(bar(Q_EMPTY + s), (uint16_t)3);
-                if (lane == 0) QK_TRACE(1, ks, 3);
+                umma2_commit_mc_elect(bar(Q_ACC), (uint16_t)3);   // also after a wait that ran out: the epilogue warps must not wait for nothing
             }
-            umma2_commit_mc_elect(bar(Q_ACC), (uint16_t)3);   // also after a wait that ran out: the epilogue warps must not wait for nothing
         }
     } else {
         // ---------------- gate multiply (A operand) and epilogue: two threads per row ----------------
@@ -220,12 +271,23 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const int quarter = warp & 3;                 // the TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
+        float *gsm = reinterpret_cast<float *>(smem + S::OFF_GATE);
+        float *ssm = reinterpret_cast<float *>(smem + S::OFF_SS);
+        const uint32_t leader_aready0 = mapa(bar(Q_AREADY), 0);
+        const uint32_t leader_accfree = mapa(bar(Q_ACCFREE), 0);
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int n_out = p.nq + 2 * p.nk;
+        bool ok = true;
+#pragma unroll 1
+        for (int it = 0; it < my_tiles; ++it) {
+        const int m0 = tile_m0(it), n0 = tile_n0(it);
+        const int g0 = it * nk_steps;
         const int r_glob = m0 + row;
         const int b = min(r_glob / p.R, p.B - 1);     // (rows past the end contribute zeros and are never stored)
-        // the gates of the streams under this CTA's 128 rows go to shared memory once: every step needs 128 fresh bytes of
-        // them per thread, and as global loads those were an L2 round trip per step on the critical path
+        // the gates of the streams under this CTA's 128 rows go to shared memory once per tile: every step needs 128 fresh bytes
+        // of them per thread, and as global loads those were an L2 round trip per step on the critical path. (Every warp is
+        // through with the last tile's gates: they are read in the step loop only, and all eight warps have met since.)
         const int b_first = min(m0 / p.R, p.B - 1), b_last = min((m0 + kQkBM - 1) / p.R, p.B - 1);
-        float *gsm = reinterpret_cast<float *>(smem + S::OFF_GATE);
         {
             const int n4 = (b_last - b_first + 1) * p.D / 4;
             const float4 *src = reinterpret_cast<const float4 *>(p.gate + (size_t)b_first * p.D);
@@ -233,18 +295,15 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             asm volatile("bar.sync 1, 256;" ::: "memory");
         }
         const float *grow = gsm + (size_t)(b - b_first) * p.D + half * 32;
-        const uint32_t leader_aready0 = mapa(bar(Q_AREADY), 0);
-        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint64_t ss2 = 0ull;
-        bool ok = true;
         for (int ks = 0; ks < nk_steps; ++ks) {
             if (threadIdx.x == 64) QK_TRACE(2, ks, 0);
-            const int s = ks % kQkStages;
+            const int s = (g0 + ks) % kQkStages;
             const ulonglong2 *g2 = reinterpret_cast<const ulonglong2 *>(grow + ks * kQkBK);
             ulonglong2 gq[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) gq[i] = g2[i];      // 32 gate values, read before the wait for the tile
-            ok = ok && wait(Q_XFULL + s, (uint32_t)(ks / kQkStages) & 1u, 4);
+            ok = ok && wait(Q_XFULL + s, (uint32_t)((g0 + ks) / kQkStages) & 1u, 4);
             if (threadIdx.x == 64) QK_TRACE(2, ks, 1);
             uint8_t *rowp = smem + S::OFF_X + s * S::X_STAGE + row * 128;
             uint4 xr[4];
@@ -273,7 +332,6 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (threadIdx.x == 64) QK_TRACE(2, ks, 4);
         }
         // the row's sum of squares: both halves meet through shared memory
-        float *ssm = reinterpret_cast<float *>(smem + S::OFF_SS);
         {
             float s0, s1;
             unpack_f32x2(ss2, s0, s1);
@@ -282,11 +340,10 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         asm volatile("bar.sync 1, 256;" ::: "memory");
         const float ss = ssm[row] + ssm[128 + row];
         if (threadIdx.x == 64) QK_TRACE(2, 31, 0);
-        ok = wait(Q_ACC, 0u, 5) && ok;
+        ok = wait(Q_ACC, (uint32_t)it & 1u, 5) && ok;
         if (threadIdx.x == 64) QK_TRACE(2, 31, 1);
         tc_fence_after();
         const float rs = rsqrtf(ss / (float)p.D + p.eps);
-        const int n_out = p.nq + 2 * p.nk;
         if (p.tma_out) {
             // The tile goes out through shared memory and TMA stores. The stage ring is idle now (every load has been consumed and
             // every MMA has completed): accumulator j is staged in the x stages (j = 0) or the weight stages (j = 1) as four
@@ -317,6 +374,12 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 #pragma unroll
                             for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(__uint_as_float(acc[i]) * rs);
                         }
+                        if (WALK && cc == 1 && g == 1 && j == (swiglu ? 0 : NACC - 1)) {
+                            // this warp's last read of the accumulators: the tensor pipe may start the next tile over them
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(leader_accfree);
+                        }
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             uint4 o;
@@ -344,8 +407,12 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                     }
                 }
             }
-            // (the staging areas have been read; the writes themselves are complete when the grid is)
-            if (quarter == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            // (the staging areas have been read -- the producer may load the next tile over them; the writes themselves are
+            // complete when the grid is)
+            if (quarter == 0 && lane == 0) {
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (WALK) mbar_arrive(bar(Q_STAGEFREE));
+            }
         } else {
         // The tile goes out through shared memory (the stage ring is idle now: every load has been consumed and every MMA
         // has completed): each thread drops its half row, scaled and rounded, as 16-byte pieces at [row][piece ^ (row % 32)]
@@ -406,6 +473,7 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (j + 1 < (swiglu ? 1 : NACC)) asm volatile("bar.sync 1, 256;" ::: "memory");   // the staging area is rewritten by the next round
         }
         }
+        }   // tiles of this pair
     }
 
     if (threadIdx.x == 64) QK_TRACE(2, 31, 2);
@@ -869,7 +937,7 @@ bool norm_qkv_tc_supported(int dtype, int B, int R, int D, int nq, int nk)
 }
 
 template <int NACC>
-static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_tiles, cudaStream_t st)
+static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, int n_tiles, int sm_count, cudaStream_t st)
 {
     // tensor maps over the outputs when every tensor's width is a multiple of the 64-column chunks the epilogue stores
     CUtensorMap mq = mx, mk = mx, mv = mx;
@@ -882,11 +950,19 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
     }
     static std::atomic<unsigned long long> attr_set{0};
     cudaError_t e0 = once_per_device(attr_set, [] {
-        return cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
+        cudaError_t e = cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
+        if (e != cudaSuccess) return e;
+        return cudaFuncSetAttribute(norm_qkv_tc_kernel<NACC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QkSmem<NACC>::TOTAL);
     });
     if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
+    // one CTA pair per tile, or per SM pair when there are more tiles than that (the pairs then walk the tiles; the
+    // hand-overs between tiles go with the TMA-store epilogue)
+    p.n_tiles = n_tiles;
+    const unsigned tiles = (unsigned)p.m_tiles * (unsigned)n_tiles;
+    const unsigned pairs_max = (unsigned)((sm_count > 0 ? sm_count : 148) / 2);
+    const bool walk = p.tma_out && tiles > pairs_max && pairs_max > 0;
+    cfg.gridDim = dim3(2u * (walk ? pairs_max : tiles));
     cfg.blockDim = dim3(kQkThreads);
     cfg.dynamicSmemBytes = QkSmem<NACC>::TOTAL;
     cfg.stream = st;
@@ -895,7 +971,8 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel<NACC>, mx, mw, mq, mk, mv, p);
+    cudaError_t e = walk ? cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel<NACC, true>, mx, mw, mq, mk, mv, p)
+                         : cudaLaunchKernelEx(&cfg, norm_qkv_tc_kernel<NACC, false>, mx, mw, mq, mk, mv, p);
     count_launch();
     return e;
 }
@@ -947,7 +1024,7 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
         if (!tensor_map_2d_bf16(&sx, x, D, M, NT) || !tensor_map_2d_bf16(&sw, W, D, w_rows, 128)) return cudaErrorInvalidValue;
         QkParams sp;
         sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
-        sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.swiglu_F = swiglu_F;
+        sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.n_tiles = 1; sp.swiglu_F = swiglu_F;
         sp.eps = eps; sp.status = status; sp.res = nullptr; sp.tma_out = 0;
         const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
         // The contraction split over 4 CTAs per feature tile where the chain of steps is long enough to pay for a cluster
@@ -970,11 +1047,12 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
     p.m_tiles = (M + 2 * kQkBM - 1) / (2 * kQkBM);
     p.swiglu_F = swiglu_F;
     p.eps = eps; p.status = status; p.res = nullptr; p.ksplit = 1; p.tma_out = 0;
-    if (swiglu_F > 0) return launch_tc<2>(mx, mw, p, (swiglu_F + kQkBN - 1) / kQkBN, st);
+    if (swiglu_F > 0) return launch_tc<2>(mx, mw, p, (swiglu_F + kQkBN - 1) / kQkBN, sm_count, st);
     int nacc = qk_choose_nacc(M, R, D, nq + 2 * nk, sm_count > 0 ? sm_count : 148);
     if (impl == 2 && nacc == 2) nacc = 1;     // (forced 256-column tiles, for tests and timing)
     const int n_out = nq + 2 * nk;
-    return nacc == 2 ? launch_tc<2>(mx, mw, p, (n_out + 2 * kQkBN - 1) / (2 * kQkBN), st) : launch_tc<1>(mx, mw, p, (n_out + kQkBN - 1) / kQkBN, st);
+    return nacc == 2 ? launch_tc<2>(mx, mw, p, (n_out + 2 * kQkBN - 1) / (2 * kQkBN), sm_count, st)
+                     : launch_tc<1>(mx, mw, p, (n_out + kQkBN - 1) / kQkBN, sm_count, st);
 }
 
 // out [M][N] = res + a [M][K] W [N][K]^T for at most 128 rows (K a multiple of 64): the few-rows kernel without its norm stage
@@ -985,7 +1063,7 @@ cudaError_t launch_linear_small(const void *a, const void *W, const void *res, v
     if (!tensor_map_2d_bf16(&sx, a, K, M, NT) || !tensor_map_2d_bf16(&sw, W, K, N, 128)) return cudaErrorInvalidValue;
     QkParams sp;
     sp.gate = nullptr; sp.q = (__nv_bfloat16 *)out; sp.k = nullptr; sp.v = nullptr;
-    sp.M = M; sp.R = M; sp.B = 1; sp.D = K; sp.nq = N; sp.nk = 0; sp.m_tiles = 1; sp.swiglu_F = 0;
+    sp.M = M; sp.R = M; sp.B = 1; sp.D = K; sp.nq = N; sp.nk = 0; sp.m_tiles = 1; sp.n_tiles = 1; sp.swiglu_F = 0;
     sp.eps = 0.f; sp.status = status; sp.res = (const __nv_bfloat16 *)res; sp.tma_out = 0;
     // split the contraction over up to 8 CTAs per feature tile while every slice keeps whole steps of two 64-column chunks and
     // the grid stays within the SMs
