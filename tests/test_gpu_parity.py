@@ -718,6 +718,29 @@ def test_norm_swiglu_bf16_ragged_hidden_width(U):
     _norm_swiglu_case(U, w, 328, 0, "norm+swiglu ragged")
 
 
+@pytest.mark.parametrize("D", [128, 640])
+def test_norm_qkv_more_tiles_than_sm_pairs(U, D):
+    """128 streams of 50 rows = 6400 rows: 25 row tiles x 5 column tiles of 512 = 125 tiles, more than the SM pairs, so every
+    CTA pair walks two tiles and hands the stage ring and the accumulators from one to the next (both accumulators are staged
+    for the TMA stores, so the next tile's weights wait for them too). D = 128 gives two contraction steps per tile, fewer
+    than the stage ring; D = 640 ten. A sample of streams from first and later tiles of a pair is compared."""
+    w = synth.CONFIGS["cfg2"].with_(B=128, D=D)
+    _norm_qkv_case(U, w, 0, f"norm+qkv 125 tiles D={D}", streams=[0, 1, 37, 63, 64, 100, 126, 127])
+
+
+def test_norm_qkv_more_tiles_than_sm_pairs_one_accumulator(U):
+    """D = 2048: the gates of a tile's four streams no longer fit beside two accumulators' stages, so the tiles are 256 columns
+    wide; 100 streams of 50 rows (20 row tiles) x 4 column tiles (2 + 1 + 1 heads of 256) = 80 tiles on 74 SM pairs."""
+    w = synth.CONFIGS["cfg2"].with_(B=100, D=2048, Hq=2, Hkv=1)
+    _norm_qkv_case(U, w, 0, "norm+qkv 80 tiles, one accumulator", streams=[0, 4, 5, 50, 94, 95, 99])
+
+
+def test_norm_swiglu_more_tiles_than_sm_pairs(U):
+    """6400 rows x 1000 hidden features (ragged last column tile) with D = 192: 25 x 4 = 100 tiles of three steps on 74 pairs."""
+    w = synth.CONFIGS["cfg2"].with_(B=128, D=192)
+    _norm_swiglu_case(U, w, 1000, 0, "norm+swiglu 100 tiles", streams=[0, 1, 63, 64, 90, 127])
+
+
 def test_norm_qkv_short_streams_and_fallback(U):
     """Rows per stream far below the tile height: with R = 13 a 128-row tile covers 11 streams (all their gates in shared
     memory); with R = 3 the gates of a tile's 44 streams no longer fit beside the stages and the call falls back to the plain
