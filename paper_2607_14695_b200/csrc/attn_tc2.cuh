@@ -35,6 +35,9 @@ namespace reflex {
 #else
 #define TC2_TRACE(role, slot, ev) do { } while (0)
 #endif
+#ifndef REFLEX_TRACE_UNIT
+#define REFLEX_TRACE_UNIT 0     // which unit of the cluster the per-tile stamps are taken in
+#endif
 
 constexpr int kTc2Keys = 128;     // keys per tile = two 64-key halves, one per CTA of the pair
 #ifndef REFLEX_TC2_NP
@@ -249,10 +252,10 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint32_t ph = (uint32_t)(gi / NKS - 1) & 1u;
                 const int h0 = 2 * (w.tile0 + c.jj), h1 = h0 + 1;
                 const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
-                if (c.ui == 0) TC2_TRACE(0, c.jj, 0);
+                if (c.ui == REFLEX_TRACE_UNIT) TC2_TRACE(0, c.jj, 0);
                 if (gi >= NKS) ok = wait(C_KEMPTY + st, ph, 1);
                 if (!ok) return;
-                if (c.ui == 0) TC2_TRACE(0, c.jj, 1);
+                if (c.ui == REFLEX_TRACE_UNIT) TC2_TRACE(0, c.jj, 1);
                 if (rank == 0) mbar_expect_tx(bar(C_KFULL + st), (uint32_t)live * L::K_STAGE);
                 const int myh = h0 + (int)rank;
                 if (myh < w.H) {
@@ -279,7 +282,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int live = (h0 < w.H ? 1 : 0) + (h1 < w.H ? 1 : 0);
                 if (gi >= NVS) ok = wait(C_VEMPTY + st, ph, 2);
                 if (!ok) return;
-                if (c.ui == 0) TC2_TRACE(0, c.jj, 2);
+                if (c.ui == REFLEX_TRACE_UNIT) TC2_TRACE(0, c.jj, 2);
                 mbar_expect_tx(bar(C_VLAND + st), (uint32_t)live * L::V_HALF);
                 for (int hh = h0; hh <= h1; ++hh) {
                     if (hh >= w.H) break;
@@ -449,7 +452,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                   }
                 }
                 const uint64_t smask = FULL ? kSliceFull : ((rmask >> koff) & kSliceFull);   // this thread's KT keys
-#define SM_EV(ev) do { if (threadIdx.x == 64 && ui_s == 0) TC2_TRACE(3, jj, ev); } while (0)
+#define SM_EV(ev) do { if (threadIdx.x == 64 && ui_s == REFLEX_TRACE_UNIT) TC2_TRACE(3, jj, ev); } while (0)
                 SM_EV(0);
                 float s[KT];
                 if constexpr (!DEAD) {
