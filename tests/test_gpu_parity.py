@@ -336,6 +336,53 @@ def test_edge_shapes(U, case, impl):
     tw.attention(0, 6, scale=0.05, what=name + " scale override")
 
 
+def _random_attention_cases(n, seed):
+    """Seeded shapes across what the kernels branch on: head_dim, queries per KV head, KV heads, prefix lengths that differ per
+    stream (0 included), ring capacity and fill (empty, partly filled, wrapped), dynamic tokens from 1 to beyond one tile."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        d = int(rng.choice([64, 128, 256]))
+        G = int(rng.choice([1, 2, 4, 8, 16]))
+        Hkv = int(rng.choice([1, 2]))
+        B = int(rng.integers(1, 5))
+        S_max = int(rng.choice([8, 70, 130, 300, 600]))
+        N = int(rng.choice([1, 7, 32, 64, 100, 200]))
+        T = int(rng.choice([1, 3, 17, 50, 64, 65, 140]))
+        S_list = [int(rng.integers(0, S_max + 1)) for _ in range(B)]
+        if i % 4 == 0:
+            S_list[0] = S_max
+        n_app = int(rng.integers(0, 4))
+        appends = [int(rng.integers(1, N + 1)) for _ in range(n_app)]
+        head0 = [int(rng.integers(0, N)) for _ in range(B)]
+        cases.append((f"r{i}_d{d}_g{G}_kv{Hkv}_B{B}_S{S_max}_N{N}_T{T}", d, G, Hkv, B, S_max, N, T, S_list, appends, head0))
+    return cases
+
+
+RANDOM_CASES = _random_attention_cases(20, 2607)
+
+
+@pytest.mark.parametrize("case", RANDOM_CASES, ids=[c[0] for c in RANDOM_CASES])
+def test_random_shapes_every_attention_kernel(U, case):
+    """Each seeded shape through every attention kernel that takes it (plain, one-CTA and two-CTA tensor-core forms, and the
+    library's own choice), both masks, against the oracle element by element; ring state and cache bytes exactly."""
+    name, d, G, Hkv, B, S_max, N, T, S_list, appends, head0 = case
+    rb = U.rb
+    w = synth.Workload(name, 99, synth.DTYPE_BF16, B=B, L=1, Hq=G * Hkv, Hkv=Hkv, d=d, S=S_max, S_max=S_max, N=N, T=T, D=64, Cd=8, Hd=8, A=4, K=2)
+    tw = U.Twin(w, head0=head0, poison=True)
+    tw.init_static(list(range(B)), S_list)
+    for i, m in enumerate(appends):
+        tw.append(list(range(B)), m, i)
+    tw.check_state()
+    tensor_core = d in (64, 128, 256) and 128 % G == 0
+    two_cta = tensor_core and d in (128, 256)
+    impls = [("auto", rb.ATTN_AUTO), ("simt", rb.ATTN_SIMT)] + ([("tc", rb.ATTN_TC)] if tensor_core else []) + ([("tc2", rb.ATTN_TC2)] if two_cta else [])
+    for iname, impl in impls:
+        rb.reflex_cache_set_attention_impl(tw.g, impl)
+        for dyn_mask in (0, 1):
+            tw.attention(0, dyn_mask, dyn_mask=dyn_mask, what=f"{name} {iname} mask {dyn_mask}")
+
+
 @pytest.mark.parametrize("impl", ["tc", "tc2"])
 def test_wide_logits_exercise_the_lazy_rescale(U, impl):
     """Queries scaled up so that row maxima keep growing by more than 2^8 from tile to tile: O and l are rescaled in
@@ -812,6 +859,38 @@ def test_linear_residual_bf16_few_rows(U, M):
     _linear_case(U, synth.DTYPE_BF16, M, 4096, 1024, 0, f"linear {M} rows K=4096 in place", in_place=True)
     _linear_case(U, synth.DTYPE_BF16, M, 192, 328, 0, f"linear {M} rows ragged", residual=False)
     _linear_case(U, synth.DTYPE_BF16, M, 2048, 1024, 2, f"linear {M} rows, 256-row tiles")
+
+
+def _random_projection_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        B = int(rng.choice([1, 2, 3, 7, 20, 45]))
+        T = int(rng.choice([1, 13, 50, 64, 100]))
+        D = int(rng.choice([64, 192, 512, 1024]))
+        Hq, d = int(rng.choice([1, 3, 8])), int(rng.choice([64, 128, 256]))
+        F = int(rng.choice([8, 72, 256, 328, 1000]))
+        N = int(rng.choice([8, 72, 256, 1000]))
+        cases.append((f"p{i}_B{B}_T{T}_D{D}_Hq{Hq}_d{d}_F{F}_N{N}", B, T, D, Hq, d, F, N))
+    return cases
+
+
+RANDOM_PROJECTIONS = _random_projection_cases(12, 14695)
+
+
+@pytest.mark.parametrize("case", RANDOM_PROJECTIONS, ids=[c[0] for c in RANDOM_PROJECTIONS])
+def test_random_shapes_projections(U, case):
+    """Seeded shapes through the three projection entry points (norm + Q/K/V, norm + gate/up, plain + residual) with the
+    kernel the library picks for them (few rows, 256-row tiles with one or two accumulators, plain kernel for what the
+    tensor-core forms refuse), a sample of streams / rows against the oracle."""
+    name, B, T, D, Hq, d, F, N = case
+    w = synth.CONFIGS["cfg2"].with_(B=B, T=T, D=D, Hq=Hq, Hkv=1, d=d)
+    streams = sorted({0, B // 2, B - 1})
+    _norm_qkv_case(U, w, 0, name + " norm+qkv", streams=streams)
+    _norm_swiglu_case(U, w, F, 0, name + " norm+swiglu", streams=streams)
+    M = B * T
+    rows = sorted({0, M // 3, M // 2, M - 1} | set(range(max(0, M - 5), M)))
+    _linear_case(U, synth.DTYPE_BF16, M, D, N, 0, name + " linear", rows=rows, seed=70)
 
 
 def test_linear_residual_error_paths(U):
