@@ -458,7 +458,7 @@ def main():
                         "roofline": roofline_of(ch_flops, ch_bytes, chained_ms * 1e-3, peaks, "sustained" if chained_sec >= 0.5 else "burst"),
                         "what": "gates of the step (one call), then per layer AdaRMSNorm + packed W_QKV projection in one launch and the partitioned attention over its "
                                 "Q / K_dyn / V_dyn, then the Euler update: 2 L + 3 launches, no stand-alone norm launch"}
-        # a whole action-expert step: the fused calls, the output / down projections with residual (this library) and library GEMMs for the two A-wide heads
+        # a whole action-expert step: the fused calls, the output / down projections with residual and the two A-wide heads (reflex_linear_residual)
         model = ex.ActionExpert(w, runner.cache, ex.random_weights_device(w, F, device=dev), F, device=dev)
         expert_ms = avg_launch_ms(lambda v: model.step(runner.xa, runner.cond[v % w.K], v % w.K), 1)
         lin = {}
@@ -481,7 +481,7 @@ def main():
                    "what": "norm_qkv / norm_swiglu: AdaRMSNorm folded into the packed Q/K/V projection resp. the fused gate/up projections, timed alone; "
                            "linear_residual: the output and down projections with their residual add (reflex_linear_residual) beside torch.addmm_ on the same shapes; "
                            "expert_step_ms: a whole action-expert denoising step (input projection, L x (norm+QKV, attention, output projection, norm+SwiGLU, "
-                           "down projection), velocity head, Euler update; F = 4 D); only the two A-wide heads are library GEMMs"}
+                           "down projection), velocity head, Euler update; F = 4 D); every contraction is this library's kernel (the two A-wide heads go through reflex_linear_residual without a residual)"}
         if not args.no_e2e:
             # end to end through the expert step: the action chunk and the conditioning vectors come from pinned host memory
             # every step and the updated chunk goes back; nothing else crosses PCIe

@@ -2,8 +2,8 @@
 packed Q/K/V projection, the partitioned attention, the output projection with its residual, the adaptive norm folded
 into the fused gate/up projections of the SwiGLU block and the down projection with its residual; then the velocity
 head and the Euler update of the action chunk (Sec. 2.1, Sec. 3.1-3.3). The output and down projections with their
-residual adds are reflex_linear_residual; only the two A-wide heads (input projection from the A = 32 action dimensions,
-velocity head back to them) are library GEMMs (torch.matmul on the current stream); everything else is this package's kernels.
+residual adds are reflex_linear_residual, and so are the two A-wide heads (input projection from the A = 32 action
+dimensions, velocity head back to them; no residual): every contraction of the step runs in this package's kernels.
 
 The paper does not print the expert's architecture; this is the usual pre-norm block of a pi0-class expert with both
 norms adaptive, no biases and no positional term (positions are outside the path), written down so that the fused calls
@@ -52,7 +52,7 @@ class ActionExpert:
         B, T, D = w.B, w.T, w.D
         rb.reflex_adarmsnorm_gate(cond, W["W1"], W["b1"], W["W2"], W["b2"], self.gates, stream=stream)   # all 2L + 1 gates
         self.a_lowp.copy_(a)
-        torch.matmul(self.a_lowp.view(B * T, w.A), W["W_in"].t(), out=self.h.view(B * T, D))
+        rb.reflex_linear_residual(self.a_lowp.view(B * T, w.A), W["W_in"], None, self.h.view(B * T, D), cache=self.cache, stream=stream)
         for l in range(w.L):
             rb.reflex_adarmsnorm_qkv(self.h, self.gate(2 * l), W["Wqkv"][l], self.q, self.k, self.v, cache=self.cache, stream=stream)
             rb.reflex_partitioned_attention(self.cache, l, self.q, self.k, self.v, self.o, stream=stream)
@@ -60,7 +60,7 @@ class ActionExpert:
             rb.reflex_adarmsnorm_swiglu(self.h, self.gate(2 * l + 1), W["Wgu"][l], self.m, cache=self.cache, stream=stream)
             rb.reflex_linear_residual(self.m.view(B * T, self.F), W["Wd"][l], self.h, self.h, cache=self.cache, stream=stream)
         rb.reflex_adarmsnorm(self.h, self.y, None, None, None, None, None, gate_buf=self.gate(2 * w.L), stream=stream)
-        torch.matmul(self.y.view(B * T, D), W["W_out"].t(), out=self.vel.view(B * T, w.A))
+        rb.reflex_linear_residual(self.y.view(B * T, D), W["W_out"], None, self.vel.view(B * T, w.A), cache=self.cache, stream=stream)
         rb.reflex_flow_step(a, self.vel, None, k, w.K, stream=stream)
         return a
 

@@ -1009,7 +1009,7 @@ def _expert_case(U, w, F, tol_v, what, streams=None):
 
 
 def test_expert_step_fp32(U):
-    """Two layers in fp32 (plain kernels + fp32 library GEMMs): the chain agrees with the double-precision chain to fp32 rounding."""
+    """Two layers in fp32 (plain kernels throughout): the chain agrees with the double-precision chain to fp32 rounding."""
     w = synth.CONFIGS["cfg1"].with_(B=2, L=2)
     _expert_case(U, w, 256, 2e-5, "expert fp32")
 
