@@ -460,7 +460,16 @@ def main():
                                 "Q / K_dyn / V_dyn, then the Euler update: 2 L + 3 launches, no stand-alone norm launch"}
         # a whole action-expert step: the fused calls, the output / down projections with residual and the two A-wide heads (reflex_linear_residual)
         model = ex.ActionExpert(w, runner.cache, ex.random_weights_device(w, F, device=dev), F, device=dev)
-        expert_ms = avg_launch_ms(lambda v: model.step(runner.xa, runner.cond[v % w.K], v % w.K), 1)
+        # (both clock regimes, like the headline: what ran just before this leg would otherwise decide which one it lands in)
+        ex_graphs = kernel_graphs(runner, lambda v: model.step(runner.xa, runner.cond[v % w.K], v % w.K))
+        cool()
+        ex_b = leg(lambda i: ex_graphs[i % len(ex_graphs)].replay(), 6, 1)
+        expert_ms = ex_b[0]
+        expert_regimes = {"burst": regime(*ex_b)}
+        if args.sustain_seconds > 0:
+            ex_s = leg(lambda i: ex_graphs[i % len(ex_graphs)].replay(), max(6, int(min(args.sustain_seconds, 1.0) / max(ex_b[0] * 1e-3, 1e-6))), 1)
+            expert_regimes["sustained"] = regime(*ex_s)
+        del ex_graphs
         lin = {}
         for name, Kc in (("output_projection", w.Hq * w.d), ("down_projection", F)):
             a_in = [runner.rnd(w.B * w.T, Kc) for _ in range(runner.variants)]
@@ -477,10 +486,10 @@ def main():
         chained = {"norm_qkv_avg_us": qkv_avg_ms * 1e3, "norm_qkv_tflops": alg["qkv_flops_per_launch"] / (qkv_avg_ms * 1e-3) / 1e12,
                    "norm_qkv_shape_mnk": [w.B * w.T, n_out, w.D], "ms_per_step": chained_ms,
                    "norm_swiglu_avg_us": swiglu_avg_ms * 1e3, "norm_swiglu_tflops": 2.0 * w.B * w.T * w.D * 2 * F / (swiglu_avg_ms * 1e-3) / 1e12,
-                   "norm_swiglu_shape_m_f_k": [w.B * w.T, F, w.D], "linear_residual": lin, "expert_step_ms": expert_ms,
+                   "norm_swiglu_shape_m_f_k": [w.B * w.T, F, w.D], "linear_residual": lin, "expert_step_ms": expert_ms, "expert_step_regimes": expert_regimes,
                    "what": "norm_qkv / norm_swiglu: AdaRMSNorm folded into the packed Q/K/V projection resp. the fused gate/up projections, timed alone; "
                            "linear_residual: the output and down projections with their residual add (reflex_linear_residual) beside torch.addmm_ on the same shapes; "
-                           "expert_step_ms: a whole action-expert denoising step (input projection, L x (norm+QKV, attention, output projection, norm+SwiGLU, "
+                           "expert_step_ms (burst clocks; expert_step_regimes has the sustained leg too): a whole action-expert denoising step (input projection, L x (norm+QKV, attention, output projection, norm+SwiGLU, "
                            "down projection), velocity head, Euler update; F = 4 D); every contraction is this library's kernel (the two A-wide heads go through reflex_linear_residual without a residual)"}
         if not args.no_e2e:
             # end to end through the expert step: the action chunk and the conditioning vectors come from pinned host memory
