@@ -755,7 +755,8 @@ bool tc2_supported(const AttnParams &p) { return tc_supported(p) && (p.d == 128 
 // Key split of the two-CTA kernel: 1, 2, 4 or 8 slices, whichever a small cost model makes cheapest. A unit (tile pair
 // of one stream and KV head) walks its 128-key tiles at about 1.3 us each, units run in waves of one per SM pair, and
 // splitting costs a fixed 3 us (merge launch) plus the fp32 partials' round trip through memory. Measured at the
-// 898-key shape: 1 stream 14.4 us with 8 slices; 2 streams 15.4 with 4; 4 streams 17.5 with 4; 8 to 32 streams 19.5 to
+// 898-key shape (before the partial tiles of a cluster's last unit were staged and written as whole rows, which took 1 us
+// off the one-stream figure): 1 stream 14.4 us with 8 slices; 2 streams 15.4 with 4; 4 streams 17.5 with 4; 8 to 32 streams 19.5 to
 // 21.7 unsplit (split in two: 21.6 to 40); at 4466 keys and 16 streams 41 us split in two, 51 unsplit, 47 in four.
 // The nsplit pairs that share a tile pair can merge inside one cluster (no partials, no merge launch) when the cluster stays
 // within the portable size of 8 CTAs, all clusters are resident at once with exactly one unit each, and a thread's share of
