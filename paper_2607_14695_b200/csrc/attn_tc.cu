@@ -45,7 +45,8 @@ struct TcParams {
     int dyn_mask;
     float scale, scale_log2;
     int nsplit;
-    int tile_tokens;  // 128 / G
+    int tile_tokens;  // 128 / G (two-CTA kernel with live_rows = 64: half of that)
+    int live_rows;    // rows of a CTA's 128-row tile that belong to its tokens: 128, or 64 (two-CTA kernel, key-split units of few streams)
     int n_qtiles;
     int cluster_merge;  // one-CTA kernel: the nsplit key slices of a query tile form a cluster and merge through shared memory
 };
@@ -828,6 +829,7 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
     tp.dyn_mask = p.dyn_mask; tp.scale = p.scale; tp.scale_log2 = p.scale * 1.4426950408889634f;
     tp.nsplit = p.nsplit;
     tp.tile_tokens = kBM / G;
+    tp.live_rows = kBM;
     tp.n_qtiles = (p.T + tp.tile_tokens - 1) / tp.tile_tokens;
     tp.cluster_merge = two_cta ? (tc2_cluster_merge_ok(p, p.nsplit, sm_count) ? 1 : 0)
                                : ((p.nsplit > 1 && p.nsplit <= 8 && (p.d / 4) % (2 * p.nsplit) == 0) ? 1 : 0);
@@ -838,6 +840,16 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
         CUtensorMap mo;
         if (!cache().get(&mo, p.out, 1, (p.B << 16) | p.T, p.Hq, p.d, G, mk_q)) return cudaErrorInvalidValue;
         tp.n_qtiles = (tp.n_qtiles + 1) / 2;
+        // Key-split units that leave fp32 partials: every CTA writes its rows x head_dim x 4 bytes, and an SM's stores leave at
+        // about 24 bytes per clock (128 KB: 2.8 us of a 10 us launch). While twice the clusters still fit the device at once,
+        // a CTA takes half a tile's tokens (64 live rows of its 128) and the partials are shared by twice the SMs.
+        if (p.nsplit > 1 && !tp.cluster_merge && tp.tile_tokens % 2 == 0) {
+            const int half_tokens = tp.tile_tokens / 2;
+            const int pairs_h = ((p.T + half_tokens - 1) / half_tokens + 1) / 2;
+            if (pairs_h > tp.n_qtiles && pairs_h * p.Hkv * p.B * p.nsplit <= tc2_active_clusters(p.d, 2)) {
+                tp.tile_tokens = half_tokens; tp.live_rows = kBM / 2; tp.n_qtiles = pairs_h;
+            }
+        }
         const int units = tp.n_qtiles * p.Hkv * p.B * p.nsplit;
         int clusters = sm_count / 2;
         if (clusters > units) clusters = units;

@@ -415,7 +415,9 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int u = u_start; u < n_units; u += u_stride, ++ui_s) {
             const Unit w = have_next ? w_next : load_unit(u);
             have_next = false;
-            const int t_row = w.t0 + row / p.G;
+            // (key-split units of a few streams may cover half a tile's tokens per CTA, rows past them idle: twice the CTAs then
+            // share the fp32 partials, which leave an SM at about 24 bytes per clock whatever else it does)
+            const int t_row = row < p.live_rows ? w.t0 + row / p.G : 0x3fffffff;
             if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 0);
             const int rows_total = p.T * p.Hq;
             const size_t n_slots = (size_t)p.B * rows_total * p.nsplit;
@@ -669,7 +671,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int rr = 0; rr < RW; ++rr) {
                         const int r = sw * RW + rr;
                         const int tr = w.t0 + r / p.G;
-                        if (tr >= p.T) continue;
+                        if (tr >= p.T || r >= p.live_rows) continue;
                         float *dst = partial_o(p.partials, partial_slot(w.b, rows_total, tr * p.Hq + w.kvh * p.G + r % p.G, p.nsplit, w.split), HD);
 #pragma unroll
                         for (int h = 0; h < PR / 32; ++h) {
