@@ -340,7 +340,7 @@ cudaError_t launch_linear_residual(const void *a, const void *W, const void *res
         if ((size_t)K * sizeof(float) > 48 * 1024) return cudaErrorInvalidValue;
         return dtype == REFLEX_DTYPE_BF16 ? launch_lin_simt<__nv_bfloat16>(a, W, res, out, M, K, N, st) : launch_lin_simt<float>(a, W, res, out, M, K, N, st);
     }
-    if (impl == 0 && M <= 128 && K % 64 == 0) return launch_linear_small(a, W, res, out, M, K, N, status, st);
+    if (impl == 0 && linear_small_takes(M, K, N)) return launch_linear_small(a, W, res, out, M, K, N, status, st);
     LinParams p;
     p.M = M; p.K = K; p.N = N; p.m_tiles = (M + 2 * kLinBM - 1) / (2 * kLinBM); p.has_res = res ? 1 : 0; p.status = status;
     // 256-column tiles unless they would leave more than half of the SM pairs without one: then 128-column tiles, twice as

@@ -30,6 +30,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+
 #include "reflex_internal.cuh"
 #include "sm100_ptx.cuh"
 
@@ -484,12 +486,13 @@ norm_qkv_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     if (warp == 1) tmem_dealloc2(tmem, NACC * kQkBN);
 }
 
-// ---- few rows (one or two streams): weights as the A operand ----------------------------------------------------------------
-// With at most 128 rows in all, tiles of 256 rows would be mostly padding and the launch a chain of sixteen dependent steps
+// ---- few rows (a handful of streams): weights as the A operand ------------------------------------------------------------
+// With a few hundred rows at most, tiles of 256 rows would be mostly padding and the launch a chain of sixteen dependent steps
 // on a handful of CTAs. Here the roles are swapped: out^T [features][rows] = W [features][D] . y'^T [D][rows]. A CTA owns 128
-// output features (the M of a cta_group::1 MMA; for SwiGLU 128 hidden features with a gate and an up accumulator), the rows
-// are the N (64 or 128), so the grid is features / 128 CTAs that each stream their own slice of the weights once (the
-// whole cost of the call) while eight warps rewrite the small x tile of every step as the gated B operand.
+// output features (the M of a cta_group::1 MMA; for SwiGLU 128 hidden features with a gate and an up accumulator) and a
+// group of rows, which are the N (64 or 128): the grid is features / 128 x row groups CTAs that each stream their slice of
+// the weights once (the whole cost of the call) while eight warps rewrite the small x tile of every step as the gated B
+// operand. Groups of 64 rows are taken while every (feature tile, group) still has an SM of its own (grid y).
 constexpr int kSmThreads = 64 + 256;   // producer warp, MMA warp, eight warps that rewrite x and run the epilogue
 
 template <int NT, int NACC>      // NT: rows (tokens) padded to 64 or 128; NACC: 1, or 2 for SwiGLU (gate and up rows)
@@ -538,6 +541,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
     const int ksplit = p.ksplit;
     const int krank = ksplit > 1 ? (int)cluster_ctarank() : 0;
     const int f0 = (blockIdx.x / ksplit) * 128;       // first output feature (hidden feature for SwiGLU) of this CTA
+    const int row0 = blockIdx.y * NT;                 // first row of this CTA's group of NT rows (grid y: row groups)
     constexpr int CPS = S::CPS;
     const int all_chunks = p.D / kQkBK;
     const int chunk0 = krank * (all_chunks / ksplit);      // this CTA's first 64-column chunk of the contraction axis
@@ -596,7 +600,7 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
 #pragma unroll
                 for (int cc = 0; cc < CPS; ++cc) {
                     const int col = (chunk0 + ks * CPS + cc) * kQkBK;
-                    tma_load_2d(base + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE, &tm_x, bar(S_XFULL + s), col, 0);
+                    tma_load_2d(base + S::OFF_X + s * S::X_STAGE + cc * S::X_TILE, &tm_x, bar(S_XFULL + s), col, row0);
 #pragma unroll
                     for (int j = 0; j < NACC; ++j)
                         tma_load_2d(base + S::OFF_W + s * S::W_STAGE + (j * CPS + cc) * S::W_TILE, &tm_w, bar(S_XFULL + s), col, j * p.swiglu_F + f0);
@@ -638,16 +642,17 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
         const int row = tid % NT;                      // row (token) this thread rewrites
         const int kpart = tid / NT;                    // which 64 / TP columns of every step
         constexpr int KW = kQkBK / TP;                 // columns per thread and step: 16 or 32
-        const int b = min(row / p.R, p.B - 1);
+        const int b = min((row0 + row) / p.R, p.B - 1);
+        const int b_first = min(row0 / p.R, p.B - 1), b_last = min((row0 + NT - 1) / p.R, p.B - 1);   // streams under this group's rows
         float *gsm = reinterpret_cast<float *>(smem + S::OFF_GATE);
         if constexpr (!PLAIN) {
-            const int n4 = p.B * p.D / 4;              // (at most 4 streams: checked by the launcher)
-            const float4 *src = reinterpret_cast<const float4 *>(p.gate);
+            const int n4 = (b_last - b_first + 1) * p.D / 4;     // (they fit: checked by the launcher)
+            const float4 *src = reinterpret_cast<const float4 *>(p.gate + (size_t)b_first * p.D);
             for (int i = tid; i < n4; i += 256) reinterpret_cast<float4 *>(gsm)[i] = __ldg(src + i);
             asm volatile("bar.sync 1, 256;" ::: "memory");
         }
         if (threadIdx.x == 64) QK_TRACE(2, 30, 2);
-        const float *grow = gsm + (size_t)b * p.D + kpart * KW;
+        const float *grow = gsm + (size_t)(b - b_first) * p.D + kpart * KW;
         uint64_t ss2 = 0ull;
         bool ok = true;
         for (int ks = 0; ks < nk_steps; ++ks) {
@@ -760,13 +765,13 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             if (!ok || f >= n_feat) continue;
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const int r = c * 32 + i;
-                if (r < p.M) {                      // (no early exit: the accumulator stays in registers)
+                const int r = c * 32 + i, rg = row0 + r;
+                if (rg < p.M) {                     // (no early exit: the accumulator stays in registers)
                     const float rs = rsm[r];
                     float val = __uint_as_float(acc[i]) * rs;
                     if (swiglu) { const float u = __uint_as_float(up[i]) * rs; val = silu_mul(val, u); }
-                    if constexpr (PLAIN) { if (p.res) val += __bfloat162float(p.res[(size_t)r * pitch + f]); }
-                    dst0[(size_t)r * pitch] = __float2bfloat16_rn(val);     // a warp writes 64 contiguous bytes per row
+                    if constexpr (PLAIN) { if (p.res) val += __bfloat162float(p.res[(size_t)rg * pitch + f]); }
+                    dst0[(size_t)rg * pitch] = __float2bfloat16_rn(val);    // a warp writes 64 contiguous bytes per row
                 }
             }
         }
@@ -802,7 +807,8 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             const int n_feat = swiglu ? p.swiglu_F : p.nq + 2 * p.nk;
             for (int e = threadIdx.x - 64; e < rows_mine * 128; e += 256) {
                 const int r = r0 + e / 128, fl = e % 128, f = f0 + fl;
-                if (r >= p.M || f >= n_feat) continue;
+                const int rg = row0 + r;
+                if (rg >= p.M || f >= n_feat) continue;
                 float sum = 0.f, sum_up = 0.f;
                 const uint32_t a0 = smem_u32(part + r * 128 + fl);
                 for (int q = 0; q < ksplit; ++q) {
@@ -816,11 +822,11 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
                     }
                 }
                 __nv_bfloat16 *dst;
-                if (swiglu || f < p.nq) dst = p.q + (size_t)r * p.nq + f;
-                else if (f < p.nq + p.nk) dst = p.k + (size_t)r * p.nk + (f - p.nq);
-                else dst = p.v + (size_t)r * p.nk + (f - p.nq - p.nk);
+                if (swiglu || f < p.nq) dst = p.q + (size_t)rg * p.nq + f;
+                else if (f < p.nq + p.nk) dst = p.k + (size_t)rg * p.nk + (f - p.nq);
+                else dst = p.v + (size_t)rg * p.nk + (f - p.nq - p.nk);
                 if constexpr (PLAIN) {
-                    if (p.res) sum += __bfloat162float(p.res[(size_t)r * p.nq + f]);
+                    if (p.res) sum += __bfloat162float(p.res[(size_t)rg * p.nq + f]);
                 } else {
                     const float rs = rs_mine[r - r0];
                     sum *= rs;
@@ -978,7 +984,7 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mw, QkPar
 }
 
 template <int NT, int NACC, bool PLAIN = false>
-static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, unsigned grid, cudaStream_t st)
+static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, QkParams p, unsigned grid, unsigned groups, cudaStream_t st)
 {
     static std::atomic<unsigned long long> attr_set{0};
     cudaError_t e0 = once_per_device(attr_set, [] {
@@ -986,7 +992,7 @@ static cudaError_t launch_small(const CUtensorMap &mx, const CUtensorMap &mw, Qk
     });
     if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
+    cfg.gridDim = dim3(grid, groups);
     cfg.blockDim = dim3(kSmThreads);
     cfg.dynamicSmemBytes = SmSmem<NT, NACC>::TOTAL;
     cfg.stream = st;
@@ -1017,27 +1023,38 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
                                           : launch_simt<float>(x, gate, W, q, k, v, M, R, D, nq, nk, swiglu_F, eps, st);
     }
     const int w_rows = swiglu_F > 0 ? 2 * swiglu_F : nq + 2 * nk;
-    if (impl == 0 && M <= 128 && (size_t)B * D * sizeof(float) <= SmSmem<64, 1>::GATE_MAX) {
-        // few rows: weights as the A operand, one CTA per 128 output features
-        const int NT = M <= 64 ? 64 : 128;
+    // Few rows: weights as the A operand, one CTA per 128 output features and group of rows. One group of 64 or 128 rows, or,
+    // while every (feature tile, group) still has an SM of its own, several groups of 64: the chain of a CTA stays as short as for
+    // one stream (100 rows as two groups of 64: 6.9 us against 10.0 as one group of 128; 200 rows: 7.x against 11.6 with the
+    // 256-row tiles).
+    const int sms = sm_count > 0 ? sm_count : 148;
+    const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
+    const int ftiles = (n_feat + 127) / 128;
+    auto gates_fit = [&](int nt) { return (size_t)std::min(B, (nt - 1) / R + 2) * D * sizeof(float) <= SmSmem<64, 1>::GATE_MAX; };
+    int NT = 0, groups = 1;
+    if (impl == 0) {
+        if (M <= 64 && gates_fit(64)) NT = 64;
+        else if (gates_fit(64) && ((M + 63) / 64) * ftiles <= sms) { NT = 64; groups = (M + 63) / 64; }
+        else if (M <= 128 && gates_fit(128)) NT = 128;
+    }
+    if (NT != 0) {
         CUtensorMap sx, sw;
         if (!tensor_map_2d_bf16(&sx, x, D, M, NT) || !tensor_map_2d_bf16(&sw, W, D, w_rows, 128)) return cudaErrorInvalidValue;
         QkParams sp;
         sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
         sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.n_tiles = 1; sp.swiglu_F = swiglu_F;
         sp.eps = eps; sp.status = status; sp.res = nullptr; sp.tma_out = 0;
-        const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
         // The contraction split over 4 CTAs per feature tile where the chain of steps is long enough to pay for a cluster
         // launch and its two barriers (16 steps or more: SwiGLU at D = 1024, 11.1 -> 10.0 us for one stream; the packed
         // projection's 8 steps got slower, 6.8 -> 8.3 us, and a split in two is slower than none for both), while every
         // slice keeps whole steps and the grid stays within the SMs.
-        const int chunks = D / kQkBK, ftiles = (n_feat + 127) / 128, cps = swiglu_F > 0 ? 1 : 2;
+        const int chunks = D / kQkBK, cps = swiglu_F > 0 ? 1 : 2;
         int ks = 1;
-        if (chunks / cps >= 16 && chunks % (4 * cps) == 0 && ftiles * 4 <= (sm_count > 0 ? sm_count : 148)) ks = 4;
+        if (chunks / cps >= 16 && chunks % (4 * cps) == 0 && ftiles * groups * 4 <= sms) ks = 4;
         sp.ksplit = ks;
         const unsigned grid = (unsigned)(ftiles * ks);
-        if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, st) : launch_small<128, 2>(sx, sw, sp, grid, st);
-        return NT == 64 ? launch_small<64, 1>(sx, sw, sp, grid, st) : launch_small<128, 1>(sx, sw, sp, grid, st);
+        if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 2>(sx, sw, sp, grid, 1u, st);
+        return NT == 64 ? launch_small<64, 1>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 1>(sx, sw, sp, grid, 1u, st);
     }
     CUtensorMap mx, mw;
     if (!tensor_map_2d_bf16(&mx, x, D, M, kQkBM) || !tensor_map_2d_bf16(&mw, W, D, w_rows, kQkBN / 2)) return cudaErrorInvalidValue;
@@ -1055,24 +1072,44 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
                      : launch_tc<1>(mx, mw, p, (n_out + kQkBN - 1) / kQkBN, sm_count, st);
 }
 
-// out [M][N] = res + a [M][K] W [N][K]^T for at most 128 rows (K a multiple of 64): the few-rows kernel without its norm stage
+// out [M][N] = res + a [M][K] W [N][K]^T for few rows (K a multiple of 64): the few-rows kernel without its norm stage
+// Row groups of the plain projection: groups of 64 rows pay while the contraction can still be split over 4 CTAs per (feature
+// tile, group) inside the SMs (a split in two is slower than none, and unsplit the chain of a long contraction loses to the
+// 256-row tiles): 200 rows x 4096 -> 1024 10.9 us against 15.4 with the tiles; x 2048 9.6 against 9.2, so only contractions of
+// 4096 and more take the groups; 300 rows and more: the tiles.
+static int linear_small_groups(int M, int K, int N)
+{
+    const int chunks = K / kQkBK, ftiles = (N + 127) / 128, groups = (M + 63) / 64;
+    if (M <= 64) return 1;
+    if (chunks % 8 == 0 && chunks >= 64 && ftiles * groups * 4 <= 148) return groups;
+    return M <= 128 ? 1 : 0;       // one group of 128 rows, or not this kernel's shape
+}
+
+bool linear_small_takes(int M, int K, int N)
+{
+    return K % kQkBK == 0 && linear_small_groups(M, K, N) > 0;
+}
+
 cudaError_t launch_linear_small(const void *a, const void *W, const void *res, void *out, int M, int K, int N, uint32_t *status, cudaStream_t st)
 {
-    const int NT = M <= 64 ? 64 : 128;
+    const int ftiles = (N + 127) / 128;
+    const int groups = linear_small_groups(M, K, N);
+    const int NT = (groups > 1 || M <= 64) ? 64 : 128;
     CUtensorMap sx, sw;
     if (!tensor_map_2d_bf16(&sx, a, K, M, NT) || !tensor_map_2d_bf16(&sw, W, K, N, 128)) return cudaErrorInvalidValue;
     QkParams sp;
     sp.gate = nullptr; sp.q = (__nv_bfloat16 *)out; sp.k = nullptr; sp.v = nullptr;
     sp.M = M; sp.R = M; sp.B = 1; sp.D = K; sp.nq = N; sp.nk = 0; sp.m_tiles = 1; sp.n_tiles = 1; sp.swiglu_F = 0;
     sp.eps = 0.f; sp.status = status; sp.res = (const __nv_bfloat16 *)res; sp.tma_out = 0;
-    // split the contraction over up to 8 CTAs per feature tile while every slice keeps whole steps of two 64-column chunks and
-    // the grid stays within the SMs
-    const int chunks = K / kQkBK, ftiles = (N + 127) / 128;
+    // split the contraction over up to 8 CTAs per (feature tile, row group) while every slice keeps whole steps of two 64-column
+    // chunks and the grid stays within the SMs
+    const int chunks = K / kQkBK;
     int ks = 1;
-    while (ks < 8 && chunks % (4 * ks) == 0 && chunks / (2 * ks) >= 2 && ftiles * 2 * ks <= 148) ks *= 2;
+    if (groups > 1) ks = 4;       // (clusters of 8 CTAs: the device holds 16 of them at once)
+    else while (ks < 8 && chunks % (4 * ks) == 0 && chunks / (2 * ks) >= 2 && ftiles * 2 * ks <= 148) ks *= 2;
     sp.ksplit = ks;
     const unsigned grid = (unsigned)(ftiles * ks);
-    return NT == 64 ? launch_small<64, 1, true>(sx, sw, sp, grid, st) : launch_small<128, 1, true>(sx, sw, sp, grid, st);
+    return NT == 64 ? launch_small<64, 1, true>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 1, true>(sx, sw, sp, grid, 1u, st);
 }
 
 }  // namespace reflex

@@ -126,6 +126,7 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
 // 1 = plain kernel, 2 = tensor cores with 256-row tiles whatever M is
 cudaError_t launch_linear_residual(const void *a, const void *W, const void *res, void *out, int M, int K, int N, int dtype, int impl,
                                    uint32_t *status, cudaStream_t st);
+bool linear_small_takes(int M, int K, int N);
 cudaError_t launch_linear_small(const void *a, const void *W, const void *res, void *out, int M, int K, int N, uint32_t *status, cudaStream_t st);
 bool gate_tc_supported(int B, int D, int Cd, int Hd);
 cudaError_t launch_gate_tc(const void *cond, const void *W1, const void *b1, const void *W2, const void *b2, float *gate_buf, int L, int B,

@@ -788,6 +788,22 @@ def test_norm_swiglu_more_tiles_than_sm_pairs(U):
     _norm_swiglu_case(U, w, 1000, 0, "norm+swiglu 100 tiles", streams=[0, 1, 63, 64, 90, 127])
 
 
+@pytest.mark.parametrize("B", [2, 5, 8])
+def test_projections_row_groups_of_the_few_rows_kernel(U, B):
+    """100, 250 and 400 rows: the few-rows kernel (weights as the A operand) on groups of 64 rows, one CTA per feature tile
+    and group; the last group ragged, streams straddling group boundaries (their gates staged per group). The fused gate/up
+    projection takes the groups up to 256 rows (32 feature tiles x 4 groups), the plain projection for a contraction of
+    4096 (split over clusters of 4), the packed Q/K/V projection up to 448 rows."""
+    w = synth.CONFIGS["cfg2"].with_(B=B)
+    streams = sorted({0, 1, B // 2, B - 1})
+    _norm_qkv_case(U, w, 0, f"norm+qkv {B * w.T} rows in groups", streams=streams)
+    _norm_swiglu_case(U, w, 4096, 0, f"norm+swiglu {B * w.T} rows in groups", streams=streams[:2])
+    M = B * w.T
+    rows = sorted({0, 63, 64, 65, M // 2, M - 1} & set(range(M)))
+    _linear_case(U, synth.DTYPE_BF16, M, 4096, 1024, 0, f"linear {M} rows in groups", rows=rows, seed=71)
+    _linear_case(U, synth.DTYPE_BF16, M, 2048, 1000, 0, f"linear {M} rows, contraction 2048", rows=rows, seed=72)
+
+
 def test_norm_qkv_short_streams_and_fallback(U):
     """Rows per stream far below the tile height: with R = 13 a 128-row tile covers 11 streams (all their gates in shared
     memory); with R = 3 the gates of a tile's 44 streams no longer fit beside the stages and the call falls back to the plain
