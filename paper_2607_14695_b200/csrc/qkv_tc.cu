@@ -1025,8 +1025,8 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
     const int w_rows = swiglu_F > 0 ? 2 * swiglu_F : nq + 2 * nk;
     // Few rows: weights as the A operand, one CTA per 128 output features and group of rows. One group of 64 or 128 rows, or,
     // while every (feature tile, group) still has an SM of its own, several groups of 64: the chain of a CTA stays as short as for
-    // one stream (100 rows as two groups of 64: 6.9 us against 10.0 as one group of 128; 200 rows: 7.x against 11.6 with the
-    // 256-row tiles).
+    // one stream (100 rows as two groups of 64: 6.6 us against 10.0 as one group of 128; 200 rows: 6.8 against 11.6 with the
+    // 256-row tiles). Beyond that, groups of 128 rows under the same condition (450-800 rows: 10.4 us against 11.7-12.2).
     const int sms = sm_count > 0 ? sm_count : 148;
     const int n_feat = swiglu_F > 0 ? swiglu_F : nq + 2 * nk;
     const int ftiles = (n_feat + 127) / 128;
@@ -1035,7 +1035,7 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
     if (impl == 0) {
         if (M <= 64 && gates_fit(64)) NT = 64;
         else if (gates_fit(64) && ((M + 63) / 64) * ftiles <= sms) { NT = 64; groups = (M + 63) / 64; }
-        else if (M <= 128 && gates_fit(128)) NT = 128;
+        else if (gates_fit(128) && ((M + 127) / 128) * ftiles <= sms) { NT = 128; groups = (M + 127) / 128; }
     }
     if (NT != 0) {
         CUtensorMap sx, sw;
@@ -1053,8 +1053,8 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
         if (chunks / cps >= 16 && chunks % (4 * cps) == 0 && ftiles * groups * 4 <= sms) ks = 4;
         sp.ksplit = ks;
         const unsigned grid = (unsigned)(ftiles * ks);
-        if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 2>(sx, sw, sp, grid, 1u, st);
-        return NT == 64 ? launch_small<64, 1>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 1>(sx, sw, sp, grid, 1u, st);
+        if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 2>(sx, sw, sp, grid, (unsigned)groups, st);
+        return NT == 64 ? launch_small<64, 1>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 1>(sx, sw, sp, grid, (unsigned)groups, st);
     }
     CUtensorMap mx, mw;
     if (!tensor_map_2d_bf16(&mx, x, D, M, kQkBM) || !tensor_map_2d_bf16(&mw, W, D, w_rows, kQkBN / 2)) return cudaErrorInvalidValue;
@@ -1082,7 +1082,7 @@ static int linear_small_groups(int M, int K, int N)
     const int chunks = K / kQkBK, ftiles = (N + 127) / 128, groups = (M + 63) / 64;
     if (M <= 64) return 1;
     if (chunks % 8 == 0 && chunks >= 64 && ftiles * groups * 4 <= 148) return groups;
-    return M <= 128 ? 1 : 0;       // one group of 128 rows, or not this kernel's shape
+    return M <= 128 ? 1 : 0;       // one group of 128 rows, or not this kernel's shape (groups of 128 rows: 16.5 us for 300 x 4096 against 15.5)
 }
 
 bool linear_small_takes(int M, int K, int N)

@@ -788,10 +788,10 @@ def test_norm_swiglu_more_tiles_than_sm_pairs(U):
     _norm_swiglu_case(U, w, 1000, 0, "norm+swiglu 100 tiles", streams=[0, 1, 63, 64, 90, 127])
 
 
-@pytest.mark.parametrize("B", [2, 5, 8])
+@pytest.mark.parametrize("B", [2, 5, 8, 13])
 def test_projections_row_groups_of_the_few_rows_kernel(U, B):
-    """100, 250 and 400 rows: the few-rows kernel (weights as the A operand) on groups of 64 rows, one CTA per feature tile
-    and group; the last group ragged, streams straddling group boundaries (their gates staged per group). The fused gate/up
+    """100, 250, 400 and 650 rows: the few-rows kernel (weights as the A operand) on groups of 64 rows (of 128 where those
+    would outnumber the SMs), one CTA per feature tile and group; the last group ragged, streams straddling group boundaries (their gates staged per group). The fused gate/up
     projection takes the groups up to 256 rows (32 feature tiles x 4 groups), the plain projection for a contraction of
     4096 (split over clusters of 4), the packed Q/K/V projection up to 448 rows."""
     w = synth.CONFIGS["cfg2"].with_(B=B)
