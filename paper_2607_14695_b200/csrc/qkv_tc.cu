@@ -792,47 +792,69 @@ norm_linear_small_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_
             if constexpr (!PLAIN) {
                 const int t = threadIdx.x - 64;
                 if (t < rows_mine) {
-                    float ss = 0.f;
+                    float ss = 0.f, sv[8];
                     const uint32_t a0 = smem_u32(rsm + r0 + t);
-                    for (int q = 0; q < ksplit; ++q) {
-                        float v;
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(mapa(a0, (uint32_t)q)) : "memory");
-                        ss += v;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {      // (all slices' loads in flight together)
+                        sv[q] = 0.f;
+                        if (q < ksplit) asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(sv[q]) : "r"(mapa(a0, (uint32_t)q)) : "memory");
                     }
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) ss += sv[q];
                     rs_mine[t] = rsqrtf(ss * (1.f / (float)p.D) + p.eps);
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             const float *part = reinterpret_cast<const float *>(smem + S::OFF_W);
             const int n_feat = swiglu ? p.swiglu_F : p.nq + 2 * p.nk;
-            for (int e = threadIdx.x - 64; e < rows_mine * 128; e += 256) {
-                const int r = r0 + e / 128, fl = e % 128, f = f0 + fl;
+            // four consecutive features of one row per thread and round: one 16-byte load from every slice's partial sums, all of
+            // them issued before the first is used. (One feature per thread, its slices read one after the other: 32 dependent
+            // round trips through distributed shared memory per thread, 7.7 k of the kernel's 10 k cycles for one stream.)
+            for (int e = threadIdx.x - 64; e < rows_mine * 32; e += 256) {
+                const int r = r0 + e / 32, fl = (e % 32) * 4, f = f0 + fl;
                 const int rg = row0 + r;
-                if (rg >= p.M || f >= n_feat) continue;
-                float sum = 0.f, sum_up = 0.f;
                 const uint32_t a0 = smem_u32(part + r * 128 + fl);
-                for (int q = 0; q < ksplit; ++q) {
-                    float v;
-                    const uint32_t aq = mapa(a0, (uint32_t)q);
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(aq) : "memory");
-                    sum += v;
-                    if (swiglu) {
-                        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(aq + (uint32_t)NT * 128 * 4) : "memory");
-                        sum_up += v;
+                float4 v[8], u[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    v[q] = make_float4(0.f, 0.f, 0.f, 0.f); u[q] = v[q];
+                    if (q < ksplit) {
+                        const uint32_t aq = mapa(a0, (uint32_t)q);
+                        asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[q].x), "=f"(v[q].y), "=f"(v[q].z), "=f"(v[q].w) : "r"(aq) : "memory");
+                        if (swiglu)
+                            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(u[q].x), "=f"(u[q].y), "=f"(u[q].z), "=f"(u[q].w)
+                                         : "r"(aq + (uint32_t)NT * 128 * 4) : "memory");
                     }
                 }
+                float sum[4] = {0.f, 0.f, 0.f, 0.f}, sum_up[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    sum[0] += v[q].x; sum[1] += v[q].y; sum[2] += v[q].z; sum[3] += v[q].w;
+                    sum_up[0] += u[q].x; sum_up[1] += u[q].y; sum_up[2] += u[q].z; sum_up[3] += u[q].w;
+                }
+                if (rg >= p.M || f >= n_feat) continue;      // (feature counts are multiples of 8: the four stand or fall together, in one tensor)
                 __nv_bfloat16 *dst;
                 if (swiglu || f < p.nq) dst = p.q + (size_t)rg * p.nq + f;
                 else if (f < p.nq + p.nk) dst = p.k + (size_t)rg * p.nk + (f - p.nq);
                 else dst = p.v + (size_t)rg * p.nk + (f - p.nq - p.nk);
                 if constexpr (PLAIN) {
-                    if (p.res) sum += __bfloat162float(p.res[(size_t)rg * p.nq + f]);
+                    if (p.res) {
+                        const uint2 rr = *reinterpret_cast<const uint2 *>(p.res + (size_t)rg * p.nq + f);
+                        sum[0] += __uint_as_float(rr.x << 16); sum[1] += __uint_as_float(rr.x & 0xFFFF0000u);
+                        sum[2] += __uint_as_float(rr.y << 16); sum[3] += __uint_as_float(rr.y & 0xFFFF0000u);
+                    }
                 } else {
                     const float rs = rs_mine[r - r0];
-                    sum *= rs;
-                    if (swiglu) sum = silu_mul(sum, sum_up * rs);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        sum[i] *= rs;
+                        if (swiglu) sum[i] = silu_mul(sum[i], sum_up[i] * rs);
+                    }
                 }
-                *dst = __float2bfloat16_rn(sum);
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(sum[0], sum[1]), h1 = __floats2bfloat162_rn(sum[2], sum[3]);
+                uint2 o;
+                o.x = *reinterpret_cast<uint32_t *>(&h0); o.y = *reinterpret_cast<uint32_t *>(&h1);
+                *reinterpret_cast<uint2 *>(dst) = o;
             }
         }
         cluster_arrive();
@@ -1044,13 +1066,16 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
         sp.gate = gate; sp.q = (__nv_bfloat16 *)q; sp.k = (__nv_bfloat16 *)k; sp.v = (__nv_bfloat16 *)v;
         sp.M = M; sp.R = R; sp.B = B; sp.D = D; sp.nq = nq; sp.nk = nk; sp.m_tiles = 1; sp.n_tiles = 1; sp.swiglu_F = swiglu_F;
         sp.eps = eps; sp.status = status; sp.res = nullptr; sp.tma_out = 0;
-        // The contraction split over 4 CTAs per feature tile where the chain of steps is long enough to pay for a cluster
-        // launch and its two barriers (16 steps or more: SwiGLU at D = 1024, 11.1 -> 10.0 us for one stream; the packed
-        // projection's 8 steps got slower, 6.8 -> 8.3 us, and a split in two is slower than none for both), while every
-        // slice keeps whole steps and the grid stays within the SMs.
+        // The contraction split over 4 CTAs per (feature tile, row group) where the chain has 8 steps or more and the grid stays
+        // within the SMs, every slice keeping whole steps: the slices' sums meet through distributed shared memory, four
+        // features per thread and all slices' loads in flight together (one stream: Q/K/V 6.4 -> 5.9 us, gate/up 11.1 -> 8.6;
+        // with one feature per thread and its slices read one after the other the reduction alone took 7.7 k cycles and
+        // the split made the Q/K/V projection slower). A split in two only pays for chains of 16 steps (gate/up, 100 rows:
+        // 10.3 -> 9.5 us; Q/K/V: 6.6 -> 6.8).
         const int chunks = D / kQkBK, cps = swiglu_F > 0 ? 1 : 2;
         int ks = 1;
-        if (chunks / cps >= 16 && chunks % (4 * cps) == 0 && ftiles * groups * 4 <= sms) ks = 4;
+        if (chunks / cps >= 8 && chunks % (4 * cps) == 0 && ftiles * groups * 4 <= sms) ks = 4;
+        else if (chunks / cps >= 16 && chunks % (2 * cps) == 0 && ftiles * groups * 2 <= sms) ks = 2;
         sp.ksplit = ks;
         const unsigned grid = (unsigned)(ftiles * ks);
         if (swiglu_F > 0) return NT == 64 ? launch_small<64, 2>(sx, sw, sp, grid, (unsigned)groups, st) : launch_small<128, 2>(sx, sw, sp, grid, (unsigned)groups, st);
@@ -1073,16 +1098,16 @@ cudaError_t launch_adarmsnorm_qkv(const void *x, const float *gate, const void *
 }
 
 // out [M][N] = res + a [M][K] W [N][K]^T for few rows (K a multiple of 64): the few-rows kernel without its norm stage
-// Row groups of the plain projection: groups of 64 rows pay while the contraction can still be split over 4 CTAs per (feature
-// tile, group) inside the SMs (a split in two is slower than none, and unsplit the chain of a long contraction loses to the
-// 256-row tiles): 200 rows x 4096 -> 1024 10.9 us against 15.4 with the tiles; x 2048 9.6 against 9.2, so only contractions of
-// 4096 and more take the groups; 300 rows and more: the tiles.
+// Row groups of the plain projection: groups of 64 rows pay while the contraction (2048 or more) can still be split over 4 CTAs
+// per (feature tile, group) inside the SMs: 200 rows x 4096 -> 1024 7.8 us against 15.4 with the 256-row tiles, x 2048 6.4
+// against 9.2 (before the slices' sums were added four features per thread with all loads in flight: 10.9 and 9.6); 300 rows
+// and more: the tiles.
 static int linear_small_groups(int M, int K, int N)
 {
     const int chunks = K / kQkBK, ftiles = (N + 127) / 128, groups = (M + 63) / 64;
     if (M <= 64) return 1;
-    if (chunks % 8 == 0 && chunks >= 64 && ftiles * groups * 4 <= 148) return groups;
-    return M <= 128 ? 1 : 0;       // one group of 128 rows, or not this kernel's shape (groups of 128 rows: 16.5 us for 300 x 4096 against 15.5)
+    if (chunks % 8 == 0 && chunks >= 32 && ftiles * groups * 4 <= 148) return groups;
+    return M <= 128 ? 1 : 0;       // one group of 128 rows, or not this kernel's shape
 }
 
 bool linear_small_takes(int M, int K, int N)
