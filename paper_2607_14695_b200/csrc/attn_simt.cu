@@ -206,23 +206,34 @@ attn_merge_kernel(AttnParams p)
     float acc[DPL];
 #pragma unroll
     for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-    for (int s = 0; s < p.nsplit; ++s) {
-        const float ws = __shfl_sync(0xffffffffu, w, s);
-        if (ws == 0.f) continue;               // an empty slice: its O row was never written
-        const float *po = partial_o(p.partials, slot0 + s, d) + lane * DPL;
-        float f[DPL];
-        if constexpr (DPL % 4 == 0) {
+    // Slices in batches of eight: all of a batch's loads are issued before the first is used (guarded one by one, every slice
+    // was an L2 round trip of its own in front of the next). An empty slice never wrote its O row: whatever is read there
+    // is dropped by the weight test, not multiplied by zero.
+    for (int s0 = 0; s0 < p.nsplit; s0 += 8) {
+        float f[8][DPL], ws[8];
 #pragma unroll
-            for (int i = 0; i < DPL; i += 4) {
-                const float4 v = *reinterpret_cast<const float4 *>(po + i);
-                f[i] = v.x; f[i + 1] = v.y; f[i + 2] = v.z; f[i + 3] = v.w;
+        for (int j = 0; j < 8; ++j) {
+            const int s = min(s0 + j, p.nsplit - 1);
+            ws[j] = s0 + j < p.nsplit ? __shfl_sync(0xffffffffu, w, s) : 0.f;
+            const float *po = partial_o(p.partials, slot0 + s, d) + lane * DPL;
+            if constexpr (DPL % 4 == 0) {
+#pragma unroll
+                for (int i = 0; i < DPL; i += 4) {
+                    const float4 v = *reinterpret_cast<const float4 *>(po + i);
+                    f[j][i] = v.x; f[j][i + 1] = v.y; f[j][i + 2] = v.z; f[j][i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < DPL; ++i) f[j][i] = po[i];
             }
-        } else {
-#pragma unroll
-            for (int i = 0; i < DPL; ++i) f[i] = po[i];
         }
 #pragma unroll
-        for (int i = 0; i < DPL; ++i) acc[i] = fmaf(f[i], ws, acc[i]);
+        for (int j = 0; j < 8; ++j) {
+            if (ws[j] != 0.f) {
+#pragma unroll
+                for (int i = 0; i < DPL; ++i) acc[i] = fmaf(f[j][i], ws[j], acc[i]);
+            }
+        }
     }
     const float inv = 1.f / l;
 #pragma unroll
