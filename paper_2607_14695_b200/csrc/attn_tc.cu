@@ -873,3 +873,10 @@ cudaError_t launch_attention_tc(const AttnParams &p, uint32_t *status, bool two_
 }
 
 }  // namespace reflex
+
+#ifdef REFLEX_TRACE
+extern "C" int reflex_debug_tc2_trace(long long *out)
+{
+    return (int)cudaMemcpyFromSymbol(out, reflex::g_tc2_trace, sizeof(long long) * 2 * 4 * 16 * 16);
+}
+#endif

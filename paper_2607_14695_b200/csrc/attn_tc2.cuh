@@ -27,11 +27,12 @@
 
 namespace reflex {
 
-// Optional timeline of the first cluster (debug builds only: -DREFLEX_TRACE): clock64 stamps into the (otherwise
-// unused) split-K partial area. Compiled out of the product library.
+// Optional timeline of the first cluster (debug builds only: -DREFLEX_TRACE): clock64 stamps into a device array that
+// reflex_debug_tc2_trace() copies out. Compiled out of the product library.
 #ifdef REFLEX_TRACE
+__device__ long long g_tc2_trace[2 * 4 * 16 * 16];
 #define TC2_TRACE(role, slot, ev) do { if (blockIdx.x < 2 && (slot) < 16 && (ev) < 16) \
-    reinterpret_cast<long long *>(p.partials)[((blockIdx.x * 4 + (role)) * 16 + (slot)) * 16 + (ev)] = clock64(); } while (0)
+    g_tc2_trace[((blockIdx.x * 4 + (role)) * 16 + (slot)) * 16 + (ev)] = clock64(); } while (0)
 #else
 #define TC2_TRACE(role, slot, ev) do { } while (0)
 #endif
@@ -642,6 +643,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (p.nsplit > 1) {
                 // key-split unit: leave (m, l, unnormalised O) for the merge kernel; m in natural-log units like the other kernels
                 if (pml && part == 0) { pml[0] = (m_ref == -INFINITY) ? -INFINITY : m_ref * p.scale; pml[1] = l; }
+                if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 6);
                 if (u + u_stride >= n_units) {
                     // The cluster's last unit (its only one when few streams are split finely): the Q tile and the K stages are
                     // idle, so the whole fp32 tile (128 rows x head_dim) is staged there, every thread dropping its half row as
@@ -697,6 +699,7 @@ attn_tc2_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 }
+                if (threadIdx.x == 64) TC2_TRACE(2, ui_s, 7);
                 asm volatile("bar.sync 1, %0;" ::"n"(SMT) : "memory");   // every thread has read the row sums before the next unit's maxima land there
                 continue;
             }
