@@ -78,11 +78,16 @@ __device__ __forceinline__ void lin_tma_store_2d(const CUtensorMap *map, uint32_
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
 }
 
-template <int BN>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kLinThreads, 1)
+// KS = 2 (128-column tiles only): the cluster holds the two pairs that share an output tile, each taking half of the contraction;
+// at the end every CTA stages the 64 columns its counterpart in the other pair finishes as fp32 in the idle stage ring, and takes
+// the counterpart's share of its own 64 columns from there through distributed shared memory. Launched with the cluster shape as
+// a launch attribute (2 KS CTAs).
+template <int BN, int KS>
+__global__ void __launch_bounds__(kLinThreads, 1)
 linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                      const __grid_constant__ CUtensorMap tm_res, const __grid_constant__ CUtensorMap tm_out, LinParams p)
 {
+    static_assert(KS == 1 || (KS == 2 && BN == 128), "contraction split");
     using S = LinSmem<BN>;
     constexpr int NST = S::NST;
     extern __shared__ uint8_t smem_raw[];
@@ -93,11 +98,15 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + S::OFF_BAR + 8 * S::C_COUNT);
     volatile uint32_t *abort_flag = tmem_slot + 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();
-    const int pair = blockIdx.x >> 1;
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t rank = crank & 1u;                                        // rank inside the pair
+    const int kq = KS > 1 ? (int)(crank >> 1) : 0;                           // which part of the contraction this pair takes
+    const uint16_t pair_mask = (uint16_t)(3u << (crank & ~1u));              // both CTAs of this pair, for multicast commits
+    const int pair = blockIdx.x / (2 * KS);                                  // output tile
     const int m0 = (pair % p.m_tiles) * (2 * kLinBM) + (int)rank * kLinBM;   // this CTA's first row
-    const int n0 = (pair / p.m_tiles) * BN;                                  // the pair's first output column
-    const int nk_steps = (p.K + kLinBK - 1) / kLinBK;                        // (columns past K come in as TMA's zeros)
+    const int n0 = (pair / p.m_tiles) * BN;                                  // the tile's first output column
+    const int nk_steps = ((p.K + kLinBK - 1) / kLinBK) / KS;                 // (columns past K come in as TMA's zeros; KS = 2: an even count)
+    const int k_first = kq * nk_steps;
     if (threadIdx.x == 64) LIN_TRACE(0);
 
     if (threadIdx.x == 0) {
@@ -135,6 +144,8 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         return false;
     };
 
+    [[maybe_unused]] bool split_ok = true;     // (KS = 2) this thread's waits all came through
+
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
@@ -145,13 +156,16 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 if (!ok) break;
                 // both CTAs' loads complete on the leader's barrier: the issuing thread there waits for all four at once
                 if (rank == 0) mbar_expect_tx(bar(S::C_FULL + s), 2 * (S::A_STAGE + S::B_STAGE));
-                lin_tma2_load_2d(base + S::OFF_A + s * S::A_STAGE, &tm_a, bar(S::C_FULL + s) & kPeerBitMask, ks * kLinBK, m0);
-                lin_tma2_load_2d(base + S::OFF_B + s * S::B_STAGE, &tm_w, bar(S::C_FULL + s) & kPeerBitMask, ks * kLinBK, n0 + (int)rank * (BN / 2));
+                lin_tma2_load_2d(base + S::OFF_A + s * S::A_STAGE, &tm_a, bar(S::C_FULL + s) & kPeerBitMask, (k_first + ks) * kLinBK, m0);
+                lin_tma2_load_2d(base + S::OFF_B + s * S::B_STAGE, &tm_w, bar(S::C_FULL + s) & kPeerBitMask, (k_first + ks) * kLinBK, n0 + (int)rank * (BN / 2));
             }
             if (ok) {
                 // the residual tile goes last: it is not needed before the epilogue, and ahead of the main loop's operands it
                 // would hold them up for the time 64 KB take to come in (measured: 0.7 us per launch)
-                if (p.has_res) {
+                if (p.has_res && KS > 1) {       // (only the 64 columns this CTA finishes)
+                    mbar_expect_tx(bar(S::C_RES), S::CHUNK);
+                    tma_load_2d(base + S::OFF_RES + kq * S::CHUNK, &tm_res, bar(S::C_RES), n0 + kq * 64, m0);
+                } else if (p.has_res) {
                     mbar_expect_tx(bar(S::C_RES), S::RES_BYTES);
 #pragma unroll
                     for (int ch = 0; ch < BN / 64; ++ch) tma_load_2d(base + S::OFF_RES + ch * S::CHUNK, &tm_res, bar(S::C_RES), n0 + ch * 64, m0);
@@ -179,9 +193,9 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     umma_desc_advance(ad, 32);
                     umma_desc_advance(bd, 32);
                 }
-                umma2_commit_mc_elect(bar(S::C_EMPTY + s), (uint16_t)3);
+                umma2_commit_mc_elect(bar(S::C_EMPTY + s), pair_mask);
             }
-            umma2_commit_mc_elect(bar(S::C_ACC), (uint16_t)3);   // also after a wait that ran out: the epilogue warps must not wait for nothing
+            umma2_commit_mc_elect(bar(S::C_ACC), pair_mask);   // also after a wait that ran out: the epilogue warps must not wait for nothing
         }
     } else {
         // ---------------- epilogue: two threads per row, each owns BN / 2 columns ----------------
@@ -195,6 +209,29 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // threads, 16 bytes per row and instruction, the residual cost the main loop 2.5 us: what an SM takes in from
         // the L2 is what limits this kernel, and half-used sectors waste it.)
         bool ok = wait(S::C_RES, 0u, 3);
+        if constexpr (KS > 1) {
+            // Contraction split: thread (row, half) holds this pair's share of columns [64 half, 64 half + 64) of its row. The
+            // half that the counterpart CTA (same rank, other pair) finishes goes to shared memory as fp32, 16-byte pieces at
+            // [row][piece ^ (row % 16)]; the other half stays in tensor memory until the cluster has met.
+            ok = wait(S::C_ACC, 0u, 4) && ok;
+            if (threadIdx.x == 64) LIN_TRACE(4);
+            tc_fence_after();
+            split_ok = ok;
+            if (half != kq) {
+                uint4 *stage = reinterpret_cast<uint4 *>(smem + S::OFF_A);     // [128 rows][16 pieces]; the stage ring is idle
+                static_assert(S::NST * S::A_STAGE >= 128u * 64u * 4u, "staging area of the split");
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    uint32_t acc[32];
+                    tmem_ld32(tmem + lane_addr + half * 64 + g * 32, acc);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        stage[row * 16 + ((g * 8 + i) ^ (row & 15))] = ok ? make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3])
+                                                                           : make_uint4(0x7fc00000u, 0x7fc00000u, 0x7fc00000u, 0x7fc00000u);
+                }
+            }
+        } else {
         constexpr int CPT = BN / 2 / 64;              // 64-column chunks per thread
         uint4 rr[CPT * 8];
 #pragma unroll
@@ -244,12 +281,73 @@ linear_res_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // (the staging buffer has been read; the writes themselves are complete when the grid is)
         if (quarter == 0 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         if (warp == 4 && lane == 0) LIN_TRACE(6);
+        }
+    }
+
+    if constexpr (KS > 1) {
+        // (cluster barriers are warp-aligned: the lanes of the producer warp that idled while lane 0 ran the loads must not
+        // reach them before lane 0 does, so the CTA meets first)
+        __syncthreads();
+        cluster_arrive();
+        cluster_wait();       // every CTA's staged half is in place
+        if (warp >= 2) {
+            // both threads of a row finish 32 of the 64 columns each
+            const int half = (warp - 2) >> 2;
+            const int quarter = warp & 3, row = quarter * 32 + lane;
+            const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+            // the counterpart's share of this thread's 32 columns: 8 loads through distributed shared memory, all in flight
+            const uint32_t peer = crank ^ 2u;
+            const uint32_t st0 = base + S::OFF_A + (uint32_t)row * 256u;
+            float4 pv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t a = mapa(st0 + (uint32_t)(((half * 8 + j) ^ (row & 15)) << 4), peer);
+                asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(pv[j].x), "=f"(pv[j].y), "=f"(pv[j].z), "=f"(pv[j].w) : "r"(a) : "memory");
+            }
+            uint8_t *rowp = smem + S::OFF_RES + kq * S::CHUNK + row * 128;     // residual in, output out: one chunk of 64 columns
+            uint4 rr[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                rr[j] = make_uint4(0u, 0u, 0u, 0u);
+                if (p.has_res) rr[j] = *reinterpret_cast<const uint4 *>(rowp + (((half * 4 + j) ^ (row & 7)) << 4));
+            }
+            tc_fence_after();
+            uint32_t acc[32];
+            tmem_ld32(tmem + lane_addr + kq * 64 + half * 32, acc);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 t = rr[i];
+                const uint32_t rv[4] = {t.x, t.y, t.z, t.w};
+                const float4 q0 = pv[2 * i], q1 = pv[2 * i + 1];
+                const float pp[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+                uint32_t ov[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float v0 = __uint_as_float(acc[8 * i + 2 * k]) + pp[2 * k] + __uint_as_float(rv[k] << 16);
+                    float v1 = __uint_as_float(acc[8 * i + 2 * k + 1]) + pp[2 * k + 1] + __uint_as_float(rv[k] & 0xFFFF0000u);
+                    if (!split_ok) v0 = v1 = __int_as_float(0x7fc00000);
+                    __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                    ov[k] = *reinterpret_cast<uint32_t *>(&h);
+                }
+                *reinterpret_cast<uint4 *>(rowp + (((half * 4 + i) ^ (row & 7)) << 4)) = make_uint4(ov[0], ov[1], ov[2], ov[3]);
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 256;" ::: "memory");     // the chunk's 256 threads
+            if (warp == 2 && lane == 0) {
+                if (m0 < p.M && n0 + kq * 64 < p.N) {
+                    lin_tma_store_2d(&tm_out, base + S::OFF_RES + kq * S::CHUNK, n0 + kq * 64, m0);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            }
+        }
     }
 
     tc_fence_before();
     __syncthreads();
     cluster_arrive();
-    cluster_wait();   // neither CTA retires while its partner can still touch its shared memory or barriers
+    cluster_wait();   // no CTA retires while another can still touch its shared memory or barriers
     if (warp == 1) tmem_dealloc2(tmem, BN);
     if (threadIdx.x == 64) LIN_TRACE(7);
 }
@@ -300,26 +398,28 @@ cudaError_t launch_lin_simt(const void *a, const void *W, const void *res, void 
     return e;
 }
 
-template <int BN>
+template <int BN, int KS>
 cudaError_t launch_lin_tc(const CUtensorMap &ma, const CUtensorMap &mw, const CUtensorMap &mr, const CUtensorMap &mo, const LinParams &p, int n_tiles,
                           cudaStream_t st)
 {
     static std::atomic<unsigned long long> attr_set{0};
     cudaError_t e0 = once_per_device(attr_set, [] {
-        return cudaFuncSetAttribute(linear_res_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LinSmem<BN>::TOTAL);
+        return cudaFuncSetAttribute(linear_res_tc_kernel<BN, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LinSmem<BN>::TOTAL);
     });
     if (e0 != cudaSuccess) return e0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2u * (unsigned)p.m_tiles * (unsigned)n_tiles);
+    cfg.gridDim = dim3(2u * KS * (unsigned)p.m_tiles * (unsigned)n_tiles);
     cfg.blockDim = dim3(kLinThreads);
     cfg.dynamicSmemBytes = LinSmem<BN>::TOTAL;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // a pair of CTAs, or the two pairs that split a tile's contraction
+    attr[1].val.clusterDim.x = 2u * KS; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_res_tc_kernel<BN>, ma, mw, mr, mo, p);
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, linear_res_tc_kernel<BN, KS>, ma, mw, mr, mo, p);
     count_launch();
     return e;
 }
@@ -351,8 +451,16 @@ cudaError_t launch_linear_residual(const void *a, const void *W, const void *res
         return cudaErrorInvalidValue;
     if (res) { if (!tensor_map_2d_bf16(&mr, res, N, M, kLinBM)) return cudaErrorInvalidValue; }
     else mr = mo;
-    if (narrow) return launch_lin_tc<128>(ma, mw, mr, mo, p, (N + 127) / 128, st);
-    return launch_lin_tc<256>(ma, mw, mr, mo, p, (N + 255) / 256, st);
+    if (narrow) {
+        // ... and the contraction in two halves on two pairs of a 4-CTA cluster while that still leaves every pair an SM pair of
+        // its own and the halves are long enough to pay for the exchange, which costs about 4 us (two cluster barriers, 32 KB
+        // per CTA through distributed shared memory, the slower pair's lag): 300-1000 rows x 4096 -> 1024 15.5-17.0 -> 12.9-15.0 us;
+        // x 2048 9.3-9.4 -> 9.8-11.0, so only contractions of 4096 and more are split
+        const int n_tiles = (N + 127) / 128, nk_all = (K + kLinBK - 1) / kLinBK;
+        if (p.m_tiles * n_tiles * 2 <= 74 && nk_all % 2 == 0 && nk_all >= 64) return launch_lin_tc<128, 2>(ma, mw, mr, mo, p, n_tiles, st);
+        return launch_lin_tc<128, 1>(ma, mw, mr, mo, p, n_tiles, st);
+    }
+    return launch_lin_tc<256, 1>(ma, mw, mr, mo, p, (N + 255) / 256, st);
 }
 
 }  // namespace reflex

@@ -909,6 +909,16 @@ def test_random_shapes_projections(U, case):
     _linear_case(U, synth.DTYPE_BF16, M, D, N, 0, name + " linear", rows=rows, seed=70)
 
 
+@pytest.mark.parametrize("M,K,N,residual", [(800, 4096, 1024, True), (800, 2048, 1024, True), (650, 4096, 1000, False), (1000, 4160, 512, True)])
+def test_linear_residual_bf16_mid_size_rows(U, M, K, N, residual):
+    """Between the few-rows form and full occupancy: 128-column tiles, and while two pairs per tile still fit the SM pairs
+    a contraction of 4096 or more split in two over a cluster of four CTAs (the halves meet through distributed shared
+    memory): 800 rows with both contractions of the expert (2048 stays unsplit), a ragged last column tile without a
+    residual in the split form, and an odd number of contraction steps (65), which stays unsplit. Rows from every row tile, both CTAs of a pair, and the ragged end."""
+    rows = sorted({0, 1, 127, 128, 255, 256, 300, M // 2, M - 130, M - 2, M - 1})
+    _linear_case(U, synth.DTYPE_BF16, M, K, N, 0, f"linear {M}x{K}->{N}", residual=residual, rows=rows, seed=73)
+
+
 def test_linear_residual_error_paths(U):
     rb = U.rb
     z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device=U.DEV)
