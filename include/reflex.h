@@ -261,8 +261,10 @@ int reflex_adarmsnorm_swiglu(reflex_cache_t *cache, const void *x, const float *
  *   res      device [M][N] dtype, or NULL for a projection without residual
  *   out      device [M][N] dtype (written); may be the same buffer as res (in-place update of the residual stream),
  *            must not overlap a
- *   impl     0: tensor cores when dtype is bf16 (256 x 256 output tiles per pair of SMs, 256 x 128 where those would leave
- *               most pairs idle; a kernel with the weights as the stationary operand when M <= 128 and K % 64 == 0),
+ *   impl     0: tensor cores when dtype is bf16 (256 x 256 output tiles per pair of SMs; 256 x 128 where those would leave
+ *               most pairs idle, a contraction of 4096 or more then split over two pairs of a cluster while they fit;
+ *               a kernel with the weights as the stationary operand when K % 64 == 0 and M <= 128, or M <= 256 in groups
+ *               of 64 rows for K >= 2048),
  *               else the plain kernel; 1: the plain kernel (fp32 FMAs, K <= 12288); 2: like 0 but always the 256-row tiles
  * Requirements: K % 8 == 0, 8 <= K <= 12288; N % 8 == 0; 16-byte aligned pointers.
  * Errors: REFLEX_ERR_INVALID_ARG (NULL pointer, unknown dtype or impl, out == a), REFLEX_ERR_SHAPE, REFLEX_ERR_ALIGN;
