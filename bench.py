@@ -16,7 +16,8 @@ Besides the headline (`value`, `ms_per_step`: exactly K steps after W warm-up st
   roofline    the attention kernel against its binding roof (tensor pipe or HBM, whichever floor is higher), sustained
               leg against the sustained peak, burst leg against the burst peak, the HBM fraction beside it
   chained_step   the step whose layers run AdaRMSNorm + packed Q/K/V projection -> attention, with its own roofline
-  extra       (default run only) the batch-1 stream of cfg3: per-tick latency over 50 ticks; the long-context attention of cfg5
+  extra       (default run only) the batch-1 stream of cfg3: per-tick latency over 50 ticks; the long-context attention of cfg5;
+              the whole expert step at 1, 4 and 16 streams
   e2e, e2e_expert   end to end from pinned host buffers: per-layer inputs of the path; and a whole expert step, where
               only the action chunk and the conditioning vectors cross PCIe
 """
@@ -632,6 +633,20 @@ def main():
         extra["cfg5_attention"]["roofline"].update({"traffic": t5, "traffic_source": src5, "bytes_per_launch": alg5["attn_bytes_per_launch"]})
         rb.reflex_cache_check_status(r5.cache)
         del r5
+        # the whole expert step at few streams (cfg4's shapes): where serving a handful of robots sits between cfg3 and cfg4
+        from paper_2607_14695_b200 import expert as ex_few
+        few = {}
+        for Bf in (1, 4, 16):
+            wf = w.with_(B=Bf)
+            rf = StepRunner(wf, device=dev)
+            mf = ex_few.ActionExpert(wf, rf.cache, ex_few.random_weights_device(wf, 4 * wf.D, device=dev), 4 * wf.D, device=dev)
+            gf = kernel_graphs(rf, lambda v: mf.step(rf.xa, rf.cond[v % wf.K], v % wf.K))
+            cool()
+            ms_f, mhz_f, _ = leg(lambda i: gf[i % len(gf)].replay(), 6, 1)
+            rb.reflex_cache_check_status(rf.cache)
+            few[str(Bf)] = {"expert_step_ms": ms_f, "sm_mhz": mhz_f, "us_per_layer": ms_f * 1e3 / wf.L}
+            del gf, mf, rf
+        extra["expert_step_by_streams"] = dict(few, what="whole action-expert step (CUDA graph, burst clocks) at 1, 4 and 16 streams of 50 tokens, cfg4's layer shapes, F = 4 D")
     sampler.stop()
 
     from paper_2607_14695_b200 import multi
